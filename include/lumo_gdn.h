@@ -1,0 +1,187 @@
+/* lumo_gdn.h - C ABI of the B200 (sm_100a) Gated DeltaNet tree verifier and committer.
+ *
+ * The library verifies every node of a speculative candidate tree through one Gated
+ * DeltaNet (GDN) layer and later replays the accepted path into the running state:
+ *
+ *   tree conv   y_i = SiLU(sum_j w[:,j] * x_{anc(i,3-j)})            (ancestry-gathered, width 4)
+ *   tree scan   R'_i = alpha_i R_parent(i);  delta_i = beta_i (v_i - R'_i k_i);
+ *               R_i = R'_i + delta_i k_i^T;  o_i = R_i q_i           (paper Eq. 2-3)
+ *   commit      the same update for the accepted nodes in path order, published in place,
+ *               plus the matching convolution history             (paper Algorithms 1 and 2)
+ *
+ * Conventions
+ *   - One GPU.  All tensor pointers are DEVICE pointers owned by the caller unless a
+ *     comment says HOST; the library never frees or reallocates caller memory.
+ *   - Row-major, innermost dimension contiguous.  B = batch, N = logical nodes per tree,
+ *     Ns >= N physical rows (padding), Hk q/k heads, Hv value heads (Hv % Hk == 0, value head
+ *     h uses q/k head h / (Hv/Hk)), d = d_k = d_v in {64, 128}, C = 2 Hk d + Hv d channels.
+ *   - Every per-node tensor is indexed by PHYSICAL row slot[b][i]; padding rows are never
+ *     read and their outputs are written as zeros.
+ *   - verify/commit/path_from_node only enqueue work on `stream` (a cudaStream_t passed as
+ *     void*); they never synchronise.  They may grow library-owned scratch on the first call
+ *     with a given shape; after that they allocate nothing.
+ *   - Host-detectable problems return a non-zero lumo_status and enqueue nothing;
+ *     lumo_last_error() then describes the problem.  Problems only the device can see are
+ *     reported per sequence in the `status` words (lumo_seq_status) and leave that sequence's
+ *     state and history untouched.  Kernels never trap and contain only bounded loops.
+ */
+#ifndef LUMO_GDN_H_
+#define LUMO_GDN_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lumo_ctx lumo_ctx;             /* device id + library-owned scratch */
+typedef struct lumo_tree_desc lumo_tree_desc; /* host + device copies of the topology tables */
+
+typedef enum {
+  LUMO_OK = 0,
+  LUMO_ERR_ARG = 1,         /* null / out-of-range argument */
+  LUMO_ERR_TREE = 2,        /* parent array or slot map violates the rules below */
+  LUMO_ERR_PATH = 3,        /* reserved for host-side path checks */
+  LUMO_ERR_UNSUPPORTED = 4, /* shape or dtype outside the supported set */
+  LUMO_ERR_CUDA = 5,        /* a CUDA runtime call failed */
+  LUMO_ERR_NOMEM = 6        /* scratch allocation failed */
+} lumo_status;
+
+typedef enum { LUMO_F32 = 0, LUMO_BF16 = 1 } lumo_dtype;
+
+/* Per-sequence device status words (first failing check wins, in this order). */
+typedef enum {
+  LUMO_SEQ_OK = 0,
+  LUMO_SEQ_BAD_LEN = 1,   /* accepted length < 0 or > lmax (or path longer than lmax) */
+  LUMO_SEQ_BAD_NODE = 2,  /* accepted entry outside [0, N) */
+  LUMO_SEQ_BAD_ROOT = 3,  /* first accepted entry is not a child of the pre-tree state */
+  LUMO_SEQ_BAD_LINK = 4,  /* accepted entry t is not a child of entry t-1 */
+  LUMO_SEQ_BAD_ROW = 5    /* state_row[b] >= n_state_rows */
+} lumo_seq_status;
+
+/* Integer tables of one tree (lumo_tree_desc_get).  The paper's tree descriptor holds parent
+ * indices, depth and the logical<->physical maps (Sec. "State and the execution boundary");
+ * the path tables are what its path-parallel schedule is built from (Sec. "Path-parallel
+ * verification and state lifetime").  All answers are unique. */
+typedef enum {
+  LUMO_TAB_DEPTH = 0,      /* [N]   1 + depth[parent]; a child of the pre-tree state has depth 1 */
+  LUMO_TAB_N_CHILD = 1,    /* [N] */
+  LUMO_TAB_CHILD_OFF = 2,  /* [N+2] CSR offsets: entry 0 = pre-tree state, entry i+1 = node i */
+  LUMO_TAB_CHILD_LIST = 3, /* [N]   children in ascending logical index */
+  LUMO_TAB_IS_LEAF = 4,    /* [N] */
+  LUMO_TAB_LEAVES = 5,     /* [P]   ascending */
+  LUMO_TAB_PATH_OFF = 6,   /* [P+1] CSR offsets of root-to-leaf paths */
+  LUMO_TAB_PATH_NODES = 7, /*       root-first node list of each path */
+  LUMO_TAB_ANC_WIN = 8,    /* [N*4] conv window: entry 3 = node, 2 = parent, ...; past the
+                                     pre-tree state -1/-2/-3 = most recent / 2nd / 3rd history row */
+  LUMO_TAB_SLOT_INV = 9,   /* [Ns]  logical node of each physical row, -1 = padding */
+  LUMO_TAB_CHAIN_HEAD = 10,  /* chain decomposition: a chain starts at each child of the pre-tree */
+  LUMO_TAB_CHAIN_OFF = 11,   /* state and at each non-lowest-index child and follows lowest-index */
+  LUMO_TAB_CHAIN_NODES = 12, /* children to a leaf; level 0 = starts at the pre-tree state, else  */
+  LUMO_TAB_CHAIN_LEVEL = 13, /* 1 + level of the chain holding the head's parent                  */
+  LUMO_TAB_CUT_NODES = 14,   /* parents (not the pre-tree state) of chain heads, ascending, unique */
+  LUMO_TAB_SCHEDULE = 15,    /* depth-first op list the scan kernel interprets, (kind<<24)|(flag<<20)|arg:
+                                kind 0 EMIT node (output from the parent's state; flag: keep delta on
+                                chip), 1 EMIT_DESCEND node (then turn the registers into the node's
+                                state), 2 DESCEND node (same, from the kept delta), 3 PUSH level,
+                                4 POP level (0xFFFF = reload the pre-tree state) */
+  LUMO_TAB_SCHEDULE_FULL = 16, /* same, materialising every node's state (snapshot modes) */
+  LUMO_TAB_COUNT = 17
+} lumo_table;
+
+/* ---- context ------------------------------------------------------------------------- */
+/* Creates a context on CUDA device `device`.  Returns LUMO_ERR_CUDA if no usable device.
+ * device = -1 creates a host-only context: descriptors can be built and their integer tables
+ * read, but every call that would launch returns LUMO_ERR_UNSUPPORTED (there is no CPU path). */
+int lumo_ctx_create(int device, lumo_ctx** out);
+void lumo_ctx_destroy(lumo_ctx* ctx);
+/* Text of the last error recorded on this context (ctx-owned, valid until the next call);
+ * with ctx == NULL, the last error of a failed lumo_ctx_create on this thread. */
+const char* lumo_last_error(const lumo_ctx* ctx);
+/* Bytes of library-owned device scratch currently held (for reporting). */
+int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx);
+
+/* Measurement aid.  While enabled, every kernel the library launches is bracketed by two CUDA
+ * events on the launch stream (up to 16384 launches between reads; later ones go untimed).
+ * lumo_ctx_timing_read waits for the recorded events, returns the launch count and summed
+ * device time of kernels of `kind` (lumo_kernel_kind) and, with reset != 0, forgets all
+ * records.  Enabling allocates the event pool; do not enable inside a stream capture. */
+typedef enum { LUMO_K_CONV = 0, LUMO_K_SCAN = 1, LUMO_K_COMMIT_STATE = 2, LUMO_K_COMMIT_HIST = 3,
+               LUMO_K_PATH = 4, LUMO_K_COUNT = 5 } lumo_kernel_kind;
+int lumo_ctx_timing_enable(lumo_ctx* ctx, int enable);
+int lumo_ctx_timing_read(lumo_ctx* ctx, int kind, int reset, int64_t* launches, double* total_ms);
+
+/* ---- tree descriptor -------------------------------------------------------------------
+ * parent, depth, slot are HOST arrays, copied.  parent[b*N+i] in {-1} U [0, i): -1 is the
+ * pre-tree state ("a previous node in the packed buffer need not be the parent", Sec. "The
+ * recurrence and path locality"; several children of -1 are allowed).  depth may be NULL
+ * (derived) and is validated if given.  slot may be NULL (identity) and must otherwise be
+ * injective into [0, n_slots).  1 <= N <= 256, N <= n_slots <= 1024.
+ * Errors: LUMO_ERR_ARG, LUMO_ERR_TREE, LUMO_ERR_CUDA.  May synchronise (host-to-device copy). */
+int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots,
+                          const int32_t* parent, const int32_t* depth, const int32_t* slot,
+                          lumo_tree_desc** out);
+void lumo_tree_desc_destroy(lumo_tree_desc* desc);
+/* HOST copy of table `which` (lumo_table) of sequence b; desc-owned memory. */
+int lumo_tree_desc_get(const lumo_tree_desc* desc, int which, int b, const int32_t** data,
+                       int64_t* count);
+/* Device helper (Sec. "One device-selected path drives native continuation": accepted node
+ * indices and path lengths are fixed-shape device products): for every sequence, the root-first
+ * node list of the path that ends at node_dev[b] (-1 = empty path) -> accepted_dev [B, lmax]
+ * (-1 padded), len_dev [B]; status_dev [B] (may be NULL) receives LUMO_SEQ_BAD_NODE /
+ * LUMO_SEQ_BAD_LEN, in which case the path is written as empty. */
+int lumo_tree_path_from_node(lumo_ctx* ctx, const lumo_tree_desc* desc, const int32_t* node_dev,
+                             int lmax, int32_t* accepted_dev, int32_t* len_dev,
+                             int32_t* status_dev, void* stream);
+
+/* ---- one GDN layer's tensors ----------------------------------------------------------- */
+typedef struct {
+  int32_t Hk, Hv, d;
+  int32_t in_dtype;    /* lumo_dtype of x, conv_w, conv_b, conv_hist, q, k, v */
+  int32_t gate_dtype;  /* lumo_dtype of alpha, beta */
+  int32_t out_dtype;   /* lumo_dtype of out */
+  float scale;         /* multiplies q (after normalisation); 1.0 = the paper's Eq. 3 */
+  int32_t qk_l2norm;   /* 1: q <- q / sqrt(sum q^2 + l2_eps), same for k, inside the kernels */
+  float l2_eps;
+  int32_t n_state_rows; /* rows of the state / history pools (bounds check of state_row) */
+  /* recorded operands: read by scan and commit; WRITTEN by verify when x != NULL */
+  void* q;              /* [B, Ns, Hk, d] */
+  void* k;              /* [B, Ns, Hk, d] */
+  void* v;              /* [B, Ns, Hv, d] */
+  const void* alpha;    /* [B, Ns, Hv] decay in (0, 1], post-activation */
+  const void* beta;     /* [B, Ns, Hv] write strength in [0, 1], post-activation */
+  /* convolution stage; x == NULL skips it in verify and skips the history update in commit */
+  const void* x;        /* [B, Ns, C] raw projections, channels [q | k | v] */
+  const void* conv_w;   /* [C, 4] tap 3 multiplies the node's own row */
+  const void* conv_b;   /* [C] or NULL */
+  void* conv_hist;      /* [rows, 3, C] committed raw inputs, oldest first; commit updates it */
+  float* state;         /* [rows, Hv, d_v, d_k] fp32 pool; read-only in verify, updated by commit */
+  const int32_t* state_row; /* [B] pool row of each sequence; -1 = skip the sequence */
+  void* out;            /* [B, Ns, Hv, d_v] verify output */
+  int32_t snapshot_mode;    /* 0 none, 1 list (snap_nodes), 2 every node */
+  int32_t n_snap;           /* E: entries per sequence in snap_nodes (mode 1) / N (mode 2) */
+  const int32_t* snap_nodes;/* [B, E] logical ids, -1 = unused (mode 1) */
+  float* snap_out;          /* [B, E, Hv, d_v, d_k] fp32 node states */
+  int32_t* status;          /* [B] lumo_seq_status, written by verify and by commit; may be NULL */
+} lumo_gdn_args;
+
+/* Verifies all nodes of every tree through n_layers independent GDN layers (Algorithm 2,
+ * "Verify paths; keep branch state temporary").  `layers` is a HOST array.  Read-only on
+ * state and conv_hist.  All layers must share Hk, Hv, d and dtypes.  n_layers <= 64. */
+int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers,
+                         int n_layers, void* stream);
+
+/* Replays accepted_dev [B, lmax] (logical ids, root first; entries at or beyond len_dev[b] are
+ * ignored) from the pre-tree state with the recorded operands and publishes state and
+ * convolution history in place (Algorithm 2, "Replay only the accepted path into native
+ * recurrent state"; Algorithm 1, "Gather the convolution history for A into the native running
+ * row").  len 0 leaves both bit-unchanged.  An invalid path sets status[b] and leaves the
+ * sequence untouched.  Calling it twice advances twice. */
+int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers,
+                    int n_layers, const int32_t* accepted_dev, const int32_t* len_dev, int lmax,
+                    void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LUMO_GDN_H_ */

@@ -1,0 +1,247 @@
+"""Thin ctypes binding of liblumo_gdn.so: argument marshalling only.
+
+Every step of the path (tree conv, tree scan, commit) runs in the CUDA kernels behind the
+C ABI declared in include/lumo_gdn.h; this module turns torch tensors into pointers and
+error codes into exceptions.  It raises at import if the shared library is missing: there
+is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblumo_gdn.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2609_23900_b200.build` "
+        "(the GDN tree verifier has no CPU fallback)")
+_lib = ctypes.CDLL(LIB_PATH)
+
+LUMO_F32, LUMO_BF16 = 0, 1
+_DTYPE = {torch.float32: LUMO_F32, torch.bfloat16: LUMO_BF16}
+
+SEQ_OK, SEQ_BAD_LEN, SEQ_BAD_NODE, SEQ_BAD_ROOT, SEQ_BAD_LINK, SEQ_BAD_ROW = range(6)
+
+TABLES = ["depth", "n_child", "child_off", "child_list", "is_leaf", "leaves", "path_off", "path_nodes",
+          "anc_win", "slot_inv", "chain_head", "chain_off", "chain_nodes", "chain_level", "cut_nodes",
+          "schedule", "schedule_full"]
+
+KERNEL_KINDS = ["conv", "scan", "commit_state", "commit_hist", "path"]
+
+EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_scratch_bytes",
+           "lumo_ctx_timing_enable", "lumo_ctx_timing_read",
+           "lumo_tree_desc_create", "lumo_tree_desc_destroy", "lumo_tree_desc_get",
+           "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit"]
+
+
+class LumoError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"lumo status {code}: {msg}")
+        self.code = code
+
+
+class _Args(ctypes.Structure):
+    """Mirror of lumo_gdn_args."""
+    _fields_ = [
+        ("Hk", ctypes.c_int32), ("Hv", ctypes.c_int32), ("d", ctypes.c_int32),
+        ("in_dtype", ctypes.c_int32), ("gate_dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+        ("scale", ctypes.c_float), ("qk_l2norm", ctypes.c_int32), ("l2_eps", ctypes.c_float),
+        ("n_state_rows", ctypes.c_int32),
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("alpha", ctypes.c_void_p), ("beta", ctypes.c_void_p),
+        ("x", ctypes.c_void_p), ("conv_w", ctypes.c_void_p), ("conv_b", ctypes.c_void_p),
+        ("conv_hist", ctypes.c_void_p),
+        ("state", ctypes.c_void_p), ("state_row", ctypes.c_void_p),
+        ("out", ctypes.c_void_p),
+        ("snapshot_mode", ctypes.c_int32), ("n_snap", ctypes.c_int32),
+        ("snap_nodes", ctypes.c_void_p), ("snap_out", ctypes.c_void_p),
+        ("status", ctypes.c_void_p),
+    ]
+
+
+_lib.lumo_ctx_create.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
+_lib.lumo_ctx_destroy.argtypes = [ctypes.c_void_p]
+_lib.lumo_ctx_destroy.restype = None
+_lib.lumo_last_error.argtypes = [ctypes.c_void_p]
+_lib.lumo_last_error.restype = ctypes.c_char_p
+_lib.lumo_ctx_scratch_bytes.argtypes = [ctypes.c_void_p]
+_lib.lumo_ctx_scratch_bytes.restype = ctypes.c_int64
+_lib.lumo_ctx_timing_enable.argtypes = [ctypes.c_void_p, ctypes.c_int]
+_lib.lumo_ctx_timing_read.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                      ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]
+_lib.lumo_tree_desc_create.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                       ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                       ctypes.POINTER(ctypes.c_void_p)]
+_lib.lumo_tree_desc_destroy.argtypes = [ctypes.c_void_p]
+_lib.lumo_tree_desc_destroy.restype = None
+_lib.lumo_tree_desc_get.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
+                                    ctypes.POINTER(ctypes.POINTER(ctypes.c_int32)),
+                                    ctypes.POINTER(ctypes.c_int64)]
+_lib.lumo_tree_path_from_node.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int,
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+_lib.lumo_gdn_tree_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
+                                      ctypes.c_void_p]
+_lib.lumo_gdn_commit.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
+                                 ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("tensors passed to the library must be contiguous CUDA tensors")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+class Context:
+    """lumo_ctx: one per device."""
+
+    def __init__(self, device: int = 0):
+        h = ctypes.c_void_p()
+        rc = _lib.lumo_ctx_create(int(device), ctypes.byref(h))
+        if rc != 0:
+            raise LumoError(rc, _lib.lumo_last_error(None).decode())
+        self._h = h
+        self.device = int(device)
+
+    def _check(self, rc: int):
+        if rc != 0:
+            raise LumoError(rc, _lib.lumo_last_error(self._h).decode())
+
+    @property
+    def scratch_bytes(self) -> int:
+        return _lib.lumo_ctx_scratch_bytes(self._h)
+
+    def timing_enable(self, on: bool = True):
+        self._check(_lib.lumo_ctx_timing_enable(self._h, int(on)))
+
+    def timing_read(self, reset: bool = True) -> dict:
+        """{kernel kind: (launches, total device ms)} of the launches recorded since the last reset."""
+        out = {}
+        for i, name in enumerate(KERNEL_KINDS):
+            n, ms = ctypes.c_int64(), ctypes.c_double()
+            last = reset and i == len(KERNEL_KINDS) - 1
+            self._check(_lib.lumo_ctx_timing_read(self._h, i, int(last), ctypes.byref(n), ctypes.byref(ms)))
+            out[name] = (n.value, ms.value)
+        return out
+
+    def close(self):
+        if self._h:
+            _lib.lumo_ctx_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- entry points -------------------------------------------------------------------
+    def tree_desc(self, parent, slot=None, n_slots: Optional[int] = None, depth=None) -> "TreeDesc":
+        return TreeDesc(self, parent, slot, n_slots, depth)
+
+    def path_from_node(self, desc: "TreeDesc", node: torch.Tensor, lmax: int, accepted: torch.Tensor,
+                       length: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None):
+        self._check(_lib.lumo_tree_path_from_node(self._h, desc._h, _ptr(node), int(lmax), _ptr(accepted),
+                                                  _ptr(length), _ptr(status), _stream(stream)))
+
+    @staticmethod
+    def pack(layers: Sequence["GdnLayer"]):
+        """ctypes array of the layers' argument blocks (reusable across calls)."""
+        return (_Args * len(layers))(*[l.args for l in layers])
+
+    def verify(self, desc: "TreeDesc", layers, stream=None):
+        arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)
+        self._check(_lib.lumo_gdn_tree_verify(self._h, desc._h, arr, len(layers), _stream(stream)))
+
+    def commit(self, desc: "TreeDesc", layers, accepted: torch.Tensor, length: torch.Tensor, stream=None):
+        arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)
+        self._check(_lib.lumo_gdn_commit(self._h, desc._h, arr, len(layers), _ptr(accepted), _ptr(length),
+                                         int(accepted.shape[1]), _stream(stream)))
+
+
+class TreeDesc:
+    """lumo_tree_desc built from host arrays parent [B, N] (and optional slot, depth)."""
+
+    def __init__(self, ctx: Context, parent, slot=None, n_slots: Optional[int] = None, depth=None):
+        parent = np.ascontiguousarray(parent, dtype=np.int32)
+        if parent.ndim != 2:
+            raise ValueError("parent must be [B, N]")
+        self.B, self.N = parent.shape
+        slot_a = None if slot is None else np.ascontiguousarray(slot, dtype=np.int32)
+        depth_a = None if depth is None else np.ascontiguousarray(depth, dtype=np.int32)
+        self.Ns = int(n_slots) if n_slots is not None else self.N
+        h = ctypes.c_void_p()
+        rc = _lib.lumo_tree_desc_create(
+            ctx._h, self.B, self.N, self.Ns, parent.ctypes.data,
+            None if depth_a is None else depth_a.ctypes.data,
+            None if slot_a is None else slot_a.ctypes.data, ctypes.byref(h))
+        ctx._check(rc)
+        self._h = h
+        self._ctx = ctx
+
+    def table(self, name: str, b: int = 0) -> np.ndarray:
+        data = ctypes.POINTER(ctypes.c_int32)()
+        count = ctypes.c_int64()
+        rc = _lib.lumo_tree_desc_get(self._h, TABLES.index(name), int(b), ctypes.byref(data), ctypes.byref(count))
+        if rc != 0:
+            raise LumoError(rc, "bad table request")
+        return np.ctypeslib.as_array(data, shape=(count.value,)).copy() if count.value else np.zeros(0, np.int32)
+
+    def close(self):
+        if self._h:
+            _lib.lumo_tree_desc_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class GdnLayer:
+    """lumo_gdn_args for one layer; keeps the tensors alive."""
+
+    def __init__(self, *, Hk: int, Hv: int, d: int, q, k, v, alpha, beta, state, state_row, out=None,
+                 x=None, conv_w=None, conv_b=None, conv_hist=None, scale: float = 1.0,
+                 qk_l2norm: bool = False, l2_eps: float = 1e-6, snapshot_mode: int = 0, snap_nodes=None,
+                 snap_out=None, status=None):
+        self.tensors = dict(q=q, k=k, v=v, alpha=alpha, beta=beta, state=state, state_row=state_row, out=out,
+                            x=x, conv_w=conv_w, conv_b=conv_b, conv_hist=conv_hist, snap_nodes=snap_nodes,
+                            snap_out=snap_out, status=status)
+        if state.dtype != torch.float32:
+            raise ValueError("state must be float32")
+        for name in ("state_row", "snap_nodes", "status"):
+            t = self.tensors[name]
+            if t is not None and t.dtype != torch.int32:
+                raise ValueError(f"{name} must be int32")
+        if alpha.dtype != beta.dtype or q.dtype != k.dtype or q.dtype != v.dtype:
+            raise ValueError("q/k/v (and alpha/beta) must share a dtype")
+        for name in ("x", "conv_w", "conv_b", "conv_hist"):
+            t = self.tensors[name]
+            if t is not None and t.dtype != q.dtype:
+                raise ValueError(f"{name} must have the dtype of q/k/v")
+        a = _Args()
+        a.Hk, a.Hv, a.d = Hk, Hv, d
+        a.in_dtype = _DTYPE[q.dtype]
+        a.gate_dtype = _DTYPE[alpha.dtype]
+        a.out_dtype = _DTYPE[out.dtype] if out is not None else LUMO_F32
+        a.scale, a.qk_l2norm, a.l2_eps = float(scale), int(qk_l2norm), float(l2_eps)
+        a.n_state_rows = int(state.shape[0])
+        a.snapshot_mode = int(snapshot_mode)
+        a.n_snap = int(snap_nodes.shape[1]) if snap_nodes is not None else 0
+        for name in ("q", "k", "v", "alpha", "beta", "x", "conv_w", "conv_b", "conv_hist", "state",
+                     "state_row", "out", "snap_nodes", "snap_out", "status"):
+            setattr(a, name, _ptr(self.tensors[name]))
+        self.args = a

@@ -1,0 +1,360 @@
+// extern "C" entry points of liblumo_gdn: argument checking and launch orchestration.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+
+using namespace lumo;
+
+namespace {
+
+thread_local std::string g_create_err;
+
+int fail(lumo_ctx* ctx, int code, const std::string& msg) {
+  if (ctx) ctx->err = msg; else g_create_err = msg;
+  return code;
+}
+
+int cuda_fail(lumo_ctx* ctx, cudaError_t e, const char* what) {
+  return fail(ctx, LUMO_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// Checks the layer array and fills the kernel-side views.  `need_out`: verify needs out.
+int prepare(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers,
+            bool for_verify, Shape* s, LayerBatch* lb) {
+  if (!ctx || !desc || !layers) return fail(ctx, LUMO_ERR_ARG, "null ctx, desc or layers");
+  if (desc->ctx != ctx) return fail(ctx, LUMO_ERR_ARG, "descriptor belongs to another context");
+  if (ctx->device < 0) return fail(ctx, LUMO_ERR_UNSUPPORTED, "host-only context cannot launch");
+  if (n_layers < 1 || n_layers > kMaxLayers)
+    return fail(ctx, LUMO_ERR_ARG, "n_layers must be in [1, " + std::to_string(kMaxLayers) + "]");
+  const lumo_gdn_args& a0 = layers[0];
+  if (a0.d != 64 && a0.d != 128) return fail(ctx, LUMO_ERR_UNSUPPORTED, "d must be 64 or 128");
+  if (a0.Hk < 1 || a0.Hv < 1 || a0.Hv % a0.Hk != 0)
+    return fail(ctx, LUMO_ERR_UNSUPPORTED, "Hv must be a positive multiple of Hk");
+  for (int dt : {a0.in_dtype, a0.gate_dtype, a0.out_dtype})
+    if (dt != LUMO_F32 && dt != LUMO_BF16) return fail(ctx, LUMO_ERR_UNSUPPORTED, "dtype must be f32 or bf16");
+  if (a0.snapshot_mode < 0 || a0.snapshot_mode > 2) return fail(ctx, LUMO_ERR_ARG, "snapshot_mode must be 0, 1 or 2");
+  if (a0.n_state_rows < 1) return fail(ctx, LUMO_ERR_ARG, "n_state_rows must be positive");
+  std::memset(s, 0, sizeof(*s));
+  s->B = desc->B; s->N = desc->N; s->Ns = desc->Ns;
+  s->Hk = a0.Hk; s->Hv = a0.Hv; s->d = a0.d; s->C = 2 * a0.Hk * a0.d + a0.Hv * a0.d;
+  s->in_dtype = a0.in_dtype; s->gate_dtype = a0.gate_dtype; s->out_dtype = a0.out_dtype;
+  s->scale = a0.scale; s->l2norm = a0.qk_l2norm; s->l2_eps = a0.l2_eps;
+  s->n_state_rows = a0.n_state_rows;
+  s->snapshot_mode = for_verify ? a0.snapshot_mode : 0;
+  s->n_snap = a0.snapshot_mode == 2 ? desc->N : a0.n_snap;
+  s->n_layers = n_layers;
+  if (for_verify && a0.snapshot_mode == 1 && (a0.n_snap < 1 || a0.n_snap > kMaxNodes))
+    return fail(ctx, LUMO_ERR_ARG, "n_snap must be in [1, 256] in snapshot list mode");
+  for (int l = 0; l < n_layers; ++l) {
+    const lumo_gdn_args& a = layers[l];
+    const std::string at = " (layer " + std::to_string(l) + ")";
+    if (a.Hk != a0.Hk || a.Hv != a0.Hv || a.d != a0.d || a.in_dtype != a0.in_dtype ||
+        a.gate_dtype != a0.gate_dtype || a.out_dtype != a0.out_dtype || a.scale != a0.scale ||
+        a.qk_l2norm != a0.qk_l2norm || a.l2_eps != a0.l2_eps || a.n_state_rows != a0.n_state_rows ||
+        a.snapshot_mode != a0.snapshot_mode || a.n_snap != a0.n_snap || (a.x == nullptr) != (a0.x == nullptr))
+      return fail(ctx, LUMO_ERR_ARG, "all layers must share shape, dtypes and options" + at);
+    if (!a.q || !a.k || !a.v || !a.alpha || !a.beta || !a.state || !a.state_row)
+      return fail(ctx, LUMO_ERR_ARG, "q, k, v, alpha, beta, state and state_row are required" + at);
+    if (for_verify && !a.out) return fail(ctx, LUMO_ERR_ARG, "out is required" + at);
+    if (a.x && (!a.conv_w || !a.conv_hist))
+      return fail(ctx, LUMO_ERR_ARG, "x needs conv_w and conv_hist" + at);
+    if (for_verify && a.snapshot_mode != 0 && !a.snap_out) return fail(ctx, LUMO_ERR_ARG, "snap_out is required" + at);
+    if (for_verify && a.snapshot_mode == 1 && !a.snap_nodes) return fail(ctx, LUMO_ERR_ARG, "snap_nodes is required" + at);
+    for (const void* p : {(const void*)a.q, (const void*)a.k, (const void*)a.v, a.x, a.conv_w, a.conv_b,
+                          (const void*)a.conv_hist, (const void*)a.state, (const void*)a.out,
+                          (const void*)a.snap_out})
+      if (p && !aligned16(p)) return fail(ctx, LUMO_ERR_ARG, "tensor pointers must be 16-byte aligned" + at);
+    LayerPtrs& p = lb->l[l];
+    p.q = a.q; p.k = a.k; p.v = a.v; p.alpha = a.alpha; p.beta = a.beta;
+    p.x = a.x; p.conv_w = a.conv_w; p.conv_b = a.conv_b; p.conv_hist = a.conv_hist;
+    p.state = a.state; p.state_row = a.state_row; p.out = a.out;
+    p.snap_nodes = a.snap_nodes; p.snap_out = a.snap_out; p.status = a.status;
+  }
+  return LUMO_OK;
+}
+
+constexpr size_t kTimingPool = 16384;
+
+// Brackets one launch with events when timing is on.
+template <typename F>
+cudaError_t timed(lumo_ctx* ctx, int kind, cudaStream_t st, F launch) {
+  const bool on = ctx->timing && ctx->ev_kind.size() < kTimingPool;
+  size_t i = ctx->ev_kind.size();
+  if (on) {
+    cudaError_t e = cudaEventRecord(ctx->ev_start[i], st);
+    if (e != cudaSuccess) return e;
+  }
+  cudaError_t e = launch();
+  if (on && e == cudaSuccess) {
+    e = cudaEventRecord(ctx->ev_stop[i], st);
+    if (e == cudaSuccess) ctx->ev_kind.push_back(kind);
+  }
+  return e;
+}
+
+TreeDev tree_view(const lumo_tree_desc* d, int which) {
+  TreeDev t;
+  t.parent = d->d_parent; t.depth = d->d_depth; t.slot = d->d_slot; t.slot_inv = d->d_slot_inv;
+  t.win = d->d_win; t.sched = d->d_sched[which]; t.nops = d->d_nops[which];
+  t.max_ops = d->max_ops[which]; t.max_levels = d->max_levels[which];
+  return t;
+}
+
+}  // namespace
+
+extern "C" {
+
+int lumo_ctx_create(int device, lumo_ctx** out) {
+  if (!out) return fail(nullptr, LUMO_ERR_ARG, "out is null");
+  *out = nullptr;
+  if (device == -1) {   // host-only context: descriptors and their integer tables, no launches
+    lumo_ctx* c = new (std::nothrow) lumo_ctx();
+    if (!c) return fail(nullptr, LUMO_ERR_NOMEM, "out of host memory");
+    c->device = -1;
+    *out = c;
+    return LUMO_OK;
+  }
+  int count = 0;
+  cudaError_t e = cudaGetDeviceCount(&count);
+  if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaGetDeviceCount");
+  if (device < 0 || device >= count) return fail(nullptr, LUMO_ERR_ARG, "no such CUDA device");
+  cudaDeviceProp prop;
+  e = cudaGetDeviceProperties(&prop, device);
+  if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaGetDeviceProperties");
+  if (prop.major != 10)
+    return fail(nullptr, LUMO_ERR_UNSUPPORTED, "this library holds sm_100a code only; device is sm_" +
+                                                   std::to_string(prop.major) + std::to_string(prop.minor));
+  lumo_ctx* c = new (std::nothrow) lumo_ctx();
+  if (!c) return fail(nullptr, LUMO_ERR_NOMEM, "out of host memory");
+  c->device = device;
+  c->sm_count = prop.multiProcessorCount;
+  *out = c;
+  return LUMO_OK;
+}
+
+void lumo_ctx_destroy(lumo_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->device >= 0) {
+    DeviceGuard g(ctx->device);
+    if (ctx->scratch) cudaFree(ctx->scratch);
+    for (cudaEvent_t e : ctx->ev_start) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->ev_stop) cudaEventDestroy(e);
+  }
+  delete ctx;
+}
+
+const char* lumo_last_error(const lumo_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_err.c_str(); }
+
+int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx) { return ctx ? (int64_t)ctx->scratch_bytes : 0; }
+
+int lumo_ctx_timing_enable(lumo_ctx* ctx, int enable) {
+  if (!ctx) return LUMO_ERR_ARG;
+  if (ctx->device < 0) return fail(ctx, LUMO_ERR_UNSUPPORTED, "host-only context cannot launch");
+  DeviceGuard g(ctx->device);
+  if (enable && ctx->ev_start.empty()) {
+    ctx->ev_start.resize(kTimingPool);
+    ctx->ev_stop.resize(kTimingPool);
+    for (size_t i = 0; i < kTimingPool; ++i) {
+      cudaError_t e = cudaEventCreate(&ctx->ev_start[i]);
+      if (e == cudaSuccess) e = cudaEventCreate(&ctx->ev_stop[i]);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventCreate");
+    }
+    ctx->ev_kind.reserve(kTimingPool);
+  }
+  ctx->timing = enable != 0;
+  return LUMO_OK;
+}
+
+int lumo_ctx_timing_read(lumo_ctx* ctx, int kind, int reset, int64_t* launches, double* total_ms) {
+  if (!ctx || !launches || !total_ms || kind < 0 || kind >= LUMO_K_COUNT) return fail(ctx, LUMO_ERR_ARG, "bad argument");
+  DeviceGuard g(ctx->device);
+  *launches = 0;
+  *total_ms = 0.0;
+  for (size_t i = 0; i < ctx->ev_kind.size(); ++i) {
+    if (ctx->ev_kind[i] != kind) continue;
+    cudaError_t e = cudaEventSynchronize(ctx->ev_stop[i]);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, ctx->ev_start[i], ctx->ev_stop[i]);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "event read");
+    *launches += 1;
+    *total_ms += ms;
+  }
+  if (reset) ctx->ev_kind.clear();
+  return LUMO_OK;
+}
+
+int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, const int32_t* parent,
+                          const int32_t* depth, const int32_t* slot, lumo_tree_desc** out) {
+  if (!ctx || !out || !parent) return fail(ctx, LUMO_ERR_ARG, "null ctx, out or parent");
+  *out = nullptr;
+  if (batch < 1 || n_nodes < 1 || n_nodes > kMaxNodes || n_slots < n_nodes || n_slots > kMaxSlots)
+    return fail(ctx, LUMO_ERR_ARG, "need batch >= 1, 1 <= n_nodes <= 256, n_nodes <= n_slots <= 1024");
+  lumo_tree_desc* d = new (std::nothrow) lumo_tree_desc();
+  if (!d) return fail(ctx, LUMO_ERR_NOMEM, "out of host memory");
+  d->ctx = ctx; d->B = batch; d->N = n_nodes; d->Ns = n_slots;
+  d->trees.resize(batch);
+  const int B = batch, N = n_nodes, Ns = n_slots;
+  for (int b = 0; b < B; ++b) {
+    std::string err;
+    int lv[2];
+    if (!build_tree(parent + (size_t)b * N, slot ? slot + (size_t)b * N : nullptr, N, Ns, &d->trees[b],
+                    &lv[0], &lv[1], &err)) {
+      delete d;
+      return fail(ctx, LUMO_ERR_TREE, "sequence " + std::to_string(b) + ": " + err);
+    }
+    if (depth)
+      for (int i = 0; i < N; ++i)
+        if (depth[(size_t)b * N + i] != d->trees[b].tab[LUMO_TAB_DEPTH][i]) {
+          delete d;
+          return fail(ctx, LUMO_ERR_TREE, "sequence " + std::to_string(b) + ": depth[" + std::to_string(i) +
+                                              "] does not match the parent array");
+        }
+    for (int w = 0; w < 2; ++w) {
+      d->max_levels[w] = std::max(d->max_levels[w], lv[w]);
+      d->max_ops[w] = std::max(d->max_ops[w], (int)d->trees[b].tab[LUMO_TAB_SCHEDULE + w].size());
+    }
+  }
+  // one device allocation holding every table
+  std::vector<int32_t> h;
+  auto reserve = [&](size_t n) { size_t off = h.size(); h.resize(off + ((n + 3) / 4) * 4, 0); return off; };
+  const size_t o_parent = reserve((size_t)B * N), o_depth = reserve((size_t)B * N), o_slot = reserve((size_t)B * N);
+  const size_t o_inv = reserve((size_t)B * Ns), o_win = reserve((size_t)B * N * 4);
+  size_t o_sched[2], o_nops[2];
+  for (int w = 0; w < 2; ++w) { o_sched[w] = reserve((size_t)B * d->max_ops[w]); o_nops[w] = reserve(B); }
+  for (int b = 0; b < B; ++b) {
+    const HostTree& t = d->trees[b];
+    for (int i = 0; i < N; ++i) {
+      h[o_parent + (size_t)b * N + i] = parent[(size_t)b * N + i];
+      h[o_depth + (size_t)b * N + i] = t.tab[LUMO_TAB_DEPTH][i];
+      h[o_slot + (size_t)b * N + i] = slot ? slot[(size_t)b * N + i] : i;
+    }
+    for (int sidx = 0; sidx < Ns; ++sidx) h[o_inv + (size_t)b * Ns + sidx] = t.tab[LUMO_TAB_SLOT_INV][sidx];
+    for (int i = 0; i < N * 4; ++i) {   // windows in physical rows
+      int w = t.tab[LUMO_TAB_ANC_WIN][i];
+      h[o_win + (size_t)b * N * 4 + i] = w < 0 ? w : h[o_slot + (size_t)b * N + w];
+    }
+    for (int w = 0; w < 2; ++w) {
+      const auto& ops = t.tab[LUMO_TAB_SCHEDULE + w];
+      std::copy(ops.begin(), ops.end(), h.begin() + o_sched[w] + (size_t)b * d->max_ops[w]);
+      h[o_nops[w] + b] = (int32_t)ops.size();
+    }
+  }
+  if (ctx->device < 0) { *out = d; return LUMO_OK; }   // host-only: tables stay on the host
+  DeviceGuard g(ctx->device);
+  cudaError_t e = cudaMalloc(&d->dev, h.size() * sizeof(int32_t));
+  if (e != cudaSuccess) { delete d; return cuda_fail(ctx, e, "cudaMalloc(tree tables)"); }
+  e = cudaMemcpy(d->dev, h.data(), h.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
+  if (e != cudaSuccess) { cudaFree(d->dev); delete d; return cuda_fail(ctx, e, "cudaMemcpy(tree tables)"); }
+  d->d_parent = d->dev + o_parent; d->d_depth = d->dev + o_depth; d->d_slot = d->dev + o_slot;
+  d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_win;
+  for (int w = 0; w < 2; ++w) { d->d_sched[w] = d->dev + o_sched[w]; d->d_nops[w] = d->dev + o_nops[w]; }
+  *out = d;
+  return LUMO_OK;
+}
+
+void lumo_tree_desc_destroy(lumo_tree_desc* desc) {
+  if (!desc) return;
+  if (desc->dev) {
+    DeviceGuard g(desc->ctx->device);
+    cudaFree(desc->dev);
+  }
+  delete desc;
+}
+
+int lumo_tree_desc_get(const lumo_tree_desc* desc, int which, int b, const int32_t** data, int64_t* count) {
+  if (!desc || !data || !count || which < 0 || which >= LUMO_TAB_COUNT || b < 0 || b >= desc->B) return LUMO_ERR_ARG;
+  const auto& v = desc->trees[b].tab[which];
+  *data = v.data();
+  *count = (int64_t)v.size();
+  return LUMO_OK;
+}
+
+int lumo_tree_path_from_node(lumo_ctx* ctx, const lumo_tree_desc* desc, const int32_t* node_dev, int lmax,
+                             int32_t* accepted_dev, int32_t* len_dev, int32_t* status_dev, void* stream) {
+  if (!ctx || !desc || !node_dev || !accepted_dev || !len_dev) return fail(ctx, LUMO_ERR_ARG, "null argument");
+  if (desc->ctx != ctx) return fail(ctx, LUMO_ERR_ARG, "descriptor belongs to another context");
+  if (lmax < 1) return fail(ctx, LUMO_ERR_ARG, "lmax must be positive");
+  if (ctx->device < 0) return fail(ctx, LUMO_ERR_UNSUPPORTED, "host-only context cannot launch");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  cudaError_t e = timed(ctx, LUMO_K_PATH, st, [&] {
+    return launch_path_from_node(tree_view(desc, 0), desc->B, desc->N, node_dev, lmax, accepted_dev, len_dev,
+                                 status_dev, st);
+  });
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "path_from_node launch");
+}
+
+int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers,
+                         void* stream) {
+  Shape s;
+  LayerBatch lb;
+  std::memset(&lb, 0, sizeof(lb));
+  int rc = prepare(ctx, desc, layers, n_layers, true, &s, &lb);
+  if (rc != LUMO_OK) return rc;
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const TreeDev t = tree_view(desc, s.snapshot_mode != 0 ? 1 : 0);
+  int grid = 0;
+  size_t stack_bytes = 0;
+  cudaError_t e = scan_plan(s, t, ctx->sm_count, &grid, &stack_bytes);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "scan_plan");
+  if (stack_bytes > ctx->scratch_bytes) {
+    // first call with this shape: grow the scratch (synchronises; later calls allocate nothing)
+    if (ctx->scratch) {
+      e = cudaDeviceSynchronize();
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaDeviceSynchronize");
+      cudaFree(ctx->scratch);
+      ctx->scratch = nullptr;
+      ctx->scratch_bytes = 0;
+    }
+    e = cudaMalloc(&ctx->scratch, stack_bytes);
+    if (e != cudaSuccess) return fail(ctx, LUMO_ERR_NOMEM, std::string("scratch allocation failed: ") + cudaGetErrorString(e));
+    ctx->scratch_bytes = stack_bytes;
+  }
+  if (layers[0].x) {
+    e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, st); });
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
+  }
+  e = timed(ctx, LUMO_K_SCAN, st, [&] {
+    return launch_scan(s, t, lb, reinterpret_cast<float*>(ctx->scratch), grid, st);
+  });
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "scan launch");
+}
+
+int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers,
+                    const int32_t* accepted_dev, const int32_t* len_dev, int lmax, void* stream) {
+  Shape s;
+  LayerBatch lb;
+  std::memset(&lb, 0, sizeof(lb));
+  int rc = prepare(ctx, desc, layers, n_layers, false, &s, &lb);
+  if (rc != LUMO_OK) return rc;
+  if (!accepted_dev || !len_dev) return fail(ctx, LUMO_ERR_ARG, "accepted_dev and len_dev are required");
+  if (lmax < 1) return fail(ctx, LUMO_ERR_ARG, "lmax must be positive");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const TreeDev t = tree_view(desc, 0);
+  cudaError_t e = timed(ctx, LUMO_K_COMMIT_STATE, st, [&] {
+    return launch_commit_state(s, t, lb, accepted_dev, len_dev, lmax, st);
+  });
+  if (e == cudaSuccess && layers[0].x)
+    e = timed(ctx, LUMO_K_COMMIT_HIST, st, [&] { return launch_commit_hist(s, t, lb, accepted_dev, len_dev, lmax, st); });
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "commit launch");
+}
+
+}  // extern "C"

@@ -1,0 +1,113 @@
+// Internal declarations shared by the host side and the kernels of liblumo_gdn.
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "lumo_gdn.h"
+
+namespace lumo {
+
+constexpr int kMaxNodes = 256;
+constexpr int kMaxSlots = 1024;
+constexpr int kMaxLayers = 64;
+
+// ---- scan schedule ------------------------------------------------------------------
+// The scan kernel walks the whole tree depth first with the state tile of the current
+// node's parent in registers.  An op is (kind << 24) | (flag << 20) | arg.
+//   EMIT c          o_c from the parent's state (no state materialised); flag=1 also caches
+//                   delta_c on chip for a later DESCEND c
+//   EMIT_DESCEND c  EMIT c, then turn the registers into S_c in place
+//   DESCEND c       turn the registers (S_parent) into S_c using the cached delta_c
+//   PUSH l          save the registers to stack level l
+//   POP l           restore the registers from stack level l; l = kPopRoot reloads the
+//                   pre-tree state from the state pool
+enum OpKind : int { OP_EMIT = 0, OP_EMIT_DESCEND = 1, OP_DESCEND = 2, OP_PUSH = 3, OP_POP = 4 };
+constexpr int kPopRoot = 0xFFFF;
+inline int make_op(int kind, int flag, int arg) { return (kind << 24) | (flag << 20) | (arg & 0xFFFF); }
+
+struct HostTree {
+  std::vector<int32_t> tab[LUMO_TAB_COUNT];
+};
+
+}  // namespace lumo
+
+struct lumo_ctx {
+  int device = 0;
+  int sm_count = 0;
+  std::string err;
+  void* scratch = nullptr;      // scan stack levels
+  size_t scratch_bytes = 0;
+  // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
+  bool timing = false;
+  std::vector<cudaEvent_t> ev_start, ev_stop;
+  std::vector<int> ev_kind;
+};
+
+struct lumo_tree_desc {
+  lumo_ctx* ctx = nullptr;
+  int B = 0, N = 0, Ns = 0;
+  std::vector<lumo::HostTree> trees;     // per sequence
+  // device tables (one allocation), all int32
+  int32_t* dev = nullptr;
+  int32_t* d_parent = nullptr;    // [B, N]
+  int32_t* d_depth = nullptr;     // [B, N]
+  int32_t* d_slot = nullptr;      // [B, N]
+  int32_t* d_slot_inv = nullptr;  // [B, Ns]
+  int32_t* d_win = nullptr;       // [B, N, 4]  physical row, or -1/-2/-3 for history rows
+  int32_t* d_sched[2] = {nullptr, nullptr};   // [B, max_ops]  lean / full (every node's state materialised)
+  int32_t* d_nops[2] = {nullptr, nullptr};    // [B]
+  int max_ops[2] = {0, 0};
+  int max_levels[2] = {0, 0};     // stack levels the schedule needs
+};
+
+namespace lumo {
+
+// ---- kernel-side views -----------------------------------------------------------------
+struct LayerPtrs {
+  void* q; void* k; void* v;
+  const void* alpha; const void* beta;
+  const void* x; const void* conv_w; const void* conv_b; void* conv_hist;
+  float* state; const int32_t* state_row;
+  void* out;
+  const int32_t* snap_nodes; float* snap_out;
+  int32_t* status;
+};
+
+struct LayerBatch {
+  LayerPtrs l[kMaxLayers];
+};
+
+struct Shape {
+  int B, N, Ns, Hk, Hv, d, C;
+  int in_dtype, gate_dtype, out_dtype;
+  float scale; int l2norm; float l2_eps;
+  int n_state_rows;
+  int snapshot_mode, n_snap;
+  int n_layers;
+};
+
+struct TreeDev {
+  const int32_t* parent; const int32_t* depth; const int32_t* slot; const int32_t* slot_inv;
+  const int32_t* win; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
+};
+
+// host-side tree tables (tree_desc.cpp)
+bool build_tree(const int32_t* parent, const int32_t* slot, int N, int Ns, HostTree* t,
+                int* levels_lean, int* levels_full, std::string* err);
+
+// launchers (kernels.cu); all return cudaError_t and only enqueue
+cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, cudaStream_t st);
+cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, float* stack,
+                        int grid, cudaStream_t st);
+// persistent grid size (CTAs resident at once) and the stack scratch it needs
+cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes);
+cudaError_t launch_commit_state(const Shape& s, const TreeDev& t, const LayerBatch& lb,
+                                const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st);
+cudaError_t launch_commit_hist(const Shape& s, const TreeDev& t, const LayerBatch& lb,
+                               const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st);
+cudaError_t launch_path_from_node(const TreeDev& t, int B, int N, const int32_t* node, int lmax,
+                                  int32_t* accepted, int32_t* len, int32_t* status, cudaStream_t st);
+
+}  // namespace lumo

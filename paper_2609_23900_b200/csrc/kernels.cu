@@ -1,0 +1,602 @@
+// sm_100a kernels of the GDN tree verifier: tree convolution, rank-1 tree scan, commit.
+//
+// Row independence is what the layout is built on: row r of the d_v x d_k state evolves
+// alone (S[r,:] <- a S[r,:] + delta_r k^T with delta_r = b (v_r - a S[r,:].k)), so a CTA
+// owns 32 rows of one (sequence, value head) and walks the WHOLE tree with them, four lanes
+// per row, each lane holding d_k/4 fp32 state values in registers (paper Eq. 2-3; Sec.
+// "Path-parallel verification and state lifetime": the working tile keeps the full key
+// dimension and is reused along the path instead of being reloaded per node).
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <type_traits>
+
+#include "internal.h"
+
+namespace lumo {
+
+namespace {
+
+constexpr int kRows = 32;        // state rows per CTA
+constexpr int kLanesPerRow = 4;
+constexpr int kScanThreads = kRows * kLanesPerRow;   // 128
+constexpr int kRingDepth = 6;    // staged node operands in flight
+
+// ---------------------------------------------------------------------------------------
+// small helpers
+// ---------------------------------------------------------------------------------------
+template <typename T> struct Vec4;   // four consecutive elements -> float4
+template <> struct Vec4<float> {
+  static __device__ __forceinline__ float4 load(const float* p) { return *reinterpret_cast<const float4*>(p); }
+};
+template <> struct Vec4<__nv_bfloat16> {
+  static __device__ __forceinline__ float4 load(const __nv_bfloat16* p) {
+    uint2 r = *reinterpret_cast<const uint2*>(p);
+    return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xFFFF0000u),
+                       __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xFFFF0000u));
+  }
+};
+
+__device__ __forceinline__ float load_scalar(const void* p, size_t i, int dtype) {
+  return dtype == LUMO_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i])
+                            : reinterpret_cast<const float*>(p)[i];
+}
+__device__ __forceinline__ void store_scalar(void* p, size_t i, int dtype, float v) {
+  if (dtype == LUMO_BF16) reinterpret_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
+  else reinterpret_cast<float*>(p)[i] = v;
+}
+
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+  unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(s), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+// Accepted-path check shared by the commit kernels; every CTA of a sequence reaches the same
+// answer.  Order of checks: length, then per entry range, root, link.
+__device__ int check_path(const int32_t* parent, int N, const int32_t* acc, int len, int lmax) {
+  if (len < 0 || len > lmax) return LUMO_SEQ_BAD_LEN;
+  int prev = -1;
+  for (int t = 0; t < len; ++t) {       // bounded by lmax
+    int a = acc[t];
+    if (a < 0 || a >= N) return LUMO_SEQ_BAD_NODE;
+    int p = parent[a];
+    if (t == 0) { if (p != -1) return LUMO_SEQ_BAD_ROOT; }
+    else if (p != prev) return LUMO_SEQ_BAD_LINK;
+    prev = a;
+  }
+  return LUMO_SEQ_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// a1: ancestry-gathered causal depthwise conv (width 4) + SiLU -> recorded operands
+// ---------------------------------------------------------------------------------------
+// One thread owns kVec consecutive channels of one physical row.  Taps are applied oldest
+// first in fp32 starting from zero, bias last, SiLU in fp32, one round-to-nearest-even cast
+// (Sec. "Precompute branch histories while preserving arithmetic": tap order and cast points
+// are part of the result).
+template <typename T, int kVec>
+__global__ void __launch_bounds__(256) conv_kernel(Shape s, TreeDev t, LayerBatch lb) {
+  const int layer = blockIdx.z / s.B, b = blockIdx.z % s.B;
+  const int ps = blockIdx.y;                                   // physical row
+  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * kVec;
+  if (c0 >= s.C) return;
+  const LayerPtrs& L = lb.l[layer];
+  const int hkd = s.Hk * s.d;
+  // destination of this channel group inside [q | k | v]
+  T* dst;
+  if (c0 < hkd) dst = reinterpret_cast<T*>(L.q) + ((size_t)b * s.Ns + ps) * hkd + c0;
+  else if (c0 < 2 * hkd) dst = reinterpret_cast<T*>(L.k) + ((size_t)b * s.Ns + ps) * hkd + (c0 - hkd);
+  else dst = reinterpret_cast<T*>(L.v) + ((size_t)b * s.Ns + ps) * (size_t)(s.Hv * s.d) + (c0 - 2 * hkd);
+
+  const int node = t.slot_inv[b * s.Ns + ps];
+  const int row = L.state_row[b];
+  float y[kVec];
+  if (node < 0 || row < 0 || row >= s.n_state_rows) {
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) y[e] = 0.f;
+  } else {
+    const T* x = reinterpret_cast<const T*>(L.x);
+    const T* hist = reinterpret_cast<const T*>(L.conv_hist);
+    const T* w = reinterpret_cast<const T*>(L.conv_w) + (size_t)c0 * 4;
+    float wv[kVec * 4];
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) {
+      float4 w4 = Vec4<T>::load(w + e * 4);
+      wv[e * 4 + 0] = w4.x; wv[e * 4 + 1] = w4.y; wv[e * 4 + 2] = w4.z; wv[e * 4 + 3] = w4.w;
+    }
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) y[e] = 0.f;
+    const int4 win = *reinterpret_cast<const int4*>(t.win + ((size_t)b * s.N + node) * 4);
+    const int wj[4] = {win.x, win.y, win.z, win.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {                    // oldest -> newest
+      const T* src = wj[j] >= 0 ? x + ((size_t)b * s.Ns + wj[j]) * s.C + c0
+                                : hist + ((size_t)row * 3 + (3 + wj[j])) * s.C + c0;
+#pragma unroll
+      for (int e4 = 0; e4 < kVec / 4; ++e4) {
+        float4 xv = Vec4<T>::load(src + e4 * 4);
+        y[e4 * 4 + 0] = fmaf(wv[(e4 * 4 + 0) * 4 + j], xv.x, y[e4 * 4 + 0]);
+        y[e4 * 4 + 1] = fmaf(wv[(e4 * 4 + 1) * 4 + j], xv.y, y[e4 * 4 + 1]);
+        y[e4 * 4 + 2] = fmaf(wv[(e4 * 4 + 2) * 4 + j], xv.z, y[e4 * 4 + 2]);
+        y[e4 * 4 + 3] = fmaf(wv[(e4 * 4 + 3) * 4 + j], xv.w, y[e4 * 4 + 3]);
+      }
+    }
+    if (L.conv_b) {
+      const T* bias = reinterpret_cast<const T*>(L.conv_b) + c0;
+#pragma unroll
+      for (int e4 = 0; e4 < kVec / 4; ++e4) {
+        float4 bv = Vec4<T>::load(bias + e4 * 4);
+        y[e4 * 4 + 0] += bv.x; y[e4 * 4 + 1] += bv.y; y[e4 * 4 + 2] += bv.z; y[e4 * 4 + 3] += bv.w;
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) y[e] = y[e] / (1.f + expf(-y[e]));   // SiLU
+  }
+  if constexpr (sizeof(T) == 2) {
+    static_assert(kVec == 8 || sizeof(T) != 2, "bf16 path stores 16 bytes");
+    uint32_t pk[kVec / 2];
+#pragma unroll
+    for (int e = 0; e < kVec / 2; ++e) {
+      __nv_bfloat162 h2 = __floats2bfloat162_rn(y[2 * e], y[2 * e + 1]);
+      pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+    }
+    *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+  } else {
+    *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// a3: rank-1 tree scan
+// ---------------------------------------------------------------------------------------
+template <int D, typename T>
+struct ScanCfg {
+  static constexpr int kChunks = D / 16;            // float4 chunks per lane
+  static constexpr int kStageElems = 2 * D + kRows; // k row, q row, v slice
+  static constexpr int kStageBytes = kStageElems * (int)sizeof(T);
+  static constexpr int kStageXfers = kStageBytes / 16;
+  static constexpr int kKXfers = D * (int)sizeof(T) / 16;
+};
+
+// dynamic shared memory layout (bytes), computed identically on host and device
+struct ScanSmem {
+  int ops, params, dcache, snaplist, ring, total;
+};
+__host__ __device__ inline ScanSmem scan_smem(int N, int max_ops, int n_snap_list, int stage_bytes) {
+  ScanSmem m;
+  int off = 0;
+  m.ops = off;      off += ((max_ops * 4 + 15) / 16) * 16;
+  m.params = off;   off += 5 * N * 4;  off = (off + 15) / 16 * 16;
+  m.dcache = off;   off += N * kRows * 4;
+  m.snaplist = off; off += ((n_snap_list * 4 + 15) / 16) * 16;
+  m.ring = off;     off += kRingDepth * stage_bytes;
+  m.total = off;
+  return m;
+}
+
+template <int D, typename T>
+__global__ void __launch_bounds__(kScanThreads)
+scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_items) {
+  using Cfg = ScanCfg<D, T>;
+  constexpr int NCH = Cfg::kChunks;
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int n_snap_list = s.snapshot_mode == 1 ? s.n_snap : 0;
+  const ScanSmem lay = scan_smem(s.N, t.max_ops, n_snap_list, Cfg::kStageBytes);
+  int32_t* s_ops = reinterpret_cast<int32_t*>(smem + lay.ops);
+  float* p_a = reinterpret_cast<float*>(smem + lay.params);
+  float* p_b = p_a + s.N;
+  float* p_ks = p_b + s.N;      // multiplies the raw key (1 / norm when normalising)
+  float* p_qs = p_ks + s.N;     // multiplies the raw query (scale / norm)
+  float* p_kq = p_qs + s.N;     // k_n . q_n with both factors applied
+  float* s_dc = reinterpret_cast<float*>(smem + lay.dcache);
+  int32_t* s_snap = reinterpret_cast<int32_t*>(smem + lay.snaplist);
+  unsigned char* s_ring = smem + lay.ring;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int j = tid & 3;               // lane within the row group
+  const int rl = tid >> 2;             // local row 0..31
+  constexpr int kTiles = D / kRows;
+  const int rep = s.Hv / s.Hk;
+  float* my_stack = stack + (size_t)blockIdx.x * t.max_levels * (kRows * D);
+
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {   // bounded: n_items
+    const int tile = item % kTiles;
+    const int hv = (item / kTiles) % s.Hv;
+    const int b = (item / (kTiles * s.Hv)) % s.B;
+    const int layer = item / (kTiles * s.Hv * s.B);
+    const LayerPtrs& L = lb.l[layer];
+    const int g = hv / rep;
+    const int row = L.state_row[b];
+    const int r0 = tile * kRows;
+    const size_t out_row_stride = (size_t)s.Hv * D;
+    __syncthreads();   // previous item's shared memory is no longer in use
+
+    if (row < 0 || row >= s.n_state_rows) {
+      // skipped sequence: zero outputs; flag a row outside the pool
+      for (int e = tid; e < s.Ns * kRows; e += kScanThreads)
+        store_scalar(L.out, ((size_t)b * s.Ns + e / kRows) * out_row_stride + hv * D + r0 + e % kRows,
+                     s.out_dtype, 0.f);
+      if (L.status && hv == 0 && tile == 0 && tid == 0) L.status[b] = row < 0 ? LUMO_SEQ_OK : LUMO_SEQ_BAD_ROW;
+      continue;
+    }
+    if (L.status && hv == 0 && tile == 0 && tid == 0) L.status[b] = LUMO_SEQ_OK;
+
+    // pre-tree state tile -> registers (issued first so the loads overlap the prologue)
+    const float* S0 = L.state + (((size_t)row * s.Hv + hv) * D + r0 + rl) * D;
+    float4 S[NCH];
+#pragma unroll
+    for (int m = 0; m < NCH; ++m) S[m] = *reinterpret_cast<const float4*>(S0 + 16 * m + 4 * j);
+
+    const int nops = t.nops[b];
+    const int32_t* ops_g = t.sched + (size_t)b * t.max_ops;
+    for (int e = tid; e < nops; e += kScanThreads) s_ops[e] = ops_g[e];
+    for (int e = tid; e < n_snap_list; e += kScanThreads) s_snap[e] = L.snap_nodes[(size_t)b * s.n_snap + e];
+    // padding rows: zero outputs
+    for (int e = tid; e < s.Ns * kRows; e += kScanThreads) {
+      int ps = e / kRows;
+      if (t.slot_inv[b * s.Ns + ps] < 0)
+        store_scalar(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * D + r0 + e % kRows, s.out_dtype, 0.f);
+    }
+    // per-node scalars: gates, normalisation factors, k.q
+    const T* qg = reinterpret_cast<const T*>(L.q);
+    const T* kg = reinterpret_cast<const T*>(L.k);
+    const T* vg = reinterpret_cast<const T*>(L.v);
+    for (int n = warp; n < s.N; n += kScanThreads / 32) {
+      const size_t pr = (size_t)b * s.Ns + t.slot[b * s.N + n];
+      const T* kr = kg + (pr * s.Hk + g) * D;
+      const T* qr = qg + (pr * s.Hk + g) * D;
+      float kk = 0.f, qq = 0.f, kq = 0.f;
+      for (int c = lane * 4; c < D; c += 128) {
+        float4 kv = Vec4<T>::load(kr + c), qv = Vec4<T>::load(qr + c);
+        kk += kv.x * kv.x + kv.y * kv.y + kv.z * kv.z + kv.w * kv.w;
+        qq += qv.x * qv.x + qv.y * qv.y + qv.z * qv.z + qv.w * qv.w;
+        kq += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        kk += __shfl_xor_sync(0xffffffffu, kk, o);
+        qq += __shfl_xor_sync(0xffffffffu, qq, o);
+        kq += __shfl_xor_sync(0xffffffffu, kq, o);
+      }
+      if (lane == 0) {
+        float ks = 1.f, qs = s.scale;
+        if (s.l2norm) { ks = rsqrtf(kk + s.l2_eps); qs = s.scale * rsqrtf(qq + s.l2_eps); }
+        p_ks[n] = ks; p_qs[n] = qs; p_kq[n] = kq * ks * qs;
+        p_a[n] = load_scalar(L.alpha, pr * s.Hv + hv, s.gate_dtype);
+        p_b[n] = load_scalar(L.beta, pr * s.Hv + hv, s.gate_dtype);
+      }
+    }
+    __syncthreads();
+
+    // operand ring: stage i holds k row, q row and this tile's v slice of op i's node
+    auto prefetch = [&](int i) {
+      if (i < nops) {
+        const int op = s_ops[i];
+        const int kind = op >> 24;
+        if (kind <= OP_DESCEND) {
+          const int n = op & 0xFFFF;
+          const size_t pr = (size_t)b * s.Ns + t.slot[b * s.N + n];
+          unsigned char* st = s_ring + (i % kRingDepth) * Cfg::kStageBytes;
+          const int nx = kind == OP_DESCEND ? Cfg::kKXfers : Cfg::kStageXfers;
+          if (tid < nx) {
+            const unsigned char* src;
+            if (tid < Cfg::kKXfers) src = reinterpret_cast<const unsigned char*>(kg + (pr * s.Hk + g) * D) + tid * 16;
+            else if (tid < 2 * Cfg::kKXfers)
+              src = reinterpret_cast<const unsigned char*>(qg + (pr * s.Hk + g) * D) + (tid - Cfg::kKXfers) * 16;
+            else
+              src = reinterpret_cast<const unsigned char*>(vg + (pr * s.Hv + hv) * D + r0) + (tid - 2 * Cfg::kKXfers) * 16;
+            cp_async16(st + tid * 16, src);
+          }
+        }
+      }
+      cp_async_commit();
+    };
+#pragma unroll
+    for (int i = 0; i < kRingDepth - 1; ++i) prefetch(i);
+
+    for (int i = 0; i < nops; ++i) {                   // bounded: nops <= max_ops
+      cp_async_wait<kRingDepth - 2>();
+      __syncthreads();
+      prefetch(i + kRingDepth - 1);
+      const int op = s_ops[i];
+      const int kind = op >> 24;
+      const int arg = op & 0xFFFF;
+      const T* st_k = reinterpret_cast<const T*>(s_ring + (i % kRingDepth) * Cfg::kStageBytes);
+      const T* st_q = st_k + D;
+      const T* st_v = st_q + D;
+      if (kind <= OP_EMIT_DESCEND) {
+        const int n = arg;
+        float u0 = 0.f, u1 = 0.f, w0 = 0.f, w1 = 0.f;
+#pragma unroll
+        for (int m = 0; m < NCH; ++m) {
+          float4 kv = Vec4<T>::load(st_k + 16 * m + 4 * j);
+          float4 qv = Vec4<T>::load(st_q + 16 * m + 4 * j);
+          u0 = fmaf(S[m].x, kv.x, u0); u1 = fmaf(S[m].y, kv.y, u1);
+          u0 = fmaf(S[m].z, kv.z, u0); u1 = fmaf(S[m].w, kv.w, u1);
+          w0 = fmaf(S[m].x, qv.x, w0); w1 = fmaf(S[m].y, qv.y, w1);
+          w0 = fmaf(S[m].z, qv.z, w0); w1 = fmaf(S[m].w, qv.w, w1);
+        }
+        float u = u0 + u1, w = w0 + w1;
+        u += __shfl_xor_sync(0xffffffffu, u, 1); w += __shfl_xor_sync(0xffffffffu, w, 1);
+        u += __shfl_xor_sync(0xffffffffu, u, 2); w += __shfl_xor_sync(0xffffffffu, w, 2);
+        const float a = p_a[n], bt = p_b[n], ks = p_ks[n];
+        float vv;
+        if constexpr (sizeof(T) == 2) vv = __bfloat162float(st_v[rl]); else vv = st_v[rl];
+        const float dl = bt * (vv - a * (ks * u));          // delta = beta (v - R' k)
+        const float o = a * (p_qs[n] * w) + dl * p_kq[n];   // o = R q = a R_p q + delta (k.q)
+        if (j == 0) {
+          const size_t pr = (size_t)b * s.Ns + t.slot[b * s.N + n];
+          store_scalar(L.out, pr * out_row_stride + hv * D + r0 + rl, s.out_dtype, o);
+          if ((op >> 20) & 1) s_dc[n * kRows + rl] = dl;
+        }
+        if (kind == OP_EMIT_DESCEND) {
+          const float gk = dl * ks;
+#pragma unroll
+          for (int m = 0; m < NCH; ++m) {
+            float4 kv = Vec4<T>::load(st_k + 16 * m + 4 * j);
+            S[m].x = fmaf(a, S[m].x, gk * kv.x); S[m].y = fmaf(a, S[m].y, gk * kv.y);
+            S[m].z = fmaf(a, S[m].z, gk * kv.z); S[m].w = fmaf(a, S[m].w, gk * kv.w);
+          }
+        }
+      } else if (kind == OP_DESCEND) {
+        const int n = arg;
+        const float a = p_a[n];
+        const float gk = s_dc[n * kRows + rl] * p_ks[n];
+#pragma unroll
+        for (int m = 0; m < NCH; ++m) {
+          float4 kv = Vec4<T>::load(st_k + 16 * m + 4 * j);
+          S[m].x = fmaf(a, S[m].x, gk * kv.x); S[m].y = fmaf(a, S[m].y, gk * kv.y);
+          S[m].z = fmaf(a, S[m].z, gk * kv.z); S[m].w = fmaf(a, S[m].w, gk * kv.w);
+        }
+      } else if (kind == OP_PUSH) {
+        float* dst = my_stack + ((size_t)arg * kRows + rl) * D;
+#pragma unroll
+        for (int m = 0; m < NCH; ++m) *reinterpret_cast<float4*>(dst + 16 * m + 4 * j) = S[m];
+      } else {  // OP_POP
+        const float* src = arg == kPopRoot ? S0 : my_stack + ((size_t)arg * kRows + rl) * D;
+#pragma unroll
+        for (int m = 0; m < NCH; ++m) S[m] = *reinterpret_cast<const float4*>(src + 16 * m + 4 * j);
+      }
+      // node states on request: the registers now hold S_n
+      if (s.snapshot_mode != 0 && (kind == OP_EMIT_DESCEND || kind == OP_DESCEND)) {
+        const int n = arg;
+        const int E = s.n_snap;
+        if (s.snapshot_mode == 2) {
+          float* dst = L.snap_out + ((((size_t)b * E + n) * s.Hv + hv) * D + r0 + rl) * D;
+#pragma unroll
+          for (int m = 0; m < NCH; ++m) *reinterpret_cast<float4*>(dst + 16 * m + 4 * j) = S[m];
+        } else {
+          for (int e = 0; e < E; ++e) {          // bounded: E
+            if (s_snap[e] != n) continue;
+            float* dst = L.snap_out + ((((size_t)b * E + e) * s.Hv + hv) * D + r0 + rl) * D;
+#pragma unroll
+            for (int m = 0; m < NCH; ++m) *reinterpret_cast<float4*>(dst + 16 * m + 4 * j) = S[m];
+          }
+        }
+      }
+    }
+    cp_async_wait<0>();
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// a4: commit - replay the accepted path into the running state, in place
+// ---------------------------------------------------------------------------------------
+// Same per-token arithmetic as the scan's EMIT_DESCEND without the output: this is the
+// "native per-token update" of Algorithm 2, applied for the accepted nodes in path order.
+template <int D, typename T>
+__global__ void __launch_bounds__(kScanThreads)
+commit_state_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ accepted,
+                    const int32_t* __restrict__ len_arr, int lmax) {
+  constexpr int NCH = D / 16;
+  constexpr int kTiles = D / kRows;
+  const int tile = blockIdx.x % kTiles, hv = blockIdx.x / kTiles;
+  const int b = blockIdx.y, layer = blockIdx.z;
+  const LayerPtrs& L = lb.l[layer];
+  const int tid = threadIdx.x, j = tid & 3, rl = tid >> 2;
+  const int row = L.state_row[b];
+  const bool lead = hv == 0 && tile == 0 && tid == 0;
+  if (row < 0) { if (lead && L.status) L.status[b] = LUMO_SEQ_OK; return; }
+  if (row >= s.n_state_rows) { if (lead && L.status) L.status[b] = LUMO_SEQ_BAD_ROW; return; }
+  const int32_t* acc = accepted + (size_t)b * lmax;
+  const int len = len_arr[b];
+  const int st = check_path(t.parent + (size_t)b * s.N, s.N, acc, len, lmax);
+  if (lead && L.status) L.status[b] = st;
+  if (st != LUMO_SEQ_OK || len == 0) return;
+
+  const int g = hv / (s.Hv / s.Hk);
+  const int r0 = tile * kRows;
+  float* Sg = L.state + (((size_t)row * s.Hv + hv) * D + r0 + rl) * D;
+  float4 S[NCH];
+#pragma unroll
+  for (int m = 0; m < NCH; ++m) S[m] = *reinterpret_cast<const float4*>(Sg + 16 * m + 4 * j);
+
+  const T* kg = reinterpret_cast<const T*>(L.k);
+  const T* vg = reinterpret_cast<const T*>(L.v);
+  auto load_node = [&](int tt, float4* kv, float* vv, float* a, float* bt) {
+    const int n = acc[tt];
+    const size_t pr = (size_t)b * s.Ns + t.slot[b * s.N + n];
+    const T* kr = kg + (pr * s.Hk + g) * D;
+#pragma unroll
+    for (int m = 0; m < NCH; ++m) kv[m] = Vec4<T>::load(kr + 16 * m + 4 * j);
+    if constexpr (sizeof(T) == 2) *vv = __bfloat162float(vg[(pr * s.Hv + hv) * D + r0 + rl]);
+    else *vv = vg[(pr * s.Hv + hv) * D + r0 + rl];
+    *a = load_scalar(L.alpha, pr * s.Hv + hv, s.gate_dtype);
+    *bt = load_scalar(L.beta, pr * s.Hv + hv, s.gate_dtype);
+  };
+  float4 kv[NCH], kn[NCH];
+  float vv, a, bt, vn = 0.f, an = 0.f, bn = 0.f;
+  load_node(0, kv, &vv, &a, &bt);
+  for (int tt = 0; tt < len; ++tt) {                      // bounded: len <= lmax
+    if (tt + 1 < len) load_node(tt + 1, kn, &vn, &an, &bn);   // next node's operands in flight
+    float u0 = 0.f, u1 = 0.f, k0 = 0.f, k1 = 0.f;
+#pragma unroll
+    for (int m = 0; m < NCH; ++m) {
+      u0 = fmaf(S[m].x, kv[m].x, u0); u1 = fmaf(S[m].y, kv[m].y, u1);
+      u0 = fmaf(S[m].z, kv[m].z, u0); u1 = fmaf(S[m].w, kv[m].w, u1);
+      k0 = fmaf(kv[m].x, kv[m].x, k0); k1 = fmaf(kv[m].y, kv[m].y, k1);
+      k0 = fmaf(kv[m].z, kv[m].z, k0); k1 = fmaf(kv[m].w, kv[m].w, k1);
+    }
+    float u = u0 + u1, kk = k0 + k1;
+    u += __shfl_xor_sync(0xffffffffu, u, 1); kk += __shfl_xor_sync(0xffffffffu, kk, 1);
+    u += __shfl_xor_sync(0xffffffffu, u, 2); kk += __shfl_xor_sync(0xffffffffu, kk, 2);
+    const float ks = s.l2norm ? rsqrtf(kk + s.l2_eps) : 1.f;
+    const float dl = bt * (vv - a * (ks * u));
+    const float gk = dl * ks;
+#pragma unroll
+    for (int m = 0; m < NCH; ++m) {
+      S[m].x = fmaf(a, S[m].x, gk * kv[m].x); S[m].y = fmaf(a, S[m].y, gk * kv[m].y);
+      S[m].z = fmaf(a, S[m].z, gk * kv[m].z); S[m].w = fmaf(a, S[m].w, gk * kv[m].w);
+    }
+#pragma unroll
+    for (int m = 0; m < NCH; ++m) kv[m] = kn[m];
+    vv = vn; a = an; bt = bn;
+  }
+#pragma unroll
+  for (int m = 0; m < NCH; ++m) *reinterpret_cast<float4*>(Sg + 16 * m + 4 * j) = S[m];
+}
+
+// a5: convolution history <- last three rows of [old history ; x of the accepted nodes]
+template <typename T>
+__global__ void __launch_bounds__(256)
+commit_hist_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ accepted,
+                   const int32_t* __restrict__ len_arr, int lmax) {
+  constexpr int kVec = 16 / (int)sizeof(T);
+  const int b = blockIdx.y, layer = blockIdx.z;
+  const LayerPtrs& L = lb.l[layer];
+  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * kVec;
+  if (c0 >= s.C) return;
+  const int row = L.state_row[b];
+  if (row < 0 || row >= s.n_state_rows) return;
+  const int32_t* acc = accepted + (size_t)b * lmax;
+  const int len = len_arr[b];
+  if (check_path(t.parent + (size_t)b * s.N, s.N, acc, len, lmax) != LUMO_SEQ_OK || len == 0) return;
+  T* hist = reinterpret_cast<T*>(L.conv_hist) + (size_t)row * 3 * s.C + c0;
+  const T* x = reinterpret_cast<const T*>(L.x);
+  uint4 v[3];
+#pragma unroll
+  for (int jj = 0; jj < 3; ++jj) {
+    const int q = len + jj;        // index into [old0 old1 old2 x_a0 x_a1 ...]
+    const T* src = q < 3 ? hist + (size_t)q * s.C
+                         : x + ((size_t)b * s.Ns + t.slot[b * s.N + acc[q - 3]]) * s.C + c0;
+    v[jj] = *reinterpret_cast<const uint4*>(src);
+  }
+#pragma unroll
+  for (int jj = 0; jj < 3; ++jj) *reinterpret_cast<uint4*>(hist + (size_t)jj * s.C) = v[jj];
+}
+
+// device helper: root-first path ending at node[b]
+__global__ void path_from_node_kernel(TreeDev t, int B, int N, const int32_t* __restrict__ node,
+                                      int lmax, int32_t* __restrict__ accepted,
+                                      int32_t* __restrict__ len, int32_t* __restrict__ status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  int32_t* acc = accepted + (size_t)b * lmax;
+  for (int e = 0; e < lmax; ++e) acc[e] = -1;
+  int n = node[b], st = LUMO_SEQ_OK, l = 0;
+  if (n != -1) {
+    if (n < 0 || n >= N) st = LUMO_SEQ_BAD_NODE;
+    else {
+      l = t.depth[(size_t)b * N + n];
+      if (l > lmax) { st = LUMO_SEQ_BAD_LEN; l = 0; }
+      else
+        for (int e = l - 1; e >= 0 && n >= 0; --e) { acc[e] = n; n = t.parent[(size_t)b * N + n]; }  // bounded: depth
+    }
+  }
+  len[b] = l;
+  if (status) status[b] = st;
+}
+
+template <typename F>
+cudaError_t dispatch(int d, int in_dtype, F f) {
+  if (d == 128 && in_dtype == LUMO_BF16) return f(std::integral_constant<int, 128>{}, __nv_bfloat16{});
+  if (d == 128 && in_dtype == LUMO_F32) return f(std::integral_constant<int, 128>{}, float{});
+  if (d == 64 && in_dtype == LUMO_BF16) return f(std::integral_constant<int, 64>{}, __nv_bfloat16{});
+  if (d == 64 && in_dtype == LUMO_F32) return f(std::integral_constant<int, 64>{}, float{});
+  return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------
+// launchers
+// ---------------------------------------------------------------------------------------
+cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, cudaStream_t st) {
+  if (s.in_dtype == LUMO_BF16) {
+    dim3 grid((s.C / 8 + 255) / 256, s.Ns, s.B * s.n_layers);
+    conv_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>(s, t, lb);
+  } else {
+    dim3 grid((s.C / 4 + 255) / 256, s.Ns, s.B * s.n_layers);
+    conv_kernel<float, 4><<<grid, 256, 0, st>>>(s, t, lb);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes) {
+  const int items = s.n_layers * s.B * s.Hv * (s.d / kRows);
+  return dispatch(s.d, s.in_dtype, [&](auto dc, auto tc) {
+    constexpr int D = decltype(dc)::value;
+    using T = decltype(tc);
+    const int n_snap_list = s.snapshot_mode == 1 ? s.n_snap : 0;
+    const ScanSmem lay = scan_smem(s.N, t.max_ops, n_snap_list, ScanCfg<D, T>::kStageBytes);
+    auto kern = scan_kernel<D, T>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, lay.total);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kScanThreads, lay.total);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const int resident = sm_count * per_sm;
+    *grid = items < resident ? items : resident;
+    *stack_bytes = (size_t)*grid * t.max_levels * kRows * D * sizeof(float);
+    return cudaSuccess;
+  });
+}
+
+cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, float* stack,
+                        int grid, cudaStream_t st) {
+  const int items = s.n_layers * s.B * s.Hv * (s.d / kRows);
+  return dispatch(s.d, s.in_dtype, [&](auto dc, auto tc) {
+    constexpr int D = decltype(dc)::value;
+    using T = decltype(tc);
+    const int n_snap_list = s.snapshot_mode == 1 ? s.n_snap : 0;
+    const ScanSmem lay = scan_smem(s.N, t.max_ops, n_snap_list, ScanCfg<D, T>::kStageBytes);
+    scan_kernel<D, T><<<grid, kScanThreads, lay.total, st>>>(s, t, lb, stack, items);
+    return cudaGetLastError();
+  });
+}
+
+cudaError_t launch_commit_state(const Shape& s, const TreeDev& t, const LayerBatch& lb,
+                                const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st) {
+  return dispatch(s.d, s.in_dtype, [&](auto dc, auto tc) {
+    constexpr int D = decltype(dc)::value;
+    using T = decltype(tc);
+    dim3 grid(s.Hv * (D / kRows), s.B, s.n_layers);
+    commit_state_kernel<D, T><<<grid, kScanThreads, 0, st>>>(s, t, lb, accepted, len, lmax);
+    return cudaGetLastError();
+  });
+}
+
+cudaError_t launch_commit_hist(const Shape& s, const TreeDev& t, const LayerBatch& lb,
+                               const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st) {
+  if (s.in_dtype == LUMO_BF16) {
+    dim3 grid((s.C / 8 + 255) / 256, s.B, s.n_layers);
+    commit_hist_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(s, t, lb, accepted, len, lmax);
+  } else {
+    dim3 grid((s.C / 4 + 255) / 256, s.B, s.n_layers);
+    commit_hist_kernel<float><<<grid, 256, 0, st>>>(s, t, lb, accepted, len, lmax);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_path_from_node(const TreeDev& t, int B, int N, const int32_t* node, int lmax,
+                                  int32_t* accepted, int32_t* len, int32_t* status, cudaStream_t st) {
+  path_from_node_kernel<<<(B + 63) / 64, 64, 0, st>>>(t, B, N, node, lmax, accepted, len, status);
+  return cudaGetLastError();
+}
+
+}  // namespace lumo

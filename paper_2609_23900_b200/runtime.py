@@ -1,0 +1,78 @@
+"""Device-side holder of one synthetic case: uploads a ``workload.Case`` and builds the
+per-layer argument blocks for the C-ABI calls.  Marshalling only; no arithmetic."""
+from __future__ import annotations
+
+from typing import List, Optional
+
+import numpy as np
+import torch
+
+from . import binding
+from .workload import Case
+
+_TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16}
+
+
+class DeviceCase:
+    def __init__(self, ctx: binding.Context, case: Case, *, out_dtype: str = "f32", use_conv: bool = True,
+                 gate_dtype: Optional[str] = None, snapshot_mode: int = 0, snap_nodes=None,
+                 scale: float = 1.0, qk_l2norm: Optional[bool] = None, l2_eps: float = 1e-6,
+                 device: Optional[torch.device] = None, pinned_host: bool = False):
+        self.ctx, self.case = ctx, case
+        # conv outputs are not unit vectors: the pipeline normalises q, k inside the kernels
+        # (Sec. "Sequential arithmetic and accepted-path replay": in-kernel query/key normalisation)
+        qk_l2norm = use_conv if qk_l2norm is None else qk_l2norm
+        self.scale, self.qk_l2norm, self.l2_eps = scale, qk_l2norm, l2_eps
+        dev = device or torch.device("cuda", ctx.device)
+        self.dev = dev
+        dt = _TORCH_DT[case.in_dtype]
+        gdt = _TORCH_DT[gate_dtype or case.in_dtype]
+        odt = _TORCH_DT[out_dtype]
+        self.desc = ctx.tree_desc(case.parent, slot=case.slot, n_slots=case.Ns)
+        up = lambda a, t: torch.from_numpy(np.ascontiguousarray(a)).to(t).to(dev)
+        self.state_row = torch.from_numpy(case.state_row.copy()).to(dev)
+        self.accepted = torch.from_numpy(case.accepted.copy()).to(dev)
+        self.accepted_len = torch.from_numpy(case.accepted_len.copy()).to(dev)
+        self.snap_nodes = None
+        E = 0
+        if snapshot_mode == 1:
+            self.snap_nodes = torch.from_numpy(np.ascontiguousarray(snap_nodes, dtype=np.int32)).to(dev)
+            E = self.snap_nodes.shape[1]
+        elif snapshot_mode == 2:
+            E = case.N
+        self.layers: List[binding.GdnLayer] = []
+        self.host = []   # pinned host copies of the per-step inputs (end-to-end timing)
+        for L in case.layers:
+            t = dict(
+                q=up(L.q, dt), k=up(L.k, dt), v=up(L.v, dt), alpha=up(L.alpha, gdt), beta=up(L.beta, gdt),
+                state=up(L.state, torch.float32), state_row=self.state_row,
+                out=torch.empty((case.B, case.Ns, case.Hv, case.d), dtype=odt, device=dev),
+                status=torch.full((case.B,), -1, dtype=torch.int32, device=dev),
+            )
+            if use_conv:
+                t.update(x=up(L.x, dt), conv_w=up(L.conv_w, dt), conv_hist=up(L.hist, dt),
+                         conv_b=None if L.conv_b is None else up(L.conv_b, dt))
+            if snapshot_mode:
+                t.update(snap_nodes=self.snap_nodes,
+                         snap_out=torch.zeros((case.B, E, case.Hv, case.d, case.d), dtype=torch.float32, device=dev))
+            self.layers.append(binding.GdnLayer(Hk=case.Hk, Hv=case.Hv, d=case.d, scale=scale, qk_l2norm=qk_l2norm,
+                                                l2_eps=l2_eps, snapshot_mode=snapshot_mode, **t))
+            if pinned_host:
+                self.host.append({n: t[n].cpu().pin_memory() for n in ("x", "alpha", "beta") if n in t})
+
+    def verify(self, stream=None):
+        self.ctx.verify(self.desc, self.layers, stream)
+
+    def commit(self, accepted=None, length=None, stream=None):
+        self.ctx.commit(self.desc, self.layers, self.accepted if accepted is None else accepted,
+                        self.accepted_len if length is None else length, stream)
+
+    def t(self, name: str, layer: int = 0) -> torch.Tensor:
+        return self.layers[layer].tensors[name]
+
+    def np(self, name: str, layer: int = 0) -> np.ndarray:
+        """Host float64 (or int) copy of a device tensor."""
+        t = self.t(name, layer)
+        if t.dtype in (torch.float32, torch.bfloat16):
+            return t.to(torch.float64).cpu().numpy()
+        return t.cpu().numpy()

@@ -1,0 +1,320 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 oracle, on the same seeded inputs.
+
+Integer products must match bit for bit; floating outputs and committed state within
+|d| <= 1e-3 (1 + |ref|) per element; bf16-typed results must be the round-to-nearest-even
+of the same kernel's fp32 results and may add half a bf16 ulp; the committed state must
+agree with the verifier's node state within 1e-5 relative (Frobenius, per value head).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gdn_oracle as O
+from oracle import tree_tables as T
+from paper_2609_23900_b200 import binding
+from paper_2609_23900_b200 import workload as W
+from paper_2609_23900_b200.runtime import DeviceCase
+from tests.harness import assert_close, ctx, oracle_commit_from_device, oracle_scan_from_device
+
+pytestmark = pytest.mark.gpu
+
+
+def small(parents, *, d=64, dtype="f32", Hk=2, Hv=4, **kw):
+    return W.make_case("small", parents, seed=99, Hk=Hk, Hv=Hv, d=d, in_dtype=dtype, **kw)
+
+
+def rand_parents(seed, n, B):
+    return [W.tree_random(W.IntStream(W.stream_key(seed, b)), n, 7) for b in range(B)]
+
+
+CASES = {
+    "cfg0": lambda: W.config0(),
+    "cfg1": lambda: W.config1(),
+    "cfg2": lambda: W.config2(),
+    "cfgP_padded_permuted": lambda: W.config_paper(B=2),
+    "d64_bf16": lambda: small(rand_parents(1, 37, 3), d=64, dtype="bf16", Ns=41, permute_slots=True),
+    "d128_f32": lambda: small(rand_parents(2, 23, 2), d=128, dtype="f32", Hk=1, Hv=3),
+    "single_node": lambda: small([[-1]], d=128, dtype="bf16"),
+    "chain16x16_b2": lambda: W.make_case("c", [W.tree_chains(16, 16)] * 2, seed=5, Hk=4, Hv=8, d=128,
+                                         in_dtype="bf16", alpha_lo=0.5, beta_uniform=True),
+    "star256_b2": lambda: W.make_case("s", [W.tree_star(256)] * 2, seed=6, Hk=4, Hv=8, d=128,
+                                      in_dtype="bf16", alpha_lo=0.5, beta_uniform=True),
+    "rand256_b2": lambda: W.make_case("r", rand_parents(3, 256, 2), seed=7, Hk=4, Hv=8, d=128,
+                                      in_dtype="bf16", alpha_lo=0.5, beta_uniform=True, with_bias=True),
+}
+
+
+# ------------------------------------------------------------------ integer products
+@pytest.mark.parametrize("name", ["cfg0", "cfg2", "cfgP_padded_permuted", "rand256_b2"])
+def test_integer_tables_bit_exact_on_device_context(name):
+    c = CASES[name]()
+    desc = ctx().tree_desc(c.parent, slot=c.slot, n_slots=c.Ns)
+    for b in range(c.B):
+        ref = T.all_tables(c.parent[b].tolist(), c.slot[b].tolist(), c.Ns)
+        for key, val in ref.items():
+            assert desc.table(key, b).tolist() == val, (name, b, key)
+
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg2", "rand256_b2"])
+def test_path_from_node_bit_exact(name):
+    c = CASES[name]()
+    dev = torch.device("cuda", 0)
+    desc = ctx().tree_desc(c.parent, slot=c.slot, n_slots=c.Ns)
+    lmax = 9
+    rs = np.random.default_rng(0)
+    for trial in range(4):
+        nodes = rs.integers(-1, c.N + 2, size=c.B).astype(np.int32)   # includes -1 and out-of-range
+        if name == "cfg0" and trial == 0:
+            nodes[:] = 6
+        acc = torch.full((c.B, lmax), 77, dtype=torch.int32, device=dev)
+        ln = torch.full((c.B,), 77, dtype=torch.int32, device=dev)
+        st = torch.full((c.B,), 77, dtype=torch.int32, device=dev)
+        ctx().path_from_node(desc, torch.from_numpy(nodes).to(dev), lmax, acc, ln, st)
+        torch.cuda.synchronize()
+        for b in range(c.B):
+            ra, rl, rst = T.path_from_node(c.parent[b].tolist(), int(nodes[b]), lmax)
+            assert acc[b].tolist() == ra and int(ln[b]) == rl and int(st[b]) == rst
+
+
+# ------------------------------------------------------------------ conv
+@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfgP_padded_permuted", "d64_bf16", "rand256_b2"])
+def test_conv_recorded_operands(name):
+    c = CASES[name]()
+    dc = DeviceCase(ctx(), c)
+    for t in ("q", "k", "v"):
+        dc.t(t).fill_(777.0)     # must be overwritten everywhere, padding rows with zeros
+    dc.verify()
+    torch.cuda.synchronize()
+    L = c.layers[0]
+    y = O.conv(c.parent, c.slot, c.state_row, L.x, L.conv_w, L.conv_b, L.hist, c.Ns, out_dtype="none")
+    hk = c.Hk * c.d
+    got = np.concatenate([dc.np("q").reshape(c.B, c.Ns, hk), dc.np("k").reshape(c.B, c.Ns, hk),
+                          dc.np("v").reshape(c.B, c.Ns, c.Hv * c.d)], axis=-1)
+    assert_close(got, y, bf16=(c.in_dtype == "bf16"), what=f"{name} conv")
+    for b in range(c.B):
+        pad = sorted(set(range(c.Ns)) - set(c.slot[b].tolist()))
+        assert np.all(got[b, pad] == 0.0)
+    if c.in_dtype == "bf16":   # values are bf16 by construction; most must be the oracle's own rounding
+        y16 = O.conv(c.parent, c.slot, c.state_row, L.x, L.conv_w, L.conv_b, L.hist, c.Ns, out_dtype="bf16")
+        assert (got == y16).mean() > 0.98
+
+
+# ------------------------------------------------------------------ scan
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("use_conv", [False, True])
+def test_scan_outputs_match_oracle(name, use_conv):
+    c = CASES[name]()
+    dc = DeviceCase(ctx(), c, use_conv=use_conv)
+    dc.t("out").fill_(float("nan"))
+    dc.verify()
+    torch.cuda.synchronize()
+    assert dc.np("status").tolist() == [0] * c.B
+    o_ref, _, _ = oracle_scan_from_device(dc)
+    got = dc.np("out")
+    worst = assert_close(got, o_ref, what=f"{name} scan")
+    assert worst < 1e-4            # fp32 arithmetic sits far inside the 1e-3 rule
+    for b in range(c.B):
+        pad = sorted(set(range(c.Ns)) - set(c.slot[b].tolist()))
+        assert np.all(got[b, pad] == 0.0)
+    # bf16-typed outputs: bitwise RNE of the same kernel's fp32 outputs
+    dc16 = DeviceCase(ctx(), c, use_conv=use_conv, out_dtype="bf16")
+    dc16.verify()
+    torch.cuda.synchronize()
+    assert torch.equal(dc16.t("out"), dc.t("out").to(torch.bfloat16))
+    assert_close(dc16.np("out"), o_ref, bf16=True, what=f"{name} scan bf16 out")
+
+
+def test_scan_twice_is_bitwise_reproducible():
+    c = CASES["cfg2"]()
+    dc = DeviceCase(ctx(), c)
+    dc.verify()
+    a = dc.t("out").clone()
+    qa = dc.t("q").clone()
+    dc.verify()
+    torch.cuda.synchronize()
+    assert torch.equal(a, dc.t("out")) and torch.equal(qa, dc.t("q"))
+
+
+def test_l2norm_flag_scale_and_f32_gates():
+    c = small(rand_parents(4, 20, 2), d=128, dtype="bf16")
+    rs = np.random.default_rng(1)
+    for L in c.layers:   # un-normalised q, k
+        L.q[:] = W.round_to(L.q * rs.uniform(0.5, 4.0, size=L.q.shape[:-1] + (1,)), "bf16")
+        L.k[:] = W.round_to(L.k * rs.uniform(0.5, 4.0, size=L.k.shape[:-1] + (1,)), "bf16")
+    dc = DeviceCase(ctx(), c, use_conv=False, gate_dtype="f32", qk_l2norm=True, l2_eps=1e-6, scale=0.5)
+    dc.verify()
+    torch.cuda.synchronize()
+    o_ref, _, _ = oracle_scan_from_device(dc)
+    assert_close(dc.np("out"), o_ref, what="l2norm scan")
+    # commit with the same options
+    dc.commit()
+    torch.cuda.synchronize()
+    st_ref, _, status, _ = oracle_commit_from_device(dc, with_hist=False)
+    assert_close(dc.np("state"), st_ref, what="l2norm commit")
+
+
+# ------------------------------------------------------------------ snapshots and commit
+@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2", "cfgP_padded_permuted", "chain16x16_b2", "rand256_b2"])
+def test_commit_state_history_and_agreement_with_verifier_state(name):
+    c = CASES[name]()
+    ends = np.array([[a[l - 1] if l else -1] for a, l in zip(c.accepted, c.accepted_len)], dtype=np.int32)
+    dc = DeviceCase(ctx(), c, snapshot_mode=1, snap_nodes=ends)
+    dc.verify()
+    torch.cuda.synchronize()
+    o_ref, snap_ref, _ = oracle_scan_from_device(dc, snap_nodes=ends)
+    assert_close(dc.np("out"), o_ref, what=f"{name} scan (snapshot schedule)")
+    snap = dc.np("snap_out")
+    assert_close(snap, snap_ref, what=f"{name} node states")
+    hist0 = dc.t("conv_hist").clone()
+    dc.commit()
+    torch.cuda.synchronize()
+    assert dc.np("status").tolist() == [0] * c.B
+    st_ref, hist_ref, status_ref, _ = oracle_commit_from_device(dc)
+    assert status_ref.tolist() == [0] * c.B
+    state = dc.np("state")
+    assert_close(state, st_ref, what=f"{name} committed state")
+    # history: a pure gather, bit-exact
+    assert np.array_equal(dc.np("conv_hist"), hist_ref)
+    # committed state vs the verifier's state at the last accepted node: 1e-5 relative
+    for b in range(c.B):
+        if c.accepted_len[b] == 0:
+            continue
+        for h in range(c.Hv):
+            a, v = state[c.state_row[b], h], snap[b, 0, h]
+            assert np.linalg.norm(a - v) <= 1e-5 * np.linalg.norm(v), (name, b, h)
+    # rows of the pool that belong to no sequence are untouched
+    other = sorted(set(range(c.rows)) - set(c.state_row.tolist()))
+    assert np.array_equal(state[other], c.layers[0].state[other].astype(np.float64))
+    assert torch.equal(dc.t("conv_hist")[other], hist0[other])
+
+
+def test_cfg0_accepted_path_is_0_2_6_and_commit_matches_leaf_state():
+    c = W.config0()
+    dev = torch.device("cuda", 0)
+    dc = DeviceCase(ctx(), c, snapshot_mode=2)
+    acc = torch.empty((1, 3), dtype=torch.int32, device=dev)
+    ln = torch.empty((1,), dtype=torch.int32, device=dev)
+    ctx().path_from_node(dc.desc, torch.tensor([6], dtype=torch.int32, device=dev), 3, acc, ln)
+    dc.verify()
+    dc.commit(acc, ln)
+    torch.cuda.synchronize()
+    assert acc.tolist() == [[0, 2, 6]] and ln.tolist() == [3]
+    state, snap = dc.np("state"), dc.np("snap_out")
+    for h in range(c.Hv):
+        assert np.linalg.norm(state[c.state_row[0], h] - snap[0, 6, h]) <= 1e-5 * np.linalg.norm(snap[0, 6, h])
+    # all seven node states against the oracle
+    _, snap_ref, _ = oracle_scan_from_device(dc, snap_nodes=[list(range(7))])
+    assert_close(snap, snap_ref, what="cfg0 all node states")
+
+
+def test_commit_controls_len0_poisoned_tail_invalid_paths_skipped_rows():
+    c = W.make_case("ctl", [W.tree_tiny()] * 6, seed=3, Hk=2, Hv=4, d=64, in_dtype="bf16", extra_rows=2)
+    dev = torch.device("cuda", 0)
+    dc = DeviceCase(ctx(), c)
+    dc.verify()
+    acc = np.array([[0, 2, 6], [0, 2, 250], [0, 4, 6], [2, 6, -1], [0, 9, 6], [1, 5, -1]], dtype=np.int32)
+    ln = np.array([0, 2, 3, 2, 3, 2], dtype=np.int32)
+    row = c.state_row.copy()
+    state0, hist0 = dc.t("state").clone(), dc.t("conv_hist").clone()
+    dc.commit(torch.from_numpy(acc).to(dev), torch.from_numpy(ln).to(dev))
+    torch.cuda.synchronize()
+    st_ref, hist_ref, status_ref, _ = oracle_commit_from_device(dc, accepted=acc, length=ln)
+    assert status_ref.tolist() == [0, 0, T.PATH_BAD_LINK, T.PATH_BAD_ROOT, T.PATH_BAD_NODE, 0]
+    assert dc.np("status").tolist() == status_ref.tolist()          # bit-exact path validation
+    state = dc.np("state")
+    assert_close(state, st_ref, what="commit controls")
+    assert np.array_equal(dc.np("conv_hist"), hist_ref)
+    for b in (0, 2, 3, 4):   # len 0 and refused paths: bit-unchanged state and history
+        assert torch.equal(dc.t("state")[row[b]], state0[row[b]])
+        assert torch.equal(dc.t("conv_hist")[row[b]], hist0[row[b]])
+    # zero-replay control: an accepted, non-empty path must have changed the row
+    assert not torch.equal(dc.t("state")[row[1]], state0[row[1]])
+    # bad length; skipped sequence; row outside the pool
+    ln2 = np.array([4, -1, 1, 1, 1, 1], dtype=np.int32)
+    dc2 = DeviceCase(ctx(), c)
+    dc2.verify()
+    dc2.state_row[2] = -1
+    dc2.state_row[3] = c.rows + 5
+    s0 = dc2.t("state").clone()
+    dc2.commit(torch.from_numpy(acc).to(dev), torch.from_numpy(ln2).to(dev))
+    torch.cuda.synchronize()
+    assert dc2.np("status").tolist() == [binding.SEQ_BAD_LEN, binding.SEQ_BAD_LEN, 0, binding.SEQ_BAD_ROW, 0, 0]
+    for b in (0, 1, 2, 3):
+        assert torch.equal(dc2.t("state")[row[b]], s0[row[b]])
+    dc2.t("out").fill_(5.0)
+    dc2.verify()
+    torch.cuda.synchronize()
+    assert dc2.np("status").tolist() == [0, 0, 0, binding.SEQ_BAD_ROW, 0, 0]
+    assert torch.all(dc2.t("out")[2] == 0) and torch.all(dc2.t("out")[3] == 0) and torch.all(dc2.t("q")[2] == 0)
+
+
+def test_off_path_poison_and_two_cycles():
+    # poisoning nodes off the accepted path must leave the committed state bitwise unchanged
+    c = W.make_case("p", [W.tree_tiny()], seed=4, Hk=2, Hv=4, d=128, in_dtype="bf16", accepted=[[0, 2, 6]])
+    dc = DeviceCase(ctx(), c, use_conv=False)
+    dc.commit()
+    good = dc.t("state").clone()
+    dc2 = DeviceCase(ctx(), c, use_conv=False)
+    for t in ("q", "k", "v", "alpha", "beta"):
+        dc2.t(t)[0, [1, 3, 4, 5]] = float("nan")
+    dc2.commit()
+    dc2.verify()
+    torch.cuda.synchronize()
+    assert torch.equal(dc2.t("state"), good)
+    # verify -> commit -> verify on a 6-chain equals one pass over the chain
+    c6 = W.make_case("c6", [W.tree_chain(6)], seed=8, Hk=2, Hv=4, d=128, in_dtype="bf16", accepted=[[0, 1, 2]])
+    full = DeviceCase(ctx(), c6, use_conv=False)
+    full.verify()
+    c3 = W.make_case("c3", [W.tree_chain(3)], seed=8, Hk=2, Hv=4, d=128, in_dtype="bf16", accepted=[[0, 1, 2]])
+    L6, L3 = c6.layers[0], c3.layers[0]
+    L3.state[:] = L6.state
+    for n in ("q", "k", "v", "alpha", "beta"):
+        getattr(L3, n)[:] = getattr(L6, n)[:, :3]
+    first = DeviceCase(ctx(), c3, use_conv=False)
+    first.verify()
+    first.commit()
+    for n in ("q", "k", "v", "alpha", "beta"):
+        first.t(n).copy_(full.t(n)[:, 3:])
+    first.verify()
+    torch.cuda.synchronize()
+    o_ref, _, _ = oracle_scan_from_device(full)
+    assert_close(first.np("out")[0], o_ref[0, 3:], what="second cycle")
+    assert_close(full.np("out"), o_ref, what="one pass")
+
+
+def test_multi_layer_launch_and_snapshot_all():
+    c = W.config3(B=2, n_layers=5)
+    dc = DeviceCase(ctx(), c, snapshot_mode=2)
+    dc.verify()
+    dc.commit()
+    torch.cuda.synchronize()
+    for l in range(5):
+        o_ref, snap_ref, _ = oracle_scan_from_device(dc, layer=l, snap_nodes=np.tile(np.arange(c.N, dtype=np.int32), (c.B, 1)))
+        assert_close(dc.np("out", l), o_ref, what=f"layer {l} out")
+        assert_close(dc.np("snap_out", l), snap_ref, what=f"layer {l} states")
+        st_ref, hist_ref, _, _ = oracle_commit_from_device(dc, layer=l)
+        assert_close(dc.np("state", l), st_ref, what=f"layer {l} state")
+        assert np.array_equal(dc.np("conv_hist", l), hist_ref)
+
+
+def test_host_detected_errors_return_codes():
+    c = W.config0()
+    with pytest.raises(binding.LumoError) as e:
+        ctx().tree_desc(np.array([[-1, 1, 0]], dtype=np.int32))
+    assert e.value.code == 2
+    with pytest.raises(binding.LumoError) as e:
+        ctx().tree_desc(c.parent, slot=np.zeros_like(c.parent), n_slots=7)
+    assert e.value.code == 2
+    with pytest.raises(binding.LumoError) as e:
+        ctx().tree_desc(c.parent, depth=np.zeros_like(c.parent))
+    assert e.value.code == 2
+    dc = DeviceCase(ctx(), c)
+    dc.layers[0].args.d = 96
+    with pytest.raises(binding.LumoError) as e:
+        dc.verify()
+    assert e.value.code == 4
+    dc.layers[0].args.d = 64
+    dc.layers[0].args.out = None
+    with pytest.raises(binding.LumoError) as e:
+        dc.verify()
+    assert e.value.code == 1
