@@ -1,0 +1,436 @@
+#!/usr/bin/env python
+"""Benchmark of the GDN tree verify + commit hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg2] [--impl reference]
+
+One "step" = the whole hot path over one batch of synthetic input: tree conv + tree scan
+(lumo_gdn_tree_verify) and accepted-path replay + conv-history gather (lumo_gdn_commit).
+The metric is tree nodes verified per second per layer, B * N * n_layers / step time, summed
+over ranks (each rank owns its own sequences: weak scaling, no collective on the data path).
+
+Prints ONE JSON line.  `value` is timed with inputs resident in HBM (CUDA-graph replay of the
+C-ABI calls, rotating over buffer sets larger than L2); `e2e` repeats the measurement through
+the C-ABI calls with the step's inputs copied from pinned host memory and its outputs copied
+back inside the timed region; `roofline` is the scan kernel's algorithmic bytes over its own
+device time (CUDA events around each launch, taken in a second pass of K steps);
+`cpu_baseline` is the fp64 oracle timed on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "gdn_tree_nodes_verified_per_s_per_layer"
+UNIT = "nodes/s"
+L2_BYTES = 126 * 2 ** 20
+
+
+def make_case(name: str, seed_offset: int = 0):
+    from paper_2609_23900_b200 import workload as W
+    if name == "cfg1":
+        return W.config1(seed=W.BASE_SEED + 1 + 1000 * seed_offset)
+    if name == "cfg2":
+        return W.config2(seed=W.BASE_SEED + 2 + 1000 * seed_offset)
+    if name == "cfg3":
+        return W.config3(seed=W.BASE_SEED + 3 + 1000 * seed_offset)
+    if name.startswith("cfg4_"):
+        return W.config4(name[5:], seed=W.BASE_SEED + 4 + 1000 * seed_offset)
+    if name == "cfgP":
+        return W.config_paper(seed=W.BASE_SEED + 5 + 1000 * seed_offset, B=8, n_layers=1)
+    raise SystemExit(f"unknown config {name}")
+
+
+WORKLOAD_TEXT = {
+    "cfg1": "config 1: batch 1, 16/32 heads, d=128, 16-node MTP-spine tree, 1 layer",
+    "cfg2": "config 2: serving batch 8, 16/32 heads, d=128, random 64-node trees (depth<=8), 1 layer",
+    "cfg3": "config 3: 48 layers back to back, batch 4, 32-node trees (depth<=6)",
+    "cfg4_chains": "config 4: batch 32, 256-node trees, 16 chains of depth 16",
+    "cfg4_star": "config 4: batch 32, 256-node trees, 255-child star",
+    "cfg4_random": "config 4: batch 32, 256-node trees, random depth<=12",
+    "cfgP": "paper geometry: 28 active rows padded to 32, batch 8, 1 layer",
+}
+
+
+def algorithmic_bytes(c, out_bytes=2):
+    """Per layer: state read once, operands read once, outputs written once (verify);
+    state read+written, accepted operands read, history rewritten (commit)."""
+    B, N, Hk, Hv, d = c.B, c.N, c.Hk, c.Hv, c.d
+    s_in = 2 if c.in_dtype == "bf16" else 4
+    C = c.C
+    state = 4 * B * Hv * d * d
+    operands = B * N * C * s_in
+    gates = 2 * B * N * Hv * s_in
+    out = B * N * Hv * d * out_bytes
+    Lsum = int(c.accepted_len.sum())
+    scan = state + operands + gates + out
+    conv = 2 * B * N * C * s_in + 4 * C * s_in + 3 * B * C * s_in
+    commit_state = 2 * state + Lsum * ((Hk * d + Hv * d) * s_in + 2 * Hv * s_in)
+    commit_hist = 2 * 3 * B * C * s_in
+    return dict(scan=scan, conv=conv, commit_state=commit_state, commit_hist=commit_hist)
+
+
+def rank1_fma(c):
+    """fp32 FMAs of the rank-1 form per layer: 2 d^2 per leaf, 3 d^2 per internal node-head."""
+    total = 0
+    for b in range(c.B):
+        par = c.parent[b]
+        internal = set(int(p) for p in par if p >= 0)
+        total += (2 * (c.N - len(internal)) + 3 * len(internal)) * c.Hv * c.d * c.d
+    return total
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the GPU is under load."""
+
+    def __init__(self, index: int, period: float = 0.01):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reasons, self.stop_flag = period, [], set(), False
+        self.max_mhz = None
+        self.windows = {}
+        self._tag = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def tag(self, name):
+        self._tag = name
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self.stop_flag:
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                if self._tag:
+                    self.windows.setdefault(self._tag, []).append(mhz)
+                    for n, bit in names.items():
+                        if r & bit:
+                            self.reasons.add(n)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def summary(self):
+        timed = self.windows.get("timed", [])
+        allw = [m for w in self.windows.values() for m in w]
+        use = timed if len(timed) >= 3 else allw
+        return {"sm_mhz": statistics.median(use) if use else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(use),
+                "window": "timed region" if use is timed and timed else "all load phases of this run"}
+
+
+def run_oracle_steps(case, seconds: float, threads: int = 0):
+    """Times the oracle, as it stands, on whole steps of the workload (conv, memo-mode scan,
+    commit) for about `seconds`; returns (nodes/s/layer, steps, cores, seconds)."""
+    from oracle import gdn_oracle as O
+    O.build()
+    n_layers = len(case.layers)
+    t0 = time.perf_counter()
+    steps, used = 0, 1
+    while True:
+        for L in case.layers:
+            y = O.conv(case.parent, case.slot, case.state_row, L.x, L.conv_w, L.conv_b, L.hist, case.Ns,
+                       out_dtype=case.in_dtype, threads=threads)
+            hk = case.Hk * case.d
+            q = y[..., :hk].reshape(case.B, case.Ns, case.Hk, case.d)
+            k = y[..., hk:2 * hk].reshape(case.B, case.Ns, case.Hk, case.d)
+            v = y[..., 2 * hk:].reshape(case.B, case.Ns, case.Hv, case.d)
+            _, _, used = O.scan(case.parent, case.slot, case.state_row, q, k, v, L.alpha, L.beta, L.state,
+                                l2norm=True, mode="memo", threads=threads)
+            O.commit(case.parent, case.slot, case.state_row, q, k, v, L.alpha, L.beta, L.state, case.accepted,
+                     case.accepted_len, l2norm=True, x=L.x, hist=L.hist, threads=threads)
+        steps += 1
+        dt = time.perf_counter() - t0
+        if dt >= seconds or steps >= 1000:
+            break
+    return case.B * case.N * n_layers * steps / dt, steps, used, dt
+
+
+def reference_arm(args, rank):
+    """The oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    case = make_case(args.config)
+    if len(case.layers) > 4:          # bounded sample: a few layers of the stack
+        case.layers = case.layers[:4]
+    per_step = []
+    cores = 1
+    for i in range(args.warmup + args.steps):
+        v, steps, cores, dt = run_oracle_steps(case, seconds=0.0)
+        if i >= args.warmup:
+            per_step.append(dt)
+        if sum(per_step) > 150:
+            break
+    ms = 1e3 * statistics.mean(per_step)
+    nodes = case.B * case.N * len(case.layers)
+    value = nodes / (ms / 1e3)
+    sample = f"whole batch of {WORKLOAD_TEXT[args.config]}" + (f", first {len(case.layers)} layers" if args.config == "cfg3" else "")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": len(per_step), "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT[args.config], "name": args.config},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--config", default="cfg2", choices=sorted(WORKLOAD_TEXT))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every step instead of graph replay")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2 twice)")
+    ap.add_argument("--out-dtype", default="bf16", choices=["bf16", "f32"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        reference_arm(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2609_23900_b200 import binding
+    from paper_2609_23900_b200.runtime import DeviceCase
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the GDN tree verifier has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    ctx = binding.Context(local)
+    # ---- buffer sets: distinct seeds per set and per rank, together larger than L2 -----------
+    case0 = make_case(args.config, seed_offset=rank * 64)
+    n_layers = len(case0.layers)
+    ab = algorithmic_bytes(case0, out_bytes=2 if args.out_dtype == "bf16" else 4)
+    set_bytes = n_layers * (ab["scan"] + ab["conv"] // 2)
+    n_sets = args.sets or max(2, min(16, -(-3 * L2_BYTES // set_bytes)))
+    cases = [case0] + [make_case(args.config, seed_offset=rank * 64 + i) for i in range(1, n_sets)]
+    sets = [DeviceCase(ctx, c, out_dtype=args.out_dtype, pinned_host=(i < 4)) for i, c in enumerate(cases)]
+    packed = [binding.Context.pack(s.layers) for s in sets]
+    nodes_per_step = case0.B * case0.N * n_layers
+
+    def run_step(i):
+        s = sets[i % n_sets]
+        ctx.verify(s.desc, packed[i % n_sets])
+        ctx.commit(s.desc, packed[i % n_sets], s.accepted, s.accepted_len)
+
+    for i in range(n_sets):          # first calls size the library scratch
+        run_step(i)
+    torch.cuda.synchronize()
+
+    launch_mode = "c_abi_direct"
+    graphs = None
+    if not args.no_graph:
+        try:
+            graphs = []
+            for i in range(n_sets):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g):
+                    run_step(i)
+                graphs.append(g)
+            launch_mode = "cuda_graph_replay_of_c_abi_calls"
+        except Exception as e:  # capture is an optimisation of the launch path only
+            graphs = None
+            launch_mode = f"c_abi_direct (graph capture failed: {type(e).__name__})"
+            torch.cuda.synchronize()
+
+    def step(i):
+        if graphs is not None:
+            graphs[i % n_sets].replay()
+        else:
+            run_step(i)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    sampler.tag("warmup")
+    for i in range(args.warmup):
+        step(i)
+    # ---- timed region: K steps, inputs resident in HBM ------------------------------------
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.tag("timed")
+    ev0.record()
+    for i in range(args.steps):
+        step(i)
+    ev1.record()
+    barrier()
+    sampler.tag("per_kernel")
+    ms_total = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * nodes_per_step / (ms_step / 1e3)
+
+    # ---- per-kernel device time: second pass, events around every launch -------------------
+    ctx.timing_enable(True)
+    ctx.timing_read(reset=True)
+    n_timed = min(args.steps, 2000)
+    for i in range(n_timed):
+        run_step(i)
+    torch.cuda.synchronize()
+    per_kernel = ctx.timing_read(reset=True)
+    ctx.timing_enable(False)
+    kern = {k: {"launches": n, "avg_us": 1e3 * ms / n} for k, (n, ms) in per_kernel.items() if n}
+
+    # ---- end to end: inputs from pinned host memory, outputs back to the host --------------
+    sampler.tag("e2e")
+    hs = [s for s in sets if s.host]
+    out_host = [[torch.empty_like(l.tensors["out"], device="cpu").pin_memory() for l in s.layers] for s in hs]
+    st_host = [torch.empty((case0.B,), dtype=torch.int32).pin_memory() for _ in hs]
+    acc_host = [(s.accepted.cpu().pin_memory(), s.accepted_len.cpu().pin_memory()) for s in hs]
+
+    def e2e_step(i):
+        j = i % len(hs)
+        s = hs[j]
+        for l, h in zip(s.layers, s.host):
+            for name, src in h.items():
+                l.tensors[name].copy_(src, non_blocking=True)
+        s.accepted.copy_(acc_host[j][0], non_blocking=True)
+        s.accepted_len.copy_(acc_host[j][1], non_blocking=True)
+        ctx.verify(s.desc, packed[j])
+        ctx.commit(s.desc, packed[j], s.accepted, s.accepted_len)
+        for l, oh in zip(s.layers, out_host[j]):
+            oh.copy_(l.tensors["out"], non_blocking=True)
+        st_host[j].copy_(s.layers[-1].tensors["status"], non_blocking=True)
+
+    h2d = sum(sum(t.numel() * t.element_size() for t in h.values()) for h in hs[0].host) \
+        + acc_host[0][0].numel() * 4 + acc_host[0][1].numel() * 4
+    d2h = sum(o.numel() * o.element_size() for o in out_host[0]) + st_host[0].numel() * 4
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_e2e = min(args.steps, 200)
+    e0.record()
+    for i in range(n_e2e):
+        e2e_step(i)
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_e2e = float(t.item())
+    e2e_value = world * nodes_per_step * n_e2e / (ms_e2e / 1e3)
+    sampler.stop_flag = True
+    sampler.join(timeout=1.0)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel -----------------------------------------------------
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        with open(peaks_path) as f:
+            peak_gbs, peak_src = float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak_gbs, peak_src = 6650.0, "fallback (earlier measurement on this pool)"
+    dominant = max(kern, key=lambda k: kern[k]["launches"] * kern[k]["avg_us"])
+    achieved = n_layers * ab[dominant] / (kern[dominant]["avg_us"] * 1e-6) / 1e9
+    clocks = sampler.summary()
+    fma = rank1_fma(case0) * n_layers
+    sm_mhz = clocks["sm_mhz"] or 1965.0
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+                "frac": achieved / peak_gbs, "peak_source": peak_src, "traffic": NCU_TRAFFIC.get(args.config),
+                "algorithmic_bytes_per_launch": n_layers * ab[dominant],
+                "avg_launch_us": kern[dominant]["avg_us"],
+                "frac_of_8TBs_nominal": achieved / 8000.0,
+                "timing": "CUDA events around each launch on the launch stream, second pass of the same steps",
+                "fp32_fma_per_launch_rank1": fma,
+                "alu_frac_at_sampled_clock": (fma / (kern["scan"]["avg_us"] * 1e-6)) / (148 * 128 * sm_mhz * 1e6)
+                if "scan" in kern else None}
+    commit_us = sum(kern[k]["avg_us"] for k in ("commit_state", "commit_hist") if k in kern) / n_layers
+    verify_us = sum(kern[k]["avg_us"] for k in ("conv", "scan") if k in kern)
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD_TEXT[args.config], "name": args.config, "batch_per_gpu": case0.B,
+                       "nodes_per_tree": case0.N, "layers": n_layers, "heads_qk_v": [case0.Hk, case0.Hv],
+                       "d": case0.d, "in_dtype": case0.in_dtype, "out_dtype": args.out_dtype, "state": "f32",
+                       "pipeline": "conv+silu -> l2norm(q,k) -> tree scan; commit state + conv history",
+                       "l2": f"rotating over {n_sets} buffer sets ({n_sets * set_bytes / 2**20:.0f} MiB) larger than L2",
+                       "launch": launch_mode, "parallelism": "replicas" if world > 1 else "single gpu",
+                       "mean_accepted_len": float(case0.accepted_len.mean())},
+            "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "window")},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                    "ms_per_step": ms_e2e / n_e2e, "steps": n_e2e},
+            "gpu_launches": int(args.steps * sum(1 for k in ("conv", "scan", "commit_state", "commit_hist") if k in kern)),
+            "roofline": roofline,
+            "kernels": kern,
+            "verify_nodes_per_s_per_layer": nodes_per_step / (verify_us * 1e-6),
+            "verify_us_per_layer": verify_us / n_layers, "commit_us_per_layer": commit_us,
+            "scratch_bytes": ctx.scratch_bytes}
+
+    if world == 1 and not args.no_cpu_baseline:
+        sample_case = case0
+        sample = "whole batch of the same workload, every step = conv + memo-mode scan + commit"
+        if n_layers > 2:
+            import copy
+            sample_case = copy.copy(case0)
+            sample_case.layers = case0.layers[:2]
+            sample += ", first 2 layers"
+        v, steps, cores, dt = run_oracle_steps(sample_case, args.cpu_seconds)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{sample}; {steps} steps in {dt:.1f} s"}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one scan launch, from the ncu captures
+# summarised under profiles/ (bytes per launch at the bench's launch configuration)
+NCU_TRAFFIC = {}
+
+if __name__ == "__main__":
+    main()

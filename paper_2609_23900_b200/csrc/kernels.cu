@@ -164,12 +164,13 @@ struct ScanCfg {
 
 // dynamic shared memory layout (bytes), computed identically on host and device
 struct ScanSmem {
-  int ops, params, dcache, snaplist, ring, total;
+  int ops, slot, params, dcache, snaplist, ring, total;
 };
 __host__ __device__ inline ScanSmem scan_smem(int N, int max_ops, int n_snap_list, int stage_bytes) {
   ScanSmem m;
   int off = 0;
   m.ops = off;      off += ((max_ops * 4 + 15) / 16) * 16;
+  m.slot = off;     off += ((N * 4 + 15) / 16) * 16;
   m.params = off;   off += 5 * N * 4;  off = (off + 15) / 16 * 16;
   m.dcache = off;   off += N * kRows * 4;
   m.snaplist = off; off += ((n_snap_list * 4 + 15) / 16) * 16;
@@ -187,6 +188,7 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
   const int n_snap_list = s.snapshot_mode == 1 ? s.n_snap : 0;
   const ScanSmem lay = scan_smem(s.N, t.max_ops, n_snap_list, Cfg::kStageBytes);
   int32_t* s_ops = reinterpret_cast<int32_t*>(smem + lay.ops);
+  int32_t* s_slot = reinterpret_cast<int32_t*>(smem + lay.slot);   // physical row of each node
   float* p_a = reinterpret_cast<float*>(smem + lay.params);
   float* p_b = p_a + s.N;
   float* p_ks = p_b + s.N;      // multiplies the raw key (1 / norm when normalising)
@@ -196,7 +198,7 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
   int32_t* s_snap = reinterpret_cast<int32_t*>(smem + lay.snaplist);
   unsigned char* s_ring = smem + lay.ring;
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   const int j = tid & 3;               // lane within the row group
   const int rl = tid >> 2;             // local row 0..31
   constexpr int kTiles = D / kRows;
@@ -234,6 +236,7 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
     const int nops = t.nops[b];
     const int32_t* ops_g = t.sched + (size_t)b * t.max_ops;
     for (int e = tid; e < nops; e += kScanThreads) s_ops[e] = ops_g[e];
+    for (int e = tid; e < s.N; e += kScanThreads) s_slot[e] = t.slot[b * s.N + e];
     for (int e = tid; e < n_snap_list; e += kScanThreads) s_snap[e] = L.snap_nodes[(size_t)b * s.n_snap + e];
     // padding rows: zero outputs
     for (int e = tid; e < s.Ns * kRows; e += kScanThreads) {
@@ -245,29 +248,40 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
     const T* qg = reinterpret_cast<const T*>(L.q);
     const T* kg = reinterpret_cast<const T*>(L.k);
     const T* vg = reinterpret_cast<const T*>(L.v);
-    for (int n = warp; n < s.N; n += kScanThreads / 32) {
-      const size_t pr = (size_t)b * s.Ns + t.slot[b * s.N + n];
-      const T* kr = kg + (pr * s.Hk + g) * D;
-      const T* qr = qg + (pr * s.Hk + g) * D;
-      float kk = 0.f, qq = 0.f, kq = 0.f;
-      for (int c = lane * 4; c < D; c += 128) {
-        float4 kv = Vec4<T>::load(kr + c), qv = Vec4<T>::load(qr + c);
-        kk += kv.x * kv.x + kv.y * kv.y + kv.z * kv.z + kv.w * kv.w;
-        qq += qv.x * qv.x + qv.y * qv.y + qv.z * qv.z + qv.w * qv.w;
-        kq += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
-      }
+    {
+      // eight lanes per node, sixteen nodes in flight per pass; the trip count is uniform over
+      // the CTA so that every lane takes part in the shuffles
+      const int grp = tid >> 3, gl = tid & 7;
+#pragma unroll 2
+      for (int n0 = 0; n0 < s.N; n0 += kScanThreads / 8) {
+        const int n = n0 + grp;
+        const bool live = n < s.N;
+        const size_t pr = (size_t)b * s.Ns + (live ? t.slot[b * s.N + n] : 0);
+        const T* kr = kg + (pr * s.Hk + g) * D;
+        const T* qr = qg + (pr * s.Hk + g) * D;
+        float kk = 0.f, qq = 0.f, kq = 0.f;
+        if (live) {
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        kk += __shfl_xor_sync(0xffffffffu, kk, o);
-        qq += __shfl_xor_sync(0xffffffffu, qq, o);
-        kq += __shfl_xor_sync(0xffffffffu, kq, o);
-      }
-      if (lane == 0) {
-        float ks = 1.f, qs = s.scale;
-        if (s.l2norm) { ks = rsqrtf(kk + s.l2_eps); qs = s.scale * rsqrtf(qq + s.l2_eps); }
-        p_ks[n] = ks; p_qs[n] = qs; p_kq[n] = kq * ks * qs;
-        p_a[n] = load_scalar(L.alpha, pr * s.Hv + hv, s.gate_dtype);
-        p_b[n] = load_scalar(L.beta, pr * s.Hv + hv, s.gate_dtype);
+          for (int c = 0; c < D / 32; ++c) {
+            float4 kv = Vec4<T>::load(kr + gl * 4 + 32 * c), qv = Vec4<T>::load(qr + gl * 4 + 32 * c);
+            kk += kv.x * kv.x + kv.y * kv.y + kv.z * kv.z + kv.w * kv.w;
+            qq += qv.x * qv.x + qv.y * qv.y + qv.z * qv.z + qv.w * qv.w;
+            kq += kv.x * qv.x + kv.y * qv.y + kv.z * qv.z + kv.w * qv.w;
+          }
+        }
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) {
+          kk += __shfl_xor_sync(0xffffffffu, kk, o);
+          qq += __shfl_xor_sync(0xffffffffu, qq, o);
+          kq += __shfl_xor_sync(0xffffffffu, kq, o);
+        }
+        if (live && gl == 0) {
+          float ks = 1.f, qs = s.scale;
+          if (s.l2norm) { ks = rsqrtf(kk + s.l2_eps); qs = s.scale * rsqrtf(qq + s.l2_eps); }
+          p_ks[n] = ks; p_qs[n] = qs; p_kq[n] = kq * ks * qs;
+          p_a[n] = load_scalar(L.alpha, pr * s.Hv + hv, s.gate_dtype);
+          p_b[n] = load_scalar(L.beta, pr * s.Hv + hv, s.gate_dtype);
+        }
       }
     }
     __syncthreads();
@@ -279,7 +293,7 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
         const int kind = op >> 24;
         if (kind <= OP_DESCEND) {
           const int n = op & 0xFFFF;
-          const size_t pr = (size_t)b * s.Ns + t.slot[b * s.N + n];
+          const size_t pr = (size_t)b * s.Ns + s_slot[n];
           unsigned char* st = s_ring + (i % kRingDepth) * Cfg::kStageBytes;
           const int nx = kind == OP_DESCEND ? Cfg::kKXfers : Cfg::kStageXfers;
           if (tid < nx) {
@@ -329,7 +343,7 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
         const float dl = bt * (vv - a * (ks * u));          // delta = beta (v - R' k)
         const float o = a * (p_qs[n] * w) + dl * p_kq[n];   // o = R q = a R_p q + delta (k.q)
         if (j == 0) {
-          const size_t pr = (size_t)b * s.Ns + t.slot[b * s.N + n];
+          const size_t pr = (size_t)b * s.Ns + s_slot[n];
           store_scalar(L.out, pr * out_row_stride + hv * D + r0 + rl, s.out_dtype, o);
           if ((op >> 20) & 1) s_dc[n * kRows + rl] = dl;
         }
