@@ -171,6 +171,32 @@ typedef struct {
 int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers,
                          int n_layers, void* stream);
 
+/* The tree scan for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this is a property of this library's scratch handling, not of the method.)
+ *
+ * lumo_gdn_tree_verify keeps the scan's state stack in memory that the context allocates the first
+ * time a shape needs it.  Some callers cannot tolerate that: code running between the capture and
+ * the replay of a CUDA graph's memory plan, a serving loop whose memory pool has already handed
+ * every byte to the KV cache and the state banks, or a process whose allocator is owned by another
+ * runtime.  This call runs the same scan kernel with the stack in a fixed array that is part of
+ * the library image (lumo_static_stack_bytes() = 64 MiB, held by every GPU that loads the library
+ * until the process exits).  It never calls cudaMalloc, cudaFree or any allocating routine.
+ *
+ *   - Runs the scan only, on the recorded operands q, k, v (the convolution stage needs no scratch;
+ *     run it through lumo_gdn_tree_verify beforehand, or pass operands directly).  `x` is ignored.
+ *   - Same arguments, outputs, snapshot modes and status words as lumo_gdn_tree_verify.
+ *   - A shape whose persistent grid needs more stack than the array holds is refused with
+ *     LUMO_ERR_UNSUPPORTED and a message that states both sizes; nothing is enqueued.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call before starting any stream capture.
+ *   - All calls share the one array.  Nothing in it has to start at zero (every stack level is
+ *     written before it is read within a call), and it keeps the previous call's contents.  Two
+ *     calls that overlap on the GPU (different streams, or graphs launched concurrently) race on
+ *     it and corrupt each other's outputs: serialise them. */
+int lumo_gdn_tree_scan_static(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers,
+                              int n_layers, void* stream);
+int64_t lumo_static_stack_bytes(void);
+
 /* Replays accepted_dev [B, lmax] (logical ids, root first; entries at or beyond len_dev[b] are
  * ignored) from the pre-tree state with the recorded operands and publishes state and
  * convolution history in place (Algorithm 2, "Replay only the accepted path into native

@@ -36,7 +36,8 @@ KERNEL_KINDS = ["conv", "scan", "commit_state", "commit_hist", "path"]
 EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_scratch_bytes",
            "lumo_ctx_timing_enable", "lumo_ctx_timing_read",
            "lumo_tree_desc_create", "lumo_tree_desc_destroy", "lumo_tree_desc_get",
-           "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit"]
+           "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit",
+           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes"]
 
 
 class LumoError(RuntimeError):
@@ -86,6 +87,9 @@ _lib.lumo_tree_path_from_node.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctyp
                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.lumo_gdn_tree_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
                                       ctypes.c_void_p]
+_lib.lumo_gdn_tree_scan_static.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
+                                           ctypes.c_void_p]
+_lib.lumo_static_stack_bytes.restype = ctypes.c_int64
 _lib.lumo_gdn_commit.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
 
@@ -163,6 +167,17 @@ class Context:
     def verify(self, desc: "TreeDesc", layers, stream=None):
         arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)
         self._check(_lib.lumo_gdn_tree_verify(self._h, desc._h, arr, len(layers), _stream(stream)))
+
+    def scan_static(self, desc: "TreeDesc", layers, stream=None):
+        """The tree scan with the library's built-in, fixed-size stack: for callers that must not
+        allocate device memory.  Scan only (no convolution); refuses shapes that need more stack than
+        ``static_stack_bytes()``.  Calls that overlap on the GPU race on the shared stack."""
+        arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)
+        self._check(_lib.lumo_gdn_tree_scan_static(self._h, desc._h, arr, len(arr), _stream(stream)))
+
+    @staticmethod
+    def static_stack_bytes() -> int:
+        return int(_lib.lumo_static_stack_bytes())
 
     def commit(self, desc: "TreeDesc", layers, accepted: torch.Tensor, length: torch.Tensor, stream=None):
         arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)

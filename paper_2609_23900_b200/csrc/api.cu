@@ -337,6 +337,33 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "scan launch");
 }
 
+int64_t lumo_static_stack_bytes(void) { return (int64_t)kStaticStackBytes; }
+
+int lumo_gdn_tree_scan_static(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers,
+                              int n_layers, void* stream) {
+  Shape s;
+  LayerBatch lb;
+  std::memset(&lb, 0, sizeof(lb));
+  int rc = prepare(ctx, desc, layers, n_layers, true, &s, &lb);
+  if (rc != LUMO_OK) return rc;
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const TreeDev t = tree_view(desc, s.snapshot_mode != 0 ? 1 : 0);
+  int grid = 0;
+  size_t stack_bytes = 0;
+  cudaError_t e = scan_plan(s, t, ctx->sm_count, &grid, &stack_bytes);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "scan_plan");
+  if (stack_bytes > kStaticStackBytes)
+    return fail(ctx, LUMO_ERR_UNSUPPORTED,
+                "this shape needs " + std::to_string(stack_bytes) + " bytes of scan stack; the built-in stack holds " +
+                    std::to_string(kStaticStackBytes) + " (use lumo_gdn_tree_verify, which allocates)");
+  float* stack = nullptr;
+  e = static_stack_address(ctx->device, &stack);
+  if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGetSymbolAddress(built-in scan stack)");
+  e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan(s, t, lb, stack, grid, st); });
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "scan launch");
+}
+
 int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers,
                     const int32_t* accepted_dev, const int32_t* len_dev, int lmax, void* stream) {
   Shape s;

@@ -12,6 +12,7 @@ namespace lumo {
 constexpr int kMaxNodes = 256;
 constexpr int kMaxSlots = 1024;
 constexpr int kMaxLayers = 64;
+constexpr size_t kStaticStackBytes = 64u << 20;   // capacity of the built-in scan stack
 
 // ---- scan schedule ------------------------------------------------------------------
 // The scan kernel walks the whole tree depth first with the state tile of the current
@@ -103,6 +104,8 @@ cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, 
                         int grid, cudaStream_t st);
 // persistent grid size (CTAs resident at once) and the stack scratch it needs
 cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes);
+// device address of the built-in stack on `device` (which must be current); looked up once per device
+cudaError_t static_stack_address(int device, float** ptr);
 cudaError_t launch_commit_state(const Shape& s, const TreeDev& t, const LayerBatch& lb,
                                 const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st);
 cudaError_t launch_commit_hist(const Shape& s, const TreeDev& t, const LayerBatch& lb,

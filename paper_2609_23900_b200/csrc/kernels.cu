@@ -9,6 +9,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <mutex>
 #include <type_traits>
 
 #include "internal.h"
@@ -569,6 +570,35 @@ cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid,
     *stack_bytes = (size_t)*grid * t.max_levels * kRows * D * sizeof(float);
     return cudaSuccess;
   });
+}
+
+// ---------------------------------------------------------------------------------------
+// fixed scratch for callers that cannot allocate (lumo_gdn_tree_scan_static)
+// ---------------------------------------------------------------------------------------
+// The scan's state stack normally lives in memory the context allocates on first use.  This
+// array is the same stack with a fixed capacity, part of the library image on every GPU that
+// loads it.  Host code must not pass `g_static_stack` itself to a kernel: on the host the name
+// is only a handle for the symbol, so its device address is looked up once per device.
+__device__ __align__(256) static float g_static_stack[kStaticStackBytes / sizeof(float)];
+
+cudaError_t static_stack_address(int device, float** ptr) {
+  constexpr int kMaxDevices = 64;
+  static float* cached[kMaxDevices] = {};
+  static std::mutex mu;
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!cached[device]) {
+    int cur = -1;
+    cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return e;
+    if (cur != device) return cudaErrorInvalidDevice;   // the caller makes `device` current first
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_static_stack);
+    if (e != cudaSuccess) return e;
+    cached[device] = static_cast<float*>(p);
+  }
+  *ptr = cached[device];
+  return cudaSuccess;
 }
 
 cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, float* stack,
