@@ -62,6 +62,31 @@ WORKLOAD_TEXT = {
 }
 
 
+def rank_seed_offset(rank: int) -> int:
+    """Each rank owns its own sequences (weak scaling): disjoint seed ranges per rank."""
+    return rank * 64
+
+
+def is_reporting_rank(rank: int) -> bool:
+    return rank == 0
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """A step is as slow as its slowest rank."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(nodes_per_rank_step: int, ms_step: float, world: int) -> float:
+    """Whole-job nodes per second: every rank processed its own batch in the (max) step time."""
+    return world * nodes_per_rank_step / (ms_step / 1e3)
+
+
 def algorithmic_bytes(c, out_bytes=2):
     """Per layer: state read once, operands read once, outputs written once (verify);
     state read+written, accepted operands read, history rewritten (commit)."""
@@ -240,12 +265,12 @@ def main():
 
     ctx = binding.Context(local)
     # ---- buffer sets: distinct seeds per set and per rank, together larger than L2 -----------
-    case0 = make_case(args.config, seed_offset=rank * 64)
+    case0 = make_case(args.config, seed_offset=rank_seed_offset(rank))
     n_layers = len(case0.layers)
     ab = algorithmic_bytes(case0, out_bytes=2 if args.out_dtype == "bf16" else 4)
     set_bytes = n_layers * (ab["scan"] + ab["conv"] // 2)
     n_sets = args.sets or max(2, min(16, -(-3 * L2_BYTES // set_bytes)))
-    cases = [case0] + [make_case(args.config, seed_offset=rank * 64 + i) for i in range(1, n_sets)]
+    cases = [case0] + [make_case(args.config, seed_offset=rank_seed_offset(rank) + i) for i in range(1, n_sets)]
     sets = [DeviceCase(ctx, c, out_dtype=args.out_dtype, pinned_host=(i < 4)) for i, c in enumerate(cases)]
     packed = [binding.Context.pack(s.layers) for s in sets]
     nodes_per_step = case0.B * case0.N * n_layers
@@ -301,13 +326,9 @@ def main():
     ev1.record()
     barrier()
     sampler.tag("per_kernel")
-    ms_total = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1), world, dev)
     ms_step = ms_total / args.steps
-    value = world * nodes_per_step / (ms_step / 1e3)
+    value = aggregate_value(nodes_per_step, ms_step, world)
 
     # ---- per-kernel device time: second pass, events around every launch -------------------
     ctx.timing_enable(True)
@@ -354,16 +375,12 @@ def main():
         e2e_step(i)
     e1.record()
     barrier()
-    ms_e2e = e0.elapsed_time(e1)
-    if world > 1:
-        t = torch.tensor([ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_e2e = float(t.item())
-    e2e_value = world * nodes_per_step * n_e2e / (ms_e2e / 1e3)
+    ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev)
+    e2e_value = aggregate_value(nodes_per_step, ms_e2e / n_e2e, world)
     sampler.stop_flag = True
     sampler.join(timeout=1.0)
 
-    if rank != 0:
+    if not is_reporting_rank(rank):
         if world > 1:
             dist.destroy_process_group()
         return
