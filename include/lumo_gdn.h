@@ -56,7 +56,8 @@ typedef enum {
   LUMO_SEQ_BAD_NODE = 2,  /* accepted entry outside [0, N) */
   LUMO_SEQ_BAD_ROOT = 3,  /* first accepted entry is not a child of the pre-tree state */
   LUMO_SEQ_BAD_LINK = 4,  /* accepted entry t is not a child of entry t-1 */
-  LUMO_SEQ_BAD_ROW = 5    /* state_row[b] >= n_state_rows */
+  LUMO_SEQ_BAD_ROW = 5,   /* state_row[b] >= n_state_rows */
+  LUMO_SEQ_TIMEOUT = 6    /* a bounded device-side wait ran out; outputs of the call are invalid */
 } lumo_seq_status;
 
 /* Integer tables of one tree (lumo_tree_desc_get).  The paper's tree descriptor holds parent
@@ -100,6 +101,11 @@ void lumo_ctx_destroy(lumo_ctx* ctx);
 const char* lumo_last_error(const lumo_ctx* ctx);
 /* Bytes of library-owned device scratch currently held (for reporting). */
 int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx);
+
+/* Which scan kernel lumo_gdn_tree_verify uses: 0 = automatic (the tensor-core Gram form when the
+ * shape allows it: d = 128, bf16 operands, N <= 64, depth <= 16, no snapshots; else rank-1),
+ * 1 = always the rank-1 fp32 kernel, 2 = Gram form or LUMO_ERR_UNSUPPORTED. */
+int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo);
 
 /* Measurement aid.  While enabled, every kernel the library launches is bracketed by two CUDA
  * events on the launch stream (up to 16384 launches between reads; later ones go untimed).

@@ -113,6 +113,7 @@ TreeDev tree_view(const lumo_tree_desc* d, int which) {
   t.parent = d->d_parent; t.depth = d->d_depth; t.slot = d->d_slot; t.slot_inv = d->d_slot_inv;
   t.win = d->d_win; t.sched = d->d_sched[which]; t.nops = d->d_nops[which];
   t.max_ops = d->max_ops[which]; t.max_levels = d->max_levels[which];
+  t.tc_meta = d->d_tc_meta; t.tc_anc = d->d_tc_anc;
   return t;
 }
 
@@ -162,6 +163,13 @@ void lumo_ctx_destroy(lumo_ctx* ctx) {
 const char* lumo_last_error(const lumo_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_err.c_str(); }
 
 int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx) { return ctx ? (int64_t)ctx->scratch_bytes : 0; }
+
+int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo) {
+  if (!ctx) return LUMO_ERR_ARG;
+  if (algo < 0 || algo > 2) return fail(ctx, LUMO_ERR_ARG, "scan algo must be 0 (auto), 1 (rank-1) or 2 (Gram form)");
+  ctx->scan_algo = algo;
+  return LUMO_OK;
+}
 
 int lumo_ctx_timing_enable(lumo_ctx* ctx, int enable) {
   if (!ctx) return LUMO_ERR_ARG;
@@ -237,6 +245,10 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   const size_t o_inv = reserve((size_t)B * Ns), o_win = reserve((size_t)B * N * 4);
   size_t o_sched[2], o_nops[2];
   for (int w = 0; w < 2; ++w) { o_sched[w] = reserve((size_t)B * d->max_ops[w]); o_nops[w] = reserve(B); }
+  for (int b = 0; b < B; ++b)
+    for (int i = 0; i < N; ++i) d->max_depth = std::max(d->max_depth, (int)d->trees[b].tab[LUMO_TAB_DEPTH][i]);
+  const bool tc = N <= 64 && d->max_depth <= 16;
+  const size_t o_tc_meta = tc ? reserve((size_t)B * N) : 0, o_tc_anc = tc ? reserve((size_t)B * N * 4) : 0;
   for (int b = 0; b < B; ++b) {
     const HostTree& t = d->trees[b];
     for (int i = 0; i < N; ++i) {
@@ -254,6 +266,27 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
       std::copy(ops.begin(), ops.end(), h.begin() + o_sched[w] + (size_t)b * d->max_ops[w]);
       h[o_nops[w] + b] = (int32_t)ops.size();
     }
+    if (tc) {
+      // depth-first preorder (children ascending); pos[node] = position
+      const auto& coff = t.tab[LUMO_TAB_CHILD_OFF];
+      const auto& clist = t.tab[LUMO_TAB_CHILD_LIST];
+      std::vector<int> order, pos(N, -1), stack;
+      for (int c = coff[1] - 1; c >= coff[0]; --c) stack.push_back(clist[c]);
+      while (!stack.empty()) {
+        int n = stack.back(); stack.pop_back();
+        pos[n] = (int)order.size();
+        order.push_back(n);
+        for (int c = coff[n + 2] - 1; c >= coff[n + 1]; --c) stack.push_back(clist[c]);
+      }
+      uint8_t* anc = reinterpret_cast<uint8_t*>(h.data() + o_tc_anc) + (size_t)b * N * 16;
+      for (int pi = 0; pi < N; ++pi) {
+        const int n = order[pi];
+        const int dep = t.tab[LUMO_TAB_DEPTH][n];
+        h[o_tc_meta + (size_t)b * N + pi] = h[o_slot + (size_t)b * N + n] | (dep << 16);
+        int cur = parent[(size_t)b * N + n];
+        for (int j = dep - 2; j >= 0; --j) { anc[pi * 16 + j] = (uint8_t)pos[cur]; cur = parent[(size_t)b * N + cur]; }
+      }
+    }
   }
   if (ctx->device < 0) { *out = d; return LUMO_OK; }   // host-only: tables stay on the host
   DeviceGuard g(ctx->device);
@@ -264,6 +297,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   d->d_parent = d->dev + o_parent; d->d_depth = d->dev + o_depth; d->d_slot = d->dev + o_slot;
   d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_win;
   for (int w = 0; w < 2; ++w) { d->d_sched[w] = d->dev + o_sched[w]; d->d_nops[w] = d->dev + o_nops[w]; }
+  if (tc) { d->d_tc_meta = d->dev + o_tc_meta; d->d_tc_anc = reinterpret_cast<uint8_t*>(d->dev + o_tc_anc); }
   *out = d;
   return LUMO_OK;
 }
@@ -310,6 +344,18 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
   DeviceGuard g(ctx->device);
   cudaStream_t st = (cudaStream_t)stream;
   const TreeDev t = tree_view(desc, s.snapshot_mode != 0 ? 1 : 0);
+  const bool gram_ok = desc->d_tc_meta != nullptr && gram_supported(s, desc->max_depth);
+  if (ctx->scan_algo == 2 && !gram_ok)
+    return fail(ctx, LUMO_ERR_UNSUPPORTED, "the Gram-form scan needs d = 128, bf16 operands, N <= 64, depth <= 16, no snapshots");
+  if (gram_ok && ctx->scan_algo != 1) {
+    cudaError_t e = cudaSuccess;
+    if (layers[0].x) {
+      e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, st); });
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
+    }
+    e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram(s, t, lb, desc->max_depth, ctx->sm_count, st); });
+    return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "Gram-form scan launch");
+  }
   int grid = 0;
   size_t stack_bytes = 0;
   cudaError_t e = scan_plan(s, t, ctx->sm_count, &grid, &stack_bytes);

@@ -41,6 +41,7 @@ struct lumo_ctx {
   void* scratch = nullptr;      // scan stack levels
   size_t scratch_bytes = 0;
   // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
+  int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form (tensor cores)
   bool timing = false;
   std::vector<cudaEvent_t> ev_start, ev_stop;
   std::vector<int> ev_kind;
@@ -61,6 +62,10 @@ struct lumo_tree_desc {
   int32_t* d_nops[2] = {nullptr, nullptr};    // [B]
   int max_ops[2] = {0, 0};
   int max_levels[2] = {0, 0};     // stack levels the schedule needs
+  int max_depth = 0;              // deepest node over the batch
+  // Gram-form scan tables (present when N <= 64 and max_depth <= 16), nodes in depth-first order
+  int32_t* d_tc_meta = nullptr;   // [B, N]  physical row | depth << 16 of the node at position pi
+  uint8_t* d_tc_anc = nullptr;    // [B, N, 16] positions of the ancestors, root first
 };
 
 namespace lumo {
@@ -92,6 +97,7 @@ struct Shape {
 struct TreeDev {
   const int32_t* parent; const int32_t* depth; const int32_t* slot; const int32_t* slot_inv;
   const int32_t* win; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
+  const int32_t* tc_meta; const uint8_t* tc_anc;
 };
 
 // host-side tree tables (tree_desc.cpp)
@@ -104,6 +110,10 @@ cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, 
                         int grid, cudaStream_t st);
 // persistent grid size (CTAs resident at once) and the stack scratch it needs
 cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes);
+// Gram-form scan on tcgen05 (scan_gram.cu)
+bool gram_supported(const Shape& s, int max_depth);
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int max_depth, int sm_count,
+                             cudaStream_t st);
 // device address of the built-in stack on `device` (which must be current); looked up once per device
 cudaError_t static_stack_address(int device, float** ptr);
 cudaError_t launch_commit_state(const Shape& s, const TreeDev& t, const LayerBatch& lb,

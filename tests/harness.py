@@ -10,11 +10,20 @@ from paper_2609_23900_b200.runtime import DeviceCase
 _ctx = None
 
 
-def ctx():
+def ctx(algo="auto"):
+    """Shared context; `algo` selects the scan kernel ("auto", "rank1", "gram") for the calls that follow."""
     global _ctx
     if _ctx is None:
         _ctx = binding.Context(0)
+    _ctx.set_scan_algo(algo)
     return _ctx
+
+
+def gram_eligible(c) -> bool:
+    """Shapes the tensor-core Gram-form scan takes: d = 128, bf16 operands, N <= 64, depth <= 16."""
+    from paper_2609_23900_b200 import workload as W
+    depth = max(max(W.tree_depths(p.tolist())) for p in c.parent)
+    return c.d == 128 and c.in_dtype == "bf16" and c.N <= 64 and depth <= 16
 
 
 def ulp_bf16(ref):

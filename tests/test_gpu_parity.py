@@ -14,7 +14,7 @@ from oracle import tree_tables as T
 from paper_2609_23900_b200 import binding
 from paper_2609_23900_b200 import workload as W
 from paper_2609_23900_b200.runtime import DeviceCase
-from tests.harness import assert_close, ctx, oracle_commit_from_device, oracle_scan_from_device
+from tests.harness import assert_close, ctx, gram_eligible, oracle_commit_from_device, oracle_scan_from_device
 
 pytestmark = pytest.mark.gpu
 
@@ -102,9 +102,15 @@ def test_conv_recorded_operands(name):
 # ------------------------------------------------------------------ scan
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("use_conv", [False, True])
-def test_scan_outputs_match_oracle(name, use_conv):
+@pytest.mark.parametrize("algo", ["rank1", "gram"])
+def test_scan_outputs_match_oracle(name, use_conv, algo):
     c = CASES[name]()
-    dc = DeviceCase(ctx(), c, use_conv=use_conv)
+    if algo == "gram" and not gram_eligible(c):
+        with pytest.raises(binding.LumoError) as e:     # refused loudly, never a silent fallback
+            DeviceCase(ctx("gram"), c, use_conv=use_conv).verify()
+        assert e.value.code == 4
+        return
+    dc = DeviceCase(ctx(algo), c, use_conv=use_conv)
     dc.t("out").fill_(float("nan"))
     dc.verify()
     torch.cuda.synchronize()
@@ -117,16 +123,17 @@ def test_scan_outputs_match_oracle(name, use_conv):
         pad = sorted(set(range(c.Ns)) - set(c.slot[b].tolist()))
         assert np.all(got[b, pad] == 0.0)
     # bf16-typed outputs: bitwise RNE of the same kernel's fp32 outputs
-    dc16 = DeviceCase(ctx(), c, use_conv=use_conv, out_dtype="bf16")
+    dc16 = DeviceCase(ctx(algo), c, use_conv=use_conv, out_dtype="bf16")
     dc16.verify()
     torch.cuda.synchronize()
     assert torch.equal(dc16.t("out"), dc.t("out").to(torch.bfloat16))
     assert_close(dc16.np("out"), o_ref, bf16=True, what=f"{name} scan bf16 out")
 
 
-def test_scan_twice_is_bitwise_reproducible():
+@pytest.mark.parametrize("algo", ["rank1", "gram"])
+def test_scan_twice_is_bitwise_reproducible(algo):
     c = CASES["cfg2"]()
-    dc = DeviceCase(ctx(), c)
+    dc = DeviceCase(ctx(algo), c)
     dc.verify()
     a = dc.t("out").clone()
     qa = dc.t("q").clone()
@@ -135,13 +142,14 @@ def test_scan_twice_is_bitwise_reproducible():
     assert torch.equal(a, dc.t("out")) and torch.equal(qa, dc.t("q"))
 
 
-def test_l2norm_flag_scale_and_f32_gates():
+@pytest.mark.parametrize("algo", ["rank1", "gram"])
+def test_l2norm_flag_scale_and_f32_gates(algo):
     c = small(rand_parents(4, 20, 2), d=128, dtype="bf16")
     rs = np.random.default_rng(1)
     for L in c.layers:   # un-normalised q, k
         L.q[:] = W.round_to(L.q * rs.uniform(0.5, 4.0, size=L.q.shape[:-1] + (1,)), "bf16")
         L.k[:] = W.round_to(L.k * rs.uniform(0.5, 4.0, size=L.k.shape[:-1] + (1,)), "bf16")
-    dc = DeviceCase(ctx(), c, use_conv=False, gate_dtype="f32", qk_l2norm=True, l2_eps=1e-6, scale=0.5)
+    dc = DeviceCase(ctx(algo), c, use_conv=False, gate_dtype="f32", qk_l2norm=True, l2_eps=1e-6, scale=0.5)
     dc.verify()
     torch.cuda.synchronize()
     o_ref, _, _ = oracle_scan_from_device(dc)
@@ -246,6 +254,36 @@ def test_commit_controls_len0_poisoned_tail_invalid_paths_skipped_rows():
     torch.cuda.synchronize()
     assert dc2.np("status").tolist() == [0, 0, 0, binding.SEQ_BAD_ROW, 0, 0]
     assert torch.all(dc2.t("out")[2] == 0) and torch.all(dc2.t("out")[3] == 0) and torch.all(dc2.t("q")[2] == 0)
+
+
+def test_gram_scan_skipped_rows_padding_and_depth_16():
+    # a 16-deep chain plus side leaves (depth limit of the Gram form), padded and permuted rows,
+    # one skipped sequence and one row outside the pool
+    parent = W.tree_chain(16) + [3, 3, 7, 11, 14]
+    c = W.make_case("g16", [parent] * 4, seed=21, Hk=2, Hv=4, d=128, in_dtype="bf16", Ns=24, permute_slots=True,
+                    alpha_lo=0.5, beta_uniform=True, extra_rows=2)
+    assert gram_eligible(c)
+    dc = DeviceCase(ctx("gram"), c)
+    dc.state_row[1] = -1
+    dc.state_row[2] = c.rows + 3
+    dc.t("out").fill_(float("nan"))
+    dc.verify()
+    torch.cuda.synchronize()
+    assert dc.np("status").tolist() == [0, 0, binding.SEQ_BAD_ROW, 0]
+    row = c.state_row.copy()
+    row[1] = row[2] = -1
+    o_ref, _, _ = O.scan(c.parent, c.slot, row, dc.np("q"), dc.np("k"), dc.np("v"), dc.np("alpha"), dc.np("beta"),
+                         c.layers[0].state, l2norm=True)
+    assert_close(dc.np("out"), o_ref, what="gram depth 16")
+    assert torch.all(dc.t("out")[1] == 0) and torch.all(dc.t("out")[2] == 0)
+    # the rank-1 kernel agrees on the same inputs
+    dr = DeviceCase(ctx("rank1"), c)
+    dr.state_row[1] = -1
+    dr.state_row[2] = c.rows + 3
+    dr.verify()
+    torch.cuda.synchronize()
+    assert_close(dr.np("out"), o_ref, what="rank-1 depth 16")
+    ctx("auto")
 
 
 def test_off_path_poison_and_two_cycles():

@@ -19,6 +19,7 @@ pytestmark = pytest.mark.gpu
 
 def test_static_stack_scan_matches_allocating_verify_twice():
     ctx = binding.Context(0)
+    ctx.set_scan_algo("rank1")      # compare like with like: the entry point under test runs the rank-1 kernel
     # a tree with several branching internal nodes so that the stack is really used
     parents = [W.tree_random(W.IntStream(W.stream_key(77, b)), 64, 8) for b in range(4)]
     case = W.make_case("noalloc", parents, seed=77, Hk=4, Hv=8, d=128, in_dtype="bf16")
