@@ -113,7 +113,7 @@ TreeDev tree_view(const lumo_tree_desc* d, int which) {
   t.parent = d->d_parent; t.depth = d->d_depth; t.slot = d->d_slot; t.slot_inv = d->d_slot_inv;
   t.win = d->d_win; t.sched = d->d_sched[which]; t.nops = d->d_nops[which];
   t.max_ops = d->max_ops[which]; t.max_levels = d->max_levels[which];
-  t.tc_meta = d->d_tc_meta; t.tc_anc = d->d_tc_anc;
+  t.tc_meta = d->d_tc_meta; t.tc_anc = d->d_tc_anc; t.tc_lvl = d->d_tc_lvl;
   return t;
 }
 
@@ -249,6 +249,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
     for (int i = 0; i < N; ++i) d->max_depth = std::max(d->max_depth, (int)d->trees[b].tab[LUMO_TAB_DEPTH][i]);
   const bool tc = N <= 64 && d->max_depth <= 16;
   const size_t o_tc_meta = tc ? reserve((size_t)B * N) : 0, o_tc_anc = tc ? reserve((size_t)B * N * 4) : 0;
+  const size_t o_tc_lvl = tc ? reserve((size_t)B * 5) : 0;
   for (int b = 0; b < B; ++b) {
     const HostTree& t = d->trees[b];
     for (int i = 0; i < N; ++i) {
@@ -267,17 +268,15 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
       h[o_nops[w] + b] = (int32_t)ops.size();
     }
     if (tc) {
-      // depth-first preorder (children ascending); pos[node] = position
-      const auto& coff = t.tab[LUMO_TAB_CHILD_OFF];
-      const auto& clist = t.tab[LUMO_TAB_CHILD_LIST];
-      std::vector<int> order, pos(N, -1), stack;
-      for (int c = coff[1] - 1; c >= coff[0]; --c) stack.push_back(clist[c]);
-      while (!stack.empty()) {
-        int n = stack.back(); stack.pop_back();
-        pos[n] = (int)order.size();
-        order.push_back(n);
-        for (int c = coff[n + 2] - 1; c >= coff[n + 1]; --c) stack.push_back(clist[c]);
+      // nodes ordered by (depth, logical index); pos[node] = position
+      std::vector<int> order, pos(N, -1);
+      uint8_t* lvl = reinterpret_cast<uint8_t*>(h.data() + o_tc_lvl) + (size_t)b * 20;
+      for (int dep = 1; dep <= 16; ++dep) {
+        for (int n = 0; n < N; ++n)
+          if (t.tab[LUMO_TAB_DEPTH][n] == dep) { pos[n] = (int)order.size(); order.push_back(n); }
+        lvl[dep] = (uint8_t)order.size();
       }
+      for (int dep = 17; dep < 20; ++dep) lvl[dep] = (uint8_t)N;
       uint8_t* anc = reinterpret_cast<uint8_t*>(h.data() + o_tc_anc) + (size_t)b * N * 16;
       for (int pi = 0; pi < N; ++pi) {
         const int n = order[pi];
@@ -297,7 +296,11 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   d->d_parent = d->dev + o_parent; d->d_depth = d->dev + o_depth; d->d_slot = d->dev + o_slot;
   d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_win;
   for (int w = 0; w < 2; ++w) { d->d_sched[w] = d->dev + o_sched[w]; d->d_nops[w] = d->dev + o_nops[w]; }
-  if (tc) { d->d_tc_meta = d->dev + o_tc_meta; d->d_tc_anc = reinterpret_cast<uint8_t*>(d->dev + o_tc_anc); }
+  if (tc) {
+    d->d_tc_meta = d->dev + o_tc_meta;
+    d->d_tc_anc = reinterpret_cast<uint8_t*>(d->dev + o_tc_anc);
+    d->d_tc_lvl = reinterpret_cast<uint8_t*>(d->dev + o_tc_lvl);
+  }
   *out = d;
   return LUMO_OK;
 }
@@ -353,7 +356,7 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
       e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, st); });
       if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
     }
-    e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram(s, t, lb, desc->max_depth, ctx->sm_count, st); });
+    e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram(s, t, lb, ctx->sm_count, st); });
     return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "Gram-form scan launch");
   }
   int grid = 0;

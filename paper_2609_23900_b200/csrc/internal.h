@@ -63,9 +63,10 @@ struct lumo_tree_desc {
   int max_ops[2] = {0, 0};
   int max_levels[2] = {0, 0};     // stack levels the schedule needs
   int max_depth = 0;              // deepest node over the batch
-  // Gram-form scan tables (present when N <= 64 and max_depth <= 16), nodes in depth-first order
+  // Gram-form scan tables (present when N <= 64 and max_depth <= 16), nodes ordered by (depth, index)
   int32_t* d_tc_meta = nullptr;   // [B, N]  physical row | depth << 16 of the node at position pi
   uint8_t* d_tc_anc = nullptr;    // [B, N, 16] positions of the ancestors, root first
+  uint8_t* d_tc_lvl = nullptr;    // [B, 20] lvl[d] = number of nodes of depth <= d (lvl[0] = 0)
 };
 
 namespace lumo {
@@ -97,7 +98,7 @@ struct Shape {
 struct TreeDev {
   const int32_t* parent; const int32_t* depth; const int32_t* slot; const int32_t* slot_inv;
   const int32_t* win; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
-  const int32_t* tc_meta; const uint8_t* tc_anc;
+  const int32_t* tc_meta; const uint8_t* tc_anc; const uint8_t* tc_lvl;
 };
 
 // host-side tree tables (tree_desc.cpp)
@@ -112,8 +113,7 @@ cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, 
 cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes);
 // Gram-form scan on tcgen05 (scan_gram.cu)
 bool gram_supported(const Shape& s, int max_depth);
-cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int max_depth, int sm_count,
-                             cudaStream_t st);
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, cudaStream_t st);
 // device address of the built-in stack on `device` (which must be current); looked up once per device
 cudaError_t static_stack_address(int device, float** ptr);
 cudaError_t launch_commit_state(const Shape& s, const TreeDev& t, const LayerBatch& lb,

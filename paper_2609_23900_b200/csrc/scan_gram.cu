@@ -12,14 +12,19 @@
 // tensor memory:
 //   P    = S0 [K | Q]^T      [128 value rows x 2*64 nodes], S0 split exactly into bf16 hi + lo
 //   Gram = [K ; Q] K^T       [2*64 x 64], exact products of bf16 inputs
-// Everything after that is O(depth) fp32 FMAs per (row, node): thread r owns value row r (= TMEM
-// lane r), keeps the deltas of the current root-to-node path in registers indexed by depth, and
-// walks the nodes in depth-first order, so sequential fp32 arithmetic along each path is kept.
+// Everything after that is O(depth) fp32 FMAs per (row, node) in sequential fp32 arithmetic along
+// each path: nodes are ordered by depth, a thread owns one value row (= TMEM lane) of one node
+// at a time, the deltas live in shared memory [node][row], and the tree is walked level by level
+// (all nodes of one depth are independent), the nodes of a level dealt out to the eight warps,
+// each lane carrying four adjacent value rows so that the per-node coefficient loads are shared.
+// Per node the CTA first builds a 224-byte record (coefficients, ancestor offsets, output
+// offset); a warp loads the record of its next node before the barrier that publishes the
+// previous level, so that only the ancestors' deltas are fetched after it.
 //
-// One CTA (128 threads) handles one (layer, sequence, value head) at a time; two CTAs per SM
-// overlap one item's loads with the other's arithmetic.  Limits of this kernel: d = 128, bf16
-// operands, N <= 64 nodes, tree depth <= 16, no state snapshots; everything else takes the
-// rank-1 kernel.
+// One CTA (256 threads) handles one (layer, sequence, value head) at a time; two CTAs per SM
+// overlap one item's loads with the other's arithmetic.  Limits of this
+// kernel: d = 128, bf16 operands, N <= 64 nodes, tree depth <= 16, no state snapshots; everything
+// else takes the rank-1 kernel.
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -31,28 +36,47 @@ namespace {
 
 constexpr int kD = 128;
 constexpr int kNT = 64;               // node tile
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
 constexpr int kTmemCols = 256;        // P: 128 columns, Gram: 64 columns (power of two allocation)
-constexpr int kWStride = 20;          // floats per coefficient row: 16 W, c0, beta/unused, depth bits, pad
-constexpr int kDumpStride = 68;       // floats per dumped Gram row (conflict-free 128-bit stores)
+constexpr int kDumpStride = 65;       // floats per dumped Gram row (odd: conflict-free scalar stores by row)
 constexpr uint32_t kSpinLimit = 1u << 24;
+
+// one record per node, built once per item, read by the warp that owns the node in the solve
+struct NodeRec {
+  float wk[16];     // -beta_t G(t,a_j) (k^_aj . k^_t), 0 beyond the node's depth
+  float wq[16];     //          G(t,a_j) (k^_aj . q^_t), 0 beyond the node's depth
+  float c0k;        // beta_t g_t |k scale|: factor of the S0 k product
+  float beta;
+  float c0q;        // g_t |q scale|: factor of the S0 q product
+  float wself;      // k^_t . q^_t
+  uint32_t out_off; // element offset of this node's output row for value row 0
+  uint32_t pad[3];
+  int32_t aoff[16]; // element offset of ancestor j's deltas in the delta array; beyond the depth: the zero row
+};
+static_assert(sizeof(NodeRec) == 224, "record layout");
 
 // shared memory map (bytes from a 1024-aligned base)
 constexpr int kOffAhi = 0;                          // S0 hi: 2 k-blocks x [128 rows x 128 B], SW128
 constexpr int kOffAlo = 32768;                      // S0 lo
 constexpr int kOffKQ = 65536;                       // rows 0..63 = K, 64..127 = Q, 2 k-blocks, SW128
 constexpr int kOffSmall = 98304;
-// after the MMAs have completed the S0 tiles are dead; their space is reused:
-constexpr int kOffDump = 0;                         // Gram [128][68] fp32
-constexpr int kOffWk = kOffDump + 128 * kDumpStride * 4;   // 34816
-constexpr int kOffWq = kOffWk + kNT * kWStride * 4;        // 39936
-constexpr int kOffV = kOffWq + kNT * kWStride * 4;         // 45056: V [64][128] bf16
+// once the MMAs have completed, the S0 tiles and later the K/Q tile are dead; their space is reused:
+constexpr int kOffDump = 0;                         // Gram [128][65] fp32; later S0 k^ products, then deltas, [65][128] fp32
+constexpr int kOffRec = 34816;                      // NodeRec[64]
+static_assert(128 * kDumpStride * 4 <= kOffRec, "Gram dump overflows its area");
+constexpr int kOffV = kOffRec + kNT * (int)sizeof(NodeRec);   // 49152: V [64][128] bf16
+constexpr int kOffPq = kOffKQ;                      // S0 q^ products [64][128] fp32
+constexpr int kZeroRow = kNT * kD;                  // element offset of the all-zero delta row
+static_assert((kNT + 1) * kD * 4 <= kOffRec, "delta array overflows the dump area");
 static_assert(kOffV + kNT * kD * 2 <= kOffKQ, "aliased region overflows the S0 tiles");
 
 struct Small {
   float alpha[kNT], beta[kNT], ks[kNT], qs[kNT];
   int32_t meta[kNT];                 // physical row | depth << 16
-  uint8_t anc[kNT][16];              // depth-first positions of the ancestors, root first
+  uint8_t anc[kNT][16];              // positions of the ancestors, root first
+  float qq[kNT];                     // |q|^2 of each node when normalising
+  uint8_t lvl[20];                   // lvl[d] = number of nodes of depth <= d
   unsigned long long mbar;
   uint32_t tmem_base;
   uint32_t timed_out;
@@ -63,9 +87,6 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* gmem) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(gmem) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit_wait_all() {
-  asm volatile("cp.async.commit_group;\ncp.async.wait_group 0;\n" ::: "memory");
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
@@ -113,16 +134,24 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a, uint64_t b, ui
 __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float* v) {
-  uint32_t r[16];
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
         "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
       : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+// 32 consecutive columns of this thread's TMEM lane -> shared memory dst[col * stride]
+__device__ __forceinline__ void tmem_cols32_to_smem(uint32_t taddr, float* dst, int stride) {
+  uint32_t r0[16], r1[16];
+  tmem_ld16_issue(taddr, r0);
+  tmem_ld16_issue(taddr + 16, r1);
+  tmem_ld_wait();
 #pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
+  for (int e = 0; e < 16; ++e) dst[e * stride] = __uint_as_float(r0[e]);
+#pragma unroll
+  for (int e = 0; e < 16; ++e) dst[(16 + e) * stride] = __uint_as_float(r1[e]);
 }
 
 __device__ __forceinline__ uint32_t sw128_offset(int row, int chunk16) {   // within one [rows x 128 B] k-block
@@ -133,20 +162,55 @@ __device__ __forceinline__ void store_out(void* out, size_t idx, int dtype, floa
   if (dtype == LUMO_BF16) reinterpret_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(v);
   else reinterpret_cast<float*>(out)[idx] = v;
 }
+__device__ __forceinline__ float load_gate(const void* p, size_t i, int dtype) {
+  return dtype == LUMO_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i])
+                            : reinterpret_cast<const float*>(p)[i];
+}
 
-template <int DMAX>
+#ifdef LUMO_GRAM_PROFILE
+__device__ long long g_prof[32];
+#define PROF(i) do { if (blockIdx.x == 0 && tid == 0 && item == blockIdx.x) g_prof[i] = clock64(); } while (0)
+#else
+#define PROF(i) do {} while (0)
+#endif
+
+// fp32 x -> bf16 hi + lo of four values, written to the two swizzled operand tiles
+__device__ __forceinline__ void split_store(unsigned char* smem, uint32_t off, float4 x) {
+  __nv_bfloat162 h01 = __floats2bfloat162_rn(x.x, x.y), h23 = __floats2bfloat162_rn(x.z, x.w);
+  const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
+  __nv_bfloat162 l01 = __floats2bfloat162_rn(x.x - f01.x, x.y - f01.y);
+  __nv_bfloat162 l23 = __floats2bfloat162_rn(x.z - f23.x, x.w - f23.y);
+  *reinterpret_cast<uint2*>(smem + kOffAhi + off) = make_uint2(*reinterpret_cast<uint32_t*>(&h01), *reinterpret_cast<uint32_t*>(&h23));
+  *reinterpret_cast<uint2*>(smem + kOffAlo + off) = make_uint2(*reinterpret_cast<uint32_t*>(&l01), *reinterpret_cast<uint32_t*>(&l23));
+}
+
+// what a warp needs for one node besides its ancestors' deltas
+struct NodeOps {
+  float4 m;        // c0k, beta, c0q, wself
+  uint32_t out_off;
+  uint2 vb;        // four bf16 values of v
+  float4 pk, pq;   // S0 k^, S0 q^ for the lane's four rows
+  float4 ck, cq;   // first four coefficients
+  int4 ao;         // first four ancestor offsets
+};
+
 __global__ void __launch_bounds__(kThreads, 2)
 scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
   extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // 1024-byte alignment for the swizzled operand tiles; plain pointer arithmetic on the shared
+  // array keeps the pointers in the shared address space
+  unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
   Small& sm = *reinterpret_cast<Small*>(smem + kOffSmall);
   float* dump = reinterpret_cast<float*>(smem + kOffDump);
-  float* Wk = reinterpret_cast<float*>(smem + kOffWk);
-  float* Wq = reinterpret_cast<float*>(smem + kOffWq);
+  float* dls = reinterpret_cast<float*>(smem + kOffDump);     // [65][128]; row 64 stays zero
+  float* Pq = reinterpret_cast<float*>(smem + kOffPq);
+  NodeRec* recs = reinterpret_cast<NodeRec*>(smem + kOffRec);
   const __nv_bfloat16* Vs = reinterpret_cast<const __nv_bfloat16*>(smem + kOffV);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int grp = tid >> 7;            // half of the CTA: 0 or 1
+  const int vrow = tid & 127;          // value row = TMEM lane
   const int rep = s.Hv / s.Hk;
   const int N = s.N;
 
@@ -159,7 +223,7 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
-  const uint32_t tmem_lane = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
+  const uint32_t tmem_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 lanes
   uint32_t phase = 0;
 
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {   // bounded: n_items
@@ -172,144 +236,112 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     const size_t out_row_stride = (size_t)s.Hv * kD;
 
     if (row < 0 || row >= s.n_state_rows) {   // skipped sequence: zero outputs
-      for (int ps = 0; ps < s.Ns; ++ps) store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + tid, s.out_dtype, 0.f);
+      for (int ps = grp; ps < s.Ns; ps += 2)
+        store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + vrow, s.out_dtype, 0.f);
       if (L.status && hv == 0 && tid == 0) L.status[b] = row < 0 ? LUMO_SEQ_OK : LUMO_SEQ_BAD_ROW;
       continue;
     }
     if (L.status && hv == 0 && tid == 0) L.status[b] = LUMO_SEQ_OK;
 
-    // ---- a. per-node tables and gates -----------------------------------------------------
+    PROF(0);
+    // ---- a. per-node tables (the addresses of everything else depend on them) -------------------
     if (tid < kNT) {
-      const int pi = tid;
-      int meta = 0;
-      float a = 1.f, bt = 0.f;
-      if (pi < N) {
-        meta = t.tc_meta[b * N + pi];
-        const size_t pr = (size_t)b * s.Ns + (meta & 0xFFFF);
-        a = s.gate_dtype == LUMO_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(L.alpha)[pr * s.Hv + hv])
-                                      : reinterpret_cast<const float*>(L.alpha)[pr * s.Hv + hv];
-        bt = s.gate_dtype == LUMO_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(L.beta)[pr * s.Hv + hv])
-                                       : reinterpret_cast<const float*>(L.beta)[pr * s.Hv + hv];
-      }
-      sm.meta[pi] = meta; sm.alpha[pi] = a; sm.beta[pi] = bt;
-    } else {
+      sm.meta[tid] = tid < N ? t.tc_meta[b * N + tid] : 0;
+    } else if (tid < 2 * kNT) {
       const int pi = tid - kNT;
       uint4 av = make_uint4(0, 0, 0, 0);
       if (pi < N) av = *reinterpret_cast<const uint4*>(t.tc_anc + ((size_t)b * N + pi) * 16);
       *reinterpret_cast<uint4*>(sm.anc[pi]) = av;
+    } else if (tid < 2 * kNT + 20) {
+      sm.lvl[tid - 2 * kNT] = t.tc_lvl[b * 20 + tid - 2 * kNT];
     }
-    // padding rows: zero outputs
-    if (s.Ns > N)
-      for (int ps = 0; ps < s.Ns; ++ps)
-        if (t.slot_inv[b * s.Ns + ps] < 0)
-        store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + tid, s.out_dtype, 0.f);
     __syncthreads();
-
-    // ---- b. K and Q rows -> swizzled operand tile (cp.async) -------------------------------
+    PROF(1);
+    // ---- b. gates (consumed much later); K and Q rows -> swizzled operand tile (cp.async);
+    //         first half of the pre-tree state rows -> registers -------------------------------------
+    float gate_a = 1.f, gate_b = 0.f;
+    if (tid < N) {
+      const size_t pr = (size_t)b * s.Ns + (sm.meta[tid] & 0xFFFF);
+      gate_a = load_gate(L.alpha, pr * s.Hv + hv, s.gate_dtype);
+      gate_b = load_gate(L.beta, pr * s.Hv + hv, s.gate_dtype);
+    }
     {
       const __nv_bfloat16* kg = reinterpret_cast<const __nv_bfloat16*>(L.k);
       const __nv_bfloat16* qg = reinterpret_cast<const __nv_bfloat16*>(L.q);
-#pragma unroll 4
-      for (int i = 0; i < 16; ++i) {
+      const __nv_bfloat16* src[2048 / kThreads];
+#pragma unroll
+      for (int i = 0; i < 2048 / kThreads; ++i) {        // addresses first, so that the copies issue back to back
         const int idx = i * kThreads + tid;
         const int R = idx >> 4, c = idx & 15;
         const int pi = R & (kNT - 1);
-        const uint32_t dst = sbase + kOffKQ + (c >> 3) * 16384 + sw128_offset(R, c & 7);
-        if (pi < N) {
-          const size_t pr = (size_t)b * s.Ns + (sm.meta[pi] & 0xFFFF);
-          const __nv_bfloat16* src = (R < kNT ? kg : qg) + (pr * s.Hk + g) * kD + c * 8;
-          cp_async16(dst, src);
-        } else {
-          asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(dst), "r"(0u) : "memory");
-        }
-      }
-    }
-    // ---- c. S0 -> bf16 hi + lo operand tiles ------------------------------------------------
-    {
-      const float* S0 = L.state + ((size_t)row * s.Hv + hv) * kD * kD;
-      const int kblock = lane >> 4, chunk = (lane & 15) >> 1, half = lane & 1;
-#pragma unroll 1
-      for (int i0 = 0; i0 < 32; i0 += 8) {
-        float4 x[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp * 32 + i0 + u) * kD + lane * 4);
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int r = warp * 32 + i0 + u;
-          __nv_bfloat162 h01 = __floats2bfloat162_rn(x[u].x, x[u].y), h23 = __floats2bfloat162_rn(x[u].z, x[u].w);
-          float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
-          __nv_bfloat162 l01 = __floats2bfloat162_rn(x[u].x - f01.x, x[u].y - f01.y);
-          __nv_bfloat162 l23 = __floats2bfloat162_rn(x[u].z - f23.x, x[u].w - f23.y);
-          const uint32_t off = kblock * 16384 + sw128_offset(r, chunk) + half * 8;
-          *reinterpret_cast<uint2*>(smem + kOffAhi + off) =
-              make_uint2(*reinterpret_cast<uint32_t*>(&h01), *reinterpret_cast<uint32_t*>(&h23));
-          *reinterpret_cast<uint2*>(smem + kOffAlo + off) =
-              make_uint2(*reinterpret_cast<uint32_t*>(&l01), *reinterpret_cast<uint32_t*>(&l23));
-        }
-      }
-    }
-    cp_async_commit_wait_all();
-    fence_async_proxy();          // generic-proxy writes -> visible to the tensor core's async proxy
-    __syncthreads();
-
-    // ---- e. MMAs: P = S0 [K|Q]^T (hi + lo), Gram = [K;Q] K^T --------------------------------
-    if (tid == 0) {
-      tc_fence_after();
-      constexpr uint32_t idesc_p = umma_idesc(128, 128), idesc_g = umma_idesc(128, 64);
-#pragma unroll
-      for (int term = 0; term < 2; ++term) {
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t koff = (ks >> 2) * 16384 + (ks & 3) * 32;
-          umma(tmem, umma_desc(sbase + (term ? kOffAlo : kOffAhi) + koff), umma_desc(sbase + kOffKQ + koff), idesc_p,
-               (term | ks) ? 1u : 0u);
-        }
+        const size_t pr = (size_t)b * s.Ns + (sm.meta[pi] & 0xFFFF);
+        src[i] = pi < N ? (R < kNT ? kg : qg) + (pr * s.Hk + g) * kD + c * 8 : nullptr;
       }
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const uint32_t koff = (ks >> 2) * 16384 + (ks & 3) * 32;
-        umma(tmem + 128, umma_desc(sbase + kOffKQ + koff), umma_desc(sbase + kOffKQ + koff), idesc_g, ks ? 1u : 0u);
-      }
-      umma_commit(&sm.mbar);
-    }
-    // ---- f. wait for the tensor core (bounded) ----------------------------------------------
-    if (!mbar_wait(&sm.mbar, phase)) sm.timed_out = 1;
-    phase ^= 1;
-    tc_fence_after();
-    __syncthreads();
-    if (sm.timed_out) {    // give up on this and all further items; report, free TMEM, leave
-      if (L.status && tid == 0) L.status[b] = LUMO_SEQ_TIMEOUT;
-      break;
-    }
-
-    // ---- g. V rows -> shared (space of the dead S0 tiles) ----------------------------------
-    {
-      const __nv_bfloat16* vg = reinterpret_cast<const __nv_bfloat16*>(L.v);
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < 2048 / kThreads; ++i) {
         const int idx = i * kThreads + tid;
-        const int pi = idx >> 4, c = idx & 15;
-        if (pi < N) {
-          const size_t pr = (size_t)b * s.Ns + (sm.meta[pi] & 0xFFFF);
-          cp_async16(sbase + kOffV + pi * 256 + c * 16, vg + (pr * s.Hv + hv) * kD + c * 8);
-        }
+        const int R = idx >> 4, c = idx & 15;
+        const uint32_t dst = sbase + kOffKQ + (c >> 3) * 16384 + sw128_offset(R, c & 7);
+        if (src[i]) cp_async16(dst, src[i]);
+        else asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(dst), "r"(0u) : "memory");
       }
       asm volatile("cp.async.commit_group;\n" ::: "memory");
     }
-    // ---- h. Gram rows out of tensor memory; |q|^2 when normalising ----------------------------
+    // warp w takes rows w, w+8, ...; a warp reads one 512-byte row per instruction
+    const float* S0 = L.state + ((size_t)row * s.Hv + hv) * kD * kD;
+    float4 x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * u) * kD + lane * 4);
+    PROF(2);
+    // ---- c. pre-tree state -> bf16 hi + lo operand tiles ------------------------------------------
     {
-      float gr[16];
+      const int kblock = lane >> 4, chunk = (lane & 15) >> 1, half = lane & 1;
 #pragma unroll
-      for (int cb = 0; cb < 4; ++cb) {
-        tmem_ld16(tmem_lane + 128 + cb * 16, gr);
-#pragma unroll
-        for (int e = 0; e < 16; e += 4)
-          *reinterpret_cast<float4*>(dump + tid * kDumpStride + cb * 16 + e) = make_float4(gr[e], gr[e + 1], gr[e + 2], gr[e + 3]);
+      for (int u = 0; u < 8; ++u) {
+        split_store(smem, kblock * 16384 + sw128_offset(warp + 8 * u, chunk) + half * 8, x[u]);
+        x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * (8 + u)) * kD + lane * 4);   // second half
       }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        split_store(smem, kblock * 16384 + sw128_offset(warp + 8 * (8 + u), chunk) + half * 8, x[u]);
     }
-    float qq = 0.f;
-    if (s.l2norm && tid >= kNT) {
-      const int R = tid;   // tile row of q_(tid-64)
+    if (tid < kNT) { sm.alpha[tid] = gate_a; sm.beta[tid] = gate_b; }
+    // padding rows: zero outputs
+    if (s.Ns > N)
+      for (int ps = grp; ps < s.Ns; ps += 2)
+        if (t.slot_inv[b * s.Ns + ps] < 0)
+          store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + vrow, s.out_dtype, 0.f);
+    PROF(3);
+    PROF(4);
+    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+    fence_async_proxy();          // generic-proxy writes -> visible to the tensor core's async proxy
+    __syncthreads();
+
+    PROF(5);
+    // ---- e. MMAs: Gram = [K;Q] K^T, P = S0 [K|Q]^T (hi + lo); meanwhile |q|^2 when normalising ----
+    if (tid == 0) {
+      tc_fence_after();
+      constexpr uint32_t idesc_p = umma_idesc(128, 128), idesc_g = umma_idesc(128, 64);
+      const uint64_t d_kq = umma_desc(sbase + kOffKQ), d_hi = umma_desc(sbase + kOffAhi), d_lo = umma_desc(sbase + kOffAlo);
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+        umma(tmem + 128, d_kq + koff, d_kq + koff, idesc_g, ks ? 1u : 0u);
+      }
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+        umma(tmem, d_hi + koff, d_kq + koff, idesc_p, ks ? 1u : 0u);
+      }
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+        umma(tmem, d_lo + koff, d_kq + koff, idesc_p, 1u);
+      }
+      umma_commit(&sm.mbar);
+    } else if (grp == 1 && s.l2norm && vrow < kNT) {
+      const int R = kNT + vrow;   // tile row of q_vrow (the tensor core only reads the tile)
+      float qq = 0.f;
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
         const uint4 w = *reinterpret_cast<const uint4*>(smem + kOffKQ + (c >> 3) * 16384 + sw128_offset(R, c & 7));
@@ -320,91 +352,160 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
           qq = fmaf(lo, lo, qq); qq = fmaf(hi, hi, qq);
         }
       }
+      sm.qq[vrow] = qq;
     }
+    PROF(6);
+    // ---- f. wait for the tensor core (bounded) ---------------------------------------------------
+    if (!mbar_wait(&sm.mbar, phase)) sm.timed_out = 1;
+    phase ^= 1;
+    tc_fence_after();
     __syncthreads();
-    // ---- i. normalisation factors ----------------------------------------------------------
-    if (tid < kNT) sm.ks[tid] = s.l2norm ? rsqrtf(dump[tid * kDumpStride + tid] + s.l2_eps) : 1.f;
-    else sm.qs[tid - kNT] = s.l2norm ? s.scale * rsqrtf(qq + s.l2_eps) : s.scale;
-    __syncthreads();
-    // ---- j. coefficient rows: one thread per (node, table) ------------------------------------
+    if (sm.timed_out) {    // give up on this and all further items; report, free TMEM, leave
+      if (L.status && tid == 0) L.status[b] = LUMO_SEQ_TIMEOUT;
+      break;
+    }
+
+    PROF(7);
+    // ---- g. V rows -> shared (space of the dead S0 tiles); Gram rows out of tensor memory ----------
     {
+      const __nv_bfloat16* vg = reinterpret_cast<const __nv_bfloat16*>(L.v);
+#pragma unroll
+      for (int i = 0; i < 1024 / kThreads; ++i) {
+        const int idx = i * kThreads + tid;
+        const int pi = idx >> 4, c = idx & 15;
+        if (pi < N) {
+          const size_t pr = (size_t)b * s.Ns + (sm.meta[pi] & 0xFFFF);
+          cp_async16(sbase + kOffV + pi * 256 + c * 16, vg + (pr * s.Hv + hv) * kD + c * 8);
+        }
+      }
+      asm volatile("cp.async.commit_group;\n" ::: "memory");
+    }
+    // both halves of the CTA read the Gram rows: 32 of the 64 columns each
+    tmem_cols32_to_smem(tmem_lane + 128 + grp * 32, dump + vrow * kDumpStride + grp * 32, 1);
+    __syncthreads();
+    PROF(8);
+    // ---- h. normalisation factors ------------------------------------------------------------------
+    if (tid < kNT) sm.ks[tid] = s.l2norm ? rsqrtf(dump[tid * kDumpStride + tid] + s.l2_eps) : 1.f;
+    else if (tid < 2 * kNT) sm.qs[tid - kNT] = s.l2norm ? s.scale * rsqrtf(sm.qq[tid - kNT] + s.l2_eps) : s.scale;
+    __syncthreads();
+    PROF(9);
+    // ---- i. first half of the CTA: node records, one thread per (node, table); second half: the
+    //         S0 q^ products move from tensor memory to shared memory [node][row] ---------------------
+    if (grp == 0) {
       const bool is_q = tid >= kNT;
       const int pi = tid & (kNT - 1);
-      float w[kWStride];
+      NodeRec& rec = recs[pi];
+      float* w = is_q ? rec.wq : rec.wk;
+      const int meta = sm.meta[pi];
+      const int D = pi < N ? (meta >> 16) : 0;                   // depth, 1..16
+      const float a_t = sm.alpha[pi], b_t = sm.beta[pi];
+      const float self = is_q ? sm.qs[pi] : -b_t * sm.ks[pi];    // factor of the node itself (k side negated)
+      const float* grow = dump + (is_q ? kNT + pi : pi) * kDumpStride;
+      float G = a_t;
 #pragma unroll
-      for (int e = 0; e < kWStride; ++e) w[e] = 0.f;
-      if (pi < N) {
-        const int D = sm.meta[pi] >> 16;                         // depth, 1..16
-        const float a_t = sm.alpha[pi], b_t = sm.beta[pi];
-        const float self = is_q ? sm.qs[pi] : b_t * sm.ks[pi];   // factor of the node itself
-        const float* grow = dump + (is_q ? kNT + pi : pi) * kDumpStride;
-        float G = a_t;
-#pragma unroll
-        for (int j = 15; j >= 0; --j) {                          // bounded: 16 depth slots
-          if (j <= D - 2) {
-            const int sidx = sm.anc[pi][j];
-            w[j] = self * G * sm.ks[sidx] * grow[sidx];
-            G *= sm.alpha[sidx];
-          }
+      for (int j = 15; j >= 0; --j) {                            // bounded: 16 depth slots
+        float val = 0.f;
+        int off = kZeroRow;
+        if (j <= D - 2) {
+          const int sidx = sm.anc[pi][j];
+          val = self * G * sm.ks[sidx] * grow[sidx];
+          G *= sm.alpha[sidx];
+          off = sidx * kD;
         }
-        if (is_q) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j)
-            if (j == D - 1) w[j] = self * sm.ks[pi] * grow[pi];   // k^_t . q^_t, G = 1
-        }
-        w[16] = self * G;                                         // factor of the S0 product
-        w[17] = b_t;
-        w[18] = __int_as_float(D);
+        w[j] = val;
+        if (!is_q) rec.aoff[j] = off;
       }
-      float* dst = (is_q ? Wq : Wk) + pi * kWStride;
-#pragma unroll
-      for (int e = 0; e < kWStride; e += 4) *reinterpret_cast<float4*>(dst + e) = make_float4(w[e], w[e + 1], w[e + 2], w[e + 3]);
+      if (is_q) {
+        rec.c0q = self * G;
+        rec.wself = self * sm.ks[pi] * grow[pi];                 // k^_t . q^_t (G = 1)
+        rec.out_off = (uint32_t)((((size_t)b * s.Ns + (meta & 0xFFFF)) * s.Hv + hv) * kD);
+      } else {
+        rec.c0k = self * G;                                      // -beta_t g_t |k scale|
+        rec.beta = b_t;
+      }
+    } else {
+      for (int cb = 0; cb < (N + 31) / 32; ++cb)                 // bounded: <= 2
+        tmem_cols32_to_smem(tmem_lane + kNT + cb * 32, Pq + (cb * 32) * kD + vrow, kD);
     }
     asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+    __syncthreads();      // records, V and Pq are in place; the Gram dump is dead from here on
+    // the S0 k^ products take the place of the dump; each delta later overwrites its own product
+    if (grp * 32 < N) tmem_cols32_to_smem(tmem_lane + grp * 32, dls + (grp * 32) * kD + vrow, kD);
+    if (tid < kD) dls[kZeroRow + tid] = 0.f;
     __syncthreads();
 
-    // ---- k. forward substitution along the depth-first walk: thread = value row --------------
+    PROF(10);
+    // ---- j. forward substitution, level by level; one warp per node, lane l carries value rows
+    //         4l .. 4l+3.  A node's record, v and S0 products are loaded before the barrier that
+    //         publishes the previous level; only the ancestors' deltas are fetched after it ----------
     {
-      float dl[DMAX];
-#pragma unroll
-      for (int j = 0; j < DMAX; ++j) dl[j] = 0.f;
-      const int nblk = (N + 15) >> 4;
-      for (int blk = 0; blk < nblk; ++blk) {                      // bounded: <= 4
-        float pk[16], pq[16];
-        tmem_ld16(tmem_lane + blk * 16, pk);
-        tmem_ld16(tmem_lane + kNT + blk * 16, pq);
-#pragma unroll
-        for (int u = 0; u < 16; ++u) {
-          const int pi = blk * 16 + u;
-          if (pi < N) {
-            const float* wk = Wk + pi * kWStride;
-            const float* wq = Wq + pi * kWStride;
-            const float4 tail = *reinterpret_cast<const float4*>(wk + 16);     // c0, beta, depth
-            const int D = __float_as_int(tail.z);
-            const float v = __bfloat162float(Vs[pi * kD + tid]);
-            float acc0 = fmaf(tail.y, v, -tail.x * pk[u]), acc1 = 0.f;
-#pragma unroll
-            for (int j4 = 0; j4 < DMAX; j4 += 4) {
-              const float4 c = *reinterpret_cast<const float4*>(wk + j4);
-              acc0 = fmaf(-c.x, dl[j4], acc0); acc1 = fmaf(-c.y, dl[j4 + 1], acc1);
-              acc0 = fmaf(-c.z, dl[j4 + 2], acc0); acc1 = fmaf(-c.w, dl[j4 + 3], acc1);
-            }
-            const float delta = acc0 + acc1;
-#pragma unroll
-            for (int j = 0; j < DMAX; ++j) dl[j] = (j == D - 1) ? delta : dl[j];
-            float o0 = wq[16] * pq[u], o1 = 0.f;
-#pragma unroll
-            for (int j4 = 0; j4 < DMAX; j4 += 4) {
-              const float4 c = *reinterpret_cast<const float4*>(wq + j4);
-              o0 = fmaf(c.x, dl[j4], o0); o1 = fmaf(c.y, dl[j4 + 1], o1);
-              o0 = fmaf(c.z, dl[j4 + 2], o0); o1 = fmaf(c.w, dl[j4 + 3], o1);
-            }
-            const size_t pr = (size_t)b * s.Ns + (sm.meta[pi] & 0xFFFF);
-            store_out(L.out, pr * out_row_stride + hv * kD + tid, s.out_dtype, o0 + o1);
+      auto load_ops = [&](NodeOps& op, int pi) {
+        const NodeRec& rec = recs[pi];
+        op.m = *reinterpret_cast<const float4*>(&rec.c0k);
+        op.out_off = rec.out_off;
+        op.vb = *reinterpret_cast<const uint2*>(Vs + pi * kD + 4 * lane);
+        op.pk = *reinterpret_cast<const float4*>(dls + pi * kD + 4 * lane);
+        op.pq = *reinterpret_cast<const float4*>(Pq + pi * kD + 4 * lane);
+        op.ck = *reinterpret_cast<const float4*>(rec.wk);
+        op.cq = *reinterpret_cast<const float4*>(rec.wq);
+        op.ao = *reinterpret_cast<const int4*>(rec.aoff);
+      };
+      auto block4 = [&](float4& acc, float4& o, const float4& ck, const float4& cq, const int4& ao) {
+        const float4 d0 = *reinterpret_cast<const float4*>(dls + ao.x + 4 * lane);
+        const float4 d1 = *reinterpret_cast<const float4*>(dls + ao.y + 4 * lane);
+        const float4 d2 = *reinterpret_cast<const float4*>(dls + ao.z + 4 * lane);
+        const float4 d3 = *reinterpret_cast<const float4*>(dls + ao.w + 4 * lane);
+        acc.x = fmaf(ck.x, d0.x, acc.x); acc.y = fmaf(ck.x, d0.y, acc.y); acc.z = fmaf(ck.x, d0.z, acc.z); acc.w = fmaf(ck.x, d0.w, acc.w);
+        o.x = fmaf(cq.x, d0.x, o.x); o.y = fmaf(cq.x, d0.y, o.y); o.z = fmaf(cq.x, d0.z, o.z); o.w = fmaf(cq.x, d0.w, o.w);
+        acc.x = fmaf(ck.y, d1.x, acc.x); acc.y = fmaf(ck.y, d1.y, acc.y); acc.z = fmaf(ck.y, d1.z, acc.z); acc.w = fmaf(ck.y, d1.w, acc.w);
+        o.x = fmaf(cq.y, d1.x, o.x); o.y = fmaf(cq.y, d1.y, o.y); o.z = fmaf(cq.y, d1.z, o.z); o.w = fmaf(cq.y, d1.w, o.w);
+        acc.x = fmaf(ck.z, d2.x, acc.x); acc.y = fmaf(ck.z, d2.y, acc.y); acc.z = fmaf(ck.z, d2.z, acc.z); acc.w = fmaf(ck.z, d2.w, acc.w);
+        o.x = fmaf(cq.z, d2.x, o.x); o.y = fmaf(cq.z, d2.y, o.y); o.z = fmaf(cq.z, d2.z, o.z); o.w = fmaf(cq.z, d2.w, o.w);
+        acc.x = fmaf(ck.w, d3.x, acc.x); acc.y = fmaf(ck.w, d3.y, acc.y); acc.z = fmaf(ck.w, d3.z, acc.z); acc.w = fmaf(ck.w, d3.w, acc.w);
+        o.x = fmaf(cq.w, d3.x, o.x); o.y = fmaf(cq.w, d3.y, o.y); o.z = fmaf(cq.w, d3.z, o.z); o.w = fmaf(cq.w, d3.w, o.w);
+      };
+      const int lvl_lane = sm.lvl[lane < 20 ? lane : 19];          // lane d holds lvl[d]
+      NodeOps op;
+      int lo = 0;
+      if (warp < __shfl_sync(0xffffffffu, lvl_lane, 1)) load_ops(op, warp);
+      for (int d = 1; d <= 16; ++d) {                              // bounded: 16 levels
+        const int hi = __shfl_sync(0xffffffffu, lvl_lane, d);      // nodes of depth d: [lo, hi)
+        const int nblk = (d + 2) >> 2;                             // blocks of four ancestors
+        for (int pi = lo + warp; pi < hi; pi += kWarps) {          // bounded: <= 64
+          if (pi != lo + warp) load_ops(op, pi);
+          const float c0k = op.m.x, beta = op.m.y, c0q = op.m.z, wself = op.m.w;
+          float4 acc, o;
+          acc.x = fmaf(beta, __uint_as_float(op.vb.x << 16), c0k * op.pk.x);
+          acc.y = fmaf(beta, __uint_as_float(op.vb.x & 0xFFFF0000u), c0k * op.pk.y);
+          acc.z = fmaf(beta, __uint_as_float(op.vb.y << 16), c0k * op.pk.z);
+          acc.w = fmaf(beta, __uint_as_float(op.vb.y & 0xFFFF0000u), c0k * op.pk.w);
+          o.x = c0q * op.pq.x; o.y = c0q * op.pq.y; o.z = c0q * op.pq.z; o.w = c0q * op.pq.w;
+          if (d > 1) block4(acc, o, op.ck, op.cq, op.ao);          // uniform over the CTA
+          for (int blk = 1; blk < nblk; ++blk) {                   // bounded: <= 3 more blocks
+            const NodeRec& rec = recs[pi];
+            block4(acc, o, *reinterpret_cast<const float4*>(rec.wk + 4 * blk), *reinterpret_cast<const float4*>(rec.wq + 4 * blk),
+                   *reinterpret_cast<const int4*>(rec.aoff + 4 * blk));
+          }
+          *reinterpret_cast<float4*>(dls + pi * kD + 4 * lane) = acc;           // delta of this node
+          o.x = fmaf(wself, acc.x, o.x); o.y = fmaf(wself, acc.y, o.y);
+          o.z = fmaf(wself, acc.z, o.z); o.w = fmaf(wself, acc.w, o.w);
+          const size_t oi = (size_t)op.out_off + 4 * lane;
+          if (s.out_dtype == LUMO_BF16) {
+            __nv_bfloat162 o01 = __floats2bfloat162_rn(o.x, o.y), o23 = __floats2bfloat162_rn(o.z, o.w);
+            *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(L.out) + oi) =
+                make_uint2(*reinterpret_cast<uint32_t*>(&o01), *reinterpret_cast<uint32_t*>(&o23));
+          } else {
+            *reinterpret_cast<float4*>(reinterpret_cast<float*>(L.out) + oi) = o;
           }
         }
+        lo = hi;
+        PROF(12 + d);
+        if (lo >= N) break;                                        // uniform
+        if (lo + warp < __shfl_sync(0xffffffffu, lvl_lane, d + 1)) load_ops(op, lo + warp);   // next level's first node
+        __syncthreads();                                           // deltas of this level visible to the next
       }
     }
+    PROF(11);
     tc_fence_before();
     __syncthreads();      // tensor memory and the aliased shared memory are free for the next item
   }
@@ -419,19 +520,25 @@ bool gram_supported(const Shape& s, int max_depth) {
   return s.d == kD && s.in_dtype == LUMO_BF16 && s.snapshot_mode == 0 && s.N <= kNT && max_depth <= 16;
 }
 
-cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int max_depth, int sm_count,
-                             cudaStream_t st) {
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, cudaStream_t st) {
   const int items = s.n_layers * s.B * s.Hv;
-  const int grid = items < 2 * sm_count ? items : 2 * sm_count;
-  auto launch = [&](auto kern) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(scan_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, kSmemBytes, st>>>(s, t, lb, items);
-    return cudaGetLastError();
-  };
-  if (max_depth <= 4) return launch(scan_gram_kernel<4>);
-  if (max_depth <= 8) return launch(scan_gram_kernel<8>);
-  return launch(scan_gram_kernel<16>);
+    configured = true;
+  }
+  // two CTAs per SM by construction: 102 KB of shared memory, 128 registers x 256 threads and 256
+  // of the 512 tensor-memory columns each
+  const int grid = items < 2 * sm_count ? items : 2 * sm_count;
+  scan_gram_kernel<<<grid, kThreads, kSmemBytes, st>>>(s, t, lb, items);
+  return cudaGetLastError();
 }
+
+#ifdef LUMO_GRAM_PROFILE
+extern "C" int lumo_debug_gram_profile(long long* out32) {
+  return (int)cudaMemcpyFromSymbol(out32, g_prof, sizeof(long long) * 32);
+}
+#endif
 
 }  // namespace lumo
