@@ -100,9 +100,8 @@ def algorithmic_bytes(c, out_bytes=2):
     Lsum = int(c.accepted_len.sum())
     scan = state + operands + gates + out
     conv = 2 * B * N * C * s_in + 4 * C * s_in + 3 * B * C * s_in
-    commit_state = 2 * state + Lsum * ((Hk * d + Hv * d) * s_in + 2 * Hv * s_in)
-    commit_hist = 2 * 3 * B * C * s_in
-    return dict(scan=scan, conv=conv, commit_state=commit_state, commit_hist=commit_hist)
+    commit = 2 * state + Lsum * ((Hk * d + Hv * d) * s_in + 2 * Hv * s_in) + 2 * 3 * B * C * s_in
+    return dict(scan=scan, conv=conv, commit=commit)
 
 
 def rank1_fma(c):
@@ -406,7 +405,7 @@ def main():
                 "fp32_fma_per_launch_rank1": fma,
                 "alu_frac_at_sampled_clock": (fma / (kern["scan"]["avg_us"] * 1e-6)) / (148 * 128 * sm_mhz * 1e6)
                 if "scan" in kern else None}
-    commit_us = sum(kern[k]["avg_us"] for k in ("commit_state", "commit_hist") if k in kern) / n_layers
+    commit_us = kern["commit"]["avg_us"] / n_layers if "commit" in kern else None
     verify_us = sum(kern[k]["avg_us"] for k in ("conv", "scan") if k in kern)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -422,7 +421,7 @@ def main():
             "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "window")},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                     "ms_per_step": ms_e2e / n_e2e, "steps": n_e2e},
-            "gpu_launches": int(args.steps * sum(1 for k in ("conv", "scan", "commit_state", "commit_hist") if k in kern)),
+            "gpu_launches": int(args.steps * sum(1 for k in ("conv", "scan", "commit") if k in kern)),
             "roofline": roofline,
             "kernels": kern,
             "verify_nodes_per_s_per_layer": nodes_per_step / (verify_us * 1e-6),

@@ -87,7 +87,11 @@ typedef enum {
                                 state), 2 DESCEND node (same, from the kept delta), 3 PUSH level,
                                 4 POP level (0xFFFF = reload the pre-tree state) */
   LUMO_TAB_SCHEDULE_FULL = 16, /* same, materialising every node's state (snapshot modes) */
-  LUMO_TAB_COUNT = 17
+  LUMO_TAB_GRAM_GROUPS = 17,   /* node groups of the tensor-core scan (empty if depth > 16): [G, then per
+                                  group: n, n node ids ordered by (depth, index), n emit flags].  A group
+                                  holds at most 64 nodes and every ancestor of each member; each node is
+                                  emitted by exactly one group */
+  LUMO_TAB_COUNT = 18
 } lumo_table;
 
 /* ---- context ------------------------------------------------------------------------- */
@@ -112,8 +116,8 @@ int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo);
  * lumo_ctx_timing_read waits for the recorded events, returns the launch count and summed
  * device time of kernels of `kind` (lumo_kernel_kind) and, with reset != 0, forgets all
  * records.  Enabling allocates the event pool; do not enable inside a stream capture. */
-typedef enum { LUMO_K_CONV = 0, LUMO_K_SCAN = 1, LUMO_K_COMMIT_STATE = 2, LUMO_K_COMMIT_HIST = 3,
-               LUMO_K_PATH = 4, LUMO_K_COUNT = 5 } lumo_kernel_kind;
+typedef enum { LUMO_K_CONV = 0, LUMO_K_SCAN = 1, LUMO_K_COMMIT = 2, LUMO_K_PATH = 3,
+               LUMO_K_COUNT = 4 } lumo_kernel_kind;
 int lumo_ctx_timing_enable(lumo_ctx* ctx, int enable);
 int lumo_ctx_timing_read(lumo_ctx* ctx, int kind, int reset, int64_t* launches, double* total_ms);
 

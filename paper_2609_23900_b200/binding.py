@@ -29,9 +29,9 @@ SEQ_OK, SEQ_BAD_LEN, SEQ_BAD_NODE, SEQ_BAD_ROOT, SEQ_BAD_LINK, SEQ_BAD_ROW, SEQ_
 
 TABLES = ["depth", "n_child", "child_off", "child_list", "is_leaf", "leaves", "path_off", "path_nodes",
           "anc_win", "slot_inv", "chain_head", "chain_off", "chain_nodes", "chain_level", "cut_nodes",
-          "schedule", "schedule_full"]
+          "schedule", "schedule_full", "gram_groups"]
 
-KERNEL_KINDS = ["conv", "scan", "commit_state", "commit_hist", "path"]
+KERNEL_KINDS = ["conv", "scan", "commit", "path"]
 
 EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_scratch_bytes",
            "lumo_ctx_timing_enable", "lumo_ctx_timing_read", "lumo_ctx_set_scan_algo",

@@ -113,7 +113,8 @@ TreeDev tree_view(const lumo_tree_desc* d, int which) {
   t.parent = d->d_parent; t.depth = d->d_depth; t.slot = d->d_slot; t.slot_inv = d->d_slot_inv;
   t.win = d->d_win; t.sched = d->d_sched[which]; t.nops = d->d_nops[which];
   t.max_ops = d->max_ops[which]; t.max_levels = d->max_levels[which];
-  t.tc_meta = d->d_tc_meta; t.tc_anc = d->d_tc_anc; t.tc_lvl = d->d_tc_lvl;
+  t.tc_group = d->d_tc_group; t.tc_meta = d->d_tc_meta; t.tc_anc = d->d_tc_anc; t.tc_lvl = d->d_tc_lvl;
+  t.n_groups = d->n_groups;
   return t;
 }
 
@@ -242,14 +243,29 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   std::vector<int32_t> h;
   auto reserve = [&](size_t n) { size_t off = h.size(); h.resize(off + ((n + 3) / 4) * 4, 0); return off; };
   const size_t o_parent = reserve((size_t)B * N), o_depth = reserve((size_t)B * N), o_slot = reserve((size_t)B * N);
-  const size_t o_inv = reserve((size_t)B * Ns), o_win = reserve((size_t)B * N * 4);
+  const size_t o_inv = reserve((size_t)B * Ns), o_win = reserve((size_t)B * Ns * 4);
   size_t o_sched[2], o_nops[2];
   for (int w = 0; w < 2; ++w) { o_sched[w] = reserve((size_t)B * d->max_ops[w]); o_nops[w] = reserve(B); }
   for (int b = 0; b < B; ++b)
     for (int i = 0; i < N; ++i) d->max_depth = std::max(d->max_depth, (int)d->trees[b].tab[LUMO_TAB_DEPTH][i]);
-  const bool tc = N <= 64 && d->max_depth <= 16;
-  const size_t o_tc_meta = tc ? reserve((size_t)B * N) : 0, o_tc_anc = tc ? reserve((size_t)B * N * 4) : 0;
-  const size_t o_tc_lvl = tc ? reserve((size_t)B * 5) : 0;
+  const bool tc = d->max_depth <= 16;
+  std::vector<std::vector<GramGroup>> groups(B);
+  if (tc)
+    for (int b = 0; b < B; ++b) {
+      build_gram_groups(parent + (size_t)b * N, N, d->trees[b], &groups[b]);
+      d->n_groups += (int)groups[b].size();
+      auto& tab = d->trees[b].tab[LUMO_TAB_GRAM_GROUPS];
+      tab.push_back((int32_t)groups[b].size());
+      for (const GramGroup& gr : groups[b]) {
+        tab.push_back((int32_t)gr.nodes.size());
+        tab.insert(tab.end(), gr.nodes.begin(), gr.nodes.end());
+        tab.insert(tab.end(), gr.emit.begin(), gr.emit.end());
+      }
+    }
+  const size_t G = (size_t)d->n_groups;
+  const size_t o_tc_group = tc ? reserve(G * 4) : 0, o_tc_meta = tc ? reserve(G * 64) : 0;
+  const size_t o_tc_anc = tc ? reserve(G * 64 * 4) : 0, o_tc_lvl = tc ? reserve(G * 5) : 0;
+  size_t gi = 0;
   for (int b = 0; b < B; ++b) {
     const HostTree& t = d->trees[b];
     for (int i = 0; i < N; ++i) {
@@ -258,9 +274,18 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
       h[o_slot + (size_t)b * N + i] = slot ? slot[(size_t)b * N + i] : i;
     }
     for (int sidx = 0; sidx < Ns; ++sidx) h[o_inv + (size_t)b * Ns + sidx] = t.tab[LUMO_TAB_SLOT_INV][sidx];
-    for (int i = 0; i < N * 4; ++i) {   // windows in physical rows
-      int w = t.tab[LUMO_TAB_ANC_WIN][i];
-      h[o_win + (size_t)b * N * 4 + i] = w < 0 ? w : h[o_slot + (size_t)b * N + w];
+    // conv windows per PHYSICAL row, entries in physical rows (or -1..-3 = history rows);
+    // a padding row holds INT32_MIN
+    for (int sidx = 0; sidx < Ns; ++sidx) {
+      const int node = t.tab[LUMO_TAB_SLOT_INV][sidx];
+      for (int j = 0; j < 4; ++j) {
+        int w = INT32_MIN;
+        if (node >= 0) {
+          w = t.tab[LUMO_TAB_ANC_WIN][node * 4 + j];
+          if (w >= 0) w = h[o_slot + (size_t)b * N + w];
+        }
+        h[o_win + ((size_t)b * Ns + sidx) * 4 + j] = w;
+      }
     }
     for (int w = 0; w < 2; ++w) {
       const auto& ops = t.tab[LUMO_TAB_SCHEDULE + w];
@@ -268,22 +293,24 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
       h[o_nops[w] + b] = (int32_t)ops.size();
     }
     if (tc) {
-      // nodes ordered by (depth, logical index); pos[node] = position
-      std::vector<int> order, pos(N, -1);
-      uint8_t* lvl = reinterpret_cast<uint8_t*>(h.data() + o_tc_lvl) + (size_t)b * 20;
-      for (int dep = 1; dep <= 16; ++dep) {
-        for (int n = 0; n < N; ++n)
-          if (t.tab[LUMO_TAB_DEPTH][n] == dep) { pos[n] = (int)order.size(); order.push_back(n); }
-        lvl[dep] = (uint8_t)order.size();
-      }
-      for (int dep = 17; dep < 20; ++dep) lvl[dep] = (uint8_t)N;
-      uint8_t* anc = reinterpret_cast<uint8_t*>(h.data() + o_tc_anc) + (size_t)b * N * 16;
-      for (int pi = 0; pi < N; ++pi) {
-        const int n = order[pi];
-        const int dep = t.tab[LUMO_TAB_DEPTH][n];
-        h[o_tc_meta + (size_t)b * N + pi] = h[o_slot + (size_t)b * N + n] | (dep << 16);
-        int cur = parent[(size_t)b * N + n];
-        for (int j = dep - 2; j >= 0; --j) { anc[pi * 16 + j] = (uint8_t)pos[cur]; cur = parent[(size_t)b * N + cur]; }
+      for (size_t k = 0; k < groups[b].size(); ++k, ++gi) {
+        const GramGroup& gr = groups[b][k];
+        const int n = (int)gr.nodes.size();
+        h[o_tc_group + gi * 4 + 0] = b;
+        h[o_tc_group + gi * 4 + 1] = n;
+        h[o_tc_group + gi * 4 + 2] = k == 0;
+        std::vector<int> pos(N, -1);
+        for (int pi = 0; pi < n; ++pi) pos[gr.nodes[pi]] = pi;
+        uint8_t* lvl = reinterpret_cast<uint8_t*>(h.data() + o_tc_lvl) + gi * 20;
+        uint8_t* anc = reinterpret_cast<uint8_t*>(h.data() + o_tc_anc) + gi * 64 * 16;
+        for (int pi = 0; pi < n; ++pi) {
+          const int node = gr.nodes[pi];
+          const int dep = t.tab[LUMO_TAB_DEPTH][node];
+          h[o_tc_meta + gi * 64 + pi] = h[o_slot + (size_t)b * N + node] | (dep << 16) | ((int)gr.emit[pi] << 24);
+          int cur = parent[(size_t)b * N + node];
+          for (int j = dep - 2; j >= 0; --j) { anc[pi * 16 + j] = (uint8_t)pos[cur]; cur = parent[(size_t)b * N + cur]; }
+          for (int dd = dep; dd < 20; ++dd) lvl[dd] += 1;      // lvl[d] = members of depth <= d
+        }
       }
     }
   }
@@ -297,6 +324,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_win;
   for (int w = 0; w < 2; ++w) { d->d_sched[w] = d->dev + o_sched[w]; d->d_nops[w] = d->dev + o_nops[w]; }
   if (tc) {
+    d->d_tc_group = d->dev + o_tc_group;
     d->d_tc_meta = d->dev + o_tc_meta;
     d->d_tc_anc = reinterpret_cast<uint8_t*>(d->dev + o_tc_anc);
     d->d_tc_lvl = reinterpret_cast<uint8_t*>(d->dev + o_tc_lvl);
@@ -349,7 +377,7 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
   const TreeDev t = tree_view(desc, s.snapshot_mode != 0 ? 1 : 0);
   const bool gram_ok = desc->d_tc_meta != nullptr && gram_supported(s, desc->max_depth);
   if (ctx->scan_algo == 2 && !gram_ok)
-    return fail(ctx, LUMO_ERR_UNSUPPORTED, "the Gram-form scan needs d = 128, bf16 operands, N <= 64, depth <= 16, no snapshots");
+    return fail(ctx, LUMO_ERR_UNSUPPORTED, "the Gram-form scan needs d = 128, bf16 operands, depth <= 16, no snapshots");
   if (gram_ok && ctx->scan_algo != 1) {
     cudaError_t e = cudaSuccess;
     if (layers[0].x) {
@@ -425,11 +453,9 @@ int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_ar
   DeviceGuard g(ctx->device);
   cudaStream_t st = (cudaStream_t)stream;
   const TreeDev t = tree_view(desc, 0);
-  cudaError_t e = timed(ctx, LUMO_K_COMMIT_STATE, st, [&] {
-    return launch_commit_state(s, t, lb, accepted_dev, len_dev, lmax, st);
+  cudaError_t e = timed(ctx, LUMO_K_COMMIT, st, [&] {
+    return launch_commit(s, t, lb, accepted_dev, len_dev, lmax, layers[0].x != nullptr, st);
   });
-  if (e == cudaSuccess && layers[0].x)
-    e = timed(ctx, LUMO_K_COMMIT_HIST, st, [&] { return launch_commit_hist(s, t, lb, accepted_dev, len_dev, lmax, st); });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "commit launch");
 }
 

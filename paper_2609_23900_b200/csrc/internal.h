@@ -32,6 +32,11 @@ struct HostTree {
   std::vector<int32_t> tab[LUMO_TAB_COUNT];
 };
 
+struct GramGroup {
+  std::vector<int> nodes;    // logical ids ordered by (depth, index); every ancestor of a member is a member
+  std::vector<char> emit;    // 1: this group writes the node's output
+};
+
 }  // namespace lumo
 
 struct lumo_ctx {
@@ -57,16 +62,19 @@ struct lumo_tree_desc {
   int32_t* d_depth = nullptr;     // [B, N]
   int32_t* d_slot = nullptr;      // [B, N]
   int32_t* d_slot_inv = nullptr;  // [B, Ns]
-  int32_t* d_win = nullptr;       // [B, N, 4]  physical row, or -1/-2/-3 for history rows
+  int32_t* d_win = nullptr;       // [B, Ns, 4] per physical row: source rows (physical), -1/-2/-3 = history rows, INT32_MIN = padding row
   int32_t* d_sched[2] = {nullptr, nullptr};   // [B, max_ops]  lean / full (every node's state materialised)
   int32_t* d_nops[2] = {nullptr, nullptr};    // [B]
   int max_ops[2] = {0, 0};
   int max_levels[2] = {0, 0};     // stack levels the schedule needs
   int max_depth = 0;              // deepest node over the batch
-  // Gram-form scan tables (present when N <= 64 and max_depth <= 16), nodes ordered by (depth, index)
-  int32_t* d_tc_meta = nullptr;   // [B, N]  physical row | depth << 16 of the node at position pi
-  uint8_t* d_tc_anc = nullptr;    // [B, N, 16] positions of the ancestors, root first
-  uint8_t* d_tc_lvl = nullptr;    // [B, 20] lvl[d] = number of nodes of depth <= d (lvl[0] = 0)
+  // Gram-form scan tables (present when max_depth <= 16): the trees are cut into groups of at most
+  // 64 nodes (prefix path + complete subtrees); G = number of groups over the batch
+  int n_groups = 0;
+  int32_t* d_tc_group = nullptr;  // [G, 4]  sequence b, node count, first-group-of-b flag, 0
+  int32_t* d_tc_meta = nullptr;   // [G, 64] physical row | depth << 16 | emit << 24 of the node at position pi
+  uint8_t* d_tc_anc = nullptr;    // [G, 64, 16] positions of the ancestors, root first
+  uint8_t* d_tc_lvl = nullptr;    // [G, 20] lvl[d] = number of group nodes of depth <= d (lvl[0] = 0)
 };
 
 namespace lumo {
@@ -98,9 +106,10 @@ struct Shape {
 struct TreeDev {
   const int32_t* parent; const int32_t* depth; const int32_t* slot; const int32_t* slot_inv;
   const int32_t* win; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
-  const int32_t* tc_meta; const uint8_t* tc_anc; const uint8_t* tc_lvl;
+  const int32_t* tc_group; const int32_t* tc_meta; const uint8_t* tc_anc; const uint8_t* tc_lvl; int n_groups;
 };
 
+void build_gram_groups(const int32_t* parent, int N, const HostTree& t, std::vector<GramGroup>* out);
 // host-side tree tables (tree_desc.cpp)
 bool build_tree(const int32_t* parent, const int32_t* slot, int N, int Ns, HostTree* t,
                 int* levels_lean, int* levels_full, std::string* err);
@@ -116,10 +125,8 @@ bool gram_supported(const Shape& s, int max_depth);
 cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, cudaStream_t st);
 // device address of the built-in stack on `device` (which must be current); looked up once per device
 cudaError_t static_stack_address(int device, float** ptr);
-cudaError_t launch_commit_state(const Shape& s, const TreeDev& t, const LayerBatch& lb,
-                                const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st);
-cudaError_t launch_commit_hist(const Shape& s, const TreeDev& t, const LayerBatch& lb,
-                               const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st);
+cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb, const int32_t* accepted,
+                          const int32_t* len, int lmax, bool with_hist, cudaStream_t st);
 cudaError_t launch_path_from_node(const TreeDev& t, int B, int N, const int32_t* node, int lmax,
                                   int32_t* accepted, int32_t* len, int32_t* status, cudaStream_t st);
 

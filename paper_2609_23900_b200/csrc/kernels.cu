@@ -9,6 +9,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <climits>
 #include <mutex>
 #include <type_traits>
 
@@ -56,17 +57,17 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
-// Accepted-path check shared by the commit kernels; every CTA of a sequence reaches the same
-// answer.  Order of checks: length, then per entry range, root, link.
-__device__ int check_path(const int32_t* parent, int N, const int32_t* acc, int len, int lmax) {
+// Accepted-path check; every CTA of a sequence reaches the same answer.  Order of checks: length,
+// then per entry range, root, link.  The path's entries and their parents were staged in shared memory
+// (parent -2 marks an entry outside [0, N)).
+__device__ int check_path_staged(const int* acc, const int* par, int N, int len, int lmax) {
   if (len < 0 || len > lmax) return LUMO_SEQ_BAD_LEN;
   int prev = -1;
   for (int t = 0; t < len; ++t) {       // bounded by lmax
-    int a = acc[t];
+    const int a = acc[t];
     if (a < 0 || a >= N) return LUMO_SEQ_BAD_NODE;
-    int p = parent[a];
-    if (t == 0) { if (p != -1) return LUMO_SEQ_BAD_ROOT; }
-    else if (p != prev) return LUMO_SEQ_BAD_LINK;
+    if (t == 0) { if (par[t] != -1) return LUMO_SEQ_BAD_ROOT; }
+    else if (par[t] != prev) return LUMO_SEQ_BAD_LINK;
     prev = a;
   }
   return LUMO_SEQ_OK;
@@ -75,79 +76,117 @@ __device__ int check_path(const int32_t* parent, int N, const int32_t* acc, int 
 // ---------------------------------------------------------------------------------------
 // a1: ancestry-gathered causal depthwise conv (width 4) + SiLU -> recorded operands
 // ---------------------------------------------------------------------------------------
-// One thread owns kVec consecutive channels of one physical row.  Taps are applied oldest
-// first in fp32 starting from zero, bias last, SiLU in fp32, one round-to-nearest-even cast
-// (Sec. "Precompute branch histories while preserving arithmetic": tap order and cast points
-// are part of the result).
+// A CTA owns kConvRows consecutive physical rows of one sequence and a slab of 256 x kVec channels;
+// a thread keeps the 4 x kVec weights of its channels in registers and walks the CTA's rows, so the
+// only per-row traffic is the four 16-byte taps, all independent and issued before the arithmetic.
+// Windows come from the host-built table (physical rows, or -1..-3 for the history rows) staged in
+// shared memory.  Taps are applied oldest first in fp32 starting from zero, bias last, SiLU in fp32,
+// one round-to-nearest-even cast (Sec. "Precompute branch histories while preserving arithmetic":
+// tap order and cast points are part of the result).
+constexpr int kConvRows = 4;
+
 template <typename T, int kVec>
 __global__ void __launch_bounds__(256) conv_kernel(Shape s, TreeDev t, LayerBatch lb) {
+  __shared__ int s_win[kConvRows][4];
   const int layer = blockIdx.z / s.B, b = blockIdx.z % s.B;
-  const int ps = blockIdx.y;                                   // physical row
+  const int ps0 = blockIdx.y * kConvRows;
   const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * kVec;
-  if (c0 >= s.C) return;
   const LayerPtrs& L = lb.l[layer];
+  const int row = L.state_row[b];
+  const bool seq_ok = row >= 0 && row < s.n_state_rows;
+  if (threadIdx.x < kConvRows * 4) {
+    const int r = threadIdx.x >> 2, j = threadIdx.x & 3;
+    const int ps = ps0 + r;
+    int w = INT_MIN;                                  // INT_MIN: this row produces zeros
+    if (ps < s.Ns) w = t.win[((size_t)b * s.Ns + ps) * 4 + j];
+    s_win[r][j] = seq_ok ? w : INT_MIN;
+  }
+  __syncthreads();
+  if (c0 >= s.C) return;
   const int hkd = s.Hk * s.d;
   // destination of this channel group inside [q | k | v]
   T* dst;
-  if (c0 < hkd) dst = reinterpret_cast<T*>(L.q) + ((size_t)b * s.Ns + ps) * hkd + c0;
-  else if (c0 < 2 * hkd) dst = reinterpret_cast<T*>(L.k) + ((size_t)b * s.Ns + ps) * hkd + (c0 - hkd);
-  else dst = reinterpret_cast<T*>(L.v) + ((size_t)b * s.Ns + ps) * (size_t)(s.Hv * s.d) + (c0 - 2 * hkd);
+  size_t dst_stride;
+  if (c0 < hkd) { dst = reinterpret_cast<T*>(L.q) + c0; dst_stride = hkd; }
+  else if (c0 < 2 * hkd) { dst = reinterpret_cast<T*>(L.k) + (c0 - hkd); dst_stride = hkd; }
+  else { dst = reinterpret_cast<T*>(L.v) + (c0 - 2 * hkd); dst_stride = (size_t)s.Hv * s.d; }
 
-  const int node = t.slot_inv[b * s.Ns + ps];
-  const int row = L.state_row[b];
-  float y[kVec];
-  if (node < 0 || row < 0 || row >= s.n_state_rows) {
-#pragma unroll
-    for (int e = 0; e < kVec; ++e) y[e] = 0.f;
-  } else {
-    const T* x = reinterpret_cast<const T*>(L.x);
-    const T* hist = reinterpret_cast<const T*>(L.conv_hist);
+  const T* x = reinterpret_cast<const T*>(L.x) + (size_t)b * s.Ns * s.C + c0;
+  const T* hist = reinterpret_cast<const T*>(L.conv_hist) + (size_t)(seq_ok ? row : 0) * 3 * s.C + c0;
+  float wv[kVec * 4];
+  {
     const T* w = reinterpret_cast<const T*>(L.conv_w) + (size_t)c0 * 4;
-    float wv[kVec * 4];
 #pragma unroll
     for (int e = 0; e < kVec; ++e) {
       float4 w4 = Vec4<T>::load(w + e * 4);
       wv[e * 4 + 0] = w4.x; wv[e * 4 + 1] = w4.y; wv[e * 4 + 2] = w4.z; wv[e * 4 + 3] = w4.w;
     }
+  }
+  float bias[kVec];
+#pragma unroll
+  for (int e = 0; e < kVec; ++e) bias[e] = 0.f;
+  if (L.conv_b) {
+    const T* bp = reinterpret_cast<const T*>(L.conv_b) + c0;
+#pragma unroll
+    for (int e4 = 0; e4 < kVec / 4; ++e4) {
+      float4 bv = Vec4<T>::load(bp + e4 * 4);
+      bias[e4 * 4 + 0] = bv.x; bias[e4 * 4 + 1] = bv.y; bias[e4 * 4 + 2] = bv.z; bias[e4 * 4 + 3] = bv.w;
+    }
+  }
+  using Raw = uint4;                                   // 16 bytes = kVec elements
+  Raw raws[kConvRows][4];
+#pragma unroll
+  for (int r = 0; r < kConvRows; ++r) {                // all taps of all rows in flight
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int wj = s_win[r][j];
+      raws[r][j] = make_uint4(0, 0, 0, 0);
+      if (wj != INT_MIN) {
+        const T* src = wj >= 0 ? x + (size_t)wj * s.C : hist + (size_t)(3 + wj) * s.C;
+        raws[r][j] = *reinterpret_cast<const Raw*>(src);
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < kConvRows; ++r) {                // bounded: kConvRows
+    const int ps = ps0 + r;
+    if (ps >= s.Ns) break;
+    float y[kVec];
 #pragma unroll
     for (int e = 0; e < kVec; ++e) y[e] = 0.f;
-    const int4 win = *reinterpret_cast<const int4*>(t.win + ((size_t)b * s.N + node) * 4);
-    const int wj[4] = {win.x, win.y, win.z, win.w};
+    if (s_win[r][3] != INT_MIN) {
+      const Raw* raw = raws[r];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {                    // oldest -> newest
-      const T* src = wj[j] >= 0 ? x + ((size_t)b * s.Ns + wj[j]) * s.C + c0
-                                : hist + ((size_t)row * 3 + (3 + wj[j])) * s.C + c0;
+      for (int j = 0; j < 4; ++j) {                    // oldest -> newest
+        const T* xv_p = reinterpret_cast<const T*>(&raw[j]);
 #pragma unroll
-      for (int e4 = 0; e4 < kVec / 4; ++e4) {
-        float4 xv = Vec4<T>::load(src + e4 * 4);
-        y[e4 * 4 + 0] = fmaf(wv[(e4 * 4 + 0) * 4 + j], xv.x, y[e4 * 4 + 0]);
-        y[e4 * 4 + 1] = fmaf(wv[(e4 * 4 + 1) * 4 + j], xv.y, y[e4 * 4 + 1]);
-        y[e4 * 4 + 2] = fmaf(wv[(e4 * 4 + 2) * 4 + j], xv.z, y[e4 * 4 + 2]);
-        y[e4 * 4 + 3] = fmaf(wv[(e4 * 4 + 3) * 4 + j], xv.w, y[e4 * 4 + 3]);
+        for (int e4 = 0; e4 < kVec / 4; ++e4) {
+          float4 xv = Vec4<T>::load(xv_p + e4 * 4);
+          y[e4 * 4 + 0] = fmaf(wv[(e4 * 4 + 0) * 4 + j], xv.x, y[e4 * 4 + 0]);
+          y[e4 * 4 + 1] = fmaf(wv[(e4 * 4 + 1) * 4 + j], xv.y, y[e4 * 4 + 1]);
+          y[e4 * 4 + 2] = fmaf(wv[(e4 * 4 + 2) * 4 + j], xv.z, y[e4 * 4 + 2]);
+          y[e4 * 4 + 3] = fmaf(wv[(e4 * 4 + 3) * 4 + j], xv.w, y[e4 * 4 + 3]);
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < kVec; ++e) {
+        const float a = y[e] + bias[e];
+        y[e] = a * __frcp_rn(1.f + __expf(-a));        // SiLU; the ~1e-6 relative error of the fast
+                                                        // exponential is far below the operand rounding
       }
     }
-    if (L.conv_b) {
-      const T* bias = reinterpret_cast<const T*>(L.conv_b) + c0;
+    T* d = dst + ((size_t)b * s.Ns + ps) * dst_stride;
+    if constexpr (sizeof(T) == 2) {
+      uint32_t pk[kVec / 2];
 #pragma unroll
-      for (int e4 = 0; e4 < kVec / 4; ++e4) {
-        float4 bv = Vec4<T>::load(bias + e4 * 4);
-        y[e4 * 4 + 0] += bv.x; y[e4 * 4 + 1] += bv.y; y[e4 * 4 + 2] += bv.z; y[e4 * 4 + 3] += bv.w;
+      for (int e = 0; e < kVec / 2; ++e) {
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(y[2 * e], y[2 * e + 1]);
+        pk[e] = *reinterpret_cast<uint32_t*>(&h2);
       }
+      *reinterpret_cast<uint4*>(d) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+    } else {
+      *reinterpret_cast<float4*>(d) = make_float4(y[0], y[1], y[2], y[3]);
     }
-#pragma unroll
-    for (int e = 0; e < kVec; ++e) y[e] = y[e] / (1.f + expf(-y[e]));   // SiLU
-  }
-  if constexpr (sizeof(T) == 2) {
-    static_assert(kVec == 8 || sizeof(T) != 2, "bf16 path stores 16 bytes");
-    uint32_t pk[kVec / 2];
-#pragma unroll
-    for (int e = 0; e < kVec / 2; ++e) {
-      __nv_bfloat162 h2 = __floats2bfloat162_rn(y[2 * e], y[2 * e + 1]);
-      pk[e] = *reinterpret_cast<uint32_t*>(&h2);
-    }
-    *reinterpret_cast<uint4*>(dst) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-  } else {
-    *reinterpret_cast<float4*>(dst) = make_float4(y[0], y[1], y[2], y[3]);
   }
 }
 
@@ -399,62 +438,115 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
 }
 
 // ---------------------------------------------------------------------------------------
-// a4: commit - replay the accepted path into the running state, in place
+// a4 + a5: commit - replay the accepted path into the running state, in place, and gather the
+// convolution history of the accepted path
 // ---------------------------------------------------------------------------------------
-// Same per-token arithmetic as the scan's EMIT_DESCEND without the output: this is the
-// "native per-token update" of Algorithm 2, applied for the accepted nodes in path order.
+// One launch.  The first Hv * d/32 CTAs of a (sequence, layer) each own a 32-row state tile: same
+// per-token arithmetic as the scan's EMIT_DESCEND without the output, i.e. the "native per-token
+// update" of Algorithm 2 applied for the accepted nodes in path order.  The remaining CTAs own
+// 128 x 16 bytes of channels of the history rows: new history = last three rows of
+// [old history ; x of the accepted nodes] (Algorithm 1).  The state tile is requested from memory
+// before the path is validated, so the two dependent chains (tile; length -> path -> operands) overlap;
+// nothing is written unless the path is valid.
+template <typename T> struct Packed4;      // four consecutive elements as loaded
+template <> struct Packed4<float> {
+  using type = float4;
+  static __device__ __forceinline__ float4 unpack(const float4& p) { return p; }
+};
+template <> struct Packed4<__nv_bfloat16> {
+  using type = uint2;
+  static __device__ __forceinline__ float4 unpack(const uint2& r) {
+    return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xFFFF0000u),
+                       __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xFFFF0000u));
+  }
+};
+
 template <int D, typename T>
-__global__ void __launch_bounds__(kScanThreads)
-commit_state_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ accepted,
-                    const int32_t* __restrict__ len_arr, int lmax) {
+__global__ void __launch_bounds__(kScanThreads, (D == 128 && sizeof(T) == 2) ? 8 : 4)
+commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ accepted,
+              const int32_t* __restrict__ len_arr, int lmax, int n_state_ctas) {
   constexpr int NCH = D / 16;
   constexpr int kTiles = D / kRows;
-  const int tile = blockIdx.x % kTiles, hv = blockIdx.x / kTiles;
+  using P4 = typename Packed4<T>::type;
   const int b = blockIdx.y, layer = blockIdx.z;
   const LayerPtrs& L = lb.l[layer];
-  const int tid = threadIdx.x, j = tid & 3, rl = tid >> 2;
+  const int tid = threadIdx.x;
   const int row = L.state_row[b];
-  const bool lead = hv == 0 && tile == 0 && tid == 0;
+  const bool lead = blockIdx.x == 0 && tid == 0;
   if (row < 0) { if (lead && L.status) L.status[b] = LUMO_SEQ_OK; return; }
   if (row >= s.n_state_rows) { if (lead && L.status) L.status[b] = LUMO_SEQ_BAD_ROW; return; }
   const int32_t* acc = accepted + (size_t)b * lmax;
+  // the whole path at once: entry t, its parent and its physical row (one level of dependent loads
+  // instead of one per step)
+  __shared__ int s_acc[kMaxNodes], s_par[kMaxNodes], s_phys[kMaxNodes];
   const int len = len_arr[b];
-  const int st = check_path(t.parent + (size_t)b * s.N, s.N, acc, len, lmax);
-  if (lead && L.status) L.status[b] = st;
-  if (st != LUMO_SEQ_OK || len == 0) return;
+  const int lcap = len < 0 ? 0 : (len > lmax ? 0 : len);
+  for (int tt = tid; tt < lcap; tt += kScanThreads) {     // bounded: lmax
+    const int a = acc[tt];
+    const bool ok = a >= 0 && a < s.N;
+    s_acc[tt] = a;
+    s_par[tt] = ok ? t.parent[(size_t)b * s.N + a] : -2;
+    s_phys[tt] = ok ? t.slot[b * s.N + a] : 0;
+  }
 
+  if ((int)blockIdx.x >= n_state_ctas) {
+    // ---- convolution history ------------------------------------------------------------------
+    constexpr int kVec = 16 / (int)sizeof(T);
+    const int c0 = ((blockIdx.x - n_state_ctas) * kScanThreads + tid) * kVec;
+    __syncthreads();
+    if (c0 >= s.C || L.x == nullptr) return;
+    if (check_path_staged(s_acc, s_par, s.N, len, lmax) != LUMO_SEQ_OK || len == 0) return;
+    T* hist = reinterpret_cast<T*>(L.conv_hist) + (size_t)row * 3 * s.C + c0;
+    const T* x = reinterpret_cast<const T*>(L.x);
+    uint4 v[3];
+#pragma unroll
+    for (int jj = 0; jj < 3; ++jj) {
+      const int q = len + jj;        // index into [old0 old1 old2 x_a0 x_a1 ...]
+      const T* src = q < 3 ? hist + (size_t)q * s.C
+                           : x + ((size_t)b * s.Ns + s_phys[q - 3]) * s.C + c0;
+      v[jj] = *reinterpret_cast<const uint4*>(src);
+    }
+#pragma unroll
+    for (int jj = 0; jj < 3; ++jj) *reinterpret_cast<uint4*>(hist + (size_t)jj * s.C) = v[jj];
+    return;
+  }
+
+  // ---- state tile ---------------------------------------------------------------------------------
+  const int tile = blockIdx.x % kTiles, hv = blockIdx.x / kTiles;
+  const int j = tid & 3, rl = tid >> 2;
   const int g = hv / (s.Hv / s.Hk);
   const int r0 = tile * kRows;
   float* Sg = L.state + (((size_t)row * s.Hv + hv) * D + r0 + rl) * D;
   float4 S[NCH];
 #pragma unroll
-  for (int m = 0; m < NCH; ++m) S[m] = *reinterpret_cast<const float4*>(Sg + 16 * m + 4 * j);
+  for (int m = 0; m < NCH; ++m) S[m] = *reinterpret_cast<const float4*>(Sg + 16 * m + 4 * j);   // in flight
+
+  __syncthreads();
+  const int st = check_path_staged(s_acc, s_par, s.N, len, lmax);
+  if (lead && L.status) L.status[b] = st;
+  if (st != LUMO_SEQ_OK || len == 0) return;
 
   const T* kg = reinterpret_cast<const T*>(L.k);
   const T* vg = reinterpret_cast<const T*>(L.v);
-  auto load_node = [&](int tt, float4* kv, float* vv, float* a, float* bt) {
-    const int n = acc[tt];
-    const size_t pr = (size_t)b * s.Ns + t.slot[b * s.N + n];
-    const T* kr = kg + (pr * s.Hk + g) * D;
-#pragma unroll
-    for (int m = 0; m < NCH; ++m) kv[m] = Vec4<T>::load(kr + 16 * m + 4 * j);
-    if constexpr (sizeof(T) == 2) *vv = __bfloat162float(vg[(pr * s.Hv + hv) * D + r0 + rl]);
-    else *vv = vg[(pr * s.Hv + hv) * D + r0 + rl];
-    *a = load_scalar(L.alpha, pr * s.Hv + hv, s.gate_dtype);
-    *bt = load_scalar(L.beta, pr * s.Hv + hv, s.gate_dtype);
-  };
-  float4 kv[NCH], kn[NCH];
-  float vv, a, bt, vn = 0.f, an = 0.f, bn = 0.f;
-  load_node(0, kv, &vv, &a, &bt);
   for (int tt = 0; tt < len; ++tt) {                      // bounded: len <= lmax
-    if (tt + 1 < len) load_node(tt + 1, kn, &vn, &an, &bn);   // next node's operands in flight
+    const size_t pr = (size_t)b * s.Ns + s_phys[tt];
+    const T* kr = kg + (pr * s.Hk + g) * D;
+    P4 kp[NCH];
+#pragma unroll
+    for (int m = 0; m < NCH; ++m) kp[m] = *reinterpret_cast<const P4*>(kr + 16 * m + 4 * j);
+    float vv;
+    if constexpr (sizeof(T) == 2) vv = __bfloat162float(vg[(pr * s.Hv + hv) * D + r0 + rl]);
+    else vv = vg[(pr * s.Hv + hv) * D + r0 + rl];
+    const float a = load_scalar(L.alpha, pr * s.Hv + hv, s.gate_dtype);
+    const float bt = load_scalar(L.beta, pr * s.Hv + hv, s.gate_dtype);
     float u0 = 0.f, u1 = 0.f, k0 = 0.f, k1 = 0.f;
 #pragma unroll
     for (int m = 0; m < NCH; ++m) {
-      u0 = fmaf(S[m].x, kv[m].x, u0); u1 = fmaf(S[m].y, kv[m].y, u1);
-      u0 = fmaf(S[m].z, kv[m].z, u0); u1 = fmaf(S[m].w, kv[m].w, u1);
-      k0 = fmaf(kv[m].x, kv[m].x, k0); k1 = fmaf(kv[m].y, kv[m].y, k1);
-      k0 = fmaf(kv[m].z, kv[m].z, k0); k1 = fmaf(kv[m].w, kv[m].w, k1);
+      const float4 kv = Packed4<T>::unpack(kp[m]);
+      u0 = fmaf(S[m].x, kv.x, u0); u1 = fmaf(S[m].y, kv.y, u1);
+      u0 = fmaf(S[m].z, kv.z, u0); u1 = fmaf(S[m].w, kv.w, u1);
+      k0 = fmaf(kv.x, kv.x, k0); k1 = fmaf(kv.y, kv.y, k1);
+      k0 = fmaf(kv.z, kv.z, k0); k1 = fmaf(kv.w, kv.w, k1);
     }
     float u = u0 + u1, kk = k0 + k1;
     u += __shfl_xor_sync(0xffffffffu, u, 1); kk += __shfl_xor_sync(0xffffffffu, kk, 1);
@@ -464,44 +556,13 @@ commit_state_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict
     const float gk = dl * ks;
 #pragma unroll
     for (int m = 0; m < NCH; ++m) {
-      S[m].x = fmaf(a, S[m].x, gk * kv[m].x); S[m].y = fmaf(a, S[m].y, gk * kv[m].y);
-      S[m].z = fmaf(a, S[m].z, gk * kv[m].z); S[m].w = fmaf(a, S[m].w, gk * kv[m].w);
+      const float4 kv = Packed4<T>::unpack(kp[m]);
+      S[m].x = fmaf(a, S[m].x, gk * kv.x); S[m].y = fmaf(a, S[m].y, gk * kv.y);
+      S[m].z = fmaf(a, S[m].z, gk * kv.z); S[m].w = fmaf(a, S[m].w, gk * kv.w);
     }
-#pragma unroll
-    for (int m = 0; m < NCH; ++m) kv[m] = kn[m];
-    vv = vn; a = an; bt = bn;
   }
 #pragma unroll
   for (int m = 0; m < NCH; ++m) *reinterpret_cast<float4*>(Sg + 16 * m + 4 * j) = S[m];
-}
-
-// a5: convolution history <- last three rows of [old history ; x of the accepted nodes]
-template <typename T>
-__global__ void __launch_bounds__(256)
-commit_hist_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ accepted,
-                   const int32_t* __restrict__ len_arr, int lmax) {
-  constexpr int kVec = 16 / (int)sizeof(T);
-  const int b = blockIdx.y, layer = blockIdx.z;
-  const LayerPtrs& L = lb.l[layer];
-  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * kVec;
-  if (c0 >= s.C) return;
-  const int row = L.state_row[b];
-  if (row < 0 || row >= s.n_state_rows) return;
-  const int32_t* acc = accepted + (size_t)b * lmax;
-  const int len = len_arr[b];
-  if (check_path(t.parent + (size_t)b * s.N, s.N, acc, len, lmax) != LUMO_SEQ_OK || len == 0) return;
-  T* hist = reinterpret_cast<T*>(L.conv_hist) + (size_t)row * 3 * s.C + c0;
-  const T* x = reinterpret_cast<const T*>(L.x);
-  uint4 v[3];
-#pragma unroll
-  for (int jj = 0; jj < 3; ++jj) {
-    const int q = len + jj;        // index into [old0 old1 old2 x_a0 x_a1 ...]
-    const T* src = q < 3 ? hist + (size_t)q * s.C
-                         : x + ((size_t)b * s.Ns + t.slot[b * s.N + acc[q - 3]]) * s.C + c0;
-    v[jj] = *reinterpret_cast<const uint4*>(src);
-  }
-#pragma unroll
-  for (int jj = 0; jj < 3; ++jj) *reinterpret_cast<uint4*>(hist + (size_t)jj * s.C) = v[jj];
 }
 
 // device helper: root-first path ending at node[b]
@@ -542,10 +603,10 @@ cudaError_t dispatch(int d, int in_dtype, F f) {
 // ---------------------------------------------------------------------------------------
 cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, cudaStream_t st) {
   if (s.in_dtype == LUMO_BF16) {
-    dim3 grid((s.C / 8 + 255) / 256, s.Ns, s.B * s.n_layers);
+    dim3 grid((s.C / 8 + 255) / 256, (s.Ns + kConvRows - 1) / kConvRows, s.B * s.n_layers);
     conv_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>(s, t, lb);
   } else {
-    dim3 grid((s.C / 4 + 255) / 256, s.Ns, s.B * s.n_layers);
+    dim3 grid((s.C / 4 + 255) / 256, (s.Ns + kConvRows - 1) / kConvRows, s.B * s.n_layers);
     conv_kernel<float, 4><<<grid, 256, 0, st>>>(s, t, lb);
   }
   return cudaGetLastError();
@@ -614,27 +675,18 @@ cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, 
   });
 }
 
-cudaError_t launch_commit_state(const Shape& s, const TreeDev& t, const LayerBatch& lb,
-                                const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st) {
+cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb, const int32_t* accepted,
+                          const int32_t* len, int lmax, bool with_hist, cudaStream_t st) {
   return dispatch(s.d, s.in_dtype, [&](auto dc, auto tc) {
     constexpr int D = decltype(dc)::value;
     using T = decltype(tc);
-    dim3 grid(s.Hv * (D / kRows), s.B, s.n_layers);
-    commit_state_kernel<D, T><<<grid, kScanThreads, 0, st>>>(s, t, lb, accepted, len, lmax);
+    const int n_state = s.Hv * (D / kRows);
+    const int per_thread = 16 / (int)sizeof(T);
+    const int n_hist = with_hist ? (s.C / per_thread + kScanThreads - 1) / kScanThreads : 0;
+    dim3 grid(n_state + n_hist, s.B, s.n_layers);
+    commit_kernel<D, T><<<grid, kScanThreads, 0, st>>>(s, t, lb, accepted, len, lmax, n_state);
     return cudaGetLastError();
   });
-}
-
-cudaError_t launch_commit_hist(const Shape& s, const TreeDev& t, const LayerBatch& lb,
-                               const int32_t* accepted, const int32_t* len, int lmax, cudaStream_t st) {
-  if (s.in_dtype == LUMO_BF16) {
-    dim3 grid((s.C / 8 + 255) / 256, s.B, s.n_layers);
-    commit_hist_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(s, t, lb, accepted, len, lmax);
-  } else {
-    dim3 grid((s.C / 4 + 255) / 256, s.B, s.n_layers);
-    commit_hist_kernel<float><<<grid, 256, 0, st>>>(s, t, lb, accepted, len, lmax);
-  }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_path_from_node(const TreeDev& t, int B, int N, const int32_t* node, int lmax,

@@ -73,7 +73,7 @@ static_assert(kOffV + kNT * kD * 2 <= kOffKQ, "aliased region overflows the S0 t
 
 struct Small {
   float alpha[kNT], beta[kNT], ks[kNT], qs[kNT];
-  int32_t meta[kNT];                 // physical row | depth << 16
+  int32_t meta[kNT];                 // physical row | depth << 16 | emit << 24
   uint8_t anc[kNT][16];              // positions of the ancestors, root first
   float qq[kNT];                     // |q|^2 of each node when normalising
   uint8_t lvl[20];                   // lvl[d] = number of nodes of depth <= d
@@ -212,7 +212,6 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
   const int grp = tid >> 7;            // half of the CTA: 0 or 1
   const int vrow = tid & 127;          // value row = TMEM lane
   const int rep = s.Hv / s.Hk;
-  const int N = s.N;
 
   if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
@@ -228,32 +227,37 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
 
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {   // bounded: n_items
     const int hv = item % s.Hv;
-    const int b = (item / s.Hv) % s.B;
-    const int layer = item / (s.Hv * s.B);
+    const int gi = (item / s.Hv) % t.n_groups;                     // node group
+    const int layer = item / (s.Hv * t.n_groups);
+    const int4 ginfo = *reinterpret_cast<const int4*>(t.tc_group + gi * 4);
+    const int b = ginfo.x, N = ginfo.y;                            // sequence, nodes in this group
+    const bool first_group = ginfo.z != 0;                         // writes the per-sequence zero rows
     const LayerPtrs& L = lb.l[layer];
     const int g = hv / rep;
     const int row = L.state_row[b];
     const size_t out_row_stride = (size_t)s.Hv * kD;
 
     if (row < 0 || row >= s.n_state_rows) {   // skipped sequence: zero outputs
-      for (int ps = grp; ps < s.Ns; ps += 2)
-        store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + vrow, s.out_dtype, 0.f);
-      if (L.status && hv == 0 && tid == 0) L.status[b] = row < 0 ? LUMO_SEQ_OK : LUMO_SEQ_BAD_ROW;
+      if (first_group) {
+        for (int ps = grp; ps < s.Ns; ps += 2)
+          store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + vrow, s.out_dtype, 0.f);
+        if (L.status && hv == 0 && tid == 0) L.status[b] = row < 0 ? LUMO_SEQ_OK : LUMO_SEQ_BAD_ROW;
+      }
       continue;
     }
-    if (L.status && hv == 0 && tid == 0) L.status[b] = LUMO_SEQ_OK;
+    if (first_group && L.status && hv == 0 && tid == 0) L.status[b] = LUMO_SEQ_OK;
 
     PROF(0);
     // ---- a. per-node tables (the addresses of everything else depend on them) -------------------
     if (tid < kNT) {
-      sm.meta[tid] = tid < N ? t.tc_meta[b * N + tid] : 0;
+      sm.meta[tid] = tid < N ? t.tc_meta[gi * kNT + tid] : 0;
     } else if (tid < 2 * kNT) {
       const int pi = tid - kNT;
       uint4 av = make_uint4(0, 0, 0, 0);
-      if (pi < N) av = *reinterpret_cast<const uint4*>(t.tc_anc + ((size_t)b * N + pi) * 16);
+      if (pi < N) av = *reinterpret_cast<const uint4*>(t.tc_anc + ((size_t)gi * kNT + pi) * 16);
       *reinterpret_cast<uint4*>(sm.anc[pi]) = av;
     } else if (tid < 2 * kNT + 20) {
-      sm.lvl[tid - 2 * kNT] = t.tc_lvl[b * 20 + tid - 2 * kNT];
+      sm.lvl[tid - 2 * kNT] = t.tc_lvl[gi * 20 + tid - 2 * kNT];
     }
     __syncthreads();
     PROF(1);
@@ -307,7 +311,7 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     }
     if (tid < kNT) { sm.alpha[tid] = gate_a; sm.beta[tid] = gate_b; }
     // padding rows: zero outputs
-    if (s.Ns > N)
+    if (first_group && s.Ns > s.N)
       for (int ps = grp; ps < s.Ns; ps += 2)
         if (t.slot_inv[b * s.Ns + ps] < 0)
           store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + vrow, s.out_dtype, 0.f);
@@ -397,7 +401,7 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
       NodeRec& rec = recs[pi];
       float* w = is_q ? rec.wq : rec.wk;
       const int meta = sm.meta[pi];
-      const int D = pi < N ? (meta >> 16) : 0;                   // depth, 1..16
+      const int D = pi < N ? ((meta >> 16) & 0xFF) : 0;          // depth, 1..16
       const float a_t = sm.alpha[pi], b_t = sm.beta[pi];
       const float self = is_q ? sm.qs[pi] : -b_t * sm.ks[pi];    // factor of the node itself (k side negated)
       const float* grow = dump + (is_q ? kNT + pi : pi) * kDumpStride;
@@ -418,7 +422,8 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
       if (is_q) {
         rec.c0q = self * G;
         rec.wself = self * sm.ks[pi] * grow[pi];                 // k^_t . q^_t (G = 1)
-        rec.out_off = (uint32_t)((((size_t)b * s.Ns + (meta & 0xFFFF)) * s.Hv + hv) * kD);
+        // a prefix node that another group emits is computed here but not written
+        rec.out_off = ((meta >> 24) & 1) ? (uint32_t)((((size_t)b * s.Ns + (meta & 0xFFFF)) * s.Hv + hv) * kD) : 0xFFFFFFFFu;
       } else {
         rec.c0k = self * G;                                      // -beta_t g_t |k scale|
         rec.beta = b_t;
@@ -490,7 +495,8 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
           o.x = fmaf(wself, acc.x, o.x); o.y = fmaf(wself, acc.y, o.y);
           o.z = fmaf(wself, acc.z, o.z); o.w = fmaf(wself, acc.w, o.w);
           const size_t oi = (size_t)op.out_off + 4 * lane;
-          if (s.out_dtype == LUMO_BF16) {
+          if (op.out_off == 0xFFFFFFFFu) {
+          } else if (s.out_dtype == LUMO_BF16) {
             __nv_bfloat162 o01 = __floats2bfloat162_rn(o.x, o.y), o23 = __floats2bfloat162_rn(o.z, o.w);
             *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(L.out) + oi) =
                 make_uint2(*reinterpret_cast<uint32_t*>(&o01), *reinterpret_cast<uint32_t*>(&o23));
@@ -517,11 +523,11 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
 }  // namespace
 
 bool gram_supported(const Shape& s, int max_depth) {
-  return s.d == kD && s.in_dtype == LUMO_BF16 && s.snapshot_mode == 0 && s.N <= kNT && max_depth <= 16;
+  return s.d == kD && s.in_dtype == LUMO_BF16 && s.snapshot_mode == 0 && max_depth <= 16;
 }
 
 cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, cudaStream_t st) {
-  const int items = s.n_layers * s.B * s.Hv;
+  const int items = s.n_layers * t.n_groups * s.Hv;
   static bool configured = false;
   if (!configured) {
     cudaError_t e = cudaFuncSetAttribute(scan_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);

@@ -161,4 +161,70 @@ bool build_tree(const int32_t* parent, const int32_t* slot, int N, int Ns, HostT
   return true;
 }
 
+// Partition of a tree into groups of at most 64 nodes for the Gram-form scan.  A group is a
+// root-first prefix path (whose deltas the group recomputes) plus complete subtrees hanging off
+// the last prefix node, so every member's ancestors are inside the group.  A node is emitted
+// (its output written) by exactly one group: as a subtree member, or by the first group that
+// carries it as a prefix node.  Members are ordered by (depth, logical index).
+void build_gram_groups(const int32_t* parent, int N, const HostTree& t, std::vector<GramGroup>* out) {
+  const auto& depth = t.tab[LUMO_TAB_DEPTH];
+  const auto& coff = t.tab[LUMO_TAB_CHILD_OFF];
+  const auto& clist = t.tab[LUMO_TAB_CHILD_LIST];
+  std::vector<int> size(N, 1);
+  for (int i = N - 1; i >= 0; --i)
+    if (parent[i] >= 0) size[parent[i]] += size[i];
+  std::vector<char> emitted(N, 0);
+  constexpr int kCap = 64;
+  auto kids = [&](int a, int* lo, int* hi) { *lo = coff[a + 1]; *hi = coff[a + 2]; };   // a = -1: children of the pre-tree state
+  auto flush = [&](const std::vector<int>& prefix, std::vector<int>& members) {
+    if (members.empty()) return;
+    GramGroup g;
+    std::vector<int> all(prefix);
+    all.insert(all.end(), members.begin(), members.end());
+    std::sort(all.begin(), all.end(), [&](int x, int y) { return depth[x] != depth[y] ? depth[x] < depth[y] : x < y; });
+    for (int n : all) {
+      g.nodes.push_back(n);
+      g.emit.push_back(emitted[n] ? 0 : 1);
+      emitted[n] = 1;
+    }
+    out->push_back(std::move(g));
+    members.clear();
+  };
+  std::function<void(int, std::vector<int>&)> pack = [&](int a, std::vector<int>& prefix) {
+    const int cap = kCap - (int)prefix.size();
+    int lo, hi;
+    kids(a, &lo, &hi);
+    std::vector<int> cur;
+    for (int ci = lo; ci < hi; ++ci) {
+      const int c = clist[ci];
+      if (size[c] <= cap) {
+        if ((int)cur.size() + size[c] > cap) flush(prefix, cur);
+        // whole subtree of c (its nodes have indices > c; walk by parent marks)
+        std::vector<int> stack{c};
+        while (!stack.empty()) {
+          int n = stack.back(); stack.pop_back();
+          cur.push_back(n);
+          int l2, h2;
+          kids(n, &l2, &h2);
+          for (int k = l2; k < h2; ++k) stack.push_back(clist[k]);
+        }
+      } else {
+        flush(prefix, cur);
+        prefix.push_back(c);
+        pack(c, prefix);
+        prefix.pop_back();
+      }
+    }
+    flush(prefix, cur);
+    if (a >= 0 && !emitted[a]) {      // every child was too large and recursed, or a has no group yet
+      std::vector<int> none;
+      GramGroup g;
+      for (int n : prefix) { g.nodes.push_back(n); g.emit.push_back(emitted[n] ? 0 : 1); emitted[n] = 1; }
+      out->push_back(std::move(g));
+    }
+  };
+  std::vector<int> prefix;
+  pack(-1, prefix);
+}
+
 }  // namespace lumo

@@ -20,10 +20,10 @@ def ctx(algo="auto"):
 
 
 def gram_eligible(c) -> bool:
-    """Shapes the tensor-core Gram-form scan takes: d = 128, bf16 operands, N <= 64, depth <= 16."""
+    """Shapes the tensor-core Gram-form scan takes: d = 128, bf16 operands, depth <= 16."""
     from paper_2609_23900_b200 import workload as W
     depth = max(max(W.tree_depths(p.tolist())) for p in c.parent)
-    return c.d == 128 and c.in_dtype == "bf16" and c.N <= 64 and depth <= 16
+    return c.d == 128 and c.in_dtype == "bf16" and depth <= 16
 
 
 def ulp_bf16(ref):

@@ -99,6 +99,38 @@ def test_scan_schedule_is_a_valid_depth_first_walk(seed):
     assert sum(1 for o in lean if (o >> 24) in (1, 2)) == len(set(p for p in parent if p >= 0))
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_gram_groups_partition_the_tree(seed):
+    rng = random.Random(300 + seed)
+    n = rng.choice([1, 40, 64, 65, 130, 256])
+    shapes = [W.tree_star(n), W.tree_chains(max(1, n // 16), 16) if n >= 16 else W.tree_chain(n),
+              W.tree_random(W.IntStream(seed), n, 12), W.tree_random(W.IntStream(seed + 50), n, 16, max_children=2)]
+    parent = shapes[seed % 4]
+    n = len(parent)
+    desc = binding.Context(-1).tree_desc(np.array([parent], dtype=np.int32))
+    tab = desc.table("gram_groups").tolist()
+    depth = T.depth(parent)
+    G, pos = tab[0], 1
+    emitted = [0] * n
+    member_once = [0] * n
+    for _ in range(G):
+        cnt = tab[pos]
+        nodes, emit = tab[pos + 1:pos + 1 + cnt], tab[pos + 1 + cnt:pos + 1 + 2 * cnt]
+        pos += 1 + 2 * cnt
+        assert 1 <= cnt <= 64
+        assert nodes == sorted(nodes, key=lambda x: (depth[x], x)) and len(set(nodes)) == cnt
+        inside = set(nodes)
+        for x, e in zip(nodes, emit):
+            assert parent[x] == -1 or parent[x] in inside       # self-contained: all ancestors are members
+            emitted[x] += e
+    assert pos == len(tab) and emitted == [1] * n               # every node is written exactly once
+    if n <= 64:
+        assert G == 1
+    # a tree deeper than 16 has no groups (the rank-1 kernel takes it)
+    deep = binding.Context(-1).tree_desc(np.array([W.tree_chain(17)], dtype=np.int32))
+    assert deep.table("gram_groups").tolist() == []
+
+
 def test_error_codes_and_no_cpu_fallback():
     ctx = binding.Context(-1)
     for bad in ([[0]], [[-1, 1]], [[-1, -2]], [[-1, 0, 3, 1]]):
