@@ -57,6 +57,19 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
+template <typename T> struct Packed4;      // four consecutive elements as loaded
+template <> struct Packed4<float> {
+  using type = float4;
+  static __device__ __forceinline__ float4 unpack(const float4& p) { return p; }
+};
+template <> struct Packed4<__nv_bfloat16> {
+  using type = uint2;
+  static __device__ __forceinline__ float4 unpack(const uint2& r) {
+    return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xFFFF0000u),
+                       __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xFFFF0000u));
+  }
+};
+
 // Accepted-path check; every CTA of a sequence reaches the same answer.  Order of checks: length,
 // then per entry range, root, link.  The path's entries and their parents were staged in shared memory
 // (parent -2 marks an entry outside [0, N)).
@@ -83,10 +96,14 @@ __device__ int check_path_staged(const int* acc, const int* par, int N, int len,
 // shared memory.  Taps are applied oldest first in fp32 starting from zero, bias last, SiLU in fp32,
 // one round-to-nearest-even cast (Sec. "Precompute branch histories while preserving arithmetic":
 // tap order and cast points are part of the result).
-constexpr int kConvRows = 4;
+constexpr int kConvRows = 8;
+
+template <typename T> struct PackedW;      // the 4 taps of one channel as loaded
+template <> struct PackedW<float> { using type = float4; };
+template <> struct PackedW<__nv_bfloat16> { using type = uint2; };
 
 template <typename T, int kVec>
-__global__ void __launch_bounds__(256) conv_kernel(Shape s, TreeDev t, LayerBatch lb) {
+__global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerBatch lb) {
   __shared__ int s_win[kConvRows][4];
   const int layer = blockIdx.z / s.B, b = blockIdx.z % s.B;
   const int ps0 = blockIdx.y * kConvRows;
@@ -101,6 +118,15 @@ __global__ void __launch_bounds__(256) conv_kernel(Shape s, TreeDev t, LayerBatc
     if (ps < s.Ns) w = t.win[((size_t)b * s.Ns + ps) * 4 + j];
     s_win[r][j] = seq_ok ? w : INT_MIN;
   }
+  using PW = typename PackedW<T>::type;
+  using P4 = typename Packed4<T>::type;
+  using Raw = uint4;                                   // 16 bytes = kVec elements
+  PW wpk[kVec];                                        // weights stay packed in registers
+  if (c0 < s.C) {
+    const T* w = reinterpret_cast<const T*>(L.conv_w) + (size_t)c0 * 4;
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) wpk[e] = *reinterpret_cast<const PW*>(w + e * 4);
+  }
   __syncthreads();
   if (c0 >= s.C) return;
   const int hkd = s.Hk * s.d;
@@ -110,69 +136,56 @@ __global__ void __launch_bounds__(256) conv_kernel(Shape s, TreeDev t, LayerBatc
   if (c0 < hkd) { dst = reinterpret_cast<T*>(L.q) + c0; dst_stride = hkd; }
   else if (c0 < 2 * hkd) { dst = reinterpret_cast<T*>(L.k) + (c0 - hkd); dst_stride = hkd; }
   else { dst = reinterpret_cast<T*>(L.v) + (c0 - 2 * hkd); dst_stride = (size_t)s.Hv * s.d; }
-
   const T* x = reinterpret_cast<const T*>(L.x) + (size_t)b * s.Ns * s.C + c0;
   const T* hist = reinterpret_cast<const T*>(L.conv_hist) + (size_t)(seq_ok ? row : 0) * 3 * s.C + c0;
-  float wv[kVec * 4];
-  {
-    const T* w = reinterpret_cast<const T*>(L.conv_w) + (size_t)c0 * 4;
-#pragma unroll
-    for (int e = 0; e < kVec; ++e) {
-      float4 w4 = Vec4<T>::load(w + e * 4);
-      wv[e * 4 + 0] = w4.x; wv[e * 4 + 1] = w4.y; wv[e * 4 + 2] = w4.z; wv[e * 4 + 3] = w4.w;
-    }
-  }
-  float bias[kVec];
-#pragma unroll
-  for (int e = 0; e < kVec; ++e) bias[e] = 0.f;
-  if (L.conv_b) {
-    const T* bp = reinterpret_cast<const T*>(L.conv_b) + c0;
-#pragma unroll
-    for (int e4 = 0; e4 < kVec / 4; ++e4) {
-      float4 bv = Vec4<T>::load(bp + e4 * 4);
-      bias[e4 * 4 + 0] = bv.x; bias[e4 * 4 + 1] = bv.y; bias[e4 * 4 + 2] = bv.z; bias[e4 * 4 + 3] = bv.w;
-    }
-  }
-  using Raw = uint4;                                   // 16 bytes = kVec elements
-  Raw raws[kConvRows][4];
-#pragma unroll
-  for (int r = 0; r < kConvRows; ++r) {                // all taps of all rows in flight
+  const T* bias = L.conv_b ? reinterpret_cast<const T*>(L.conv_b) + c0 : nullptr;
+
+  auto load_row = [&](int r, Raw* raw) {               // the four taps of row r, all in flight
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int wj = s_win[r][j];
-      raws[r][j] = make_uint4(0, 0, 0, 0);
+      raw[j] = make_uint4(0, 0, 0, 0);
       if (wj != INT_MIN) {
         const T* src = wj >= 0 ? x + (size_t)wj * s.C : hist + (size_t)(3 + wj) * s.C;
-        raws[r][j] = *reinterpret_cast<const Raw*>(src);
+        raw[j] = *reinterpret_cast<const Raw*>(src);
       }
     }
-  }
-#pragma unroll
+  };
+  Raw cur[4], nxt[4];
+  load_row(0, cur);
+#pragma unroll 1
   for (int r = 0; r < kConvRows; ++r) {                // bounded: kConvRows
     const int ps = ps0 + r;
     if (ps >= s.Ns) break;
+    if (r + 1 < kConvRows && ps + 1 < s.Ns) load_row(r + 1, nxt);    // next row's taps fly during this row's math
     float y[kVec];
 #pragma unroll
     for (int e = 0; e < kVec; ++e) y[e] = 0.f;
     if (s_win[r][3] != INT_MIN) {
-      const Raw* raw = raws[r];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {                    // oldest -> newest
-        const T* xv_p = reinterpret_cast<const T*>(&raw[j]);
+        const P4* xp = reinterpret_cast<const P4*>(&cur[j]);
 #pragma unroll
         for (int e4 = 0; e4 < kVec / 4; ++e4) {
-          float4 xv = Vec4<T>::load(xv_p + e4 * 4);
-          y[e4 * 4 + 0] = fmaf(wv[(e4 * 4 + 0) * 4 + j], xv.x, y[e4 * 4 + 0]);
-          y[e4 * 4 + 1] = fmaf(wv[(e4 * 4 + 1) * 4 + j], xv.y, y[e4 * 4 + 1]);
-          y[e4 * 4 + 2] = fmaf(wv[(e4 * 4 + 2) * 4 + j], xv.z, y[e4 * 4 + 2]);
-          y[e4 * 4 + 3] = fmaf(wv[(e4 * 4 + 3) * 4 + j], xv.w, y[e4 * 4 + 3]);
+          const float4 xv = Packed4<T>::unpack(xp[e4]);
+          const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float4 wv = Packed4<T>::unpack(*reinterpret_cast<const P4*>(&wpk[e4 * 4 + e]));
+            const float wj = j == 0 ? wv.x : (j == 1 ? wv.y : (j == 2 ? wv.z : wv.w));
+            y[e4 * 4 + e] = fmaf(wj, xs[e], y[e4 * 4 + e]);
+          }
         }
       }
 #pragma unroll
       for (int e = 0; e < kVec; ++e) {
-        const float a = y[e] + bias[e];
-        y[e] = a * __frcp_rn(1.f + __expf(-a));        // SiLU; the ~1e-6 relative error of the fast
-                                                        // exponential is far below the operand rounding
+        float a = y[e];
+        if (bias) {                                    // bias last
+          if constexpr (sizeof(T) == 2) a += __bfloat162float(bias[e]); else a += bias[e];
+        }
+        // SiLU with the hardware exponential and reciprocal: ~1e-6 relative error, far below the
+        // rounding of the recorded operand
+        y[e] = __fdividef(a, 1.f + __expf(-a));
       }
     }
     T* d = dst + ((size_t)b * s.Ns + ps) * dst_stride;
@@ -187,6 +200,8 @@ __global__ void __launch_bounds__(256) conv_kernel(Shape s, TreeDev t, LayerBatc
     } else {
       *reinterpret_cast<float4*>(d) = make_float4(y[0], y[1], y[2], y[3]);
     }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
   }
 }
 
@@ -448,19 +463,6 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
 // [old history ; x of the accepted nodes] (Algorithm 1).  The state tile is requested from memory
 // before the path is validated, so the two dependent chains (tile; length -> path -> operands) overlap;
 // nothing is written unless the path is valid.
-template <typename T> struct Packed4;      // four consecutive elements as loaded
-template <> struct Packed4<float> {
-  using type = float4;
-  static __device__ __forceinline__ float4 unpack(const float4& p) { return p; }
-};
-template <> struct Packed4<__nv_bfloat16> {
-  using type = uint2;
-  static __device__ __forceinline__ float4 unpack(const uint2& r) {
-    return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xFFFF0000u),
-                       __uint_as_float(r.y << 16), __uint_as_float(r.y & 0xFFFF0000u));
-  }
-};
-
 template <int D, typename T>
 __global__ void __launch_bounds__(kScanThreads, (D == 128 && sizeof(T) == 2) ? 8 : 4)
 commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ accepted,
