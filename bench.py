@@ -235,6 +235,7 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch through the C ABI every step instead of graph replay")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true", help="plain stream order instead of programmatic dependent launch")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2 twice)")
     ap.add_argument("--out-dtype", default="bf16", choices=["bf16", "f32"])
@@ -263,6 +264,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     ctx = binding.Context(local)
+    ctx.set_overlap(not args.no_overlap)
     # ---- buffer sets: distinct seeds per set and per rank, together larger than L2 -----------
     case0 = make_case(args.config, seed_offset=rank_seed_offset(rank))
     n_layers = len(case0.layers)
@@ -416,7 +418,7 @@ def main():
                        "d": case0.d, "in_dtype": case0.in_dtype, "out_dtype": args.out_dtype, "state": "f32",
                        "pipeline": "conv+silu -> l2norm(q,k) -> tree scan; commit state + conv history",
                        "l2": f"rotating over {n_sets} buffer sets ({n_sets * set_bytes / 2**20:.0f} MiB) larger than L2",
-                       "launch": launch_mode, "parallelism": "replicas" if world > 1 else "single gpu",
+                       "launch": launch_mode, "kernel_overlap": "programmatic dependent launch" if not args.no_overlap else "off", "parallelism": "replicas" if world > 1 else "single gpu",
                        "mean_accepted_len": float(case0.accepted_len.mean())},
             "clocks": {k: clocks[k] for k in ("sm_mhz", "sm_max_mhz", "reasons", "samples", "window")},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),

@@ -111,6 +111,13 @@ int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx);
  * 1 = always the rank-1 fp32 kernel, 2 = Gram form or LUMO_ERR_UNSUPPORTED. */
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo);
 
+/* Kernel overlap (default on): conv, scan and commit are launched with programmatic dependent launch,
+ * so each kernel's set-up (and, for commit, its whole read phase) runs under the tail of the kernel
+ * before it; each waits on the device before touching data its predecessor produces or still reads.
+ * Applied only to small launches (n_layers * B * Hv <= 4 x SM count), where it measured faster.
+ * Results are identical either way; 0 restores plain stream order. */
+int lumo_ctx_set_overlap(lumo_ctx* ctx, int on);
+
 /* Measurement aid.  While enabled, every kernel the library launches is bracketed by two CUDA
  * events on the launch stream (up to 16384 launches between reads; later ones go untimed).
  * lumo_ctx_timing_read waits for the recorded events, returns the launch count and summed

@@ -108,6 +108,13 @@ cudaError_t timed(lumo_ctx* ctx, int kind, cudaStream_t st, F launch) {
   return e;
 }
 
+// Overlapping a kernel with its predecessor pays when both are a single wave of CTAs (the set-up and
+// dependent-load chains hide under the predecessor's tail); with many waves it measured slower (the
+// early CTAs only take slots from the predecessor), so it is limited to small launches.
+bool use_overlap(const lumo_ctx* ctx, const Shape& s) {
+  return ctx->overlap && (long long)s.n_layers * s.B * s.Hv <= 4LL * ctx->sm_count;
+}
+
 TreeDev tree_view(const lumo_tree_desc* d, int which) {
   TreeDev t;
   t.parent = d->d_parent; t.depth = d->d_depth; t.slot = d->d_slot; t.slot_inv = d->d_slot_inv;
@@ -169,6 +176,12 @@ int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo) {
   if (!ctx) return LUMO_ERR_ARG;
   if (algo < 0 || algo > 2) return fail(ctx, LUMO_ERR_ARG, "scan algo must be 0 (auto), 1 (rank-1) or 2 (Gram form)");
   ctx->scan_algo = algo;
+  return LUMO_OK;
+}
+
+int lumo_ctx_set_overlap(lumo_ctx* ctx, int on) {
+  if (!ctx) return LUMO_ERR_ARG;
+  ctx->overlap = on != 0;
   return LUMO_OK;
 }
 
@@ -381,10 +394,10 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
   if (gram_ok && ctx->scan_algo != 1) {
     cudaError_t e = cudaSuccess;
     if (layers[0].x) {
-      e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, st); });
+      e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, use_overlap(ctx, s), st); });
       if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
     }
-    e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram(s, t, lb, ctx->sm_count, st); });
+    e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram(s, t, lb, ctx->sm_count, use_overlap(ctx, s), st); });
     return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "Gram-form scan launch");
   }
   int grid = 0;
@@ -405,7 +418,7 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
     ctx->scratch_bytes = stack_bytes;
   }
   if (layers[0].x) {
-    e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, st); });
+    e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, use_overlap(ctx, s), st); });
     if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
   }
   e = timed(ctx, LUMO_K_SCAN, st, [&] {
@@ -454,7 +467,7 @@ int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_ar
   cudaStream_t st = (cudaStream_t)stream;
   const TreeDev t = tree_view(desc, 0);
   cudaError_t e = timed(ctx, LUMO_K_COMMIT, st, [&] {
-    return launch_commit(s, t, lb, accepted_dev, len_dev, lmax, layers[0].x != nullptr, st);
+    return launch_commit(s, t, lb, accepted_dev, len_dev, lmax, layers[0].x != nullptr, use_overlap(ctx, s), st);
   });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "commit launch");
 }

@@ -47,6 +47,7 @@ struct lumo_ctx {
   size_t scratch_bytes = 0;
   // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
   int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form (tensor cores)
+  bool overlap = true;          // programmatic dependent launch between conv -> scan -> commit
   bool timing = false;
   std::vector<cudaEvent_t> ev_start, ev_stop;
   std::vector<int> ev_kind;
@@ -114,19 +115,43 @@ void build_gram_groups(const int32_t* parent, int N, const HostTree& t, std::vec
 bool build_tree(const int32_t* parent, const int32_t* slot, int N, int Ns, HostTree* t,
                 int* levels_lean, int* levels_full, std::string* err);
 
+// Programmatic dependent launch (sm_90+): a kernel launched with the attribute may start while its
+// predecessor in the stream is still running; it must call pdl_wait() before touching anything the
+// predecessor writes (or writing anything the predecessor reads), and the predecessor lets it in with
+// pdl_trigger().  Rule used here: a kernel triggers only AFTER its own wait, so that everything older
+// than its predecessor has completed by the time its dependent starts.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
+                          Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+#endif
+
 // launchers (kernels.cu); all return cudaError_t and only enqueue
-cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, cudaStream_t st);
+cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st);
 cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, float* stack,
                         int grid, cudaStream_t st);
 // persistent grid size (CTAs resident at once) and the stack scratch it needs
 cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes);
 // Gram-form scan on tcgen05 (scan_gram.cu)
 bool gram_supported(const Shape& s, int max_depth);
-cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, cudaStream_t st);
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
+                             cudaStream_t st);
 // device address of the built-in stack on `device` (which must be current); looked up once per device
 cudaError_t static_stack_address(int device, float** ptr);
 cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb, const int32_t* accepted,
-                          const int32_t* len, int lmax, bool with_hist, cudaStream_t st);
+                          const int32_t* len, int lmax, bool with_hist, bool pdl, cudaStream_t st);
 cudaError_t launch_path_from_node(const TreeDev& t, int B, int N, const int32_t* node, int lmax,
                                   int32_t* accepted, int32_t* len, int32_t* status, cudaStream_t st);
 

@@ -109,6 +109,8 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
   const int ps0 = blockIdx.y * kConvRows;
   const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * kVec;
   const LayerPtrs& L = lb.l[layer];
+  pdl_wait();       // x, history and the operand buffers belong to earlier kernels until here
+  pdl_trigger();
   const int row = L.state_row[b];
   const bool seq_ok = row >= 0 && row < s.n_state_rows;
   if (threadIdx.x < kConvRows * 4) {
@@ -475,8 +477,11 @@ commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ acc
   const int tid = threadIdx.x;
   const int row = L.state_row[b];
   const bool lead = blockIdx.x == 0 && tid == 0;
-  if (row < 0) { if (lead && L.status) L.status[b] = LUMO_SEQ_OK; return; }
-  if (row >= s.n_state_rows) { if (lead && L.status) L.status[b] = LUMO_SEQ_BAD_ROW; return; }
+  // Everything this kernel READS (state, operands, path) is complete once its predecessor passed its
+  // own dependency wait; what it WRITES (state, history, status) may still be read by the predecessor
+  // (the scan reads the pre-tree state), so every write sits behind pdl_wait().
+  if (row < 0) { pdl_wait(); if (lead && L.status) L.status[b] = LUMO_SEQ_OK; return; }
+  if (row >= s.n_state_rows) { pdl_wait(); if (lead && L.status) L.status[b] = LUMO_SEQ_BAD_ROW; return; }
   const int32_t* acc = accepted + (size_t)b * lmax;
   // the whole path at once: entry t, its parent and its physical row (one level of dependent loads
   // instead of one per step)
@@ -508,6 +513,7 @@ commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ acc
                            : x + ((size_t)b * s.Ns + s_phys[q - 3]) * s.C + c0;
       v[jj] = *reinterpret_cast<const uint4*>(src);
     }
+    pdl_wait();
 #pragma unroll
     for (int jj = 0; jj < 3; ++jj) *reinterpret_cast<uint4*>(hist + (size_t)jj * s.C) = v[jj];
     return;
@@ -525,7 +531,7 @@ commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ acc
 
   __syncthreads();
   const int st = check_path_staged(s_acc, s_par, s.N, len, lmax);
-  if (lead && L.status) L.status[b] = st;
+  if (lead && L.status) { pdl_wait(); L.status[b] = st; }
   if (st != LUMO_SEQ_OK || len == 0) return;
 
   const T* kg = reinterpret_cast<const T*>(L.k);
@@ -563,6 +569,7 @@ commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ acc
       S[m].z = fmaf(a, S[m].z, gk * kv.z); S[m].w = fmaf(a, S[m].w, gk * kv.w);
     }
   }
+  pdl_wait();
 #pragma unroll
   for (int m = 0; m < NCH; ++m) *reinterpret_cast<float4*>(Sg + 16 * m + 4 * j) = S[m];
 }
@@ -603,13 +610,13 @@ cudaError_t dispatch(int d, int in_dtype, F f) {
 // ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
-cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, cudaStream_t st) {
+cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st) {
   if (s.in_dtype == LUMO_BF16) {
     dim3 grid((s.C / 8 + 255) / 256, (s.Ns + kConvRows - 1) / kConvRows, s.B * s.n_layers);
-    conv_kernel<__nv_bfloat16, 8><<<grid, 256, 0, st>>>(s, t, lb);
+    return launch_kernel(conv_kernel<__nv_bfloat16, 8>, grid, dim3(256), 0, st, pdl, s, t, lb);
   } else {
     dim3 grid((s.C / 4 + 255) / 256, (s.Ns + kConvRows - 1) / kConvRows, s.B * s.n_layers);
-    conv_kernel<float, 4><<<grid, 256, 0, st>>>(s, t, lb);
+    return launch_kernel(conv_kernel<float, 4>, grid, dim3(256), 0, st, pdl, s, t, lb);
   }
   return cudaGetLastError();
 }
@@ -678,7 +685,7 @@ cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, 
 }
 
 cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb, const int32_t* accepted,
-                          const int32_t* len, int lmax, bool with_hist, cudaStream_t st) {
+                          const int32_t* len, int lmax, bool with_hist, bool pdl, cudaStream_t st) {
   return dispatch(s.d, s.in_dtype, [&](auto dc, auto tc) {
     constexpr int D = decltype(dc)::value;
     using T = decltype(tc);
@@ -686,8 +693,7 @@ cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb
     const int per_thread = 16 / (int)sizeof(T);
     const int n_hist = with_hist ? (s.C / per_thread + kScanThreads - 1) / kScanThreads : 0;
     dim3 grid(n_state + n_hist, s.B, s.n_layers);
-    commit_kernel<D, T><<<grid, kScanThreads, 0, st>>>(s, t, lb, accepted, len, lmax, n_state);
-    return cudaGetLastError();
+    return launch_kernel(commit_kernel<D, T>, grid, dim3(kScanThreads), 0, st, pdl, s, t, lb, accepted, len, lmax, n_state);
   });
 }
 

@@ -263,6 +263,11 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     PROF(1);
     // ---- b. gates (consumed much later); K and Q rows -> swizzled operand tile (cp.async);
     //         first half of the pre-tree state rows -> registers -------------------------------------
+    // K, Q, V may still be in the making (the convolution runs right before this kernel): everything
+    // above touched only the descriptor tables.  The dependent kernel (commit) is let in afterwards:
+    // it reads freely and writes only behind its own wait.
+    pdl_wait();
+    pdl_trigger();
     float gate_a = 1.f, gate_b = 0.f;
     if (tid < N) {
       const size_t pr = (size_t)b * s.Ns + (sm.meta[tid] & 0xFFFF);
@@ -526,7 +531,8 @@ bool gram_supported(const Shape& s, int max_depth) {
   return s.d == kD && s.in_dtype == LUMO_BF16 && s.snapshot_mode == 0 && max_depth <= 16;
 }
 
-cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, cudaStream_t st) {
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
+                             cudaStream_t st) {
   const int items = s.n_layers * t.n_groups * s.Hv;
   static bool configured = false;
   if (!configured) {
@@ -537,8 +543,7 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
   // two CTAs per SM by construction: 102 KB of shared memory, 128 registers x 256 threads and 256
   // of the 512 tensor-memory columns each
   const int grid = items < 2 * sm_count ? items : 2 * sm_count;
-  scan_gram_kernel<<<grid, kThreads, kSmemBytes, st>>>(s, t, lb, items);
-  return cudaGetLastError();
+  return launch_kernel(scan_gram_kernel, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
 }
 
 #ifdef LUMO_GRAM_PROFILE

@@ -320,6 +320,32 @@ def test_off_path_poison_and_two_cycles():
     assert_close(full.np("out"), o_ref, what="one pass")
 
 
+@pytest.mark.parametrize("name", ["cfg2", "rand256_b2", "d64_bf16"])
+def test_kernel_overlap_changes_nothing(name):
+    """conv -> scan -> commit launched back to back with programmatic dependent launch must give
+    bitwise the results of plain stream order, cycle after cycle (commit rewrites the state the next
+    scan reads)."""
+    c = CASES[name]()
+    res = {}
+    for on in (False, True):
+        cx = ctx("auto")
+        cx.set_overlap(on)
+        dc = DeviceCase(cx, c)
+        outs = []
+        for cycle in range(4):
+            dc.verify()
+            dc.commit()
+            outs.append(dc.t("out").clone())
+        torch.cuda.synchronize()
+        res[on] = (outs, dc.t("state").clone(), dc.t("conv_hist").clone(), dc.t("q").clone())
+    ctx("auto").set_overlap(True)
+    for a, b in zip(res[False][0], res[True][0]):
+        assert torch.equal(a, b)
+    for i in (1, 2, 3):
+        assert torch.equal(res[False][i], res[True][i])
+    assert not torch.equal(res[True][0][0], res[True][0][1])      # the cycles really advanced the state
+
+
 def test_multi_layer_launch_and_snapshot_all():
     c = W.config3(B=2, n_layers=5)
     dc = DeviceCase(ctx(), c, snapshot_mode=2)
