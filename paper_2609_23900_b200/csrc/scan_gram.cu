@@ -52,9 +52,11 @@ struct NodeRec {
   float wself;      // k^_t . q^_t
   uint32_t out_off; // element offset of this node's output row for value row 0
   uint32_t pad[3];
-  int32_t aoff[16]; // element offset of ancestor j's deltas in the delta array; beyond the depth: the zero row
+  uint16_t aoff[16]; // element offset of ancestor j's deltas in the delta array; beyond the depth: the zero row
+  uint32_t pad2[4];  // 208 bytes = 13 x 16: consecutive records start 13 bank groups apart, so the
+                     // 128-bit stores of eight neighbouring threads never meet in a bank
 };
-static_assert(sizeof(NodeRec) == 224, "record layout");
+static_assert(sizeof(NodeRec) == 208, "record layout");
 
 // shared memory map (bytes from a 1024-aligned base)
 constexpr int kOffAhi = 0;                          // S0 hi: 2 k-blocks x [128 rows x 128 B], SW128
@@ -191,7 +193,7 @@ struct NodeOps {
   uint2 vb;        // four bf16 values of v
   float4 pk, pq;   // S0 k^, S0 q^ for the lane's four rows
   float4 ck, cq;   // first four coefficients
-  int4 ao;         // first four ancestor offsets
+  uint2 ao;        // first four ancestor offsets (16 bits each)
 };
 
 __global__ void __launch_bounds__(kThreads, 2)
@@ -404,17 +406,18 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
       const bool is_q = tid >= kNT;
       const int pi = tid & (kNT - 1);
       NodeRec& rec = recs[pi];
-      float* w = is_q ? rec.wq : rec.wk;
       const int meta = sm.meta[pi];
       const int D = pi < N ? ((meta >> 16) & 0xFF) : 0;          // depth, 1..16
       const float a_t = sm.alpha[pi], b_t = sm.beta[pi];
       const float self = is_q ? sm.qs[pi] : -b_t * sm.ks[pi];    // factor of the node itself (k side negated)
       const float* grow = dump + (is_q ? kNT + pi : pi) * kDumpStride;
       float G = a_t;
+      float w[16];
+      uint32_t ao[8];
 #pragma unroll
       for (int j = 15; j >= 0; --j) {                            // bounded: 16 depth slots
         float val = 0.f;
-        int off = kZeroRow;
+        uint32_t off = kZeroRow;
         if (j <= D - 2) {
           const int sidx = sm.anc[pi][j];
           val = self * G * sm.ks[sidx] * grow[sidx];
@@ -422,8 +425,11 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
           off = sidx * kD;
         }
         w[j] = val;
-        if (!is_q) rec.aoff[j] = off;
+        if (j & 1) ao[j >> 1] = off << 16; else ao[j >> 1] |= off;
       }
+      float4* wdst = reinterpret_cast<float4*>(is_q ? rec.wq : rec.wk);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) wdst[e] = make_float4(w[4 * e], w[4 * e + 1], w[4 * e + 2], w[4 * e + 3]);
       if (is_q) {
         rec.c0q = self * G;
         rec.wself = self * sm.ks[pi] * grow[pi];                 // k^_t . q^_t (G = 1)
@@ -432,6 +438,9 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
       } else {
         rec.c0k = self * G;                                      // -beta_t g_t |k scale|
         rec.beta = b_t;
+        uint4* adst = reinterpret_cast<uint4*>(rec.aoff);
+        adst[0] = make_uint4(ao[0], ao[1], ao[2], ao[3]);
+        adst[1] = make_uint4(ao[4], ao[5], ao[6], ao[7]);
       }
     } else {
       for (int cb = 0; cb < (N + 31) / 32; ++cb)                 // bounded: <= 2
@@ -458,13 +467,13 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
         op.pq = *reinterpret_cast<const float4*>(Pq + pi * kD + 4 * lane);
         op.ck = *reinterpret_cast<const float4*>(rec.wk);
         op.cq = *reinterpret_cast<const float4*>(rec.wq);
-        op.ao = *reinterpret_cast<const int4*>(rec.aoff);
+        op.ao = *reinterpret_cast<const uint2*>(rec.aoff);
       };
-      auto block4 = [&](float4& acc, float4& o, const float4& ck, const float4& cq, const int4& ao) {
-        const float4 d0 = *reinterpret_cast<const float4*>(dls + ao.x + 4 * lane);
-        const float4 d1 = *reinterpret_cast<const float4*>(dls + ao.y + 4 * lane);
-        const float4 d2 = *reinterpret_cast<const float4*>(dls + ao.z + 4 * lane);
-        const float4 d3 = *reinterpret_cast<const float4*>(dls + ao.w + 4 * lane);
+      auto block4 = [&](float4& acc, float4& o, const float4& ck, const float4& cq, const uint2& ao) {
+        const float4 d0 = *reinterpret_cast<const float4*>(dls + (ao.x & 0xFFFFu) + 4 * lane);
+        const float4 d1 = *reinterpret_cast<const float4*>(dls + (ao.x >> 16) + 4 * lane);
+        const float4 d2 = *reinterpret_cast<const float4*>(dls + (ao.y & 0xFFFFu) + 4 * lane);
+        const float4 d3 = *reinterpret_cast<const float4*>(dls + (ao.y >> 16) + 4 * lane);
         acc.x = fmaf(ck.x, d0.x, acc.x); acc.y = fmaf(ck.x, d0.y, acc.y); acc.z = fmaf(ck.x, d0.z, acc.z); acc.w = fmaf(ck.x, d0.w, acc.w);
         o.x = fmaf(cq.x, d0.x, o.x); o.y = fmaf(cq.x, d0.y, o.y); o.z = fmaf(cq.x, d0.z, o.z); o.w = fmaf(cq.x, d0.w, o.w);
         acc.x = fmaf(ck.y, d1.x, acc.x); acc.y = fmaf(ck.y, d1.y, acc.y); acc.z = fmaf(ck.y, d1.z, acc.z); acc.w = fmaf(ck.y, d1.w, acc.w);
@@ -494,7 +503,7 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
           for (int blk = 1; blk < nblk; ++blk) {                   // bounded: <= 3 more blocks
             const NodeRec& rec = recs[pi];
             block4(acc, o, *reinterpret_cast<const float4*>(rec.wk + 4 * blk), *reinterpret_cast<const float4*>(rec.wq + 4 * blk),
-                   *reinterpret_cast<const int4*>(rec.aoff + 4 * blk));
+                   *reinterpret_cast<const uint2*>(rec.aoff + 4 * blk));
           }
           *reinterpret_cast<float4*>(dls + pi * kD + 4 * lane) = acc;           // delta of this node
           o.x = fmaf(wself, acc.x, o.x); o.y = fmaf(wself, acc.y, o.y);
