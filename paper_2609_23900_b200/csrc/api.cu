@@ -118,7 +118,7 @@ bool use_overlap(const lumo_ctx* ctx, const Shape& s) {
 TreeDev tree_view(const lumo_tree_desc* d, int which) {
   TreeDev t;
   t.parent = d->d_parent; t.depth = d->d_depth; t.slot = d->d_slot; t.slot_inv = d->d_slot_inv;
-  t.win = d->d_win; t.sched = d->d_sched[which]; t.nops = d->d_nops[which];
+  t.win = d->d_win; t.conv_prog = d->d_conv_prog; t.sched = d->d_sched[which]; t.nops = d->d_nops[which];
   t.max_ops = d->max_ops[which]; t.max_levels = d->max_levels[which];
   t.tc_group = d->d_tc_group; t.tc_meta = d->d_tc_meta; t.tc_anc = d->d_tc_anc; t.tc_lvl = d->d_tc_lvl;
   t.n_groups = d->n_groups;
@@ -257,6 +257,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   auto reserve = [&](size_t n) { size_t off = h.size(); h.resize(off + ((n + 3) / 4) * 4, 0); return off; };
   const size_t o_parent = reserve((size_t)B * N), o_depth = reserve((size_t)B * N), o_slot = reserve((size_t)B * N);
   const size_t o_inv = reserve((size_t)B * Ns), o_win = reserve((size_t)B * Ns * 4);
+  const size_t o_prog = reserve((size_t)B * Ns);
   size_t o_sched[2], o_nops[2];
   for (int w = 0; w < 2; ++w) { o_sched[w] = reserve((size_t)B * d->max_ops[w]); o_nops[w] = reserve(B); }
   for (int b = 0; b < B; ++b)
@@ -300,6 +301,33 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
         h[o_win + ((size_t)b * Ns + sidx) * 4 + j] = w;
       }
     }
+    {
+      // conv visiting order: depth-first preorder, so that most rows find three of their four taps
+      // already in the registers of the thread that handled the previous row
+      const auto& coff = t.tab[LUMO_TAB_CHILD_OFF];
+      const auto& clist = t.tab[LUMO_TAB_CHILD_LIST];
+      std::vector<int> stack, order;
+      for (int c = coff[1] - 1; c >= coff[0]; --c) stack.push_back(clist[c]);
+      while (!stack.empty()) {
+        const int n = stack.back(); stack.pop_back();
+        order.push_back(n);
+        for (int c = coff[n + 2] - 1; c >= coff[n + 1]; --c) stack.push_back(clist[c]);
+      }
+      size_t k = 0;
+      for (size_t pidx = 0; pidx < order.size(); ++pidx, ++k) {
+        const int n = order[pidx];
+        int flag = 0;
+        if (pidx > 0) {
+          const int prev = order[pidx - 1];
+          const int pn = parent[(size_t)b * N + n], pp = parent[(size_t)b * N + prev];
+          if (pn == prev) flag = 1;
+          else if (pn == pp) flag = 2;
+        }
+        h[o_prog + (size_t)b * Ns + k] = h[o_slot + (size_t)b * N + n] | (flag << 16);
+      }
+      for (int sidx = 0; sidx < Ns; ++sidx)
+        if (t.tab[LUMO_TAB_SLOT_INV][sidx] < 0) h[o_prog + (size_t)b * Ns + k++] = sidx | (3 << 16);
+    }
     for (int w = 0; w < 2; ++w) {
       const auto& ops = t.tab[LUMO_TAB_SCHEDULE + w];
       std::copy(ops.begin(), ops.end(), h.begin() + o_sched[w] + (size_t)b * d->max_ops[w]);
@@ -334,7 +362,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   e = cudaMemcpy(d->dev, h.data(), h.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) { cudaFree(d->dev); delete d; return cuda_fail(ctx, e, "cudaMemcpy(tree tables)"); }
   d->d_parent = d->dev + o_parent; d->d_depth = d->dev + o_depth; d->d_slot = d->dev + o_slot;
-  d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_win;
+  d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_win; d->d_conv_prog = d->dev + o_prog;
   for (int w = 0; w < 2; ++w) { d->d_sched[w] = d->dev + o_sched[w]; d->d_nops[w] = d->dev + o_nops[w]; }
   if (tc) {
     d->d_tc_group = d->dev + o_tc_group;

@@ -64,6 +64,9 @@ struct lumo_tree_desc {
   int32_t* d_slot = nullptr;      // [B, N]
   int32_t* d_slot_inv = nullptr;  // [B, Ns]
   int32_t* d_win = nullptr;       // [B, Ns, 4] per physical row: source rows (physical), -1/-2/-3 = history rows, INT32_MIN = padding row
+  int32_t* d_conv_prog = nullptr; // [B, Ns] conv visiting order (depth first): physical row | flag << 16; flag 0 = fetch the whole
+                                  // window, 1 = previous row is the parent (window slides), 2 = same parent as the previous row
+                                  // (only the own row changes), 3 = padding row (zeros)
   int32_t* d_sched[2] = {nullptr, nullptr};   // [B, max_ops]  lean / full (every node's state materialised)
   int32_t* d_nops[2] = {nullptr, nullptr};    // [B]
   int max_ops[2] = {0, 0};
@@ -106,7 +109,7 @@ struct Shape {
 
 struct TreeDev {
   const int32_t* parent; const int32_t* depth; const int32_t* slot; const int32_t* slot_inv;
-  const int32_t* win; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
+  const int32_t* win; const int32_t* conv_prog; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
   const int32_t* tc_group; const int32_t* tc_meta; const uint8_t* tc_anc; const uint8_t* tc_lvl; int n_groups;
 };
 

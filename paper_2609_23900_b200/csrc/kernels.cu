@@ -89,11 +89,13 @@ __device__ int check_path_staged(const int* acc, const int* par, int N, int len,
 // ---------------------------------------------------------------------------------------
 // a1: ancestry-gathered causal depthwise conv (width 4) + SiLU -> recorded operands
 // ---------------------------------------------------------------------------------------
-// A CTA owns kConvRows consecutive physical rows of one sequence and a slab of 256 x kVec channels;
-// a thread keeps the 4 x kVec weights of its channels in registers and walks the CTA's rows, so the
-// only per-row traffic is the four 16-byte taps, all independent and issued before the arithmetic.
-// Windows come from the host-built table (physical rows, or -1..-3 for the history rows) staged in
-// shared memory.  Taps are applied oldest first in fp32 starting from zero, bias last, SiLU in fp32,
+// A CTA owns kConvRows consecutive entries of one sequence's visiting order (depth-first, built on
+// the host) and a slab of 256 x kVec channels; a thread keeps the packed taps of its channels and the
+// current 4-row window in registers.  In depth-first order most rows either follow their parent (the
+// window slides by one) or share the parent of the previous row (only the own row changes), so one
+// 16-byte load per row replaces four; the own rows of the next two entries are always in flight.
+// Windows that cannot be derived come from the per-row table (physical rows, or -1..-3 for the
+// history rows).  Taps are applied oldest first in fp32 starting from zero, bias last, SiLU in fp32,
 // one round-to-nearest-even cast (Sec. "Precompute branch histories while preserving arithmetic":
 // tap order and cast points are part of the result).
 constexpr int kConvRows = 8;
@@ -105,8 +107,9 @@ template <> struct PackedW<__nv_bfloat16> { using type = uint2; };
 template <typename T, int kVec>
 __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerBatch lb) {
   __shared__ int s_win[kConvRows][4];
+  __shared__ int s_prog[kConvRows];
   const int layer = blockIdx.z / s.B, b = blockIdx.z % s.B;
-  const int ps0 = blockIdx.y * kConvRows;
+  const int e0 = blockIdx.y * kConvRows;               // first entry of the visiting order
   const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * kVec;
   const LayerPtrs& L = lb.l[layer];
   pdl_wait();       // x, history and the operand buffers belong to earlier kernels until here
@@ -115,10 +118,14 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
   const bool seq_ok = row >= 0 && row < s.n_state_rows;
   if (threadIdx.x < kConvRows * 4) {
     const int r = threadIdx.x >> 2, j = threadIdx.x & 3;
-    const int ps = ps0 + r;
-    int w = INT_MIN;                                  // INT_MIN: this row produces zeros
-    if (ps < s.Ns) w = t.win[((size_t)b * s.Ns + ps) * 4 + j];
-    s_win[r][j] = seq_ok ? w : INT_MIN;
+    int prog = 3 << 16, w = INT_MIN;
+    if (e0 + r < s.Ns) {
+      prog = t.conv_prog[(size_t)b * s.Ns + e0 + r];
+      if (!seq_ok) prog = (prog & 0xFFFF) | (3 << 16);        // skipped sequence: every row is a zero row
+      w = t.win[((size_t)b * s.Ns + (prog & 0xFFFF)) * 4 + j];
+    }
+    s_win[r][j] = w;
+    if (j == 0) s_prog[r] = (e0 + r < s.Ns) ? prog : -1;
   }
   using PW = typename PackedW<T>::type;
   using P4 = typename Packed4<T>::type;
@@ -138,35 +145,41 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
   if (c0 < hkd) { dst = reinterpret_cast<T*>(L.q) + c0; dst_stride = hkd; }
   else if (c0 < 2 * hkd) { dst = reinterpret_cast<T*>(L.k) + (c0 - hkd); dst_stride = hkd; }
   else { dst = reinterpret_cast<T*>(L.v) + (c0 - 2 * hkd); dst_stride = (size_t)s.Hv * s.d; }
+  dst += (size_t)b * s.Ns * dst_stride;
   const T* x = reinterpret_cast<const T*>(L.x) + (size_t)b * s.Ns * s.C + c0;
   const T* hist = reinterpret_cast<const T*>(L.conv_hist) + (size_t)(seq_ok ? row : 0) * 3 * s.C + c0;
   const T* bias = L.conv_b ? reinterpret_cast<const T*>(L.conv_b) + c0 : nullptr;
 
-  auto load_row = [&](int r, Raw* raw) {               // the four taps of row r, all in flight
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int wj = s_win[r][j];
-      raw[j] = make_uint4(0, 0, 0, 0);
-      if (wj != INT_MIN) {
-        const T* src = wj >= 0 ? x + (size_t)wj * s.C : hist + (size_t)(3 + wj) * s.C;
-        raw[j] = *reinterpret_cast<const Raw*>(src);
-      }
-    }
+  auto load_src = [&](int wj) -> Raw {                 // one window entry: a row of x or of the history
+    const T* src = wj >= 0 ? x + (size_t)wj * s.C : hist + (size_t)(3 + wj) * s.C;
+    return *reinterpret_cast<const Raw*>(src);
   };
-  Raw cur[4], nxt[4];
-  load_row(0, cur);
-#pragma unroll 1
+  auto load_own = [&](int r) -> Raw {                  // the entry's own row (padding rows: zeros)
+    const int prog = r < kConvRows ? s_prog[r] : -1;
+    if (prog < 0 || (prog >> 16) == 3) return make_uint4(0, 0, 0, 0);
+    return *reinterpret_cast<const Raw*>(x + (size_t)(prog & 0xFFFF) * s.C);
+  };
+  Raw win[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+  Raw pf[2] = {load_own(0), load_own(1)};
+#pragma unroll
   for (int r = 0; r < kConvRows; ++r) {                // bounded: kConvRows
-    const int ps = ps0 + r;
-    if (ps >= s.Ns) break;
-    if (r + 1 < kConvRows && ps + 1 < s.Ns) load_row(r + 1, nxt);    // next row's taps fly during this row's math
+    const int prog = s_prog[r];
+    if (prog < 0) break;
+    const int ps = prog & 0xFFFF;
+    int flag = prog >> 16;
+    if (r == 0 && flag != 3) flag = 0;                 // the first row of a CTA has nothing to reuse
+    const Raw own = pf[r & 1];
+    pf[r & 1] = load_own(r + 2);                       // keeps two own rows in flight
     float y[kVec];
 #pragma unroll
     for (int e = 0; e < kVec; ++e) y[e] = 0.f;
-    if (s_win[r][3] != INT_MIN) {
+    if (flag != 3) {
+      if (flag == 0) { win[0] = load_src(s_win[r][0]); win[1] = load_src(s_win[r][1]); win[2] = load_src(s_win[r][2]); }
+      else if (flag == 1) { win[0] = win[1]; win[1] = win[2]; win[2] = win[3]; }
+      win[3] = own;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {                    // oldest -> newest
-        const P4* xp = reinterpret_cast<const P4*>(&cur[j]);
+        const P4* xp = reinterpret_cast<const P4*>(&win[j]);
 #pragma unroll
         for (int e4 = 0; e4 < kVec / 4; ++e4) {
           const float4 xv = Packed4<T>::unpack(xp[e4]);
@@ -190,7 +203,7 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
         y[e] = __fdividef(a, 1.f + __expf(-a));
       }
     }
-    T* d = dst + ((size_t)b * s.Ns + ps) * dst_stride;
+    T* d = dst + (size_t)ps * dst_stride;
     if constexpr (sizeof(T) == 2) {
       uint32_t pk[kVec / 2];
 #pragma unroll
@@ -202,8 +215,6 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
     } else {
       *reinterpret_cast<float4*>(d) = make_float4(y[0], y[1], y[2], y[3]);
     }
-#pragma unroll
-    for (int j = 0; j < 4; ++j) cur[j] = nxt[j];
   }
 }
 
