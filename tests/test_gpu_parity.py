@@ -286,6 +286,32 @@ def test_gram_scan_skipped_rows_padding_and_depth_16():
     ctx("auto")
 
 
+def test_gram_groups_with_long_prefix_paths():
+    # caterpillar: a 10-node spine with 24 leaves under every spine node (250 nodes).  The tree is cut
+    # into groups that each carry a prefix path of up to 10 recomputed nodes; every node must still be
+    # written exactly once and match the oracle.
+    spine = 10
+    parent = [i - 1 for i in range(spine)]
+    for sp in range(spine):
+        parent += [sp] * 24
+    c = W.make_case("cat", [parent] * 2, seed=31, Hk=2, Hv=4, d=128, in_dtype="bf16", alpha_lo=0.5, beta_uniform=True)
+    assert gram_eligible(c)
+    desc = ctx("gram").tree_desc(c.parent)
+    tab = desc.table("gram_groups").tolist()
+    assert tab[0] >= 5                                            # several groups
+    dc = DeviceCase(ctx("gram"), c)
+    dc.t("out").fill_(float("nan"))
+    dc.verify()
+    torch.cuda.synchronize()
+    o_ref, _, _ = oracle_scan_from_device(dc)
+    assert_close(dc.np("out"), o_ref, what="caterpillar, Gram form in groups")
+    dr = DeviceCase(ctx("rank1"), c)
+    dr.verify()
+    torch.cuda.synchronize()
+    assert_close(dr.np("out"), o_ref, what="caterpillar, rank-1")
+    ctx("auto")
+
+
 def test_off_path_poison_and_two_cycles():
     # poisoning nodes off the accepted path must leave the committed state bitwise unchanged
     c = W.make_case("p", [W.tree_tiny()], seed=4, Hk=2, Hv=4, d=128, in_dtype="bf16", accepted=[[0, 2, 6]])
