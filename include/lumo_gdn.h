@@ -151,6 +151,37 @@ int lumo_tree_path_from_node(lumo_ctx* ctx, const lumo_tree_desc* desc, const in
                              int lmax, int32_t* accepted_dev, int32_t* len_dev,
                              int32_t* status_dev, void* stream);
 
+/* ---- acceptance walk ---------------------------------------------------------------------
+ * The step between verify and commit (paper Algorithm 1, "Select one continuation": the accepted
+ * materialized path and the pending token from sampling with the target probabilities p and the
+ * proposal probabilities q; Sec. "One device-selected path drives native continuation": accepted
+ * node indices, path lengths, emitted tokens and the selected final row are device products).
+ * Starting at the pre-tree state the walk tries the children of the current node in ascending
+ * logical index.  mode 0, greedy: the child whose token equals argmax of the current target row is
+ * accepted (lowest token index on ties); otherwise the walk stops and the pending token is that
+ * argmax.  mode 1, rejection sampling (accepted mass min(p, q), residual mass proportional to
+ * (p - q)+, Appendix "Serving configuration and measurement"): child c with token x is accepted iff
+ * u_c q_c(x) < r(x) / Z with r the unnormalised residual target (p at first), Z its sum; a rejection
+ * replaces r by (r - Z q_c)+; when no child is accepted the pending token is argmax_i r_i / e_i over
+ * the caller's Exp(1) variates (an exact draw from r / Z), lowest index on ties.  All device pointers. */
+typedef struct {
+  int32_t V;               /* vocabulary size */
+  int32_t mode;            /* 0 greedy, 1 rejection sampling */
+  const int32_t* token;    /* [B, Ns] candidate token of each physical row */
+  const float* p_target;   /* [B, Ns+1, V] target probabilities after the node in physical row s;
+                              row Ns: after the pre-tree state */
+  const float* q_draft;    /* [B, Ns, V] proposal distribution the row's token was drawn from (mode 1) */
+  const float* uniforms;   /* [B, Ns] one U[0,1) number per physical row (mode 1) */
+  const float* noise;      /* [B, V] Exp(1) variates for the pending-token draw (mode 1) */
+  float* work;             /* [B, V] scratch for the residual (mode 1); contents undefined afterwards */
+} lumo_accept_args;
+/* accepted_dev [B, lmax] (-1 padded, root first), len_dev [B], next_token_dev [B] (the correction or
+ * bonus token: emitted, not yet materialised), final_node_dev [B] (last accepted node, -1 = none):
+ * the inputs of lumo_gdn_commit and of the next drafting step.  lmax >= tree depth.  Enqueues only. */
+int lumo_tree_accept(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_accept_args* args, int lmax,
+                     int32_t* accepted_dev, int32_t* len_dev, int32_t* next_token_dev,
+                     int32_t* final_node_dev, void* stream);
+
 /* ---- one GDN layer's tensors ----------------------------------------------------------- */
 typedef struct {
   int32_t Hk, Hv, d;

@@ -37,7 +37,7 @@ EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_s
            "lumo_ctx_timing_enable", "lumo_ctx_timing_read", "lumo_ctx_set_scan_algo", "lumo_ctx_set_overlap",
            "lumo_tree_desc_create", "lumo_tree_desc_destroy", "lumo_tree_desc_get",
            "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit",
-           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes"]
+           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_tree_accept"]
 
 
 class LumoError(RuntimeError):
@@ -63,6 +63,13 @@ class _Args(ctypes.Structure):
         ("snap_nodes", ctypes.c_void_p), ("snap_out", ctypes.c_void_p),
         ("status", ctypes.c_void_p),
     ]
+
+
+class _AcceptArgs(ctypes.Structure):
+    """Mirror of lumo_accept_args."""
+    _fields_ = [("V", ctypes.c_int32), ("mode", ctypes.c_int32), ("token", ctypes.c_void_p),
+                ("p_target", ctypes.c_void_p), ("q_draft", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
+                ("noise", ctypes.c_void_p), ("work", ctypes.c_void_p)]
 
 
 _lib.lumo_ctx_create.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
@@ -92,6 +99,8 @@ _lib.lumo_gdn_tree_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.P
 _lib.lumo_gdn_tree_scan_static.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
                                            ctypes.c_void_p]
 _lib.lumo_static_stack_bytes.restype = ctypes.c_int64
+_lib.lumo_tree_accept.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_AcceptArgs), ctypes.c_int,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.lumo_gdn_commit.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
 
@@ -188,6 +197,17 @@ class Context:
     @staticmethod
     def static_stack_bytes() -> int:
         return int(_lib.lumo_static_stack_bytes())
+
+    def accept(self, desc: "TreeDesc", *, token, p_target, accepted, length, next_token, final_node,
+               mode: str = "greedy", q_draft=None, uniforms=None, noise=None, work=None, stream=None):
+        """Acceptance walk on the device: fills accepted [B, lmax], length, next_token, final_node."""
+        a = _AcceptArgs()
+        a.V, a.mode = int(p_target.shape[-1]), {"greedy": 0, "rejection": 1}[mode]
+        for name, t in (("token", token), ("p_target", p_target), ("q_draft", q_draft), ("uniforms", uniforms),
+                        ("noise", noise), ("work", work)):
+            setattr(a, name, _ptr(t))
+        self._check(_lib.lumo_tree_accept(self._h, desc._h, ctypes.byref(a), int(accepted.shape[1]), _ptr(accepted),
+                                          _ptr(length), _ptr(next_token), _ptr(final_node), _stream(stream)))
 
     def commit(self, desc: "TreeDesc", layers, accepted: torch.Tensor, length: torch.Tensor, stream=None):
         arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)

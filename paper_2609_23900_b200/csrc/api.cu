@@ -118,6 +118,7 @@ bool use_overlap(const lumo_ctx* ctx, const Shape& s) {
 TreeDev tree_view(const lumo_tree_desc* d, int which) {
   TreeDev t;
   t.parent = d->d_parent; t.depth = d->d_depth; t.slot = d->d_slot; t.slot_inv = d->d_slot_inv;
+  t.child_off = d->d_child_off; t.child_list = d->d_child_list;
   t.win = d->d_win; t.conv_prog = d->d_conv_prog; t.sched = d->d_sched[which]; t.nops = d->d_nops[which];
   t.max_ops = d->max_ops[which]; t.max_levels = d->max_levels[which];
   t.tc_group = d->d_tc_group; t.tc_meta = d->d_tc_meta; t.tc_anc = d->d_tc_anc; t.tc_lvl = d->d_tc_lvl;
@@ -258,6 +259,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   const size_t o_parent = reserve((size_t)B * N), o_depth = reserve((size_t)B * N), o_slot = reserve((size_t)B * N);
   const size_t o_inv = reserve((size_t)B * Ns), o_win = reserve((size_t)B * Ns * 4);
   const size_t o_prog = reserve((size_t)B * Ns);
+  const size_t o_coff = reserve((size_t)B * (N + 2)), o_clist = reserve((size_t)B * N);
   size_t o_sched[2], o_nops[2];
   for (int w = 0; w < 2; ++w) { o_sched[w] = reserve((size_t)B * d->max_ops[w]); o_nops[w] = reserve(B); }
   for (int b = 0; b < B; ++b)
@@ -301,6 +303,8 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
         h[o_win + ((size_t)b * Ns + sidx) * 4 + j] = w;
       }
     }
+    for (int i = 0; i < N + 2; ++i) h[o_coff + (size_t)b * (N + 2) + i] = t.tab[LUMO_TAB_CHILD_OFF][i];
+    for (int i = 0; i < N; ++i) h[o_clist + (size_t)b * N + i] = t.tab[LUMO_TAB_CHILD_LIST][i];
     {
       // conv visiting order: depth-first preorder, so that most rows find three of their four taps
       // already in the registers of the thread that handled the previous row
@@ -363,6 +367,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   if (e != cudaSuccess) { cudaFree(d->dev); delete d; return cuda_fail(ctx, e, "cudaMemcpy(tree tables)"); }
   d->d_parent = d->dev + o_parent; d->d_depth = d->dev + o_depth; d->d_slot = d->dev + o_slot;
   d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_win; d->d_conv_prog = d->dev + o_prog;
+  d->d_child_off = d->dev + o_coff; d->d_child_list = d->dev + o_clist;
   for (int w = 0; w < 2; ++w) { d->d_sched[w] = d->dev + o_sched[w]; d->d_nops[w] = d->dev + o_nops[w]; }
   if (tc) {
     d->d_tc_group = d->dev + o_tc_group;
@@ -404,6 +409,28 @@ int lumo_tree_path_from_node(lumo_ctx* ctx, const lumo_tree_desc* desc, const in
                                  status_dev, st);
   });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "path_from_node launch");
+}
+
+int lumo_tree_accept(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_accept_args* a, int lmax,
+                     int32_t* accepted_dev, int32_t* len_dev, int32_t* next_token_dev, int32_t* final_node_dev,
+                     void* stream) {
+  if (!ctx || !desc || !a || !accepted_dev || !len_dev || !next_token_dev || !final_node_dev)
+    return fail(ctx, LUMO_ERR_ARG, "null argument");
+  if (desc->ctx != ctx) return fail(ctx, LUMO_ERR_ARG, "descriptor belongs to another context");
+  if (ctx->device < 0) return fail(ctx, LUMO_ERR_UNSUPPORTED, "host-only context cannot launch");
+  if (a->V < 1) return fail(ctx, LUMO_ERR_ARG, "V must be positive");
+  if (a->mode != 0 && a->mode != 1) return fail(ctx, LUMO_ERR_ARG, "mode must be 0 (greedy) or 1 (rejection sampling)");
+  if (lmax < desc->max_depth) return fail(ctx, LUMO_ERR_ARG, "lmax must be at least the tree depth");
+  if (!a->token || !a->p_target) return fail(ctx, LUMO_ERR_ARG, "token and p_target are required");
+  if (a->mode == 1 && (!a->q_draft || !a->uniforms || !a->noise || !a->work))
+    return fail(ctx, LUMO_ERR_ARG, "rejection sampling needs q_draft, uniforms, noise and work");
+  DeviceGuard g(ctx->device);
+  AcceptView v;
+  v.V = a->V; v.mode = a->mode; v.token = a->token; v.p_target = a->p_target; v.q_draft = a->q_draft;
+  v.uniforms = a->uniforms; v.noise = a->noise; v.work = a->work;
+  cudaError_t e = launch_accept(tree_view(desc, 0), desc->B, desc->N, desc->Ns, v, lmax, accepted_dev, len_dev,
+                                next_token_dev, final_node_dev, (cudaStream_t)stream);
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "accept launch");
 }
 
 int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers,

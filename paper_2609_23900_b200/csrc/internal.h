@@ -64,6 +64,8 @@ struct lumo_tree_desc {
   int32_t* d_slot = nullptr;      // [B, N]
   int32_t* d_slot_inv = nullptr;  // [B, Ns]
   int32_t* d_win = nullptr;       // [B, Ns, 4] per physical row: source rows (physical), -1/-2/-3 = history rows, INT32_MIN = padding row
+  int32_t* d_child_off = nullptr; // [B, N+2]
+  int32_t* d_child_list = nullptr;// [B, N]
   int32_t* d_conv_prog = nullptr; // [B, Ns] conv visiting order (depth first): physical row | flag << 16; flag 0 = fetch the whole
                                   // window, 1 = previous row is the parent (window slides), 2 = same parent as the previous row
                                   // (only the own row changes), 3 = padding row (zeros)
@@ -110,6 +112,7 @@ struct Shape {
 struct TreeDev {
   const int32_t* parent; const int32_t* depth; const int32_t* slot; const int32_t* slot_inv;
   const int32_t* win; const int32_t* conv_prog; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
+  const int32_t* child_off; const int32_t* child_list;   // [B, N+2] CSR (entry 0 = pre-tree state), [B, N]
   const int32_t* tc_group; const int32_t* tc_meta; const uint8_t* tc_anc; const uint8_t* tc_lvl; int n_groups;
 };
 
@@ -147,6 +150,14 @@ cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, 
                         int grid, cudaStream_t st);
 // persistent grid size (CTAs resident at once) and the stack scratch it needs
 cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes);
+// acceptance walk (accept.cu)
+struct AcceptView {
+  int V, mode;
+  const int32_t* token; const float* p_target; const float* q_draft; const float* uniforms; const float* noise;
+  float* work;
+};
+cudaError_t launch_accept(const TreeDev& t, int B, int N, int Ns, const AcceptView& a, int lmax, int32_t* accepted,
+                          int32_t* len, int32_t* next_token, int32_t* final_node, cudaStream_t st);
 // Gram-form scan on tcgen05 (scan_gram.cu)
 bool gram_supported(const Shape& s, int max_depth);
 cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
