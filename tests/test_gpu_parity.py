@@ -312,6 +312,32 @@ def test_gram_groups_with_long_prefix_paths():
     ctx("auto")
 
 
+def test_deep_tree_falls_back_to_rank1_and_wide_padding():
+    # depth 24 > 16: the automatic choice is the rank-1 kernel; the Gram form refuses it
+    deep = W.tree_chain(24) + [5, 5, 17, 23]
+    c = W.make_case("deep", [deep] * 2, seed=41, Hk=2, Hv=4, d=128, in_dtype="bf16", alpha_lo=0.5, beta_uniform=True)
+    assert not gram_eligible(c)
+    dc = DeviceCase(ctx("auto"), c)
+    dc.verify()
+    torch.cuda.synchronize()
+    assert_close(dc.np("out"), oracle_scan_from_device(dc)[0], what="depth 24, automatic kernel choice")
+    with pytest.raises(binding.LumoError):
+        DeviceCase(ctx("gram"), c).verify()
+    # 256 nodes scattered over 300 physical rows: padding rows are zero, every node is written once
+    wide = W.make_case("wide", rand_parents(9, 256, 1), seed=42, Hk=2, Hv=4, d=128, in_dtype="bf16", Ns=300,
+                       permute_slots=True, alpha_lo=0.5, beta_uniform=True)
+    dw = DeviceCase(ctx("auto"), wide)
+    dw.t("out").fill_(float("nan"))
+    dw.verify()
+    torch.cuda.synchronize()
+    o_ref, _, _ = oracle_scan_from_device(dw)
+    got = dw.np("out")
+    assert_close(got, o_ref, what="256 nodes in 300 rows")
+    pad = sorted(set(range(300)) - set(wide.slot[0].tolist()))
+    assert len(pad) == 44 and np.all(got[0, pad] == 0.0)
+    ctx("auto")
+
+
 def test_off_path_poison_and_two_cycles():
     # poisoning nodes off the accepted path must leave the committed state bitwise unchanged
     c = W.make_case("p", [W.tree_tiny()], seed=4, Hk=2, Hv=4, d=128, in_dtype="bf16", accepted=[[0, 2, 6]])
