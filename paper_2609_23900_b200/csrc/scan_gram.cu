@@ -265,9 +265,15 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     PROF(1);
     // ---- b. gates (consumed much later); K and Q rows -> swizzled operand tile (cp.async);
     //         first half of the pre-tree state rows -> registers -------------------------------------
+    // warp w takes rows w, w+8, ...; a warp reads one 512-byte row per instruction.  The state is not
+    // written by the kernel before this one, so its first half is requested ahead of the dependency wait.
+    const float* S0 = L.state + ((size_t)row * s.Hv + hv) * kD * kD;
+    float4 x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * u) * kD + lane * 4);
     // K, Q, V may still be in the making (the convolution runs right before this kernel): everything
-    // above touched only the descriptor tables.  The dependent kernel (commit) is let in afterwards:
-    // it reads freely and writes only behind its own wait.
+    // above touched only the descriptor tables and the state.  The dependent kernel (commit) is let in
+    // afterwards: it reads freely and writes only behind its own wait.
     pdl_wait();
     pdl_trigger();
     float gate_a = 1.f, gate_b = 0.f;
@@ -298,11 +304,6 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
       }
       asm volatile("cp.async.commit_group;\n" ::: "memory");
     }
-    // warp w takes rows w, w+8, ...; a warp reads one 512-byte row per instruction
-    const float* S0 = L.state + ((size_t)row * s.Hv + hv) * kD * kD;
-    float4 x[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * u) * kD + lane * 4);
     PROF(2);
     // ---- c. pre-tree state -> bf16 hi + lo operand tiles ------------------------------------------
     {
