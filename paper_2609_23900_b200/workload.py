@@ -165,8 +165,11 @@ def tree_mtp_spine(rs: IntStream, n: int = 16, spine: int = 4) -> List[int]:
 def tree_random(rs: IntStream, n: int, max_depth: int, max_children: int = 4) -> List[int]:
     """Frontier expansion: pop a uniformly random frontier node; if it is above
     ``max_depth`` give it U{1..max_children} children; stop at ``n`` nodes.
-    Restarts (continuing the same stream) if the frontier empties first."""
-    while True:
+    Restarts (continuing the same stream) if the frontier empties first; gives up with ValueError
+    when the shape cannot hold ``n`` nodes or after 1000 restarts."""
+    if sum(max_children ** k for k in range(1, max_depth + 1)) < n:
+        raise ValueError(f"a tree of depth <= {max_depth} with fan-out <= {max_children} cannot hold {n} nodes")
+    for _ in range(1000):
         parent: List[int] = []
         depth: List[int] = []
         frontier = [-1]
@@ -184,6 +187,7 @@ def tree_random(rs: IntStream, n: int, max_depth: int, max_children: int = 4) ->
                 frontier.append(len(parent) - 1)
         if len(parent) == n:
             return parent
+    raise ValueError("tree_random: the frontier kept emptying before the tree was full")
 
 
 def tree_paper_geometry() -> List[int]:

@@ -312,6 +312,55 @@ def test_gram_groups_with_long_prefix_paths():
     ctx("auto")
 
 
+def test_randomized_shapes_both_kernels():
+    """Seeded sweep over node counts around the 64-node group size, depths up to 16, padded and
+    permuted rows, head ratios and gate ranges: both scan kernels and the commit against the oracle."""
+    import random
+    rng = random.Random(2024)
+    for it in range(24):
+        N = rng.choice([1, 2, 31, 32, 33, 63, 64, 65, 100, 129, 255, 256])
+        B = rng.choice([1, 2])
+        kind = rng.choice(["frontier", "uniform_parent", "narrow"])
+        parents = []
+        for b in range(B):
+            if kind == "frontier":
+                parents.append(W.tree_random(W.IntStream(rng.getrandbits(40)), N, 9, max_children=rng.choice([4, 8])))
+            elif kind == "narrow":
+                parents.append(W.tree_random(W.IntStream(rng.getrandbits(40)), N, 16, max_children=3))
+            else:
+                par, dep = [], []
+                for i in range(N):
+                    while True:
+                        q = rng.randint(-1, i - 1)
+                        dq = 0 if q < 0 else dep[q]
+                        if dq < 16:
+                            break
+                    par.append(q)
+                    dep.append(dq + 1)
+                parents.append(par)
+        Ns = N + rng.choice([0, 0, 7])
+        Hk = rng.choice([1, 2])
+        c = W.make_case("rnd", parents, seed=rng.getrandbits(30), Hk=Hk, Hv=Hk * rng.choice([1, 2, 3]), d=128,
+                        in_dtype="bf16", Ns=Ns, permute_slots=True, alpha_lo=rng.choice([0.5, 0.9]),
+                        beta_uniform=rng.random() < 0.5, with_bias=rng.random() < 0.3)
+        use_conv = rng.random() < 0.5
+        ref = None
+        for algo in ("gram", "rank1"):
+            dc = DeviceCase(ctx(algo), c, use_conv=use_conv)
+            dc.t("out").fill_(float("nan"))
+            dc.verify()
+            dc.commit()
+            torch.cuda.synchronize()
+            if ref is None:
+                ref = (oracle_scan_from_device(dc)[0], oracle_commit_from_device(dc, with_hist=use_conv))
+            what = f"case {it} ({kind}, N={N}, Ns={Ns}, conv={use_conv}, {algo})"
+            assert assert_close(dc.np("out"), ref[0], what=what) < 1e-5
+            assert_close(dc.np("state"), ref[1][0], what=what + " committed state")
+            if use_conv:
+                assert np.array_equal(dc.np("conv_hist"), ref[1][1])
+    ctx("auto")
+
+
 def test_deep_tree_falls_back_to_rank1_and_wide_padding():
     # depth 24 > 16: the automatic choice is the rank-1 kernel; the Gram form refuses it
     deep = W.tree_chain(24) + [5, 5, 17, 23]
