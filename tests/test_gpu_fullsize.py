@@ -1,0 +1,68 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times (conv + scan with
+in-kernel q/k normalisation, bf16 outputs, then commit): the oracle is run on sampled (sequence,
+value head) pairs and sampled layers, one by one, on the operands the GPU recorded."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gdn_oracle as O
+from paper_2609_23900_b200 import workload as W
+from paper_2609_23900_b200.runtime import DeviceCase
+from tests.harness import assert_close, ctx
+
+pytestmark = pytest.mark.gpu
+
+
+def check_samples(dc, case, layer, pairs):
+    L = case.layers[layer]
+    rep = case.Hv // case.Hk
+    f = lambda name: dc.t(name, layer)
+    out = f("out")
+    state = f("state")
+    for b, h in pairs:
+        g = h // rep
+        sl = lambda t, hh: t[b:b + 1, :, hh:hh + 1].to(torch.float64).cpu().numpy()
+        q, k, v = sl(f("q"), g), sl(f("k"), g), sl(f("v"), h)
+        al, be = sl(f("alpha"), h), sl(f("beta"), h)
+        row = case.state_row[b:b + 1]
+        S0 = L.state[:, h:h + 1]
+        o_ref, _, _ = O.scan(case.parent[b:b + 1], case.slot[b:b + 1], row, q, k, v, al, be, S0, l2norm=True, threads=4)
+        assert_close(out[b, :, h].to(torch.float64).cpu().numpy(), o_ref[0, :, 0], bf16=True,
+                     what=f"{case.name} layer {layer} b={b} h={h} outputs")
+        st_ref, _, status, _ = O.commit(case.parent[b:b + 1], case.slot[b:b + 1], row, q, k, v, al, be, S0,
+                                        case.accepted[b:b + 1], case.accepted_len[b:b + 1], l2norm=True, threads=4)
+        assert status[0] == 0
+        assert_close(state[row[0], h].to(torch.float64).cpu().numpy(), st_ref[row[0], 0],
+                     what=f"{case.name} layer {layer} b={b} h={h} committed state")
+
+
+@pytest.mark.parametrize("shape", ["chains", "star", "random"])
+def test_config4_full_size_sampled(shape):
+    case = W.config4(shape)                       # batch 32, 256 nodes, 16/32 heads
+    dc = DeviceCase(ctx("auto"), case, out_dtype="bf16")
+    dc.verify()
+    dc.commit()
+    torch.cuda.synchronize()
+    assert dc.np("status").tolist() == [0] * case.B
+    rs = np.random.default_rng(4)
+    pairs = [(int(rs.integers(case.B)), int(rs.integers(case.Hv))) for _ in range(5)] + [(0, 0), (case.B - 1, case.Hv - 1)]
+    check_samples(dc, case, 0, pairs)
+    # properties that hold at any size: finite everywhere, rows of the pool that belong to nobody untouched
+    assert torch.isfinite(dc.t("out").float()).all()
+    other = sorted(set(range(case.rows)) - set(case.state_row.tolist()))
+    assert torch.equal(dc.t("state")[other].cpu(), torch.from_numpy(case.layers[0].state[other]))
+
+
+def test_config3_full_stack_sampled():
+    case = W.config3()                            # 48 layers, batch 4, 32 nodes
+    dc = DeviceCase(ctx("auto"), case, out_dtype="bf16")
+    dc.verify()
+    dc.commit()
+    torch.cuda.synchronize()
+    rs = np.random.default_rng(3)
+    for layer in (0, 23, 47):
+        assert dc.np("status", layer).tolist() == [0] * case.B
+        pairs = [(int(rs.integers(case.B)), int(rs.integers(case.Hv))) for _ in range(4)]
+        check_samples(dc, case, layer, pairs)
+    for layer in range(48):
+        assert torch.isfinite(dc.t("out", layer).float()).all()
