@@ -1,8 +1,9 @@
 // Device-resident acceptance walk: accepted path, its length, the pending token and the final row
 // as fixed-shape device products (paper Algorithm 1, "Select one continuation"; Sec. "One
 // device-selected path drives native continuation"), so that verify -> select -> commit needs no
-// host round trip.  One CTA per sequence walks from the pre-tree state through the children of the
-// current node in ascending logical index.
+// host round trip.  One thread-block cluster per sequence (the vocabulary is split over its CTAs,
+// partial results meet through distributed shared memory) walks from the pre-tree state through the
+// children of the current node in ascending logical index.
 //
 //   greedy     accept the child whose token equals argmax of the current target row (lowest token
 //              index on ties); otherwise stop, the pending token is that argmax.
@@ -14,137 +15,249 @@
 // Decisions that turn floats into integers use fixed precisions: the acceptance test and the residual
 // update in float64 (separate multiply and subtract, no contraction), the residual stored in float32,
 // the race keys as correctly rounded float32 quotients; sums are float64 in a fixed order.
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 
 #include "internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace lumo {
 
 namespace {
 
 constexpr int kAcceptThreads = 512;
+constexpr int kAcceptCluster = 8;       // CTAs per sequence: the vocabulary is split over a cluster
 
-__device__ double block_sum(double v, double* red) {
+// A CTA's partial result, read by its peers through distributed shared memory.
+struct ClusterSlot { double sum; float val; int idx; int flag; };
+
+// Visit this CTA's slice [lo, hi) of the vocabulary with kAcceptUnroll independent loads in flight per
+// thread; each thread sees its indices in ascending order.
+constexpr int kAcceptUnroll = 8;
+template <class Load, class Use>
+__device__ __forceinline__ void for_slice(int lo, int hi, Load load, Use use) {
+  for (int base = lo + (int)threadIdx.x; base < hi; base += kAcceptUnroll * kAcceptThreads) {
+    decltype(load(0)) vals[kAcceptUnroll];
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
-  __syncthreads();                       // red may still be read from the previous reduction
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-  __syncthreads();
-  double t = 0.0;
-  for (int w = 0; w < kAcceptThreads / 32; ++w) t += red[w];     // fixed order, every thread the same
-  return t;
+    for (int k = 0; k < kAcceptUnroll; ++k) {
+      const int i = base + k * kAcceptThreads;
+      if (i < hi) vals[k] = load(i);
+    }
+#pragma unroll
+    for (int k = 0; k < kAcceptUnroll; ++k) {
+      const int i = base + k * kAcceptThreads;
+      if (i < hi) use(i, vals[k]);
+    }
+  }
 }
 
-// argmax with the lowest index on ties; every thread returns the result
-__device__ int block_argmax(float v, int i, float* redv, int* redi) {
+// Cluster-wide reductions.  Each CTA reduces its slice, publishes the partial in one of two alternating
+// slots of its shared memory, and after one cluster barrier warp 0 of every CTA combines all partials
+// with the same shuffle tree, so all CTAs reach bit-identical results and take the same branches.  The
+// slot written in reduction k is next written in reduction k + 2, i.e. after the barrier of reduction
+// k + 1, which no CTA passes before it has read slot k.
+struct Exchange {
+  double red[kAcceptThreads / 32];
+  float redv[kAcceptThreads / 32];
+  int redi[kAcceptThreads / 32];
+  ClusterSlot slot[2];
+  ClusterSlot result;
+  int parity;
+};
+
+__device__ double cluster_sum(cg::cluster_group& cl, double v, Exchange* x) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_down_sync(0xffffffffu, v, o);
-    const int oi = __shfl_down_sync(0xffffffffu, i, o);
-    if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if (lane == 0) x->red[warp] = v;
+  __syncthreads();
+  const int par = x->parity;
+  if (warp == 0) {
+    double t = lane < kAcceptThreads / 32 ? x->red[lane] : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (lane == 0) x->slot[par].sum = t;
+  }
+  cl.sync();
+  if (warp == 0) {
+    double t = lane < (int)cl.num_blocks() ? cl.map_shared_rank(&x->slot[par], lane)->sum : 0.0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (lane == 0) { x->result.sum = t; x->parity = par ^ 1; }
   }
   __syncthreads();
-  if ((threadIdx.x & 31) == 0) { redv[threadIdx.x >> 5] = v; redi[threadIdx.x >> 5] = i; }
+  return x->result.sum;
+}
+
+__device__ __forceinline__ void argmax_step(float& v, int& i, int o) {
+  const float ov = __shfl_xor_sync(0xffffffffu, v, o);
+  const int oi = __shfl_xor_sync(0xffffffffu, i, o);
+  if (ov > v || (ov == v && oi < i)) { v = ov; i = oi; }
+}
+
+// argmax with the lowest index on ties over the whole cluster; every thread returns the result
+__device__ int cluster_argmax(cg::cluster_group& cl, float v, int i, Exchange* x) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) argmax_step(v, i, o);
+  if (lane == 0) { x->redv[warp] = v; x->redi[warp] = i; }
   __syncthreads();
-  float bv = redv[0];
-  int bi = redi[0];
-  for (int w = 1; w < kAcceptThreads / 32; ++w)
-    if (redv[w] > bv || (redv[w] == bv && redi[w] < bi)) { bv = redv[w]; bi = redi[w]; }
-  return bi;
+  const int par = x->parity;
+  if (warp == 0) {
+    float bv = lane < kAcceptThreads / 32 ? x->redv[lane] : -2.f;
+    int bi = lane < kAcceptThreads / 32 ? x->redi[lane] : 0x7fffffff;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) argmax_step(bv, bi, o);
+    if (lane == 0) { x->slot[par].val = bv; x->slot[par].idx = bi; }
+  }
+  cl.sync();
+  if (warp == 0) {
+    float bv = -2.f;
+    int bi = 0x7fffffff;
+    if (lane < (int)cl.num_blocks()) {
+      const ClusterSlot* o = cl.map_shared_rank(&x->slot[par], lane);
+      bv = o->val;
+      bi = o->idx;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) argmax_step(bv, bi, o);
+    if (lane == 0) { x->result.idx = bi; x->parity = par ^ 1; }
+  }
+  __syncthreads();
+  return x->result.idx;
 }
 
 __global__ void __launch_bounds__(kAcceptThreads)
 accept_kernel(TreeDev t, int N, int Ns, AcceptView a, int lmax, int32_t* __restrict__ accepted,
               int32_t* __restrict__ len_out, int32_t* __restrict__ next_token, int32_t* __restrict__ final_node) {
-  __shared__ double red[kAcceptThreads / 32];
-  __shared__ float redv[kAcceptThreads / 32];
-  __shared__ int redi[kAcceptThreads / 32];
-  __shared__ int s_take;
-  const int b = blockIdx.x, tid = threadIdx.x, V = a.V;
-  const int32_t* parent_child_off = t.child_off + (size_t)b * (N + 2);
-  const int32_t* child_list = t.child_list + (size_t)b * N;
-  const int32_t* slot = t.slot + (size_t)b * N;
-  const int32_t* token = a.token + (size_t)b * Ns;
+  // this sequence's tree, staged once: the walk's dependent lookups then stay on chip
+  __shared__ int32_t parent_child_off[kMaxNodes + 2], child_list[kMaxNodes], slot_map[kMaxNodes], tok_of_node[kMaxNodes];
+  __shared__ Exchange xch;
+  cg::cluster_group cl = cg::this_cluster();
+  const int rank = (int)cl.block_rank(), nblk = (int)cl.num_blocks();
+  const int b = blockIdx.y, tid = threadIdx.x, V = a.V;
+  // this CTA's slice of the vocabulary
+  const int chunk = (V + nblk - 1) / nblk;
+  const int v_lo = rank * chunk, v_hi = min(V, v_lo + chunk);
+  for (int e = tid; e < N + 2; e += kAcceptThreads) parent_child_off[e] = t.child_off[(size_t)b * (N + 2) + e];
+  for (int e = tid; e < N; e += kAcceptThreads) {
+    child_list[e] = t.child_list[(size_t)b * N + e];
+    const int row = t.slot[(size_t)b * N + e];
+    slot_map[e] = row;
+    tok_of_node[e] = a.token[(size_t)b * Ns + row];
+  }
+  if (tid == 0) xch.parity = 0;
+  __syncthreads();
   float* r = a.work + (size_t)b * V;
   int32_t* acc = accepted + (size_t)b * lmax;
-  for (int e = tid; e < lmax; e += kAcceptThreads) acc[e] = -1;
+  if (rank == 0)
+    for (int e = tid; e < lmax; e += kAcceptThreads) acc[e] = -1;
   int cur = -1, len = 0, nxt = 0;
 
   for (int step = 0; step <= lmax; ++step) {                 // bounded: a path has at most lmax nodes
-    const int prow = cur < 0 ? Ns : slot[cur];
+    const int prow = cur < 0 ? Ns : slot_map[cur];
     const float* p = a.p_target + ((size_t)b * (Ns + 1) + prow) * V;
     const int c_lo = parent_child_off[cur + 1], c_hi = parent_child_off[cur + 2];
     int took = -1;
     if (a.mode == 0) {
       float bv = -1.f;
       int bi = 0x7fffffff;
-      for (int i = tid; i < V; i += kAcceptThreads) {         // strided, ascending per thread
-        const float v = p[i];
-        if (v > bv) { bv = v; bi = i; }
-      }
-      nxt = block_argmax(bv, bi, redv, redi);
+      for_slice(v_lo, v_hi, [&](int i) { return p[i]; },
+                [&](int i, float v) { if (v > bv) { bv = v; bi = i; } });
+      nxt = cluster_argmax(cl, bv, bi, &xch);
       if (len < lmax)
         for (int ci = c_lo; ci < c_hi; ++ci) {                // bounded: children of one node
           const int c = child_list[ci];
-          if (token[slot[c]] == nxt) { took = c; break; }
+          if (tok_of_node[c] == nxt) { took = c; break; }
         }
     } else {
       double zp = 0.0;
-      for (int i = tid; i < V; i += kAcceptThreads) { const float v = p[i]; r[i] = v; zp += (double)v; }
-      double Z = block_sum(zp, red);
+      for_slice(v_lo, v_hi, [&](int i) { return p[i]; }, [&](int i, float v) { r[i] = v; zp += (double)v; });
+      double Z = cluster_sum(cl, zp, &xch);            // its cluster barriers also publish r
       for (int ci = c_lo; ci < c_hi && len < lmax; ++ci) {    // bounded: children of one node
         const int c = child_list[ci];
-        const int sc = slot[c];
-        const int x = token[sc];
+        const int sc = slot_map[c];
+        const int x = tok_of_node[c];
         const float* q = a.q_draft + ((size_t)b * Ns + sc) * V;
-        __syncthreads();                                       // r is complete
-        if (tid == 0) {
-          const double lhs = __dmul_rn(__dmul_rn((double)a.uniforms[(size_t)b * Ns + sc], (double)q[x]), Z);
-          s_take = lhs < (double)r[x];
-        }
-        __syncthreads();
-        if (s_take) { took = c; break; }
+        // every CTA evaluates the same test on the same values (r[x] was published by a cluster barrier)
+        const double lhs = __dmul_rn(__dmul_rn((double)a.uniforms[(size_t)b * Ns + sc], (double)q[x]), Z);
+        const float rx = *reinterpret_cast<volatile const float*>(r + x);
+        cl.sync();                                             // everyone has read r[x] before it changes
+        if (lhs < (double)rx) { took = c; break; }
         double zn = 0.0;
-        for (int i = tid; i < V; i += kAcceptThreads) {
-          const double d = __dsub_rn((double)r[i], __dmul_rn(Z, (double)q[i]));
-          const float rn = (float)(d > 0.0 ? d : 0.0);
-          r[i] = rn;
-          zn += (double)rn;
-        }
-        const double Zn = block_sum(zn, red);
+        for_slice(v_lo, v_hi, [&](int i) { return make_float2(r[i], q[i]); },
+                  [&](int i, float2 rq) {
+                    const double d = __dsub_rn((double)rq.x, __dmul_rn(Z, (double)rq.y));
+                    const float rn = (float)(d > 0.0 ? d : 0.0);
+                    r[i] = rn;
+                    zn += (double)rn;
+                  });
+        const double Zn = cluster_sum(cl, zn, &xch);
         if (Zn > 0.0) Z = Zn;
         else {                                                 // empty residual: restore the target row
           double z2 = 0.0;
-          for (int i = tid; i < V; i += kAcceptThreads) { const float v = p[i]; r[i] = v; z2 += (double)v; }
-          Z = block_sum(z2, red);
+          for_slice(v_lo, v_hi, [&](int i) { return p[i]; }, [&](int i, float v) { r[i] = v; z2 += (double)v; });
+          Z = cluster_sum(cl, z2, &xch);
         }
       }
       if (took < 0) {                                          // draw the pending token from r / Z
-        __syncthreads();
         const float* noise = a.noise + (size_t)b * V;
         float bv = -1.f;
         int bi = 0x7fffffff;
-        for (int i = tid; i < V; i += kAcceptThreads) {
-          const float key = __fdiv_rn(r[i], noise[i]);
-          if (key > bv) { bv = key; bi = i; }
-        }
-        nxt = block_argmax(bv, bi, redv, redi);
+        for_slice(v_lo, v_hi, [&](int i) { return make_float2(r[i], noise[i]); },   // own slice of r
+                  [&](int i, float2 rn) {
+                    const float key = __fdiv_rn(rn.x, rn.y);
+                    if (key > bv) { bv = key; bi = i; }
+                  });
+        nxt = cluster_argmax(cl, bv, bi, &xch);
       }
     }
-    if (took < 0) break;                                       // uniform over the CTA
-    if (tid == 0) acc[len] = took;
+    if (took < 0) break;                                       // uniform over the cluster
+    if (rank == 0 && tid == 0) acc[len] = took;
     cur = took;
     ++len;
   }
-  if (tid == 0) { len_out[b] = len; next_token[b] = nxt; final_node[b] = cur; }
+  if (rank == 0 && tid == 0) { len_out[b] = len; next_token[b] = nxt; final_node[b] = cur; }
+  cl.sync();                                                   // no CTA leaves while a peer may still read its slots
 }
 
 }  // namespace
 
 cudaError_t launch_accept(const TreeDev& t, int B, int N, int Ns, const AcceptView& a, int lmax, int32_t* accepted,
                           int32_t* len, int32_t* next_token, int32_t* final_node, cudaStream_t st) {
-  accept_kernel<<<B, kAcceptThreads, 0, st>>>(t, N, Ns, a, lmax, accepted, len, next_token, final_node);
-  return cudaGetLastError();
+  // largest cluster this device schedules, found once per device (16 CTAs needs the opt-in attribute)
+  static int max_cluster[64] = {};
+  int dev = 0, sms = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  cfg.blockDim = dim3(kAcceptThreads);
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  if (dev >= 0 && dev < 64 && max_cluster[dev] == 0) {
+    int c = cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess
+                ? 16 : kAcceptCluster;
+    for (; c > 1; c >>= 1) {                               // bounded: at most four sizes
+      int fit = 0;
+      cfg.gridDim = dim3(c, 1);
+      attr[0].val.clusterDim.x = c;
+      if (cudaOccupancyMaxActiveClusters(&fit, accept_kernel, &cfg) == cudaSuccess && fit > 0) break;
+    }
+    (void)cudaGetLastError();
+    max_cluster[dev] = c;
+  }
+  int cluster = (dev >= 0 && dev < 64) ? max_cluster[dev] : 1;
+  if (cluster > kAcceptCluster && B * cluster > sms) cluster = kAcceptCluster;   // many sequences: smaller clusters
+  while (cluster > 1 && a.V < cluster * kAcceptThreads) cluster >>= 1;           // small vocabularies
+  cfg.gridDim = dim3(cluster, B);
+  attr[0].val.clusterDim.x = cluster;
+  return cudaLaunchKernelEx(&cfg, accept_kernel, t, N, Ns, a, lmax, accepted, len, next_token, final_node);
 }
 
 }  // namespace lumo

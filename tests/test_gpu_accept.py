@@ -48,7 +48,7 @@ def run_device(desc, Ns, token, p, q, u, noise, mode, lmax):
 
 
 @pytest.mark.parametrize("mode", ["greedy", "rejection"])
-@pytest.mark.parametrize("shape", ["tiny", "cfg2", "paper", "star"])
+@pytest.mark.parametrize("shape", ["tiny", "cfg2", "paper", "star", "chains"])
 def test_accept_matches_oracle_bit_exactly(mode, shape):
     if shape == "tiny":
         c, V = W.make_case("t", [W.tree_tiny()] * 3, seed=1, Hk=1, Hv=1, d=64, in_dtype="f32"), 37
@@ -56,9 +56,11 @@ def test_accept_matches_oracle_bit_exactly(mode, shape):
         c, V = W.config2(B=4), 4099
     elif shape == "paper":
         c, V = W.config_paper(B=3), 32000
+    elif shape == "chains":  # the largest tree; a vocabulary that does not divide over the cluster
+        c, V = W.make_case("w", [W.tree_chains(32, 8)] * 2, seed=3, Hk=1, Hv=1, d=64, in_dtype="f32"), 8191
     else:
         c, V = W.make_case("s", [W.tree_star(40)] * 2, seed=2, Hk=1, Hv=1, d=64, in_dtype="f32", Ns=48, permute_slots=True), 1000
-    token, p, q, u, noise = make_inputs(c.parent, c.slot, c.Ns, V, seed={"tiny": 11, "cfg2": 12, "paper": 13, "star": 14}[shape])
+    token, p, q, u, noise = make_inputs(c.parent, c.slot, c.Ns, V, seed={"tiny": 11, "cfg2": 12, "paper": 13, "star": 14, "chains": 15}[shape])
     lmax = max(max(W.tree_depths(pp.tolist())) for pp in c.parent) + 1
     desc = ctx().tree_desc(c.parent, slot=c.slot, n_slots=c.Ns)
     acc, ln, nxt, fin = run_device(desc, c.Ns, token, p, q, u, noise, mode, lmax)
