@@ -470,19 +470,26 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
         op.cq = *reinterpret_cast<const float4*>(rec.wq);
         op.ao = *reinterpret_cast<const uint2*>(rec.aoff);
       };
+      // packed fp32 FMAs (two correctly rounded fp32 lanes per instruction: same bits as scalar fmaf)
       auto block4 = [&](float4& acc, float4& o, const float4& ck, const float4& cq, const uint2& ao) {
         const float4 d0 = *reinterpret_cast<const float4*>(dls + (ao.x & 0xFFFFu) + 4 * lane);
         const float4 d1 = *reinterpret_cast<const float4*>(dls + (ao.x >> 16) + 4 * lane);
         const float4 d2 = *reinterpret_cast<const float4*>(dls + (ao.y & 0xFFFFu) + 4 * lane);
         const float4 d3 = *reinterpret_cast<const float4*>(dls + (ao.y >> 16) + 4 * lane);
-        acc.x = fmaf(ck.x, d0.x, acc.x); acc.y = fmaf(ck.x, d0.y, acc.y); acc.z = fmaf(ck.x, d0.z, acc.z); acc.w = fmaf(ck.x, d0.w, acc.w);
-        o.x = fmaf(cq.x, d0.x, o.x); o.y = fmaf(cq.x, d0.y, o.y); o.z = fmaf(cq.x, d0.z, o.z); o.w = fmaf(cq.x, d0.w, o.w);
-        acc.x = fmaf(ck.y, d1.x, acc.x); acc.y = fmaf(ck.y, d1.y, acc.y); acc.z = fmaf(ck.y, d1.z, acc.z); acc.w = fmaf(ck.y, d1.w, acc.w);
-        o.x = fmaf(cq.y, d1.x, o.x); o.y = fmaf(cq.y, d1.y, o.y); o.z = fmaf(cq.y, d1.z, o.z); o.w = fmaf(cq.y, d1.w, o.w);
-        acc.x = fmaf(ck.z, d2.x, acc.x); acc.y = fmaf(ck.z, d2.y, acc.y); acc.z = fmaf(ck.z, d2.z, acc.z); acc.w = fmaf(ck.z, d2.w, acc.w);
-        o.x = fmaf(cq.z, d2.x, o.x); o.y = fmaf(cq.z, d2.y, o.y); o.z = fmaf(cq.z, d2.z, o.z); o.w = fmaf(cq.z, d2.w, o.w);
-        acc.x = fmaf(ck.w, d3.x, acc.x); acc.y = fmaf(ck.w, d3.y, acc.y); acc.z = fmaf(ck.w, d3.z, acc.z); acc.w = fmaf(ck.w, d3.w, acc.w);
-        o.x = fmaf(cq.w, d3.x, o.x); o.y = fmaf(cq.w, d3.y, o.y); o.z = fmaf(cq.w, d3.z, o.z); o.w = fmaf(cq.w, d3.w, o.w);
+        float2 a01 = make_float2(acc.x, acc.y), a23 = make_float2(acc.z, acc.w);
+        float2 o01 = make_float2(o.x, o.y), o23 = make_float2(o.z, o.w);
+        auto step = [&](float k, float q, const float4& dd) {
+          const float2 kk = make_float2(k, k), qq = make_float2(q, q);
+          const float2 lo2 = make_float2(dd.x, dd.y), hi2 = make_float2(dd.z, dd.w);
+          a01 = __ffma2_rn(kk, lo2, a01); a23 = __ffma2_rn(kk, hi2, a23);
+          o01 = __ffma2_rn(qq, lo2, o01); o23 = __ffma2_rn(qq, hi2, o23);
+        };
+        step(ck.x, cq.x, d0);
+        step(ck.y, cq.y, d1);
+        step(ck.z, cq.z, d2);
+        step(ck.w, cq.w, d3);
+        acc = make_float4(a01.x, a01.y, a23.x, a23.y);
+        o = make_float4(o01.x, o01.y, o23.x, o23.y);
       };
       const int lvl_lane = sm.lvl[lane < 20 ? lane : 19];          // lane d holds lvl[d]
       NodeOps op;
