@@ -90,27 +90,25 @@ __device__ int check_path_staged(const int* acc, const int* par, int N, int len,
 // a1: ancestry-gathered causal depthwise conv (width 4) + SiLU -> recorded operands
 // ---------------------------------------------------------------------------------------
 // A CTA owns kConvRows consecutive entries of one sequence's visiting order (depth-first, built on
-// the host) and a slab of 256 x kVec channels; a thread keeps the packed taps of its channels and the
-// current 4-row window in registers.  In depth-first order most rows either follow their parent (the
-// window slides by one) or share the parent of the previous row (only the own row changes), so one
-// 16-byte load per row replaces four; the own rows of the next two entries are always in flight.
-// Windows that cannot be derived come from the per-row table (physical rows, or -1..-3 for the
-// history rows).  Taps are applied oldest first in fp32 starting from zero, bias last, SiLU in fp32,
-// one round-to-nearest-even cast (Sec. "Precompute branch histories while preserving arithmetic":
-// tap order and cast points are part of the result).
-constexpr int kConvRows = 8;
+// the host) and a slab of 256 x 4 channels; a thread keeps the taps (as pairs of neighbouring
+// channels), the bias and the current 4-row window of its channels unpacked in fp32 registers.  In
+// depth-first order most rows either follow their parent (the window slides by one) or share the
+// parent of the previous row (only the own row changes), so one load per row replaces four; the own
+// rows of the next eight entries are always in flight (the kernel is bound by the special-function
+// unit, two operations per element for the SiLU, and by load latency, not by bandwidth).  Windows
+// that cannot be derived come from the per-row table (physical rows, or -1..-3 for the history rows).
+// Taps are applied oldest first in fp32 starting from zero (packed FMAs: two correctly rounded fp32
+// lanes per instruction, same bits as scalar fmaf), bias last, SiLU in fp32, one round-to-nearest-even
+// cast (Sec. "Precompute branch histories while preserving arithmetic": tap order and cast points are
+// part of the result).
 
-template <typename T> struct PackedW;      // the 4 taps of one channel as loaded
-template <> struct PackedW<float> { using type = float4; };
-template <> struct PackedW<__nv_bfloat16> { using type = uint2; };
-
-template <typename T, int kVec>
+template <typename T, int kConvRows>
 __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerBatch lb) {
   __shared__ int s_win[kConvRows][4];
   __shared__ int s_prog[kConvRows];
   const int layer = blockIdx.z / s.B, b = blockIdx.z % s.B;
   const int e0 = blockIdx.y * kConvRows;               // first entry of the visiting order
-  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * kVec;
+  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   const LayerPtrs& L = lb.l[layer];
   pdl_wait();       // x, history and the operand buffers belong to earlier kernels until here
   pdl_trigger();
@@ -127,19 +125,28 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
     s_win[r][j] = w;
     if (j == 0) s_prog[r] = (e0 + r < s.Ns) ? prog : -1;
   }
-  using PW = typename PackedW<T>::type;
-  using P4 = typename Packed4<T>::type;
-  using Raw = uint4;                                   // 16 bytes = kVec elements
-  PW wpk[kVec];                                        // weights stay packed in registers
+  using P4 = typename Packed4<T>::type;                // four elements as loaded
+  float2 wp[4][2];                                     // tap j of channel pairs (0,1) and (2,3)
+  float2 bp[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
   if (c0 < s.C) {
     const T* w = reinterpret_cast<const T*>(L.conv_w) + (size_t)c0 * 4;
+    float4 wc[4];
 #pragma unroll
-    for (int e = 0; e < kVec; ++e) wpk[e] = *reinterpret_cast<const PW*>(w + e * 4);
+    for (int e = 0; e < 4; ++e) wc[e] = Packed4<T>::unpack(*reinterpret_cast<const P4*>(w + e * 4));
+    wp[0][0] = make_float2(wc[0].x, wc[1].x); wp[0][1] = make_float2(wc[2].x, wc[3].x);
+    wp[1][0] = make_float2(wc[0].y, wc[1].y); wp[1][1] = make_float2(wc[2].y, wc[3].y);
+    wp[2][0] = make_float2(wc[0].z, wc[1].z); wp[2][1] = make_float2(wc[2].z, wc[3].z);
+    wp[3][0] = make_float2(wc[0].w, wc[1].w); wp[3][1] = make_float2(wc[2].w, wc[3].w);
+    if (L.conv_b) {
+      const float4 bv = Packed4<T>::unpack(*reinterpret_cast<const P4*>(reinterpret_cast<const T*>(L.conv_b) + c0));
+      bp[0] = make_float2(bv.x, bv.y);
+      bp[1] = make_float2(bv.z, bv.w);
+    }
   }
   __syncthreads();
   if (c0 >= s.C) return;
+  const bool has_bias = L.conv_b != nullptr;
   const int hkd = s.Hk * s.d;
-  // destination of this channel group inside [q | k | v]
   T* dst;
   size_t dst_stride;
   if (c0 < hkd) { dst = reinterpret_cast<T*>(L.q) + c0; dst_stride = hkd; }
@@ -148,19 +155,22 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
   dst += (size_t)b * s.Ns * dst_stride;
   const T* x = reinterpret_cast<const T*>(L.x) + (size_t)b * s.Ns * s.C + c0;
   const T* hist = reinterpret_cast<const T*>(L.conv_hist) + (size_t)(seq_ok ? row : 0) * 3 * s.C + c0;
-  const T* bias = L.conv_b ? reinterpret_cast<const T*>(L.conv_b) + c0 : nullptr;
 
-  auto load_src = [&](int wj) -> Raw {                 // one window entry: a row of x or of the history
+  auto load_src = [&](int wj) -> float4 {              // one window entry: a row of x or of the history
     const T* src = wj >= 0 ? x + (size_t)wj * s.C : hist + (size_t)(3 + wj) * s.C;
-    return *reinterpret_cast<const Raw*>(src);
+    return Packed4<T>::unpack(*reinterpret_cast<const P4*>(src));
   };
-  auto load_own = [&](int r) -> Raw {                  // the entry's own row (padding rows: zeros)
+  auto load_own = [&](int r) -> P4 {                   // the entry's own row (padding rows: zeros)
     const int prog = r < kConvRows ? s_prog[r] : -1;
-    if (prog < 0 || (prog >> 16) == 3) return make_uint4(0, 0, 0, 0);
-    return *reinterpret_cast<const Raw*>(x + (size_t)(prog & 0xFFFF) * s.C);
+    P4 z = {};
+    if (prog < 0 || (prog >> 16) == 3) return z;
+    return *reinterpret_cast<const P4*>(x + (size_t)(prog & 0xFFFF) * s.C);
   };
-  Raw win[4] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
-  Raw pf[2] = {load_own(0), load_own(1)};
+  float4 win[4] = {};
+  constexpr int kAhead = sizeof(T) == 2 ? (kConvRows < 8 ? kConvRows : 8) : 4;   // own rows in flight (a register budget)
+  P4 pf[kAhead];
+#pragma unroll
+  for (int r = 0; r < kAhead; ++r) pf[r] = load_own(r);
 #pragma unroll
   for (int r = 0; r < kConvRows; ++r) {                // bounded: kConvRows
     const int prog = s_prog[r];
@@ -168,50 +178,28 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
     const int ps = prog & 0xFFFF;
     int flag = prog >> 16;
     if (r == 0 && flag != 3) flag = 0;                 // the first row of a CTA has nothing to reuse
-    const Raw own = pf[r & 1];
-    pf[r & 1] = load_own(r + 2);                       // keeps two own rows in flight
-    float y[kVec];
-#pragma unroll
-    for (int e = 0; e < kVec; ++e) y[e] = 0.f;
+    const float4 own = Packed4<T>::unpack(pf[r % kAhead]);
+    pf[r % kAhead] = load_own(r + kAhead);
+    float y[4] = {0.f, 0.f, 0.f, 0.f};
     if (flag != 3) {
       if (flag == 0) { win[0] = load_src(s_win[r][0]); win[1] = load_src(s_win[r][1]); win[2] = load_src(s_win[r][2]); }
       else if (flag == 1) { win[0] = win[1]; win[1] = win[2]; win[2] = win[3]; }
       win[3] = own;
+      float2 y01 = make_float2(0.f, 0.f), y23 = make_float2(0.f, 0.f);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {                    // oldest -> newest
-        const P4* xp = reinterpret_cast<const P4*>(&win[j]);
-#pragma unroll
-        for (int e4 = 0; e4 < kVec / 4; ++e4) {
-          const float4 xv = Packed4<T>::unpack(xp[e4]);
-          const float xs[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float4 wv = Packed4<T>::unpack(*reinterpret_cast<const P4*>(&wpk[e4 * 4 + e]));
-            const float wj = j == 0 ? wv.x : (j == 1 ? wv.y : (j == 2 ? wv.z : wv.w));
-            y[e4 * 4 + e] = fmaf(wj, xs[e], y[e4 * 4 + e]);
-          }
-        }
+        y01 = __ffma2_rn(wp[j][0], make_float2(win[j].x, win[j].y), y01);
+        y23 = __ffma2_rn(wp[j][1], make_float2(win[j].z, win[j].w), y23);
       }
+      if (has_bias) { y01 = __fadd2_rn(y01, bp[0]); y23 = __fadd2_rn(y23, bp[1]); }   // bias last
+      y[0] = y01.x; y[1] = y01.y; y[2] = y23.x; y[3] = y23.y;
 #pragma unroll
-      for (int e = 0; e < kVec; ++e) {
-        float a = y[e];
-        if (bias) {                                    // bias last
-          if constexpr (sizeof(T) == 2) a += __bfloat162float(bias[e]); else a += bias[e];
-        }
-        // SiLU with the hardware exponential and reciprocal: ~1e-6 relative error, far below the
-        // rounding of the recorded operand
-        y[e] = __fdividef(a, 1.f + __expf(-a));
-      }
+      for (int e = 0; e < 4; ++e) y[e] = __fdividef(y[e], 1.f + __expf(-y[e]));        // SiLU
     }
     T* d = dst + (size_t)ps * dst_stride;
     if constexpr (sizeof(T) == 2) {
-      uint32_t pk[kVec / 2];
-#pragma unroll
-      for (int e = 0; e < kVec / 2; ++e) {
-        __nv_bfloat162 h2 = __floats2bfloat162_rn(y[2 * e], y[2 * e + 1]);
-        pk[e] = *reinterpret_cast<uint32_t*>(&h2);
-      }
-      *reinterpret_cast<uint4*>(d) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+      __nv_bfloat162 h01 = __floats2bfloat162_rn(y[0], y[1]), h23 = __floats2bfloat162_rn(y[2], y[3]);
+      *reinterpret_cast<uint2*>(d) = make_uint2(*reinterpret_cast<uint32_t*>(&h01), *reinterpret_cast<uint32_t*>(&h23));
     } else {
       *reinterpret_cast<float4*>(d) = make_float4(y[0], y[1], y[2], y[3]);
     }
@@ -621,15 +609,25 @@ cudaError_t dispatch(int d, int in_dtype, F f) {
 // ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
+template <typename T>
+static cudaError_t launch_conv_t(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st) {
+  // sixteen entries per CTA amortise the window set-up; small launches take fewer so that the grid
+  // still covers the GPU
+  const int slabs = (s.C / 4 + 255) / 256, seqs = s.B * s.n_layers;
+  auto ctas = [&](int rows) { return (long long)slabs * ((s.Ns + rows - 1) / rows) * seqs; };
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (ctas(16) >= 2LL * sms)
+    return launch_kernel(conv_kernel<T, 16>, dim3(slabs, (s.Ns + 15) / 16, seqs), dim3(256), 0, st, pdl, s, t, lb);
+  if (ctas(8) >= 2LL * sms)
+    return launch_kernel(conv_kernel<T, 8>, dim3(slabs, (s.Ns + 7) / 8, seqs), dim3(256), 0, st, pdl, s, t, lb);
+  return launch_kernel(conv_kernel<T, 4>, dim3(slabs, (s.Ns + 3) / 4, seqs), dim3(256), 0, st, pdl, s, t, lb);
+}
+
 cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st) {
-  if (s.in_dtype == LUMO_BF16) {
-    dim3 grid((s.C / 8 + 255) / 256, (s.Ns + kConvRows - 1) / kConvRows, s.B * s.n_layers);
-    return launch_kernel(conv_kernel<__nv_bfloat16, 8>, grid, dim3(256), 0, st, pdl, s, t, lb);
-  } else {
-    dim3 grid((s.C / 4 + 255) / 256, (s.Ns + kConvRows - 1) / kConvRows, s.B * s.n_layers);
-    return launch_kernel(conv_kernel<float, 4>, grid, dim3(256), 0, st, pdl, s, t, lb);
-  }
-  return cudaGetLastError();
+  if (s.in_dtype == LUMO_BF16) return launch_conv_t<__nv_bfloat16>(s, t, lb, pdl, st);
+  return launch_conv_t<float>(s, t, lb, pdl, st);
 }
 
 cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes) {
