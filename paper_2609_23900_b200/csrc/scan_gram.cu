@@ -250,6 +250,13 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     if (first_group && L.status && hv == 0 && tid == 0) L.status[b] = LUMO_SEQ_OK;
 
     PROF(0);
+    // The pre-tree state is not written by the kernel before this one and its address needs no
+    // table: its first half (warp w takes rows w, w+8, ...; one 512-byte row per instruction) is
+    // requested first of all, ahead of the table loads and of the dependency wait.
+    const float* S0 = L.state + ((size_t)row * s.Hv + hv) * kD * kD;
+    float4 x[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * u) * kD + lane * 4);
     // ---- a. per-node tables (the addresses of everything else depend on them) -------------------
     if (tid < kNT) {
       sm.meta[tid] = tid < N ? t.tc_meta[gi * kNT + tid] : 0;
@@ -263,14 +270,7 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     }
     __syncthreads();
     PROF(1);
-    // ---- b. gates (consumed much later); K and Q rows -> swizzled operand tile (cp.async);
-    //         first half of the pre-tree state rows -> registers -------------------------------------
-    // warp w takes rows w, w+8, ...; a warp reads one 512-byte row per instruction.  The state is not
-    // written by the kernel before this one, so its first half is requested ahead of the dependency wait.
-    const float* S0 = L.state + ((size_t)row * s.Hv + hv) * kD * kD;
-    float4 x[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * u) * kD + lane * 4);
+    // ---- b. gates (consumed much later); K and Q rows -> swizzled operand tile (cp.async) ---------
     // K, Q, V may still be in the making (the convolution runs right before this kernel): everything
     // above touched only the descriptor tables and the state.  The dependent kernel (commit) is let in
     // afterwards: it reads freely and writes only behind its own wait.
