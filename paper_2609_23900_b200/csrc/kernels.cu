@@ -57,6 +57,9 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
   asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
+__device__ __forceinline__ float ex2_approx(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float rcp_approx(float x) { float y; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+
 template <typename T> struct Packed4;      // four consecutive elements as loaded
 template <> struct Packed4<float> {
   using type = float4;
@@ -192,9 +195,15 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
         y23 = __ffma2_rn(wp[j][1], make_float2(win[j].z, win[j].w), y23);
       }
       if (has_bias) { y01 = __fadd2_rn(y01, bp[0]); y23 = __fadd2_rn(y23, bp[1]); }   // bias last
+      // SiLU a / (1 + 2^(-a log2 e)) with the hardware exponential and reciprocal (1e-6 relative, far
+      // below the rounding of the recorded operand); the multiplies and the add are packed
+      const float2 nl2e = make_float2(-1.4426950408889634f, -1.4426950408889634f), one = make_float2(1.f, 1.f);
+      float2 e01 = __fmul2_rn(y01, nl2e), e23 = __fmul2_rn(y23, nl2e);
+      e01 = __fadd2_rn(make_float2(ex2_approx(e01.x), ex2_approx(e01.y)), one);
+      e23 = __fadd2_rn(make_float2(ex2_approx(e23.x), ex2_approx(e23.y)), one);
+      y01 = __fmul2_rn(y01, make_float2(rcp_approx(e01.x), rcp_approx(e01.y)));
+      y23 = __fmul2_rn(y23, make_float2(rcp_approx(e23.x), rcp_approx(e23.y)));
       y[0] = y01.x; y[1] = y01.y; y[2] = y23.x; y[3] = y23.y;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) y[e] = __fdividef(y[e], 1.f + __expf(-y[e]));        // SiLU
     }
     T* d = dst + (size_t)ps * dst_stride;
     if constexpr (sizeof(T) == 2) {
