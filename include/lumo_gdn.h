@@ -182,6 +182,27 @@ int lumo_tree_accept(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_accep
                      int32_t* accepted_dev, int32_t* len_dev, int32_t* next_token_dev,
                      int32_t* final_node_dev, void* stream);
 
+/* ---- fused draft selection ------------------------------------------------------------------
+ * Upstream of the tree (paper Sec. "Fuse draft selection without changing proposals"): from one
+ * full-vocabulary logits row per drafting position, the spine token and three ordered sibling
+ * candidates, written into caller-owned (graph-reusable) device buffers in one pass.
+ *   spine[r]      = argmax_i logits[r, i], the lowest index among equal maxima;
+ *   cand[r, 0..2] = the three largest entries, larger value first, among equal values the higher
+ *                   index first (the paper states only that the two conventions differ; this is the
+ *                   reading taken); duplicates of the spine token are kept.
+ * logits: device [rows, V] contiguous, lumo_dtype f32 or bf16 (bf16 is widened exactly), no NaN
+ * (entries of -inf are ordinary values).  rows >= 1, V >= 3.  split = CTAs that share one row:
+ * 0 lets the library choose, else 1, 2, 4, 8 or 16; the result does not depend on it.  Enqueues
+ * only; allocates nothing.  LUMO_ERR_ARG on bad sizes, dtype or split. */
+typedef struct {
+  int32_t rows, V;
+  int32_t dtype;           /* lumo_dtype of logits */
+  int32_t split;
+  const void* logits;
+} lumo_select_args;
+int lumo_select_spine_top3(lumo_ctx* ctx, const lumo_select_args* args, int32_t* spine_dev /* [rows] */,
+                           int32_t* cand_dev /* [rows, 3] */, void* stream);
+
 /* ---- one GDN layer's tensors ----------------------------------------------------------- */
 typedef struct {
   int32_t Hk, Hv, d;

@@ -37,7 +37,7 @@ EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_s
            "lumo_ctx_timing_enable", "lumo_ctx_timing_read", "lumo_ctx_set_scan_algo", "lumo_ctx_set_overlap",
            "lumo_tree_desc_create", "lumo_tree_desc_destroy", "lumo_tree_desc_get",
            "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit",
-           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_tree_accept"]
+           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_tree_accept", "lumo_select_spine_top3"]
 
 
 class LumoError(RuntimeError):
@@ -72,6 +72,12 @@ class _AcceptArgs(ctypes.Structure):
                 ("noise", ctypes.c_void_p), ("work", ctypes.c_void_p)]
 
 
+class _SelectArgs(ctypes.Structure):
+    """Mirror of lumo_select_args."""
+    _fields_ = [("rows", ctypes.c_int32), ("V", ctypes.c_int32), ("dtype", ctypes.c_int32), ("split", ctypes.c_int32),
+                ("logits", ctypes.c_void_p)]
+
+
 _lib.lumo_ctx_create.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
 _lib.lumo_ctx_destroy.argtypes = [ctypes.c_void_p]
 _lib.lumo_ctx_destroy.restype = None
@@ -99,6 +105,8 @@ _lib.lumo_gdn_tree_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.P
 _lib.lumo_gdn_tree_scan_static.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
                                            ctypes.c_void_p]
 _lib.lumo_static_stack_bytes.restype = ctypes.c_int64
+_lib.lumo_select_spine_top3.argtypes = [ctypes.c_void_p, ctypes.POINTER(_SelectArgs), ctypes.c_void_p, ctypes.c_void_p,
+                                        ctypes.c_void_p]
 _lib.lumo_tree_accept.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_AcceptArgs), ctypes.c_int,
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.lumo_gdn_commit.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
@@ -208,6 +216,16 @@ class Context:
             setattr(a, name, _ptr(t))
         self._check(_lib.lumo_tree_accept(self._h, desc._h, ctypes.byref(a), int(accepted.shape[1]), _ptr(accepted),
                                           _ptr(length), _ptr(next_token), _ptr(final_node), _stream(stream)))
+
+    def select_spine_top3(self, logits: torch.Tensor, spine: torch.Tensor, cand: torch.Tensor, split: int = 0,
+                          stream=None):
+        """Fused draft selection: spine [R] and cand [R, 3] (int32, device) from logits [R, V] (f32 or bf16)."""
+        a = _SelectArgs()
+        a.rows, a.V = int(logits.shape[0]), int(logits.shape[1])
+        a.dtype = {torch.float32: 0, torch.bfloat16: 1}[logits.dtype]
+        a.split = int(split)
+        a.logits = _ptr(logits)
+        self._check(_lib.lumo_select_spine_top3(self._h, ctypes.byref(a), _ptr(spine), _ptr(cand), _stream(stream)))
 
     def commit(self, desc: "TreeDesc", layers, accepted: torch.Tensor, length: torch.Tensor, stream=None):
         arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)

@@ -433,6 +433,25 @@ int lumo_tree_accept(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_accep
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "accept launch");
 }
 
+int lumo_select_spine_top3(lumo_ctx* ctx, const lumo_select_args* a, int32_t* spine_dev, int32_t* cand_dev,
+                           void* stream) {
+  if (!ctx || !a || !a->logits || !spine_dev || !cand_dev) return fail(ctx, LUMO_ERR_ARG, "null argument");
+  if (ctx->device < 0) return fail(ctx, LUMO_ERR_UNSUPPORTED, "host-only context cannot launch");
+  if (a->rows < 1 || a->V < 3) return fail(ctx, LUMO_ERR_ARG, "need rows >= 1 and V >= 3");
+  if (a->rows > 65535) return fail(ctx, LUMO_ERR_ARG, "at most 65535 rows per call");
+  if (a->dtype != LUMO_F32 && a->dtype != LUMO_BF16) return fail(ctx, LUMO_ERR_ARG, "logits must be f32 or bf16");
+  const int sp = a->split;
+  if (sp != 0 && sp != 1 && sp != 2 && sp != 4 && sp != 8 && sp != 16)
+    return fail(ctx, LUMO_ERR_ARG, "split must be 0, 1, 2, 4, 8 or 16");
+  DeviceGuard g(ctx->device);
+  cudaError_t e = launch_select(a->logits, a->dtype, a->rows, a->V, sp, spine_dev, cand_dev, (cudaStream_t)stream);
+  if (e == cudaErrorInvalidConfiguration) {
+    (void)cudaGetLastError();
+    return fail(ctx, LUMO_ERR_UNSUPPORTED, "this device does not schedule clusters of that size");
+  }
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "select launch");
+}
+
 int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers,
                          void* stream) {
   Shape s;

@@ -158,6 +158,9 @@ struct AcceptView {
 };
 cudaError_t launch_accept(const TreeDev& t, int B, int N, int Ns, const AcceptView& a, int lmax, int32_t* accepted,
                           int32_t* len, int32_t* next_token, int32_t* final_node, cudaStream_t st);
+// fused draft selection (select.cu)
+cudaError_t launch_select(const void* logits, int dtype, int rows, int V, int split, int32_t* spine, int32_t* cand,
+                          cudaStream_t st);
 // Gram-form scan on tcgen05 (scan_gram.cu)
 bool gram_supported(const Shape& s, int max_depth);
 cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
