@@ -217,8 +217,8 @@ typedef struct {
   void* q;              /* [B, Ns, Hk, d] */
   void* k;              /* [B, Ns, Hk, d] */
   void* v;              /* [B, Ns, Hv, d] */
-  const void* alpha;    /* [B, Ns, Hv] decay in (0, 1], post-activation */
-  const void* beta;     /* [B, Ns, Hv] write strength in [0, 1], post-activation */
+  const void* alpha;    /* [B, Ns, Hv] decay in (0, 1], post-activation (raw input if gate_mode = 1) */
+  const void* beta;     /* [B, Ns, Hv] write strength in [0, 1], post-activation (raw input if gate_mode = 1) */
   /* convolution stage; x == NULL skips it in verify and skips the history update in commit */
   const void* x;        /* [B, Ns, C] raw projections, channels [q | k | v] */
   const void* conv_w;   /* [C, 4] tap 3 multiplies the node's own row */
@@ -232,6 +232,14 @@ typedef struct {
   const int32_t* snap_nodes;/* [B, E] logical ids, -1 = unused (mode 1) */
   float* snap_out;          /* [B, E, Hv, d_v, d_k] fp32 node states */
   int32_t* status;          /* [B] lumo_seq_status, written by verify and by commit; may be NULL */
+  /* Gate form.  0: alpha and beta hold post-activation values (above).  1: they hold the raw gate
+   * inputs (Sec. "Sequential arithmetic and accepted-path replay": the verifier takes raw gate
+   * inputs; the paper prints no formula, the reading taken is the Gated DeltaNet parametrisation)
+   *   alpha = exp(-exp(a_log[h]) * softplus(alpha_in + dt_bias[h])),  beta = sigmoid(beta_in),
+   * evaluated in fp32 inside verify and commit with the same code, so both see the same gates. */
+  int32_t gate_mode;
+  const float* a_log;       /* [Hv] fp32 (gate_mode 1) */
+  const float* dt_bias;     /* [Hv] fp32 (gate_mode 1) */
 } lumo_gdn_args;
 
 /* Verifies all nodes of every tree through n_layers independent GDN layers (Algorithm 2,

@@ -58,6 +58,21 @@ def round_bf16(x: float) -> float:
     return _load().oracle_round_bf16(float(x))
 
 
+def gates_from_raw(alpha_in, beta_in, a_log, dt_bias) -> Tuple[np.ndarray, np.ndarray]:
+    """Raw gate inputs [B, Ns, Hv] -> the decay and write strength the recurrence consumes (fp64).
+
+    Sec. "Sequential arithmetic and accepted-path replay" says the verifier takes raw gate inputs
+    but prints no formula; the reading taken is the Gated DeltaNet parametrisation, per value head h:
+    alpha = exp(-exp(a_log[h]) * softplus(alpha_in + dt_bias[h])), beta = 1 / (1 + exp(-beta_in)).
+    Pins (tests/test_oracle_scan.py): closed-form values, limits, the softplus and sigmoid
+    reflection identities, monotonicity."""
+    x = _f64(alpha_in) + _f64(dt_bias)[None, None, :]
+    softplus = np.where(x > 0, x, 0.0) + np.log1p(np.exp(-np.abs(x)))
+    alpha = np.exp(-np.exp(_f64(a_log))[None, None, :] * softplus)
+    beta = 1.0 / (1.0 + np.exp(-_f64(beta_in)))
+    return alpha, beta
+
+
 def conv(parent, slot, state_row, x, w, bias, hist, Ns: int, out_dtype: str = "none",
          threads: int = 0) -> np.ndarray:
     """Recorded operands y [B, Ns, C] (physical rows) of the ancestry-gathered conv + SiLU."""

@@ -62,6 +62,7 @@ class _Args(ctypes.Structure):
         ("snapshot_mode", ctypes.c_int32), ("n_snap", ctypes.c_int32),
         ("snap_nodes", ctypes.c_void_p), ("snap_out", ctypes.c_void_p),
         ("status", ctypes.c_void_p),
+        ("gate_mode", ctypes.c_int32), ("a_log", ctypes.c_void_p), ("dt_bias", ctypes.c_void_p),
     ]
 
 
@@ -279,10 +280,17 @@ class GdnLayer:
     def __init__(self, *, Hk: int, Hv: int, d: int, q, k, v, alpha, beta, state, state_row, out=None,
                  x=None, conv_w=None, conv_b=None, conv_hist=None, scale: float = 1.0,
                  qk_l2norm: bool = False, l2_eps: float = 1e-6, snapshot_mode: int = 0, snap_nodes=None,
-                 snap_out=None, status=None):
+                 snap_out=None, status=None, a_log=None, dt_bias=None):
+        """a_log and dt_bias ([Hv] float32) switch to raw gate inputs: alpha and beta are then activated in
+        the kernels."""
         self.tensors = dict(q=q, k=k, v=v, alpha=alpha, beta=beta, state=state, state_row=state_row, out=out,
                             x=x, conv_w=conv_w, conv_b=conv_b, conv_hist=conv_hist, snap_nodes=snap_nodes,
-                            snap_out=snap_out, status=status)
+                            snap_out=snap_out, status=status, a_log=a_log, dt_bias=dt_bias)
+        if (a_log is None) != (dt_bias is None):
+            raise ValueError("a_log and dt_bias go together")
+        for t in (a_log, dt_bias):
+            if t is not None and t.dtype != torch.float32:
+                raise ValueError("a_log and dt_bias must be float32")
         if state.dtype != torch.float32:
             raise ValueError("state must be float32")
         for name in ("state_row", "snap_nodes", "status"):
@@ -304,7 +312,8 @@ class GdnLayer:
         a.n_state_rows = int(state.shape[0])
         a.snapshot_mode = int(snapshot_mode)
         a.n_snap = int(snap_nodes.shape[1]) if snap_nodes is not None else 0
+        a.gate_mode = 0 if a_log is None else 1
         for name in ("q", "k", "v", "alpha", "beta", "x", "conv_w", "conv_b", "conv_hist", "state",
-                     "state_row", "out", "snap_nodes", "snap_out", "status"):
+                     "state_row", "out", "snap_nodes", "snap_out", "status", "a_log", "dt_bias"):
             setattr(a, name, _ptr(self.tensors[name]))
         self.args = a

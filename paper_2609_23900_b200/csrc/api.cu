@@ -50,6 +50,7 @@ int prepare(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* laye
     if (dt != LUMO_F32 && dt != LUMO_BF16) return fail(ctx, LUMO_ERR_UNSUPPORTED, "dtype must be f32 or bf16");
   if (a0.snapshot_mode < 0 || a0.snapshot_mode > 2) return fail(ctx, LUMO_ERR_ARG, "snapshot_mode must be 0, 1 or 2");
   if (a0.n_state_rows < 1) return fail(ctx, LUMO_ERR_ARG, "n_state_rows must be positive");
+  if (a0.gate_mode != 0 && a0.gate_mode != 1) return fail(ctx, LUMO_ERR_ARG, "gate_mode must be 0 or 1");
   std::memset(s, 0, sizeof(*s));
   s->B = desc->B; s->N = desc->N; s->Ns = desc->Ns;
   s->Hk = a0.Hk; s->Hv = a0.Hv; s->d = a0.d; s->C = 2 * a0.Hk * a0.d + a0.Hv * a0.d;
@@ -59,6 +60,7 @@ int prepare(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* laye
   s->snapshot_mode = for_verify ? a0.snapshot_mode : 0;
   s->n_snap = a0.snapshot_mode == 2 ? desc->N : a0.n_snap;
   s->n_layers = n_layers;
+  s->gate_mode = a0.gate_mode;
   if (for_verify && a0.snapshot_mode == 1 && (a0.n_snap < 1 || a0.n_snap > kMaxNodes))
     return fail(ctx, LUMO_ERR_ARG, "n_snap must be in [1, 256] in snapshot list mode");
   for (int l = 0; l < n_layers; ++l) {
@@ -67,10 +69,13 @@ int prepare(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* laye
     if (a.Hk != a0.Hk || a.Hv != a0.Hv || a.d != a0.d || a.in_dtype != a0.in_dtype ||
         a.gate_dtype != a0.gate_dtype || a.out_dtype != a0.out_dtype || a.scale != a0.scale ||
         a.qk_l2norm != a0.qk_l2norm || a.l2_eps != a0.l2_eps || a.n_state_rows != a0.n_state_rows ||
-        a.snapshot_mode != a0.snapshot_mode || a.n_snap != a0.n_snap || (a.x == nullptr) != (a0.x == nullptr))
+        a.snapshot_mode != a0.snapshot_mode || a.n_snap != a0.n_snap || (a.x == nullptr) != (a0.x == nullptr) ||
+        a.gate_mode != a0.gate_mode)
       return fail(ctx, LUMO_ERR_ARG, "all layers must share shape, dtypes and options" + at);
     if (!a.q || !a.k || !a.v || !a.alpha || !a.beta || !a.state || !a.state_row)
       return fail(ctx, LUMO_ERR_ARG, "q, k, v, alpha, beta, state and state_row are required" + at);
+    if (a.gate_mode == 1 && (!a.a_log || !a.dt_bias))
+      return fail(ctx, LUMO_ERR_ARG, "raw gates need a_log and dt_bias" + at);
     if (for_verify && !a.out) return fail(ctx, LUMO_ERR_ARG, "out is required" + at);
     if (a.x && (!a.conv_w || !a.conv_hist))
       return fail(ctx, LUMO_ERR_ARG, "x needs conv_w and conv_hist" + at);
@@ -82,6 +87,7 @@ int prepare(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* laye
       if (p && !aligned16(p)) return fail(ctx, LUMO_ERR_ARG, "tensor pointers must be 16-byte aligned" + at);
     LayerPtrs& p = lb->l[l];
     p.q = a.q; p.k = a.k; p.v = a.v; p.alpha = a.alpha; p.beta = a.beta;
+    p.a_log = a.a_log; p.dt_bias = a.dt_bias;
     p.x = a.x; p.conv_w = a.conv_w; p.conv_b = a.conv_b; p.conv_hist = a.conv_hist;
     p.state = a.state; p.state_row = a.state_row; p.out = a.out;
     p.snap_nodes = a.snap_nodes; p.snap_out = a.snap_out; p.status = a.status;

@@ -89,6 +89,7 @@ namespace lumo {
 struct LayerPtrs {
   void* q; void* k; void* v;
   const void* alpha; const void* beta;
+  const float* a_log; const float* dt_bias;
   const void* x; const void* conv_w; const void* conv_b; void* conv_hist;
   float* state; const int32_t* state_row;
   void* out;
@@ -107,6 +108,7 @@ struct Shape {
   int n_state_rows;
   int snapshot_mode, n_snap;
   int n_layers;
+  int gate_mode;
 };
 
 struct TreeDev {
@@ -127,6 +129,27 @@ bool build_tree(const int32_t* parent, const int32_t* slot, int N, int Ns, HostT
 // pdl_trigger().  Rule used here: a kernel triggers only AFTER its own wait, so that everything older
 // than its predecessor has completed by the time its dependent starts.
 #ifdef __CUDACC__
+// Gates of one (physical row, value head) as the recurrence consumes them: the stored values, or in
+// raw-gate mode alpha = exp(-exp(a_log) softplus(g + dt_bias)), beta = sigmoid(b), in fp32.  Every
+// kernel goes through this one function, so verify and commit see bit-identical gates.
+__device__ __forceinline__ float2 load_gates(const LayerPtrs& L, const Shape& s, size_t i, int hv) {
+  float a, b;
+  if (s.gate_dtype == LUMO_BF16) {
+    a = __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(L.alpha)[i] << 16);
+    b = __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(L.beta)[i] << 16);
+  } else {
+    a = reinterpret_cast<const float*>(L.alpha)[i];
+    b = reinterpret_cast<const float*>(L.beta)[i];
+  }
+  if (s.gate_mode == 1) {
+    const float x = a + L.dt_bias[hv];
+    const float sp = x > 20.f ? x : log1pf(expf(x));
+    a = expf(-expf(L.a_log[hv]) * sp);
+    b = 1.f / (1.f + expf(-b));
+  }
+  return make_float2(a, b);
+}
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 

@@ -39,10 +39,6 @@ template <> struct Vec4<__nv_bfloat16> {
   }
 };
 
-__device__ __forceinline__ float load_scalar(const void* p, size_t i, int dtype) {
-  return dtype == LUMO_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i])
-                            : reinterpret_cast<const float*>(p)[i];
-}
 __device__ __forceinline__ void store_scalar(void* p, size_t i, int dtype, float v) {
   if (dtype == LUMO_BF16) reinterpret_cast<__nv_bfloat16*>(p)[i] = __float2bfloat16_rn(v);
   else reinterpret_cast<float*>(p)[i] = v;
@@ -344,8 +340,9 @@ scan_kernel(Shape s, TreeDev t, LayerBatch lb, float* __restrict__ stack, int n_
           float ks = 1.f, qs = s.scale;
           if (s.l2norm) { ks = rsqrtf(kk + s.l2_eps); qs = s.scale * rsqrtf(qq + s.l2_eps); }
           p_ks[n] = ks; p_qs[n] = qs; p_kq[n] = kq * ks * qs;
-          p_a[n] = load_scalar(L.alpha, pr * s.Hv + hv, s.gate_dtype);
-          p_b[n] = load_scalar(L.beta, pr * s.Hv + hv, s.gate_dtype);
+          const float2 gates = load_gates(L, s, pr * s.Hv + hv, hv);
+          p_a[n] = gates.x;
+          p_b[n] = gates.y;
         }
       }
     }
@@ -553,8 +550,8 @@ commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ acc
     float vv;
     if constexpr (sizeof(T) == 2) vv = __bfloat162float(vg[(pr * s.Hv + hv) * D + r0 + rl]);
     else vv = vg[(pr * s.Hv + hv) * D + r0 + rl];
-    const float a = load_scalar(L.alpha, pr * s.Hv + hv, s.gate_dtype);
-    const float bt = load_scalar(L.beta, pr * s.Hv + hv, s.gate_dtype);
+    const float2 gates = load_gates(L, s, pr * s.Hv + hv, hv);
+    const float a = gates.x, bt = gates.y;
     float u0 = 0.f, u1 = 0.f, k0 = 0.f, k1 = 0.f;
 #pragma unroll
     for (int m = 0; m < NCH; ++m) {

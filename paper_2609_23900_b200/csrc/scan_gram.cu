@@ -164,11 +164,6 @@ __device__ __forceinline__ void store_out(void* out, size_t idx, int dtype, floa
   if (dtype == LUMO_BF16) reinterpret_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(v);
   else reinterpret_cast<float*>(out)[idx] = v;
 }
-__device__ __forceinline__ float load_gate(const void* p, size_t i, int dtype) {
-  return dtype == LUMO_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i])
-                            : reinterpret_cast<const float*>(p)[i];
-}
-
 #ifdef LUMO_GRAM_PROFILE
 __device__ long long g_prof[32];
 #define PROF(i) do { if (blockIdx.x == 0 && tid == 0 && item == blockIdx.x) g_prof[i] = clock64(); } while (0)
@@ -279,8 +274,9 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     float gate_a = 1.f, gate_b = 0.f;
     if (tid < N) {
       const size_t pr = (size_t)b * s.Ns + (sm.meta[tid] & 0xFFFF);
-      gate_a = load_gate(L.alpha, pr * s.Hv + hv, s.gate_dtype);
-      gate_b = load_gate(L.beta, pr * s.Hv + hv, s.gate_dtype);
+      const float2 gates = load_gates(L, s, pr * s.Hv + hv, hv);
+      gate_a = gates.x;
+      gate_b = gates.y;
     }
     {
       const __nv_bfloat16* kg = reinterpret_cast<const __nv_bfloat16*>(L.k);

@@ -17,7 +17,10 @@ class DeviceCase:
     def __init__(self, ctx: binding.Context, case: Case, *, out_dtype: str = "f32", use_conv: bool = True,
                  gate_dtype: Optional[str] = None, snapshot_mode: int = 0, snap_nodes=None,
                  scale: float = 1.0, qk_l2norm: Optional[bool] = None, l2_eps: float = 1e-6,
-                 device: Optional[torch.device] = None, pinned_host: bool = False):
+                 device: Optional[torch.device] = None, pinned_host: bool = False, raw_gates=None):
+        """raw_gates: optional list (one entry per layer) of dicts with host arrays alpha_in, beta_in
+        [B, Ns, Hv] and a_log, dt_bias [Hv]; the layer then takes raw gate inputs instead of the case's
+        post-activation gates."""
         self.ctx, self.case = ctx, case
         # conv outputs are not unit vectors: the pipeline normalises q, k inside the kernels
         # (Sec. "Sequential arithmetic and accepted-path replay": in-kernel query/key normalisation)
@@ -49,6 +52,10 @@ class DeviceCase:
                 out=torch.empty((case.B, case.Ns, case.Hv, case.d), dtype=odt, device=dev),
                 status=torch.full((case.B,), -1, dtype=torch.int32, device=dev),
             )
+            if raw_gates is not None:
+                rg = raw_gates[len(self.layers)]
+                t.update(alpha=up(rg["alpha_in"], gdt), beta=up(rg["beta_in"], gdt),
+                         a_log=up(rg["a_log"], torch.float32), dt_bias=up(rg["dt_bias"], torch.float32))
             if use_conv:
                 t.update(x=up(L.x, dt), conv_w=up(L.conv_w, dt), conv_hist=up(L.hist, dt),
                          conv_b=None if L.conv_b is None else up(L.conv_b, dt))

@@ -45,11 +45,20 @@ def assert_close(got, ref, *, bf16=False, what=""):
     return float((err / (1.0 + np.abs(ref))).max())
 
 
+def device_gates(dc: DeviceCase, layer=0):
+    """The gates the recurrence consumes, from the arrays the GPU reads (raw-gate layers: activated in fp64)."""
+    a, b = dc.np("alpha", layer), dc.np("beta", layer)
+    if dc.t("a_log", layer) is not None:
+        a, b = O.gates_from_raw(a, b, dc.np("a_log", layer), dc.np("dt_bias", layer))
+    return a, b
+
+
 def oracle_scan_from_device(dc: DeviceCase, layer=0, **kw):
     """Oracle scan on the operands the GPU recorded (same rounded arrays on both sides)."""
     c = dc.case
+    alpha, beta = device_gates(dc, layer)
     return O.scan(c.parent, c.slot, c.state_row, dc.np("q", layer), dc.np("k", layer), dc.np("v", layer),
-                  dc.np("alpha", layer), dc.np("beta", layer), c.layers[layer].state, scale=dc.scale,
+                  alpha, beta, c.layers[layer].state, scale=dc.scale,
                   l2norm=dc.qk_l2norm, eps=dc.l2_eps, **kw)
 
 
@@ -59,6 +68,7 @@ def oracle_commit_from_device(dc: DeviceCase, layer=0, accepted=None, length=Non
     acc = c.accepted if accepted is None else accepted
     ln = c.accepted_len if length is None else length
     x, hist = (L.x, L.hist) if with_hist else (None, None)
+    alpha, beta = device_gates(dc, layer)
     return O.commit(c.parent, c.slot, c.state_row, dc.np("q", layer), dc.np("k", layer), dc.np("v", layer),
-                    dc.np("alpha", layer), dc.np("beta", layer), L.state, acc, ln, x=x, hist=hist,
+                    alpha, beta, L.state, acc, ln, x=x, hist=hist,
                     l2norm=dc.qk_l2norm, eps=dc.l2_eps, **kw)

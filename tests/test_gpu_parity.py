@@ -483,3 +483,47 @@ def test_host_detected_errors_return_codes():
     with pytest.raises(binding.LumoError) as e:
         dc.verify()
     assert e.value.code == 1
+
+
+# ------------------------------------------------------------------ raw gate inputs
+def _raw_gates(c, seed):
+    rs = np.random.default_rng(seed)
+    out = []
+    for _ in c.layers:
+        out.append(dict(alpha_in=(rs.standard_normal((c.B, c.Ns, c.Hv)) * 2 - 2).astype(np.float32),
+                        beta_in=(rs.standard_normal((c.B, c.Ns, c.Hv)) * 1.5).astype(np.float32),
+                        a_log=rs.uniform(-1.0, 1.0, c.Hv).astype(np.float32),
+                        dt_bias=rs.uniform(-1.0, 1.0, c.Hv).astype(np.float32)))
+    return out
+
+
+@pytest.mark.parametrize("name,algo", [("cfg0", "rank1"), ("cfg1", "rank1"), ("cfg1", "gram"), ("d64_bf16", "rank1"),
+                                       ("cfgP_padded_permuted", "rank1"), ("cfgP_padded_permuted", "gram")])
+def test_raw_gate_inputs_verify_and_commit(name, algo):
+    """Raw gate inputs activated inside the kernels: scan outputs and the committed state against the
+    oracle fed with the fp64 activation of the same (rounded) inputs."""
+    c = CASES[name]()
+    assert algo == "rank1" or gram_eligible(c)
+    dc = DeviceCase(ctx(algo), c, raw_gates=_raw_gates(c, 17))
+    dc.verify()
+    torch.cuda.synchronize()
+    o_ref, _, _ = oracle_scan_from_device(dc)
+    assert_close(dc.np("out"), o_ref, what=f"{name} raw-gate scan")
+    dc.commit()
+    torch.cuda.synchronize()
+    st_ref, _, status_ref, _ = oracle_commit_from_device(dc)
+    assert_close(dc.np("state"), st_ref, what=f"{name} raw-gate commit")
+    assert np.array_equal(dc.t("status").cpu().numpy(), status_ref)
+    # the activation is live: the same call with the inputs read as post-activation gates differs
+    dc2 = DeviceCase(ctx(algo), c)
+    dc2.verify()
+    torch.cuda.synchronize()
+    assert np.abs(dc2.np("out") - dc.np("out")).max() > 1e-3
+
+
+def test_raw_gates_need_both_parameter_vectors():
+    c = CASES["cfg0"]()
+    with pytest.raises(ValueError):
+        binding.GdnLayer(Hk=c.Hk, Hv=c.Hv, d=c.d, q=torch.zeros(1), k=torch.zeros(1), v=torch.zeros(1),
+                         alpha=torch.zeros(1), beta=torch.zeros(1), state=torch.zeros(1),
+                         state_row=torch.zeros(1, dtype=torch.int32), a_log=torch.zeros(c.Hv))

@@ -352,3 +352,33 @@ def test_commit_history_is_last_three_of_old_plus_accepted_inputs():
     assert np.array_equal(h[r], np.stack([h0[r, 2], x[0, 1], x[0, 5]]))
     _, h, _, _ = O.commit(*args, [[1, -1, -1]], [1], x=L.x, hist=L.hist)
     assert np.array_equal(h[r], np.stack([h0[r, 1], h0[r, 2], x[0, 1]]))
+
+
+# ------------------------------------------------------------------ raw gate inputs
+def test_raw_gate_activation_closed_forms_and_identities():
+    import scipy.special
+    one = lambda v: np.full((1, 1, 1), v)
+    # softplus(0) = ln 2, a_log = 0: alpha = exp(-ln 2) = 1/2; sigmoid(0) = 1/2
+    a, b = O.gates_from_raw(one(0.3), one(0.0), [0.0], [-0.3])
+    assert a[0, 0, 0] == pytest.approx(0.5, abs=1e-15) and b[0, 0, 0] == 0.5
+    # a_log = ln 3: alpha = 2^-3
+    a, _ = O.gates_from_raw(one(0.0), one(0.0), [np.log(3.0)], [0.0])
+    assert a[0, 0, 0] == pytest.approx(0.125, rel=1e-14)
+    # limits: a very negative input leaves the state undecayed, a large one decays like exp(-x e^a_log)
+    a, b = O.gates_from_raw(np.array([[[-60.0], [40.0]]]), np.array([[[-60.0], [60.0]]]), [0.5], [0.0])
+    assert a[0, 0, 0] == pytest.approx(1.0, abs=1e-15) and a[0, 1, 0] == pytest.approx(np.exp(-40.0 * np.exp(0.5)), rel=1e-12)
+    assert b[0, 0, 0] < 1e-25 and b[0, 1, 0] == pytest.approx(1.0, abs=1e-15)
+    # identities and the library routines, per head (a_log and dt_bias index the last axis)
+    rs = np.random.default_rng(3)
+    g, r = rs.standard_normal((2, 5, 3)) * 4, rs.standard_normal((2, 5, 3)) * 4
+    a_log, dt = rs.uniform(-1, 1, 3), rs.uniform(-1, 1, 3)
+    a, b = O.gates_from_raw(g, r, a_log, dt)
+    assert np.all((a > 0) & (a <= 1)) and np.all((b > 0) & (b < 1))
+    np.testing.assert_allclose(b, scipy.special.expit(r), rtol=1e-14)
+    np.testing.assert_allclose(-np.log(a) / np.exp(a_log), np.logaddexp(0.0, g + dt), rtol=1e-9, atol=1e-14)
+    b_neg = O.gates_from_raw(g, -r, a_log, dt)[1]
+    np.testing.assert_allclose(b + b_neg, 1.0, rtol=1e-14)                       # sigmoid(x) + sigmoid(-x) = 1
+    sp = lambda x: -np.log(O.gates_from_raw(x, r, np.zeros(3), np.zeros(3))[0])
+    np.testing.assert_allclose(sp(g) - sp(-g), g, rtol=1e-9, atol=1e-12)        # softplus(x) - softplus(-x) = x
+    a_up = O.gates_from_raw(g + 0.1, r, a_log, dt)[0]
+    assert np.all(a_up < a)                                                      # decay is monotone in the input
