@@ -5,6 +5,7 @@
 // (dependent path groups, cut states; Sec. "Path-parallel verification and state
 // lifetime").  The depth-first op list is this library's own schedule.
 #include <algorithm>
+#include <bitset>
 #include <functional>
 
 #include "internal.h"
@@ -161,70 +162,78 @@ bool build_tree(const int32_t* parent, const int32_t* slot, int N, int Ns, HostT
   return true;
 }
 
-// Partition of a tree into groups of at most 64 nodes for the Gram-form scan.  A group is a
-// root-first prefix path (whose deltas the group recomputes) plus complete subtrees hanging off
-// the last prefix node, so every member's ancestors are inside the group.  A node is emitted
-// (its output written) by exactly one group: as a subtree member, or by the first group that
-// carries it as a prefix node.  Members are ordered by (depth, logical index).
+// Node groups of the tensor-core scan.  A group is a set of at most 64 nodes closed under "parent
+// of", so that it can be solved from the pre-tree state alone; every node is emitted (written) by
+// exactly one group and may be recomputed, unwritten, in others.  Fewer groups mean fewer passes
+// over the state, so the tree is first cut into atoms (a complete subtree if it fits together with
+// its ancestors, else the node alone and its children in turn) and the atoms are packed, largest
+// closure first, each into the group whose node set grows least (groups that already hold the
+// atom's ancestors take it for little), or into a new group.  Members are ordered by (depth, index).
 void build_gram_groups(const int32_t* parent, int N, const HostTree& t, std::vector<GramGroup>* out) {
   const auto& depth = t.tab[LUMO_TAB_DEPTH];
   const auto& coff = t.tab[LUMO_TAB_CHILD_OFF];
   const auto& clist = t.tab[LUMO_TAB_CHILD_LIST];
+  constexpr int kCap = 64;
+  using Mask = std::bitset<kMaxNodes>;
   std::vector<int> size(N, 1);
   for (int i = N - 1; i >= 0; --i)
     if (parent[i] >= 0) size[parent[i]] += size[i];
-  std::vector<char> emitted(N, 0);
-  constexpr int kCap = 64;
-  auto kids = [&](int a, int* lo, int* hi) { *lo = coff[a + 1]; *hi = coff[a + 2]; };   // a = -1: children of the pre-tree state
-  auto flush = [&](const std::vector<int>& prefix, std::vector<int>& members) {
-    if (members.empty()) return;
+  struct Atom { Mask emit, closure; int count; };
+  std::vector<Atom> atoms;
+  // depth-first over the tree with an explicit stack (a = -1: children of the pre-tree state)
+  std::vector<int> todo;
+  for (int ci = coff[1] - 1; ci >= coff[0]; --ci) todo.push_back(clist[ci]);
+  while (!todo.empty()) {
+    const int c = todo.back();
+    todo.pop_back();
+    Atom at;
+    if (size[c] + depth[c] - 1 <= kCap) {            // the whole subtree and its ancestors fit
+      std::vector<int> st{c};
+      while (!st.empty()) {
+        const int n = st.back();
+        st.pop_back();
+        at.emit.set(n);
+        for (int k = coff[n + 1]; k < coff[n + 2]; ++k) st.push_back(clist[k]);
+      }
+    } else {
+      at.emit.set(c);
+      for (int k = coff[c + 2] - 1; k >= coff[c + 1]; --k) todo.push_back(clist[k]);
+    }
+    at.closure = at.emit;
+    for (int a = parent[c]; a >= 0; a = parent[a]) at.closure.set(a);
+    at.count = (int)at.closure.count();
+    atoms.push_back(at);
+  }
+  std::stable_sort(atoms.begin(), atoms.end(), [](const Atom& x, const Atom& y) { return x.count > y.count; });
+  std::vector<Atom> bins;
+  for (const Atom& at : atoms) {
+    int best = -1, best_growth = 0;
+    for (int b = 0; b < (int)bins.size(); ++b) {
+      const int total = (int)(bins[b].closure | at.closure).count();
+      if (total > kCap) continue;
+      const int growth = total - bins[b].count;
+      if (best < 0 || growth < best_growth) { best = b; best_growth = growth; }
+    }
+    if (best < 0) {
+      bins.push_back(at);
+    } else {
+      bins[best].emit |= at.emit;
+      bins[best].closure |= at.closure;
+      bins[best].count = (int)bins[best].closure.count();
+    }
+  }
+  for (const Atom& bin : bins) {
     GramGroup g;
-    std::vector<int> all(prefix);
-    all.insert(all.end(), members.begin(), members.end());
+    std::vector<int> all;
+    for (int n = 0; n < N; ++n)
+      if (bin.closure.test(n)) all.push_back(n);
     std::sort(all.begin(), all.end(), [&](int x, int y) { return depth[x] != depth[y] ? depth[x] < depth[y] : x < y; });
     for (int n : all) {
       g.nodes.push_back(n);
-      g.emit.push_back(emitted[n] ? 0 : 1);
-      emitted[n] = 1;
+      g.emit.push_back(bin.emit.test(n) ? 1 : 0);
     }
     out->push_back(std::move(g));
-    members.clear();
-  };
-  std::function<void(int, std::vector<int>&)> pack = [&](int a, std::vector<int>& prefix) {
-    const int cap = kCap - (int)prefix.size();
-    int lo, hi;
-    kids(a, &lo, &hi);
-    std::vector<int> cur;
-    for (int ci = lo; ci < hi; ++ci) {
-      const int c = clist[ci];
-      if (size[c] <= cap) {
-        if ((int)cur.size() + size[c] > cap) flush(prefix, cur);
-        // whole subtree of c (its nodes have indices > c; walk by parent marks)
-        std::vector<int> stack{c};
-        while (!stack.empty()) {
-          int n = stack.back(); stack.pop_back();
-          cur.push_back(n);
-          int l2, h2;
-          kids(n, &l2, &h2);
-          for (int k = l2; k < h2; ++k) stack.push_back(clist[k]);
-        }
-      } else {
-        flush(prefix, cur);
-        prefix.push_back(c);
-        pack(c, prefix);
-        prefix.pop_back();
-      }
-    }
-    flush(prefix, cur);
-    if (a >= 0 && !emitted[a]) {      // every child was too large and recursed, or a has no group yet
-      std::vector<int> none;
-      GramGroup g;
-      for (int n : prefix) { g.nodes.push_back(n); g.emit.push_back(emitted[n] ? 0 : 1); emitted[n] = 1; }
-      out->push_back(std::move(g));
-    }
-  };
-  std::vector<int> prefix;
-  pack(-1, prefix);
+  }
 }
 
 }  // namespace lumo
