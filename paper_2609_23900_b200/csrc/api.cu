@@ -129,6 +129,7 @@ TreeDev tree_view(const lumo_tree_desc* d, int which) {
   t.max_ops = d->max_ops[which]; t.max_levels = d->max_levels[which];
   t.tc_group = d->d_tc_group; t.tc_meta = d->d_tc_meta; t.tc_anc = d->d_tc_anc; t.tc_lvl = d->d_tc_lvl;
   t.n_groups = d->n_groups;
+  t.max_group_nodes = d->max_group_nodes;
   return t;
 }
 
@@ -279,6 +280,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
       auto& tab = d->trees[b].tab[LUMO_TAB_GRAM_GROUPS];
       tab.push_back((int32_t)groups[b].size());
       for (const GramGroup& gr : groups[b]) {
+        d->max_group_nodes = std::max(d->max_group_nodes, (int)gr.nodes.size());
         tab.push_back((int32_t)gr.nodes.size());
         tab.insert(tab.end(), gr.nodes.begin(), gr.nodes.end());
         tab.insert(tab.end(), gr.emit.begin(), gr.emit.end());

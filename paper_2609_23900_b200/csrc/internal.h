@@ -77,6 +77,7 @@ struct lumo_tree_desc {
   // Gram-form scan tables (present when max_depth <= 16): the trees are cut into groups of at most
   // 64 nodes (prefix path + complete subtrees); G = number of groups over the batch
   int n_groups = 0;
+  int max_group_nodes = 0;        // largest group (the scan picks a 32-node tile when every group fits it)
   int32_t* d_tc_group = nullptr;  // [G, 4]  sequence b, node count, first-group-of-b flag, 0
   int32_t* d_tc_meta = nullptr;   // [G, 64] physical row | depth << 16 | emit << 24 of the node at position pi
   uint8_t* d_tc_anc = nullptr;    // [G, 64, 16] positions of the ancestors, root first
@@ -115,7 +116,7 @@ struct TreeDev {
   const int32_t* parent; const int32_t* depth; const int32_t* slot; const int32_t* slot_inv;
   const int32_t* win; const int32_t* conv_prog; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
   const int32_t* child_off; const int32_t* child_list;   // [B, N+2] CSR (entry 0 = pre-tree state), [B, N]
-  const int32_t* tc_group; const int32_t* tc_meta; const uint8_t* tc_anc; const uint8_t* tc_lvl; int n_groups;
+  const int32_t* tc_group; const int32_t* tc_meta; const uint8_t* tc_anc; const uint8_t* tc_lvl; int n_groups; int max_group_nodes;
 };
 
 void build_gram_groups(const int32_t* parent, int N, const HostTree& t, std::vector<GramGroup>* out);

@@ -191,6 +191,9 @@ struct NodeOps {
   uint2 ao;        // first four ancestor offsets (16 bits each)
 };
 
+// NT = node tile of the MMAs: 64, or 32 when no group of the launch has more than 32 nodes (K rows
+// 0..NT-1 and Q rows NT..2NT-1 of the operand tile; the products occupy NT + NT + NT columns)
+template <int NT>
 __global__ void __launch_bounds__(kThreads, 2)
 scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
   extern __shared__ unsigned char smem_raw[];
@@ -281,17 +284,18 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     {
       const __nv_bfloat16* kg = reinterpret_cast<const __nv_bfloat16*>(L.k);
       const __nv_bfloat16* qg = reinterpret_cast<const __nv_bfloat16*>(L.q);
-      const __nv_bfloat16* src[2048 / kThreads];
+      constexpr int kCopies = 2 * NT * 16 / kThreads;   // 16-byte pieces of the 2 NT rows, per thread
+      const __nv_bfloat16* src[kCopies];
 #pragma unroll
-      for (int i = 0; i < 2048 / kThreads; ++i) {        // addresses first, so that the copies issue back to back
+      for (int i = 0; i < kCopies; ++i) {                // addresses first, so that the copies issue back to back
         const int idx = i * kThreads + tid;
         const int R = idx >> 4, c = idx & 15;
-        const int pi = R & (kNT - 1);
+        const int pi = R & (NT - 1);
         const size_t pr = (size_t)b * s.Ns + (sm.meta[pi] & 0xFFFF);
-        src[i] = pi < N ? (R < kNT ? kg : qg) + (pr * s.Hk + g) * kD + c * 8 : nullptr;
+        src[i] = pi < N ? (R < NT ? kg : qg) + (pr * s.Hk + g) * kD + c * 8 : nullptr;
       }
 #pragma unroll
-      for (int i = 0; i < 2048 / kThreads; ++i) {
+      for (int i = 0; i < kCopies; ++i) {
         const int idx = i * kThreads + tid;
         const int R = idx >> 4, c = idx & 15;
         const uint32_t dst = sbase + kOffKQ + (c >> 3) * 16384 + sw128_offset(R, c & 7);
@@ -329,7 +333,7 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     // ---- e. MMAs: Gram = [K;Q] K^T, P = S0 [K|Q]^T (hi + lo); meanwhile |q|^2 when normalising ----
     if (tid == 0) {
       tc_fence_after();
-      constexpr uint32_t idesc_p = umma_idesc(128, 128), idesc_g = umma_idesc(128, 64);
+      constexpr uint32_t idesc_p = umma_idesc(128, 2 * NT), idesc_g = umma_idesc(128, NT);
       const uint64_t d_kq = umma_desc(sbase + kOffKQ), d_hi = umma_desc(sbase + kOffAhi), d_lo = umma_desc(sbase + kOffAlo);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
@@ -347,8 +351,8 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
         umma(tmem, d_lo + koff, d_kq + koff, idesc_p, 1u);
       }
       umma_commit(&sm.mbar);
-    } else if (grp == 1 && s.l2norm && vrow < kNT) {
-      const int R = kNT + vrow;   // tile row of q_vrow (the tensor core only reads the tile)
+    } else if (grp == 1 && s.l2norm && vrow < NT) {
+      const int R = NT + vrow;   // tile row of q_vrow (the tensor core only reads the tile)
       float qq = 0.f;
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
@@ -378,7 +382,7 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     {
       const __nv_bfloat16* vg = reinterpret_cast<const __nv_bfloat16*>(L.v);
 #pragma unroll
-      for (int i = 0; i < 1024 / kThreads; ++i) {
+      for (int i = 0; i < NT * 16 / kThreads; ++i) {
         const int idx = i * kThreads + tid;
         const int pi = idx >> 4, c = idx & 15;
         if (pi < N) {
@@ -388,26 +392,27 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
       }
       asm volatile("cp.async.commit_group;\n" ::: "memory");
     }
-    // both halves of the CTA read the Gram rows: 32 of the 64 columns each
-    tmem_cols32_to_smem(tmem_lane + 128 + grp * 32, dump + vrow * kDumpStride + grp * 32, 1);
+    // both halves of the CTA read the Gram rows: 32 of the NT columns each (one half is enough for NT = 32)
+    if (grp * 32 < NT) tmem_cols32_to_smem(tmem_lane + 128 + grp * 32, dump + vrow * kDumpStride + grp * 32, 1);
     __syncthreads();
     PROF(8);
     // ---- h. normalisation factors ------------------------------------------------------------------
-    if (tid < kNT) sm.ks[tid] = s.l2norm ? rsqrtf(dump[tid * kDumpStride + tid] + s.l2_eps) : 1.f;
-    else if (tid < 2 * kNT) sm.qs[tid - kNT] = s.l2norm ? s.scale * rsqrtf(sm.qq[tid - kNT] + s.l2_eps) : s.scale;
+    if (tid < NT) sm.ks[tid] = s.l2norm ? rsqrtf(dump[tid * kDumpStride + tid] + s.l2_eps) : 1.f;
+    else if (tid < 2 * NT) sm.qs[tid - NT] = s.l2norm ? s.scale * rsqrtf(sm.qq[tid - NT] + s.l2_eps) : s.scale;
     __syncthreads();
     PROF(9);
     // ---- i. first half of the CTA: node records, one thread per (node, table); second half: the
     //         S0 q^ products move from tensor memory to shared memory [node][row] ---------------------
     if (grp == 0) {
-      const bool is_q = tid >= kNT;
-      const int pi = tid & (kNT - 1);
+      if (tid < 2 * NT) {
+      const bool is_q = tid >= NT;
+      const int pi = tid & (NT - 1);
       NodeRec& rec = recs[pi];
       const int meta = sm.meta[pi];
       const int D = pi < N ? ((meta >> 16) & 0xFF) : 0;          // depth, 1..16
       const float a_t = sm.alpha[pi], b_t = sm.beta[pi];
       const float self = is_q ? sm.qs[pi] : -b_t * sm.ks[pi];    // factor of the node itself (k side negated)
-      const float* grow = dump + (is_q ? kNT + pi : pi) * kDumpStride;
+      const float* grow = dump + (is_q ? NT + pi : pi) * kDumpStride;
       float G = a_t;
       float w[16];
       uint32_t ao[8];
@@ -439,9 +444,10 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
         adst[0] = make_uint4(ao[0], ao[1], ao[2], ao[3]);
         adst[1] = make_uint4(ao[4], ao[5], ao[6], ao[7]);
       }
+      }
     } else {
       for (int cb = 0; cb < (N + 31) / 32; ++cb)                 // bounded: <= 2
-        tmem_cols32_to_smem(tmem_lane + kNT + cb * 32, Pq + (cb * 32) * kD + vrow, kD);
+        tmem_cols32_to_smem(tmem_lane + NT + cb * 32, Pq + (cb * 32) * kD + vrow, kD);
     }
     asm volatile("cp.async.wait_group 0;\n" ::: "memory");
     __syncthreads();      // records, V and Pq are in place; the Gram dump is dead from here on
@@ -549,14 +555,18 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
   const int items = s.n_layers * t.n_groups * s.Hv;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(scan_gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(scan_gram_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(scan_gram_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     configured = true;
   }
   // two CTAs per SM by construction: 102 KB of shared memory, 128 registers x 256 threads and 256
   // of the 512 tensor-memory columns each
   const int grid = items < 2 * sm_count ? items : 2 * sm_count;
-  return launch_kernel(scan_gram_kernel, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
+  if (t.max_group_nodes <= 32)
+    return launch_kernel(scan_gram_kernel<32>, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
+  return launch_kernel(scan_gram_kernel<64>, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
 }
 
 #ifdef LUMO_GRAM_PROFILE
