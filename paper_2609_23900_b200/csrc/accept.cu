@@ -226,38 +226,15 @@ accept_kernel(TreeDev t, int N, int Ns, AcceptView a, int lmax, int32_t* __restr
 
 cudaError_t launch_accept(const TreeDev& t, int B, int N, int Ns, const AcceptView& a, int lmax, int32_t* accepted,
                           int32_t* len, int32_t* next_token, int32_t* final_node, cudaStream_t st) {
-  // largest cluster this device schedules, found once per device (16 CTAs needs the opt-in attribute)
-  static int max_cluster[64] = {};
+  static int cache[64] = {};
   int dev = 0, sms = 0;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  cfg.blockDim = dim3(kAcceptThreads);
-  cfg.stream = st;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  if (dev >= 0 && dev < 64 && max_cluster[dev] == 0) {
-    int c = cudaFuncSetAttribute(accept_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess
-                ? 16 : kAcceptCluster;
-    for (; c > 1; c >>= 1) {                               // bounded: at most four sizes
-      int fit = 0;
-      cfg.gridDim = dim3(c, 1);
-      attr[0].val.clusterDim.x = c;
-      if (cudaOccupancyMaxActiveClusters(&fit, accept_kernel, &cfg) == cudaSuccess && fit > 0) break;
-    }
-    (void)cudaGetLastError();
-    max_cluster[dev] = c;
-  }
-  int cluster = (dev >= 0 && dev < 64) ? max_cluster[dev] : 1;
+  int cluster = max_cluster_ctas(accept_kernel, kAcceptThreads, cache);
   if (cluster > kAcceptCluster && B * cluster > sms) cluster = kAcceptCluster;   // many sequences: smaller clusters
   while (cluster > 1 && a.V < cluster * kAcceptThreads) cluster >>= 1;           // small vocabularies
-  cfg.gridDim = dim3(cluster, B);
-  attr[0].val.clusterDim.x = cluster;
-  return cudaLaunchKernelEx(&cfg, accept_kernel, t, N, Ns, a, lmax, accepted, len, next_token, final_node);
+  return launch_cluster_kernel(accept_kernel, dim3(cluster, B), dim3(kAcceptThreads), cluster, st, t, N, Ns, a, lmax,
+                               accepted, len, next_token, final_node);
 }
 
 }  // namespace lumo

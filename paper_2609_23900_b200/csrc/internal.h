@@ -154,6 +154,49 @@ __device__ __forceinline__ float2 load_gates(const LayerPtrs& L, const Shape& s,
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 
+// Largest thread-block cluster (16, 8, 4, 2 or 1 CTAs of `threads` threads along x) that the current
+// device schedules for `kern`; 16 needs the non-portable opt-in.  Looked up once per device and kernel
+// (`cache` is the caller's static table, zero-initialised).
+template <typename K>
+int max_cluster_ctas(K kern, int threads, int (&cache)[64]) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= 64) return 1;
+  if (cache[dev] == 0) {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    cfg.blockDim = dim3(threads);
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    int c = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess ? 16 : 8;
+    for (; c > 1; c >>= 1) {                               // bounded: at most four sizes
+      int fit = 0;
+      cfg.gridDim = dim3(c, 1);
+      attr[0].val.clusterDim.x = c;
+      if (cudaOccupancyMaxActiveClusters(&fit, kern, &cfg) == cudaSuccess && fit > 0) break;
+    }
+    (void)cudaGetLastError();
+    cache[dev] = c;
+  }
+  return cache[dev];
+}
+
+// launch of a kernel whose CTAs form clusters of `cluster` along x
+template <typename... KArgs, typename... Args>
+cudaError_t launch_cluster_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, int cluster, cudaStream_t st, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = cluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool pdl,
                           Args... args) {

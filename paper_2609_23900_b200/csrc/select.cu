@@ -225,33 +225,9 @@ cudaError_t launch_select(const void* logits, int dtype, int rows, int V, int sp
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  static int max_cluster[64] = {};
-  cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  cfg.blockDim = dim3(kSelThreads);
-  cfg.stream = st;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  auto kernel_f = select_kernel<float>;
-  auto kernel_h = select_kernel<__nv_bfloat16>;
-  if (dev >= 0 && dev < 64 && max_cluster[dev] == 0) {   // largest schedulable cluster, found once per device
-    int c = 8;
-    if (cudaFuncSetAttribute(kernel_f, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess &&
-        cudaFuncSetAttribute(kernel_h, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess)
-      c = 16;
-    for (; c > 1; c >>= 1) {                             // bounded: at most four sizes
-      int fit = 0;
-      cfg.gridDim = dim3(c, 1);
-      attr[0].val.clusterDim.x = c;
-      if (cudaOccupancyMaxActiveClusters(&fit, kernel_f, &cfg) == cudaSuccess && fit > 0) break;
-    }
-    (void)cudaGetLastError();
-    max_cluster[dev] = c;
-  }
-  const int cap = (dev >= 0 && dev < 64) ? max_cluster[dev] : 1;
+  static int cache_f[64] = {}, cache_h[64] = {};
+  const int cap = dtype == LUMO_BF16 ? max_cluster_ctas(select_kernel<__nv_bfloat16>, kSelThreads, cache_h)
+                                     : max_cluster_ctas(select_kernel<float>, kSelThreads, cache_f);
   int cluster = split;
   if (cluster == 0) {                                    // few rows: spread each over more SMs
     cluster = cap;
@@ -260,11 +236,11 @@ cudaError_t launch_select(const void* logits, int dtype, int rows, int V, int sp
     while (cluster > 1 && V < cluster * kSelThreads * unit) cluster >>= 1;
   }
   if (cluster > cap) return cudaErrorInvalidConfiguration;
-  cfg.gridDim = dim3(cluster, rows);
-  attr[0].val.clusterDim.x = cluster;
   if (dtype == LUMO_BF16)
-    return cudaLaunchKernelEx(&cfg, kernel_h, reinterpret_cast<const __nv_bfloat16*>(logits), V, spine, cand);
-  return cudaLaunchKernelEx(&cfg, kernel_f, reinterpret_cast<const float*>(logits), V, spine, cand);
+    return launch_cluster_kernel(select_kernel<__nv_bfloat16>, dim3(cluster, rows), dim3(kSelThreads), cluster, st,
+                                 reinterpret_cast<const __nv_bfloat16*>(logits), V, spine, cand);
+  return launch_cluster_kernel(select_kernel<float>, dim3(cluster, rows), dim3(kSelThreads), cluster, st,
+                               reinterpret_cast<const float*>(logits), V, spine, cand);
 }
 
 }  // namespace lumo
