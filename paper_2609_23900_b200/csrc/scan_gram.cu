@@ -17,7 +17,7 @@
 // at a time, the deltas live in shared memory [node][row], and the tree is walked level by level
 // (all nodes of one depth are independent), the nodes of a level dealt out to the eight warps,
 // each lane carrying four adjacent value rows so that the per-node coefficient loads are shared.
-// Per node the CTA first builds a 224-byte record (coefficients, ancestor offsets, output
+// Per node the CTA first builds a 208-byte record (coefficients, ancestor offsets, output
 // offset); a warp loads the record of its next node before the barrier that publishes the
 // previous level, so that only the ancestors' deltas are fetched after it.
 //
