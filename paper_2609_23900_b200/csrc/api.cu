@@ -266,6 +266,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   const size_t o_parent = reserve((size_t)B * N), o_depth = reserve((size_t)B * N), o_slot = reserve((size_t)B * N);
   const size_t o_inv = reserve((size_t)B * Ns), o_win = reserve((size_t)B * Ns * 4);
   const size_t o_prog = reserve((size_t)B * Ns);
+  const size_t o_winv = reserve((size_t)B * Ns * 4);
   const size_t o_coff = reserve((size_t)B * (N + 2)), o_clist = reserve((size_t)B * N);
   size_t o_sched[2], o_nops[2];
   for (int w = 0; w < 2; ++w) { o_sched[w] = reserve((size_t)B * d->max_ops[w]); o_nops[w] = reserve(B); }
@@ -339,6 +340,11 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
       }
       for (int sidx = 0; sidx < Ns; ++sidx)
         if (t.tab[LUMO_TAB_SLOT_INV][sidx] < 0) h[o_prog + (size_t)b * Ns + k++] = sidx | (3 << 16);
+      // the windows in the same visiting order, so that the kernel fetches order and window together
+      for (int e = 0; e < Ns; ++e) {
+        const int sidx = h[o_prog + (size_t)b * Ns + e] & 0xFFFF;
+        for (int j = 0; j < 4; ++j) h[o_winv + ((size_t)b * Ns + e) * 4 + j] = h[o_win + ((size_t)b * Ns + sidx) * 4 + j];
+      }
     }
     for (int w = 0; w < 2; ++w) {
       const auto& ops = t.tab[LUMO_TAB_SCHEDULE + w];
@@ -374,7 +380,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   e = cudaMemcpy(d->dev, h.data(), h.size() * sizeof(int32_t), cudaMemcpyHostToDevice);
   if (e != cudaSuccess) { cudaFree(d->dev); delete d; return cuda_fail(ctx, e, "cudaMemcpy(tree tables)"); }
   d->d_parent = d->dev + o_parent; d->d_depth = d->dev + o_depth; d->d_slot = d->dev + o_slot;
-  d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_win; d->d_conv_prog = d->dev + o_prog;
+  d->d_slot_inv = d->dev + o_inv; d->d_win = d->dev + o_winv; d->d_conv_prog = d->dev + o_prog;
   d->d_child_off = d->dev + o_coff; d->d_child_list = d->dev + o_clist;
   for (int w = 0; w < 2; ++w) { d->d_sched[w] = d->dev + o_sched[w]; d->d_nops[w] = d->dev + o_nops[w]; }
   if (tc) {

@@ -63,7 +63,7 @@ struct lumo_tree_desc {
   int32_t* d_depth = nullptr;     // [B, N]
   int32_t* d_slot = nullptr;      // [B, N]
   int32_t* d_slot_inv = nullptr;  // [B, Ns]
-  int32_t* d_win = nullptr;       // [B, Ns, 4] per physical row: source rows (physical), -1/-2/-3 = history rows, INT32_MIN = padding row
+  int32_t* d_win = nullptr;       // [B, Ns, 4] per entry of the conv visiting order: source rows (physical), -1/-2/-3 = history rows, INT32_MIN = padding row
   int32_t* d_child_off = nullptr; // [B, N+2]
   int32_t* d_child_list = nullptr;// [B, N]
   int32_t* d_conv_prog = nullptr; // [B, Ns] conv visiting order (depth first): physical row | flag << 16; flag 0 = fetch the whole

@@ -95,7 +95,8 @@ __device__ int check_path_staged(const int* acc, const int* par, int N, int len,
 // parent of the previous row (only the own row changes), so one load per row replaces four; the own
 // rows of the next eight entries are always in flight (the kernel is bound by the special-function
 // unit, two operations per element for the SiLU, and by load latency, not by bandwidth).  Windows
-// that cannot be derived come from the per-row table (physical rows, or -1..-3 for the history rows).
+// that cannot be derived come from a table in the same visiting order (physical rows, or -1..-3 for
+// the history rows), fetched together with the order itself.
 // Taps are applied oldest first in fp32 starting from zero (packed FMAs: two correctly rounded fp32
 // lanes per instruction, same bits as scalar fmaf), bias last, SiLU in fp32, one round-to-nearest-even
 // cast (Sec. "Precompute branch histories while preserving arithmetic": tap order and cast points are
@@ -119,7 +120,7 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
     if (e0 + r < s.Ns) {
       prog = t.conv_prog[(size_t)b * s.Ns + e0 + r];
       if (!seq_ok) prog = (prog & 0xFFFF) | (3 << 16);        // skipped sequence: every row is a zero row
-      w = t.win[((size_t)b * s.Ns + (prog & 0xFFFF)) * 4 + j];
+      w = t.win[((size_t)b * s.Ns + e0 + r) * 4 + j];
     }
     s_win[r][j] = w;
     if (j == 0) s_prog[r] = (e0 + r < s.Ns) ? prog : -1;
