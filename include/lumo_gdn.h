@@ -284,6 +284,23 @@ int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_ar
                     int n_layers, const int32_t* accepted_dev, const int32_t* len_dev, int lmax,
                     void* stream);
 
+/* Commit of the previous cycle folded into this cycle's verify: the same result as
+ *   lumo_gdn_commit(ctx, prev_desc, prev_layers, n_layers, accepted_dev, len_dev, lmax, stream);
+ *   lumo_gdn_tree_verify(ctx, desc, layers, n_layers, stream);
+ * with the running state read once: the scan replays the accepted path of the previous tree into
+ * the state rows as it loads them, writes them back in place and verifies the new tree from there
+ * (the paper's own design replays at once with a native update, Sec. "Sequential arithmetic and
+ * accepted-path replay"; it names the fusion with the next verification as another system's choice,
+ * Sec. "Temporary state versus recomputation").  prev_layers[l] and layers[l] must name the same
+ * state, state_row and conv_hist and must share shapes, dtypes and options; the previous cycle's
+ * q/k/v/x/gates must live in buffers of their own (they are read while the new ones are written).
+ * prev_layers[l].status receives the commit's per-sequence status, layers[l].status the verify's.
+ * The fused kernel serves d = 128, bf16 operands, trees of at most 64 nodes and depth 16,
+ * lmax <= 16; every other case runs the two calls above one after the other.  Enqueues only. */
+int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const lumo_gdn_args* prev_layers,
+                           const int32_t* accepted_dev, const int32_t* len_dev, int lmax,
+                           const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -37,7 +37,7 @@ EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_s
            "lumo_ctx_timing_enable", "lumo_ctx_timing_read", "lumo_ctx_set_scan_algo", "lumo_ctx_set_overlap",
            "lumo_tree_desc_create", "lumo_tree_desc_destroy", "lumo_tree_desc_get",
            "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit",
-           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_tree_accept", "lumo_select_spine_top3"]
+           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_tree_accept", "lumo_select_spine_top3", "lumo_gdn_commit_verify"]
 
 
 class LumoError(RuntimeError):
@@ -106,6 +106,8 @@ _lib.lumo_gdn_tree_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.P
 _lib.lumo_gdn_tree_scan_static.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
                                            ctypes.c_void_p]
 _lib.lumo_static_stack_bytes.restype = ctypes.c_int64
+_lib.lumo_gdn_commit_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                        ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
 _lib.lumo_select_spine_top3.argtypes = [ctypes.c_void_p, ctypes.POINTER(_SelectArgs), ctypes.c_void_p, ctypes.c_void_p,
                                         ctypes.c_void_p]
 _lib.lumo_tree_accept.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_AcceptArgs), ctypes.c_int,
@@ -217,6 +219,14 @@ class Context:
             setattr(a, name, _ptr(t))
         self._check(_lib.lumo_tree_accept(self._h, desc._h, ctypes.byref(a), int(accepted.shape[1]), _ptr(accepted),
                                           _ptr(length), _ptr(next_token), _ptr(final_node), _stream(stream)))
+
+    def commit_verify(self, prev_desc: "TreeDesc", prev_layers, accepted: torch.Tensor, length: torch.Tensor,
+                      desc: "TreeDesc", layers, stream=None):
+        """commit(prev_desc, prev_layers, accepted, length) then verify(desc, layers), the state read once."""
+        parr = prev_layers if isinstance(prev_layers, ctypes.Array) else self.pack(prev_layers)
+        arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)
+        self._check(_lib.lumo_gdn_commit_verify(self._h, prev_desc._h, parr, _ptr(accepted), _ptr(length),
+                                                int(accepted.shape[1]), desc._h, arr, len(layers), _stream(stream)))
 
     def select_spine_top3(self, logits: torch.Tensor, spine: torch.Tensor, cand: torch.Tensor, split: int = 0,
                           stream=None):

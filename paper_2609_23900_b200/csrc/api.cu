@@ -555,9 +555,64 @@ int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_ar
   cudaStream_t st = (cudaStream_t)stream;
   const TreeDev t = tree_view(desc, 0);
   cudaError_t e = timed(ctx, LUMO_K_COMMIT, st, [&] {
-    return launch_commit(s, t, lb, accepted_dev, len_dev, lmax, layers[0].x != nullptr, use_overlap(ctx, s), st);
+    return launch_commit(s, t, lb, accepted_dev, len_dev, lmax, true, layers[0].x != nullptr, use_overlap(ctx, s), st);
   });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "commit launch");
+}
+
+int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const lumo_gdn_args* prev_layers,
+                           const int32_t* accepted_dev, const int32_t* len_dev, int lmax,
+                           const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers, void* stream) {
+  Shape ps, s;
+  LayerBatch lb;
+  FusedPrev fp;
+  std::memset(&lb, 0, sizeof(lb));
+  std::memset(&fp, 0, sizeof(fp));
+  int rc = prepare(ctx, prev_desc, prev_layers, n_layers, false, &ps, &fp.lb);
+  if (rc != LUMO_OK) return rc;
+  rc = prepare(ctx, desc, layers, n_layers, true, &s, &lb);
+  if (rc != LUMO_OK) return rc;
+  if (!accepted_dev || !len_dev) return fail(ctx, LUMO_ERR_ARG, "accepted_dev and len_dev are required");
+  if (lmax < 1) return fail(ctx, LUMO_ERR_ARG, "lmax must be positive");
+  if (prev_desc->B != desc->B) return fail(ctx, LUMO_ERR_ARG, "both trees must cover the same batch");
+  if (ps.Hk != s.Hk || ps.Hv != s.Hv || ps.d != s.d || ps.in_dtype != s.in_dtype || ps.gate_dtype != s.gate_dtype ||
+      ps.l2norm != s.l2norm || ps.l2_eps != s.l2_eps || ps.gate_mode != s.gate_mode || ps.n_state_rows != s.n_state_rows)
+    return fail(ctx, LUMO_ERR_ARG, "both cycles must share shapes, dtypes and options");
+  for (int l = 0; l < n_layers; ++l) {
+    const lumo_gdn_args &p = prev_layers[l], &c = layers[l];
+    if (p.state != c.state || p.state_row != c.state_row || p.conv_hist != c.conv_hist)
+      return fail(ctx, LUMO_ERR_ARG, "both cycles must name the same state, state_row and conv_hist");
+    if (p.k == c.k || p.v == c.v || (p.x && p.x == c.x))
+      return fail(ctx, LUMO_ERR_ARG, "the previous cycle's operands must live in their own buffers");
+    if (p.gate_mode == 1 && (p.a_log != c.a_log || p.dt_bias != c.dt_bias))
+      return fail(ctx, LUMO_ERR_ARG, "both cycles must share a_log and dt_bias");
+  }
+  const bool gram_ok = desc->d_tc_meta != nullptr && gram_supported(s, desc->max_depth);
+  const bool fused = gram_ok && ctx->scan_algo != 1 && desc->n_groups == desc->B && lmax <= kFusedMaxPath;
+  if (!fused) {   // same result from the two separate calls
+    rc = lumo_gdn_commit(ctx, prev_desc, prev_layers, n_layers, accepted_dev, len_dev, lmax, stream);
+    if (rc != LUMO_OK) return rc;
+    return lumo_gdn_tree_verify(ctx, desc, layers, n_layers, stream);
+  }
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const TreeDev pt = tree_view(prev_desc, 0);
+  const TreeDev t = tree_view(desc, 0);
+  fp.parent = pt.parent; fp.slot = pt.slot; fp.N = prev_desc->N; fp.Ns = prev_desc->Ns;
+  fp.accepted = accepted_dev; fp.len = len_dev; fp.lmax = lmax;
+  cudaError_t e = cudaSuccess;
+  if (prev_layers[0].x) {   // convolution history of the accepted path, ahead of the convolution that reads it
+    e = timed(ctx, LUMO_K_COMMIT, st, [&] {
+      return launch_commit(ps, pt, fp.lb, accepted_dev, len_dev, lmax, false, true, use_overlap(ctx, s), st);
+    });
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "history launch");
+  }
+  if (layers[0].x) {
+    e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, use_overlap(ctx, s), st); });
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
+  }
+  e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, use_overlap(ctx, s), st); });
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "fused scan launch");
 }
 
 }  // extern "C"

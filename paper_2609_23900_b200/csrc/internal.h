@@ -112,6 +112,15 @@ struct Shape {
   int gate_mode;
 };
 
+// What the fused commit + verify scan needs of the previous cycle: its layers (recorded k, v, gates,
+// status), its tree (parent, slot) and the device-resident accepted path.
+constexpr int kFusedMaxPath = 16;
+struct FusedPrev {
+  LayerBatch lb;
+  const int32_t* parent; const int32_t* slot; int N, Ns;
+  const int32_t* accepted; const int32_t* len; int lmax;
+};
+
 struct TreeDev {
   const int32_t* parent; const int32_t* depth; const int32_t* slot; const int32_t* slot_inv;
   const int32_t* win; const int32_t* conv_prog; const int32_t* sched; const int32_t* nops; int max_ops; int max_levels;
@@ -149,6 +158,22 @@ __device__ __forceinline__ float2 load_gates(const LayerPtrs& L, const Shape& s,
     b = 1.f / (1.f + expf(-b));
   }
   return make_float2(a, b);
+}
+
+// Accepted-path check; every CTA of a sequence reaches the same answer.  Order of checks: length,
+// then per entry range, root, link.  The path's entries and their parents were staged in shared memory
+// (parent -2 marks an entry outside [0, N)).
+__device__ __forceinline__ int check_path_staged(const int* acc, const int* par, int N, int len, int lmax) {
+  if (len < 0 || len > lmax) return LUMO_SEQ_BAD_LEN;
+  int prev = -1;
+  for (int t = 0; t < len; ++t) {       // bounded by lmax
+    const int a = acc[t];
+    if (a < 0 || a >= N) return LUMO_SEQ_BAD_NODE;
+    if (t == 0) { if (par[t] != -1) return LUMO_SEQ_BAD_ROOT; }
+    else if (par[t] != prev) return LUMO_SEQ_BAD_LINK;
+    prev = a;
+  }
+  return LUMO_SEQ_OK;
 }
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
@@ -232,10 +257,13 @@ cudaError_t launch_select(const void* logits, int dtype, int rows, int V, int sp
 bool gram_supported(const Shape& s, int max_depth);
 cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
                              cudaStream_t st);
+// same scan, first replaying the previous cycle's accepted path into the state it has just loaded
+cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
+                                   int sm_count, bool pdl, cudaStream_t st);
 // device address of the built-in stack on `device` (which must be current); looked up once per device
 cudaError_t static_stack_address(int device, float** ptr);
 cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb, const int32_t* accepted,
-                          const int32_t* len, int lmax, bool with_hist, bool pdl, cudaStream_t st);
+                          const int32_t* len, int lmax, bool with_state, bool with_hist, bool pdl, cudaStream_t st);
 cudaError_t launch_path_from_node(const TreeDev& t, int B, int N, const int32_t* node, int lmax,
                                   int32_t* accepted, int32_t* len, int32_t* status, cudaStream_t st);
 

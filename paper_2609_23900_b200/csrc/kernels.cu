@@ -69,22 +69,6 @@ template <> struct Packed4<__nv_bfloat16> {
   }
 };
 
-// Accepted-path check; every CTA of a sequence reaches the same answer.  Order of checks: length,
-// then per entry range, root, link.  The path's entries and their parents were staged in shared memory
-// (parent -2 marks an entry outside [0, N)).
-__device__ int check_path_staged(const int* acc, const int* par, int N, int len, int lmax) {
-  if (len < 0 || len > lmax) return LUMO_SEQ_BAD_LEN;
-  int prev = -1;
-  for (int t = 0; t < len; ++t) {       // bounded by lmax
-    const int a = acc[t];
-    if (a < 0 || a >= N) return LUMO_SEQ_BAD_NODE;
-    if (t == 0) { if (par[t] != -1) return LUMO_SEQ_BAD_ROOT; }
-    else if (par[t] != prev) return LUMO_SEQ_BAD_LINK;
-    prev = a;
-  }
-  return LUMO_SEQ_OK;
-}
-
 // ---------------------------------------------------------------------------------------
 // a1: ancestry-gathered causal depthwise conv (width 4) + SiLU -> recorded operands
 // ---------------------------------------------------------------------------------------
@@ -701,11 +685,12 @@ cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, 
 }
 
 cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb, const int32_t* accepted,
-                          const int32_t* len, int lmax, bool with_hist, bool pdl, cudaStream_t st) {
+                          const int32_t* len, int lmax, bool with_state, bool with_hist, bool pdl, cudaStream_t st) {
+  if (!with_state && !with_hist) return cudaSuccess;
   return dispatch(s.d, s.in_dtype, [&](auto dc, auto tc) {
     constexpr int D = decltype(dc)::value;
     using T = decltype(tc);
-    const int n_state = s.Hv * (D / kRows);
+    const int n_state = with_state ? s.Hv * (D / kRows) : 0;
     const int per_thread = 16 / (int)sizeof(T);
     const int n_hist = with_hist ? (s.C / per_thread + kScanThreads - 1) / kScanThreads : 0;
     dim3 grid(n_state + n_hist, s.B, s.n_layers);

@@ -85,6 +85,17 @@ struct Small {
 };
 constexpr int kSmemBytes = kOffSmall + (int)sizeof(Small) + 1024;   // + alignment slack
 
+// fused commit + verify: the previous cycle's accepted path and its operands for this (sequence, head)
+struct PrevStage {
+  int32_t acc[kFusedMaxPath], par[kFusedMaxPath], phys[kFusedMaxPath];
+  float ks[kFusedMaxPath];           // key normalisation factor of each accepted node
+  float2 gates[kFusedMaxPath];       // alpha, beta
+  __align__(16) __nv_bfloat16 k[kFusedMaxPath][kD];
+  __align__(16) __nv_bfloat16 v[kFusedMaxPath][kD];
+};
+constexpr int kOffPrev = kOffSmall + (((int)sizeof(Small) + 15) / 16) * 16;
+constexpr int kSmemBytesFused = kOffPrev + (int)sizeof(PrevStage) + 1024;
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* gmem) {
@@ -193,9 +204,12 @@ struct NodeOps {
 
 // NT = node tile of the MMAs: 64, or 32 when no group of the launch has more than 32 nodes (K rows
 // 0..NT-1 and Q rows NT..2NT-1 of the operand tile; the products occupy NT + NT + NT columns)
-template <int NT>
-__global__ void __launch_bounds__(kThreads, 2)
-scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
+// kFused: before anything else the previous cycle's accepted path is replayed into the state rows as
+// they pass through the registers (same per-token update as the commit kernel), and the rows are
+// written back in place; the scan then runs from the updated state.  One group per sequence only.
+template <int NT, bool kFused>
+__device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t, const LayerBatch& lb, int n_items,
+                                               const FusedPrev* fp) {
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment for the swizzled operand tiles; plain pointer arithmetic on the shared
   // array keeps the pointers in the shared address space
@@ -242,6 +256,10 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
         for (int ps = grp; ps < s.Ns; ps += 2)
           store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + vrow, s.out_dtype, 0.f);
         if (L.status && hv == 0 && tid == 0) L.status[b] = row < 0 ? LUMO_SEQ_OK : LUMO_SEQ_BAD_ROW;
+        if constexpr (kFused) {
+          int32_t* pst = fp->lb.l[layer].status;
+          if (pst && hv == 0 && tid == 0) pst[b] = row < 0 ? LUMO_SEQ_OK : LUMO_SEQ_BAD_ROW;
+        }
       }
       continue;
     }
@@ -266,7 +284,58 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     } else if (tid < 2 * kNT + 20) {
       sm.lvl[tid - 2 * kNT] = t.tc_lvl[gi * 20 + tid - 2 * kNT];
     }
+    bool replay = false;
+    int plen = 0;
+    if constexpr (kFused) {
+      // the accepted path of the previous cycle: entries, parents, physical rows (one level of dependent loads)
+      PrevStage& ps = *reinterpret_cast<PrevStage*>(smem + kOffPrev);
+      plen = fp->len[b];
+      const int lcap = plen < 0 ? 0 : (plen > fp->lmax ? 0 : plen);
+      if (tid >= 2 * kNT + 32 && tid < 2 * kNT + 32 + lcap) {
+        const int tt = tid - (2 * kNT + 32);
+        const int a = fp->accepted[(size_t)b * fp->lmax + tt];
+        const bool ok = a >= 0 && a < fp->N;
+        ps.acc[tt] = a;
+        ps.par[tt] = ok ? fp->parent[(size_t)b * fp->N + a] : -2;
+        ps.phys[tt] = ok ? fp->slot[(size_t)b * fp->N + a] : 0;
+      }
+    }
     __syncthreads();
+    if constexpr (kFused) {
+      PrevStage& ps = *reinterpret_cast<PrevStage*>(smem + kOffPrev);
+      const LayerPtrs& PL = fp->lb.l[layer];
+      const int st = check_path_staged(ps.acc, ps.par, fp->N, plen, fp->lmax);    // same answer in every thread
+      if (PL.status && hv == 0 && tid == 0) PL.status[b] = st;
+      replay = st == LUMO_SEQ_OK && plen > 0;
+      if (replay) {
+        // recorded key and value rows of the accepted nodes, gates; these were complete long before
+        // this kernel's predecessor started
+        const __nv_bfloat16* pk = reinterpret_cast<const __nv_bfloat16*>(PL.k);
+        const __nv_bfloat16* pv = reinterpret_cast<const __nv_bfloat16*>(PL.v);
+        for (int e = tid; e < plen * 32; e += kThreads) {            // bounded: <= 512
+          const int tt = e >> 5, c = e & 15;
+          const size_t pr = (size_t)b * fp->Ns + ps.phys[tt];
+          if ((e & 16) == 0)
+            *reinterpret_cast<uint4*>(&ps.k[tt][c * 8]) = *reinterpret_cast<const uint4*>(pk + (pr * s.Hk + g) * kD + c * 8);
+          else
+            *reinterpret_cast<uint4*>(&ps.v[tt][c * 8]) = *reinterpret_cast<const uint4*>(pv + (pr * s.Hv + hv) * kD + c * 8);
+        }
+        if (tid < plen) ps.gates[tid] = load_gates(PL, s, ((size_t)b * fp->Ns + ps.phys[tid]) * s.Hv + hv, hv);
+      }
+      __syncthreads();
+      if (replay) {
+        for (int tt = warp; tt < plen; tt += kWarps) {               // bounded: <= 16
+          const uint2 w = *reinterpret_cast<const uint2*>(&ps.k[tt][4 * lane]);
+          const float k0 = __uint_as_float(w.x << 16), k1 = __uint_as_float(w.x & 0xFFFF0000u);
+          const float k2 = __uint_as_float(w.y << 16), k3 = __uint_as_float(w.y & 0xFFFF0000u);
+          float kk = fmaf(k0, k0, fmaf(k1, k1, fmaf(k2, k2, k3 * k3)));
+#pragma unroll
+          for (int o = 16; o > 0; o >>= 1) kk += __shfl_xor_sync(0xffffffffu, kk, o);
+          if (lane == 0) ps.ks[tt] = s.l2norm ? rsqrtf(kk + s.l2_eps) : 1.f;
+        }
+      }
+      __syncthreads();
+    }
     PROF(1);
     // ---- b. gates (consumed much later); K and Q rows -> swizzled operand tile (cp.async) ---------
     // K, Q, V may still be in the making (the convolution runs right before this kernel): everything
@@ -308,11 +377,44 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
     // ---- c. pre-tree state -> bf16 hi + lo operand tiles ------------------------------------------
     {
       const int kblock = lane >> 4, chunk = (lane & 15) >> 1, half = lane & 1;
+      // fused mode: rows r0 + 8u of the state, held as x[u], take the accepted path's updates
+      // (u_r = S_r . k, delta_r = beta (v_r - alpha ks u_r), S_r <- alpha S_r + delta_r ks k) and go back to memory
+      auto replay_rows = [&](int r0) {
+        if constexpr (kFused) {
+          if (!replay) return;
+          const PrevStage& ps = *reinterpret_cast<const PrevStage*>(smem + kOffPrev);
+          for (int tt = 0; tt < plen; ++tt) {                        // bounded: <= 16
+            const uint2 w = *reinterpret_cast<const uint2*>(&ps.k[tt][4 * lane]);
+            const float4 kv = make_float4(__uint_as_float(w.x << 16), __uint_as_float(w.x & 0xFFFF0000u),
+                                          __uint_as_float(w.y << 16), __uint_as_float(w.y & 0xFFFF0000u));
+            const float a = ps.gates[tt].x, bt = ps.gates[tt].y, ks = ps.ks[tt];
+            float p[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) p[u] = fmaf(x[u].x, kv.x, fmaf(x[u].y, kv.y, fmaf(x[u].z, kv.z, x[u].w * kv.w)));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+              for (int u = 0; u < 8; ++u) p[u] += __shfl_xor_sync(0xffffffffu, p[u], o);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+              const float vv = __bfloat162float(ps.v[tt][r0 + 8 * u]);
+              const float gk = bt * (vv - a * (ks * p[u])) * ks;
+              x[u].x = fmaf(a, x[u].x, gk * kv.x); x[u].y = fmaf(a, x[u].y, gk * kv.y);
+              x[u].z = fmaf(a, x[u].z, gk * kv.z); x[u].w = fmaf(a, x[u].w, gk * kv.w);
+            }
+          }
+          float* Sw = const_cast<float*>(S0);
+#pragma unroll
+          for (int u = 0; u < 8; ++u) *reinterpret_cast<float4*>(Sw + (size_t)(r0 + 8 * u) * kD + lane * 4) = x[u];
+        }
+      };
+      replay_rows(warp);
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
         split_store(smem, kblock * 16384 + sw128_offset(warp + 8 * u, chunk) + half * 8, x[u]);
         x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * (8 + u)) * kD + lane * 4);   // second half
       }
+      replay_rows(warp + 64);
 #pragma unroll
       for (int u = 0; u < 8; ++u)
         split_store(smem, kblock * 16384 + sw128_offset(warp + 8 * (8 + u), chunk) + half * 8, x[u]);
@@ -544,6 +646,18 @@ scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
+template <int NT>
+__global__ void __launch_bounds__(kThreads, 2)
+scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
+  scan_gram_body<NT, false>(s, t, lb, n_items, nullptr);
+}
+
+template <int NT>
+__global__ void __launch_bounds__(kThreads, 2)
+scan_gram_fused_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items, FusedPrev fp) {
+  scan_gram_body<NT, true>(s, t, lb, n_items, &fp);
+}
+
 }  // namespace
 
 bool gram_supported(const Shape& s, int max_depth) {
@@ -567,6 +681,23 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
   if (t.max_group_nodes <= 32)
     return launch_kernel(scan_gram_kernel<32>, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
   return launch_kernel(scan_gram_kernel<64>, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
+}
+
+cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
+                                   int sm_count, bool pdl, cudaStream_t st) {
+  const int items = s.n_layers * t.n_groups * s.Hv;
+  static bool configured = false;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(scan_gram_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesFused);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(scan_gram_fused_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesFused);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  const int grid = items < 2 * sm_count ? items : 2 * sm_count;
+  if (t.max_group_nodes <= 32)
+    return launch_kernel(scan_gram_fused_kernel<32>, dim3(grid), dim3(kThreads), kSmemBytesFused, st, pdl, s, t, lb, items, fp);
+  return launch_kernel(scan_gram_fused_kernel<64>, dim3(grid), dim3(kThreads), kSmemBytesFused, st, pdl, s, t, lb, items, fp);
 }
 
 #ifdef LUMO_GRAM_PROFILE

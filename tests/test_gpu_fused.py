@@ -1,0 +1,132 @@
+"""lumo_gdn_commit_verify: the previous cycle's commit folded into this cycle's verify must equal the
+two separate steps: committed state, history, statuses and the new tree's outputs against the oracle
+(commit oracle, then conv and scan oracles from the committed state), and against the unfused calls."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import gdn_oracle as O
+from paper_2609_23900_b200 import binding, workload as W
+from paper_2609_23900_b200.runtime import DeviceCase
+from tests.harness import assert_close, ctx
+
+pytestmark = pytest.mark.gpu
+
+
+def _cycles(kind):
+    """Previous and current cycle over the same sequences: same heads and state pool, different trees."""
+    if kind == "cfg2":
+        P, C = W.config2(B=4), W.config2(B=4, seed=W.BASE_SEED + 77)
+    elif kind == "two_layers":
+        P, C = W.config2(B=3, n_layers=2), W.config2(B=3, n_layers=2, seed=W.BASE_SEED + 78)
+    elif kind == "paper_then_cfg3":     # padded permuted 28-of-32 tree, then 32-node trees (32-node MMA tile)
+        P, C = W.config_paper(B=4), W.config3(B=4, n_layers=1)
+    else:                               # 256-node trees: several groups per sequence, served by the two separate calls
+        P, C = W.config2(B=2), W.make_case("big", [W.tree_star(200)] * 2, seed=9, Hk=16, Hv=32, d=128, in_dtype="bf16")
+    C.state_row = P.state_row.copy()
+    C.rows = P.rows
+    for LP, LC in zip(P.layers, C.layers):
+        LC.state = LP.state.copy()
+        LC.hist = LP.hist.copy()
+    return P, C
+
+
+def _share_state(dcP, dcC):
+    """Layers of the current cycle that name the previous cycle's state, history and row tensors."""
+    c = dcC.case
+    out = []
+    for l, layer in enumerate(dcC.layers):
+        t = dict(layer.tensors)
+        t.update(state=dcP.t("state", l), conv_hist=dcP.t("conv_hist", l), state_row=dcP.state_row)
+        out.append(binding.GdnLayer(Hk=c.Hk, Hv=c.Hv, d=c.d, scale=dcC.scale, qk_l2norm=dcC.qk_l2norm, l2_eps=dcC.l2_eps, **t))
+    return out
+
+
+def _oracle(P, C, dcP, layersC, l, accepted, length):
+    """commit(P) then conv + scan(C) in fp64, on the operands the GPU recorded."""
+    LP, LC = P.layers[l], C.layers[l]
+    f = lambda t: t.to(torch.float64).cpu().numpy()
+    st1, hist1, status, _ = O.commit(P.parent, P.slot, P.state_row, dcP.np("q", l), dcP.np("k", l), dcP.np("v", l),
+                                     LP.alpha, LP.beta, LP.state, accepted, length, x=LP.x, hist=LP.hist,
+                                     l2norm=dcP.qk_l2norm, eps=dcP.l2_eps)
+    y = O.conv(C.parent, C.slot, C.state_row, LC.x, LC.conv_w, LC.conv_b, hist1, C.Ns, out_dtype="bf16")
+    tc = layersC[l].tensors
+    o_ref, _, _ = O.scan(C.parent, C.slot, C.state_row, f(tc["q"]), f(tc["k"]), f(tc["v"]), LC.alpha, LC.beta, st1,
+                         l2norm=True, eps=1e-6)
+    return st1, hist1, status, y, o_ref
+
+
+@pytest.mark.parametrize("kind", ["cfg2", "two_layers", "paper_then_cfg3", "fallback_many_groups"])
+def test_commit_verify_equals_commit_then_verify(kind):
+    P, C = _cycles(kind)
+    c = ctx()
+    dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
+    dcP.verify()                                    # records the previous cycle's operands
+    layersC = _share_state(dcP, dcC)
+    c.commit_verify(dcP.desc, dcP.layers, dcP.accepted, dcP.accepted_len, dcC.desc, layersC)
+    torch.cuda.synchronize()
+    hk = C.Hk * C.d
+    for l in range(len(C.layers)):
+        st1, hist1, status, y, o_ref = _oracle(P, C, dcP, layersC, l, P.accepted, P.accepted_len)
+        assert_close(dcP.np("state", l), st1, what=f"{kind} committed state, layer {l}")
+        assert np.array_equal(dcP.np("conv_hist", l), hist1), "history"
+        assert dcP.t("status", l).cpu().numpy().tolist() == status.tolist()
+        f = lambda t: t.to(torch.float64).cpu().numpy()
+        tc = layersC[l].tensors
+        got = np.concatenate([f(tc["q"]).reshape(C.B, C.Ns, hk), f(tc["k"]).reshape(C.B, C.Ns, hk),
+                              f(tc["v"]).reshape(C.B, C.Ns, C.Hv * C.d)], axis=-1)
+        assert (got == y).mean() > 0.98             # the new conv saw the committed history
+        assert_close(f(tc["out"]), o_ref, what=f"{kind} outputs of the new tree, layer {l}")
+        assert tc["status"].cpu().numpy().tolist() == [0] * C.B
+    # against the two separate calls on fresh copies
+    dcP2, dcC2 = DeviceCase(c, P), DeviceCase(c, C)
+    dcP2.verify()
+    layersC2 = _share_state(dcP2, dcC2)
+    dcP2.commit()
+    c.verify(dcC2.desc, layersC2)
+    torch.cuda.synchronize()
+    for l in range(len(C.layers)):
+        a, b = dcP.np("state", l), dcP2.np("state", l)
+        assert np.abs(a - b).max() <= 1e-5 * max(1.0, np.abs(b).max())
+        assert torch.equal(dcP.t("conv_hist", l), dcP2.t("conv_hist", l))
+        o1 = layersC[l].tensors["out"].to(torch.float64).cpu().numpy()
+        o2 = layersC2[l].tensors["out"].to(torch.float64).cpu().numpy()
+        assert np.abs(o1 - o2).max() <= 1e-4 * (1.0 + np.abs(o2).max())
+
+
+def test_commit_verify_rejects_a_bad_path_and_skips_empty_ones():
+    P, C = _cycles("cfg2")
+    acc, ln = P.accepted.copy(), P.accepted_len.copy()
+    ln[1] = 0                                       # nothing accepted: state stays
+    depth = W.tree_depths(P.parent[2].tolist())
+    root = int(np.flatnonzero(P.parent[2] < 0)[0])
+    acc[2, :2] = [root, next(i for i in range(P.N) if depth[i] == 3)]   # second entry is no child of the first
+    ln[2] = 2
+    c = ctx()
+    dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
+    dcP.verify()
+    layersC = _share_state(dcP, dcC)
+    dev = dcP.accepted.device
+    c.commit_verify(dcP.desc, dcP.layers, torch.from_numpy(acc).to(dev), torch.from_numpy(ln).to(dev), dcC.desc, layersC)
+    torch.cuda.synchronize()
+    st1, hist1, status, y, o_ref = _oracle(P, C, dcP, layersC, 0, acc, ln)
+    assert status[2] != 0 and status[1] == 0
+    assert dcP.t("status").cpu().numpy().tolist() == status.tolist()
+    assert_close(dcP.np("state"), st1, what="state")
+    row1, row2 = P.state_row[1], P.state_row[2]
+    assert np.array_equal(dcP.np("state")[row1], P.layers[0].state[row1])      # bitwise untouched
+    assert np.array_equal(dcP.np("state")[row2], P.layers[0].state[row2])
+    assert np.array_equal(dcP.np("conv_hist"), hist1)
+    assert_close(layersC[0].tensors["out"].to(torch.float64).cpu().numpy(), o_ref, what="outputs")
+
+
+def test_commit_verify_argument_checks():
+    P, C = _cycles("cfg2")
+    c = ctx()
+    dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
+    with pytest.raises(binding.LumoError) as e:     # the two cycles name different state tensors
+        c.commit_verify(dcP.desc, dcP.layers, dcP.accepted, dcP.accepted_len, dcC.desc, dcC.layers)
+    assert e.value.code == 1
+    with pytest.raises(binding.LumoError) as e:     # the previous operands must not be the new ones
+        c.commit_verify(dcP.desc, dcP.layers, dcP.accepted, dcP.accepted_len, dcP.desc, dcP.layers)
+    assert e.value.code == 1
