@@ -601,14 +601,21 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
   fp.parent = pt.parent; fp.slot = pt.slot; fp.N = prev_desc->N; fp.Ns = prev_desc->Ns;
   fp.accepted = accepted_dev; fp.len = len_dev; fp.lmax = lmax;
   cudaError_t e = cudaSuccess;
-  if (prev_layers[0].x) {   // convolution history of the accepted path, ahead of the convolution that reads it
+  // Convolution history of the accepted path.  With a convolution in this cycle the two kernels take
+  // care of it (the conv reads the committed rows through the path, the scan writes them back);
+  // a scan-only verify needs the history CTAs of the commit kernel.
+  fp.hist_in_kernels = prev_layers[0].x != nullptr && layers[0].x != nullptr;
+  if (prev_layers[0].x && !fp.hist_in_kernels) {
     e = timed(ctx, LUMO_K_COMMIT, st, [&] {
       return launch_commit(ps, pt, fp.lb, accepted_dev, len_dev, lmax, false, true, use_overlap(ctx, s), st);
     });
     if (e != cudaSuccess) return cuda_fail(ctx, e, "history launch");
   }
   if (layers[0].x) {
-    e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, use_overlap(ctx, s), st); });
+    e = timed(ctx, LUMO_K_CONV, st, [&] {
+      return fp.hist_in_kernels ? launch_conv_fused(s, t, lb, fp, use_overlap(ctx, s), st)
+                                : launch_conv(s, t, lb, use_overlap(ctx, s), st);
+    });
     if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
   }
   e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, use_overlap(ctx, s), st); });

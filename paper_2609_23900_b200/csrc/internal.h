@@ -119,6 +119,7 @@ struct FusedPrev {
   LayerBatch lb;
   const int32_t* parent; const int32_t* slot; int N, Ns;
   const int32_t* accepted; const int32_t* len; int lmax;
+  int hist_in_kernels;   // 1: the conv reads the committed history through the path and the scan writes it back
 };
 
 struct TreeDev {
@@ -238,6 +239,9 @@ cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t 
 
 // launchers (kernels.cu); all return cudaError_t and only enqueue
 cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st);
+// same convolution reading the history the previous cycle's accepted path would commit (not yet in memory)
+cudaError_t launch_conv_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp, bool pdl,
+                              cudaStream_t st);
 cudaError_t launch_scan(const Shape& s, const TreeDev& t, const LayerBatch& lb, float* stack,
                         int grid, cudaStream_t st);
 // persistent grid size (CTAs resident at once) and the stack scratch it needs

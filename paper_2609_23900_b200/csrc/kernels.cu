@@ -86,10 +86,15 @@ template <> struct Packed4<__nv_bfloat16> {
 // cast (Sec. "Precompute branch histories while preserving arithmetic": tap order and cast points are
 // part of the result).
 
-template <typename T, int kConvRows>
-__global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerBatch lb) {
+// kFused: the three history rows are the ones the previous cycle's accepted path will commit, i.e. the
+// last three of [old history ; raw inputs of the accepted nodes], read in place through the path (the
+// scan that follows writes them to the history buffer once every CTA of this kernel has finished).
+template <typename T, int kConvRows, bool kFused>
+__device__ __forceinline__ void conv_body(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev* fp) {
   __shared__ int s_win[kConvRows][4];
   __shared__ int s_prog[kConvRows];
+  __shared__ int f_acc[kFusedMaxPath], f_par[kFusedMaxPath], f_phys[kFusedMaxPath];
+  __shared__ const T* f_hsrc[3];
   const int layer = blockIdx.z / s.B, b = blockIdx.z % s.B;
   const int e0 = blockIdx.y * kConvRows;               // first entry of the visiting order
   const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
@@ -108,6 +113,19 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
     }
     s_win[r][j] = w;
     if (j == 0) s_prog[r] = (e0 + r < s.Ns) ? prog : -1;
+  }
+  int plen = 0;
+  if constexpr (kFused) {
+    plen = fp->len[b];
+    const int lcap = plen < 0 ? 0 : (plen > fp->lmax ? 0 : plen);
+    const int tt = (int)threadIdx.x - 128;
+    if (tt >= 0 && tt < lcap) {
+      const int a = fp->accepted[(size_t)b * fp->lmax + tt];
+      const bool ok = a >= 0 && a < fp->N;
+      f_acc[tt] = a;
+      f_par[tt] = ok ? fp->parent[(size_t)b * fp->N + a] : -2;
+      f_phys[tt] = ok ? fp->slot[(size_t)b * fp->N + a] : 0;
+    }
   }
   using P4 = typename Packed4<T>::type;                // four elements as loaded
   float2 wp[4][2];                                     // tap j of channel pairs (0,1) and (2,3)
@@ -128,6 +146,20 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
     }
   }
   __syncthreads();
+  if constexpr (kFused) {
+    if (threadIdx.x == 0) {
+      // an invalid or empty path commits nothing: the history in memory is the history
+      const bool ok = seq_ok && check_path_staged(f_acc, f_par, fp->N, plen, fp->lmax) == LUMO_SEQ_OK;
+      const int leff = ok ? plen : 0;
+      const T* hbase = reinterpret_cast<const T*>(L.conv_hist) + (size_t)(seq_ok ? row : 0) * 3 * s.C;
+      const T* xprev = reinterpret_cast<const T*>(fp->lb.l[layer].x) + (size_t)b * fp->Ns * s.C;
+      for (int j = 0; j < 3; ++j) {
+        const int q = leff + j;        // index into [old0 old1 old2 x_a0 x_a1 ...]
+        f_hsrc[j] = q < 3 ? hbase + (size_t)q * s.C : xprev + (size_t)f_phys[q - 3] * s.C;
+      }
+    }
+    __syncthreads();
+  }
   if (c0 >= s.C) return;
   const bool has_bias = L.conv_b != nullptr;
   const int hkd = s.Hk * s.d;
@@ -141,7 +173,10 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
   const T* hist = reinterpret_cast<const T*>(L.conv_hist) + (size_t)(seq_ok ? row : 0) * 3 * s.C + c0;
 
   auto load_src = [&](int wj) -> float4 {              // one window entry: a row of x or of the history
-    const T* src = wj >= 0 ? x + (size_t)wj * s.C : hist + (size_t)(3 + wj) * s.C;
+    const T* src;
+    if (wj >= 0) src = x + (size_t)wj * s.C;
+    else if constexpr (kFused) src = f_hsrc[3 + wj] + c0;
+    else src = hist + (size_t)(3 + wj) * s.C;
     return Packed4<T>::unpack(*reinterpret_cast<const P4*>(src));
   };
   auto load_own = [&](int r) -> P4 {                   // the entry's own row (padding rows: zeros)
@@ -194,6 +229,15 @@ __global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerB
       *reinterpret_cast<float4*>(d) = make_float4(y[0], y[1], y[2], y[3]);
     }
   }
+}
+
+template <typename T, int kConvRows>
+__global__ void __launch_bounds__(256, 3) conv_kernel(Shape s, TreeDev t, LayerBatch lb) {
+  conv_body<T, kConvRows, false>(s, t, lb, nullptr);
+}
+template <typename T, int kConvRows>
+__global__ void __launch_bounds__(256, 3) conv_fused_kernel(Shape s, TreeDev t, LayerBatch lb, FusedPrev fp) {
+  conv_body<T, kConvRows, true>(s, t, lb, &fp);
 }
 
 // ---------------------------------------------------------------------------------------
@@ -614,6 +658,22 @@ static cudaError_t launch_conv_t(const Shape& s, const TreeDev& t, const LayerBa
   if (ctas(8) >= 2LL * sms)
     return launch_kernel(conv_kernel<T, 8>, dim3(slabs, (s.Ns + 7) / 8, seqs), dim3(256), 0, st, pdl, s, t, lb);
   return launch_kernel(conv_kernel<T, 4>, dim3(slabs, (s.Ns + 3) / 4, seqs), dim3(256), 0, st, pdl, s, t, lb);
+}
+
+cudaError_t launch_conv_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp, bool pdl,
+                              cudaStream_t st) {
+  if (s.in_dtype != LUMO_BF16) return cudaErrorInvalidValue;      // the fused path serves bf16 operands only
+  using T = __nv_bfloat16;
+  const int slabs = (s.C / 4 + 255) / 256, seqs = s.B * s.n_layers;
+  auto ctas = [&](int rows) { return (long long)slabs * ((s.Ns + rows - 1) / rows) * seqs; };
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (ctas(16) >= 2LL * sms)
+    return launch_kernel(conv_fused_kernel<T, 16>, dim3(slabs, (s.Ns + 15) / 16, seqs), dim3(256), 0, st, pdl, s, t, lb, fp);
+  if (ctas(8) >= 2LL * sms)
+    return launch_kernel(conv_fused_kernel<T, 8>, dim3(slabs, (s.Ns + 7) / 8, seqs), dim3(256), 0, st, pdl, s, t, lb, fp);
+  return launch_kernel(conv_fused_kernel<T, 4>, dim3(slabs, (s.Ns + 3) / 4, seqs), dim3(256), 0, st, pdl, s, t, lb, fp);
 }
 
 cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st) {

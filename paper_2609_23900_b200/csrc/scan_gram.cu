@@ -343,6 +343,30 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     // afterwards: it reads freely and writes only behind its own wait.
     pdl_wait();
     pdl_trigger();
+    if constexpr (kFused) {
+      // The convolution before this kernel read the committed history through the path; now that it has
+      // finished, the history buffer itself is brought up to date: the value heads of a sequence share
+      // out the channels, a thread moves its 16 bytes of all three rows (reads before writes).
+      if (fp->hist_in_kernels && replay && warp == kWarps - 1) {
+        const PrevStage& ps = *reinterpret_cast<const PrevStage*>(smem + kOffPrev);
+        const LayerPtrs& PL = fp->lb.l[layer];
+        const int chunks = s.C / 8;                                    // 16-byte pieces of a row of bf16 channels
+        const int per_head = (chunks + s.Hv - 1) / s.Hv;
+        __nv_bfloat16* hist = reinterpret_cast<__nv_bfloat16*>(L.conv_hist) + (size_t)row * 3 * s.C;
+        const __nv_bfloat16* xprev = reinterpret_cast<const __nv_bfloat16*>(PL.x) + (size_t)b * fp->Ns * s.C;
+        for (int c = hv * per_head + lane; c < min(chunks, (hv + 1) * per_head); c += 32) {   // bounded: per_head
+          uint4 rows3[3];
+#pragma unroll
+          for (int j = 0; j < 3; ++j) {
+            const int q = plen + j;    // index into [old0 old1 old2 x_a0 x_a1 ...]
+            const __nv_bfloat16* src = q < 3 ? hist + (size_t)q * s.C : xprev + (size_t)ps.phys[q - 3] * s.C;
+            rows3[j] = *reinterpret_cast<const uint4*>(src + c * 8);
+          }
+#pragma unroll
+          for (int j = 0; j < 3; ++j) *reinterpret_cast<uint4*>(hist + (size_t)j * s.C + c * 8) = rows3[j];
+        }
+      }
+    }
     float gate_a = 1.f, gate_b = 0.f;
     if (tid < N) {
       const size_t pr = (size_t)b * s.Ns + (sm.meta[tid] & 0xFFFF);
