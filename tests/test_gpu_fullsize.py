@@ -66,3 +66,38 @@ def test_config3_full_stack_sampled():
         check_samples(dc, case, layer, pairs)
     for layer in range(48):
         assert torch.isfinite(dc.t("out", layer).float()).all()
+
+
+def test_config3_fused_commit_verify_matches_the_separate_calls():
+    """48 layers in the launch configuration bench.py times: lumo_gdn_commit_verify against
+    lumo_gdn_commit followed by lumo_gdn_tree_verify, every layer, state and outputs."""
+    from paper_2609_23900_b200 import binding
+    from tests.test_gpu_fused import _share_state
+    P, C = W.config3(seed=W.BASE_SEED + 303), W.config3()
+    C.state_row = P.state_row.copy()
+    for LP, LC in zip(P.layers, C.layers):
+        LC.state = LP.state.copy()
+        LC.hist = LP.hist.copy()
+    c = ctx()
+    results = []
+    for fused in (True, False):
+        dcP, dcC = DeviceCase(c, P, out_dtype="bf16"), DeviceCase(c, C, out_dtype="bf16")
+        dcP.verify()
+        layersC = _share_state(dcP, dcC)
+        if fused:
+            c.commit_verify(dcP.desc, dcP.layers, dcP.accepted, dcP.accepted_len, dcC.desc, layersC)
+        else:
+            dcP.commit()
+            c.verify(dcC.desc, layersC)
+        torch.cuda.synchronize()
+        results.append((dcP, layersC))
+    (pf, lf), (pu, lu) = results
+    for l in range(len(C.layers)):
+        sf, su = pf.t("state", l), pu.t("state", l)
+        assert torch.isfinite(sf).all()
+        assert (sf - su).abs().max().item() <= 1e-5 * max(1.0, su.abs().max().item())
+        assert torch.equal(pf.t("conv_hist", l), pu.t("conv_hist", l))
+        assert torch.equal(pf.t("status", l), pu.t("status", l))
+        of, ou = lf[l].tensors["out"].float(), lu[l].tensors["out"].float()
+        assert bool(((of - ou).abs() <= 2.0 ** -7 * ou.abs() + 1e-3).all())   # bf16 outputs: one ulp apart at most
+        assert torch.equal(lf[l].tensors["k"], lu[l].tensors["k"]) and torch.equal(lf[l].tensors["v"], lu[l].tensors["v"])
