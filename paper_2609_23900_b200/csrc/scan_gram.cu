@@ -266,6 +266,21 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     if (first_group && L.status && hv == 0 && tid == 0) L.status[b] = LUMO_SEQ_OK;
 
     PROF(0);
+    int plen = 0;
+    if constexpr (kFused) {
+      // the accepted path of the previous cycle: entries, parents, physical rows (one level of dependent loads)
+      PrevStage& ps = *reinterpret_cast<PrevStage*>(smem + kOffPrev);
+      plen = fp->len[b];
+      const int lcap = plen < 0 ? 0 : (plen > fp->lmax ? 0 : plen);
+      if (tid >= 2 * kNT + 32 && tid < 2 * kNT + 32 + lcap) {
+        const int tt = tid - (2 * kNT + 32);
+        const int a = fp->accepted[(size_t)b * fp->lmax + tt];
+        const bool ok = a >= 0 && a < fp->N;
+        ps.acc[tt] = a;
+        ps.par[tt] = ok ? fp->parent[(size_t)b * fp->N + a] : -2;
+        ps.phys[tt] = ok ? fp->slot[(size_t)b * fp->N + a] : 0;
+      }
+    }
     // The pre-tree state is not written by the kernel before this one and its address needs no
     // table: its first half (warp w takes rows w, w+8, ...; one 512-byte row per instruction) is
     // requested first of all, ahead of the table loads and of the dependency wait.
@@ -285,21 +300,6 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       sm.lvl[tid - 2 * kNT] = t.tc_lvl[gi * 20 + tid - 2 * kNT];
     }
     bool replay = false;
-    int plen = 0;
-    if constexpr (kFused) {
-      // the accepted path of the previous cycle: entries, parents, physical rows (one level of dependent loads)
-      PrevStage& ps = *reinterpret_cast<PrevStage*>(smem + kOffPrev);
-      plen = fp->len[b];
-      const int lcap = plen < 0 ? 0 : (plen > fp->lmax ? 0 : plen);
-      if (tid >= 2 * kNT + 32 && tid < 2 * kNT + 32 + lcap) {
-        const int tt = tid - (2 * kNT + 32);
-        const int a = fp->accepted[(size_t)b * fp->lmax + tt];
-        const bool ok = a >= 0 && a < fp->N;
-        ps.acc[tt] = a;
-        ps.par[tt] = ok ? fp->parent[(size_t)b * fp->N + a] : -2;
-        ps.phys[tt] = ok ? fp->slot[(size_t)b * fp->N + a] : 0;
-      }
-    }
     __syncthreads();
     if constexpr (kFused) {
       PrevStage& ps = *reinterpret_cast<PrevStage*>(smem + kOffPrev);
