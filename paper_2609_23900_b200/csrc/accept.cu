@@ -163,8 +163,33 @@ accept_kernel(TreeDev t, int N, int Ns, AcceptView a, int lmax, int32_t* __restr
     if (a.mode == 0) {
       float bv = -1.f;
       int bi = 0x7fffffff;
-      for_slice(v_lo, v_hi, [&](int i) { return p[i]; },
-                [&](int i, float v) { if (v > bv) { bv = v; bi = i; } });
+      auto look = [&](int i, float v) { if (v > bv) { bv = v; bi = i; } };     // ascending i per thread
+      if ((V & 3) == 0 && (reinterpret_cast<uintptr_t>(p) & 15) == 0) {
+        // rows on 16-byte boundaries: the body of the slice in 16-byte loads, all of a thread's loads
+        // of one round in flight together; ragged ends element by element
+        const int a4 = (v_lo + 3) & ~3, b4 = max(a4, v_hi & ~3);
+        constexpr int kU4 = 5;
+        for (int q0 = a4 / 4 + tid; q0 < b4 / 4; q0 += kU4 * kAcceptThreads) {   // bounded: slice
+          float4 vals[kU4];
+#pragma unroll
+          for (int k = 0; k < kU4; ++k) {
+            const int q = q0 + k * kAcceptThreads;
+            if (q < b4 / 4) vals[k] = *reinterpret_cast<const float4*>(p + 4 * (size_t)q);
+          }
+#pragma unroll
+          for (int k = 0; k < kU4; ++k) {
+            const int q = q0 + k * kAcceptThreads;
+            if (q < b4 / 4) { look(4 * q, vals[k].x); look(4 * q + 1, vals[k].y); look(4 * q + 2, vals[k].z); look(4 * q + 3, vals[k].w); }
+          }
+        }
+        // the ragged ends hold lower (head) or higher (tail) indices than the body: ties are settled
+        // by index in the reduction, and within a thread the head is visited last but compared with >
+        // against a body value of higher index, so an equal head value must win explicitly
+        for (int i = v_lo + tid; i < min(a4, v_hi); i += kAcceptThreads) { const float v = p[i]; if (v > bv || (v == bv && i < bi)) { bv = v; bi = i; } }
+        for (int i = b4 + tid; i < v_hi; i += kAcceptThreads) look(i, p[i]);
+      } else {
+        for_slice(v_lo, v_hi, [&](int i) { return p[i]; }, look);
+      }
       nxt = cluster_argmax(cl, bv, bi, &xch);
       if (len < lmax)
         for (int ci = c_lo; ci < c_hi; ++ci) {                // bounded: children of one node

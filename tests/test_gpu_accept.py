@@ -90,3 +90,32 @@ def test_verify_accept_commit_without_host_round_trip():
                                       dc.np("beta"), L.state, ref[0], ref[1], l2norm=True, x=L.x, hist=L.hist)
     assert_close(dc.np("state"), st_ref, what="state committed along the device-selected path")
     assert np.array_equal(dc.np("conv_hist"), hist_ref)
+
+
+@pytest.mark.parametrize("V", [4096, 4099, 151936])
+def test_greedy_ties_take_the_lowest_token_on_every_load_path(V):
+    """Target rows whose maximum occurs several times, spread over the slices of the cluster and over
+    the ragged ends of the 16-byte body: the pending token must be the lowest such index."""
+    c = W.make_case("t", [W.tree_tiny()] * 3, seed=1, Hk=1, Hv=1, d=64, in_dtype="f32")
+    rs = np.random.default_rng(V)
+    p = rs.uniform(0.0, 0.5, size=(c.B, c.Ns + 1, V)).astype(np.float32)
+    for b in range(c.B):
+        for r in range(c.Ns + 1):
+            pos = rs.choice(V, size=5, replace=False)
+            if r % 3 == 0:
+                pos = np.concatenate([pos, [1, V - 1, V - 2]])      # ragged ends
+            p[b, r, pos] = 0.75
+    token = rs.integers(0, V, size=(c.B, c.Ns)).astype(np.int32)
+    for b in range(c.B):                                            # let the walk take a few steps
+        for i in range(c.N):
+            prow = c.Ns if c.parent[b, i] < 0 else c.slot[b, c.parent[b, i]]
+            token[b, c.slot[b, i]] = int(np.flatnonzero(p[b, prow] == p[b, prow].max())[0]) if i % 2 == 0 else token[b, c.slot[b, i]]
+    lmax = max(W.tree_depths(c.parent[0].tolist())) + 1
+    desc = ctx().tree_desc(c.parent, slot=c.slot, n_slots=c.Ns)
+    q = np.zeros((c.B, c.Ns, 1), np.float32)
+    acc, ln, nxt, fin = run_device(desc, c.Ns, token, p, q, np.zeros((c.B, c.Ns), np.float32), np.ones((c.B, V), np.float32), "greedy", lmax)
+    torch.cuda.synchronize()
+    ref = A.accept(c.parent, c.slot, c.Ns, token, p, None, None, None, mode=A.GREEDY, lmax=lmax)
+    assert acc.cpu().numpy().tolist() == ref[0].tolist() and ln.cpu().numpy().tolist() == ref[1].tolist()
+    assert nxt.cpu().numpy().tolist() == ref[2].tolist() and fin.cpu().numpy().tolist() == ref[3].tolist()
+    assert (ref[1] > 0).any()
