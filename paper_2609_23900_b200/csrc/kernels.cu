@@ -644,41 +644,36 @@ cudaError_t dispatch(int d, int in_dtype, F f) {
 // ---------------------------------------------------------------------------------------
 // launchers
 // ---------------------------------------------------------------------------------------
+// sixteen entries per CTA amortise the window set-up; small launches take fewer so that the grid still
+// covers the GPU
 template <typename T>
-static cudaError_t launch_conv_t(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st) {
-  // sixteen entries per CTA amortise the window set-up; small launches take fewer so that the grid
-  // still covers the GPU
+static cudaError_t launch_conv_t(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev* fp, bool pdl,
+                                 cudaStream_t st) {
   const int slabs = (s.C / 4 + 255) / 256, seqs = s.B * s.n_layers;
   auto ctas = [&](int rows) { return (long long)slabs * ((s.Ns + rows - 1) / rows) * seqs; };
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (ctas(16) >= 2LL * sms)
-    return launch_kernel(conv_kernel<T, 16>, dim3(slabs, (s.Ns + 15) / 16, seqs), dim3(256), 0, st, pdl, s, t, lb);
-  if (ctas(8) >= 2LL * sms)
-    return launch_kernel(conv_kernel<T, 8>, dim3(slabs, (s.Ns + 7) / 8, seqs), dim3(256), 0, st, pdl, s, t, lb);
-  return launch_kernel(conv_kernel<T, 4>, dim3(slabs, (s.Ns + 3) / 4, seqs), dim3(256), 0, st, pdl, s, t, lb);
+  auto go = [&](auto rows_c) {
+    constexpr int kRowsPerCta = decltype(rows_c)::value;
+    const dim3 grid(slabs, (s.Ns + kRowsPerCta - 1) / kRowsPerCta, seqs);
+    if (fp) return launch_kernel(conv_fused_kernel<T, kRowsPerCta>, grid, dim3(256), 0, st, pdl, s, t, lb, *fp);
+    return launch_kernel(conv_kernel<T, kRowsPerCta>, grid, dim3(256), 0, st, pdl, s, t, lb);
+  };
+  if (ctas(16) >= 2LL * sms) return go(std::integral_constant<int, 16>{});
+  if (ctas(8) >= 2LL * sms) return go(std::integral_constant<int, 8>{});
+  return go(std::integral_constant<int, 4>{});
+}
+
+cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st) {
+  if (s.in_dtype == LUMO_BF16) return launch_conv_t<__nv_bfloat16>(s, t, lb, nullptr, pdl, st);
+  return launch_conv_t<float>(s, t, lb, nullptr, pdl, st);
 }
 
 cudaError_t launch_conv_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp, bool pdl,
                               cudaStream_t st) {
   if (s.in_dtype != LUMO_BF16) return cudaErrorInvalidValue;      // the fused path serves bf16 operands only
-  using T = __nv_bfloat16;
-  const int slabs = (s.C / 4 + 255) / 256, seqs = s.B * s.n_layers;
-  auto ctas = [&](int rows) { return (long long)slabs * ((s.Ns + rows - 1) / rows) * seqs; };
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (ctas(16) >= 2LL * sms)
-    return launch_kernel(conv_fused_kernel<T, 16>, dim3(slabs, (s.Ns + 15) / 16, seqs), dim3(256), 0, st, pdl, s, t, lb, fp);
-  if (ctas(8) >= 2LL * sms)
-    return launch_kernel(conv_fused_kernel<T, 8>, dim3(slabs, (s.Ns + 7) / 8, seqs), dim3(256), 0, st, pdl, s, t, lb, fp);
-  return launch_kernel(conv_fused_kernel<T, 4>, dim3(slabs, (s.Ns + 3) / 4, seqs), dim3(256), 0, st, pdl, s, t, lb, fp);
-}
-
-cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st) {
-  if (s.in_dtype == LUMO_BF16) return launch_conv_t<__nv_bfloat16>(s, t, lb, pdl, st);
-  return launch_conv_t<float>(s, t, lb, pdl, st);
+  return launch_conv_t<__nv_bfloat16>(s, t, lb, &fp, pdl, st);
 }
 
 cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid, size_t* stack_bytes) {
