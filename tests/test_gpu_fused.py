@@ -130,3 +130,29 @@ def test_commit_verify_argument_checks():
     with pytest.raises(binding.LumoError) as e:     # the previous operands must not be the new ones
         c.commit_verify(dcP.desc, dcP.layers, dcP.accepted, dcP.accepted_len, dcP.desc, dcP.layers)
     assert e.value.code == 1
+
+
+def test_commit_verify_scan_only_cycle_updates_history_with_the_commit_kernel():
+    """The new cycle has no convolution (operands given): the history of the accepted path is then
+    gathered by the commit kernel's history CTAs ahead of the fused scan."""
+    P, C = _cycles("cfg2")
+    c = ctx()
+    dcP, dcC = DeviceCase(c, P), DeviceCase(c, C, use_conv=False, qk_l2norm=True)
+    dcP.verify()
+    layersC = []
+    for l, layer in enumerate(dcC.layers):
+        t = dict(layer.tensors)
+        t.update(state=dcP.t("state", l), state_row=dcP.state_row, conv_hist=dcP.t("conv_hist", l))
+        layersC.append(binding.GdnLayer(Hk=C.Hk, Hv=C.Hv, d=C.d, scale=dcC.scale, qk_l2norm=True, l2_eps=dcC.l2_eps, **t))
+    c.commit_verify(dcP.desc, dcP.layers, dcP.accepted, dcP.accepted_len, dcC.desc, layersC)
+    torch.cuda.synchronize()
+    LP, LC = P.layers[0], C.layers[0]
+    st1, hist1, status, _ = O.commit(P.parent, P.slot, P.state_row, dcP.np("q"), dcP.np("k"), dcP.np("v"), LP.alpha, LP.beta,
+                                     LP.state, P.accepted, P.accepted_len, x=LP.x, hist=LP.hist, l2norm=True, eps=dcP.l2_eps)
+    f = lambda t: t.to(torch.float64).cpu().numpy()
+    tc = layersC[0].tensors
+    o_ref, _, _ = O.scan(C.parent, C.slot, C.state_row, f(tc["q"]), f(tc["k"]), f(tc["v"]), LC.alpha, LC.beta, st1,
+                         l2norm=True, eps=dcC.l2_eps)
+    assert_close(dcP.np("state"), st1, what="state")
+    assert np.array_equal(dcP.np("conv_hist"), hist1)
+    assert_close(f(tc["out"]), o_ref, what="outputs")
