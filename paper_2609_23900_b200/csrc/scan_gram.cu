@@ -342,7 +342,9 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     // above touched only the descriptor tables and the state.  The dependent kernel (commit) is let in
     // afterwards: it reads freely and writes only behind its own wait.
     pdl_wait();
-    pdl_trigger();
+    // A fused launch rewrites the state, which a dependent (a commit, the next scan) requests ahead of
+    // its own wait: it lets nobody in before it has finished.
+    if constexpr (!kFused) pdl_trigger();
     if constexpr (kFused) {
       // The convolution before this kernel read the committed history through the path; now that it has
       // finished, the history buffer itself is brought up to date: the value heads of a sequence share

@@ -156,3 +156,24 @@ def test_commit_verify_scan_only_cycle_updates_history_with_the_commit_kernel():
     assert_close(dcP.np("state"), st1, what="state")
     assert np.array_equal(dcP.np("conv_hist"), hist1)
     assert_close(f(tc["out"]), o_ref, what="outputs")
+
+
+def test_commit_after_commit_verify_sees_the_rewritten_state():
+    """A plain commit right after a fused call (the last cycle of a generation) under kernel overlap:
+    it must start from the state the fused scan wrote, cycle after cycle, bitwise as without overlap."""
+    P, C = _cycles("cfg2")
+    res = {}
+    for on in (False, True):
+        c = ctx()
+        c.set_overlap(on)
+        dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
+        dcP.verify()
+        layersC = _share_state(dcP, dcC)
+        for _ in range(3):
+            c.commit_verify(dcP.desc, dcP.layers, dcP.accepted, dcP.accepted_len, dcC.desc, layersC)
+            c.commit(dcC.desc, layersC, dcC.accepted, dcC.accepted_len)
+        torch.cuda.synchronize()
+        res[on] = (dcP.t("state").clone(), dcP.t("conv_hist").clone(), layersC[0].tensors["out"].clone())
+    ctx().set_overlap(True)
+    for a, b in zip(res[False], res[True]):
+        assert torch.equal(a, b)
