@@ -226,6 +226,23 @@ def reference_arm(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def fused_arm(args):
+    """The same workload through lumo_gdn_commit_verify (the previous cycle's commit folded into the
+    verify), timed by a run of this script of its own; reported beside the headline, never as it."""
+    import subprocess
+    cmd = [sys.executable, os.path.abspath(__file__), "--config", args.config, "--steps", str(args.steps), "--warmup",
+           str(args.warmup), "--out-dtype", args.out_dtype, "--no-cpu-baseline", "--fused-commit"]
+    if args.no_overlap:
+        cmd.append("--no-overlap")
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK")}
+    try:
+        out = subprocess.run(cmd, capture_output=True, text=True, timeout=600, env=env).stdout
+        d = json.loads([l for l in out.splitlines() if l.startswith("{")][-1])
+        return {"value": d["value"], "unit": d["unit"], "ms_per_step": d["ms_per_step"], "step": d["config"]["step"]}
+    except Exception as e:      # an extra figure only: its failure must not cost the headline
+        return {"unavailable": f"{type(e).__name__}: {e}"[:200]}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -513,6 +530,8 @@ def main():
         v, steps, cores, dt = run_oracle_steps(sample_case, args.cpu_seconds)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                 "sample": f"{sample}; {steps} steps in {dt:.1f} s"}
+    if world == 1 and not args.fused_commit and not args.no_cpu_baseline:
+        line["fused_commit_verify"] = fused_arm(args)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
