@@ -177,3 +177,66 @@ def test_commit_after_commit_verify_sees_the_rewritten_state():
     ctx().set_overlap(True)
     for a, b in zip(res[False], res[True]):
         assert torch.equal(a, b)
+
+
+def test_commit_verify_randomized_sweep():
+    """Seeded sweep: tree sizes around the tile sizes, depths up to 16, padded and permuted slots, bias,
+    head ratios 1..3, empty and invalid accepted paths; state, history, status, recorded operands and
+    outputs against the composed oracles."""
+    import random
+    rng = random.Random(2024)
+
+    def rand_tree(N, maxd):
+        p, d = [], []
+        for i in range(N):
+            while True:
+                q = rng.randint(-1, i - 1)
+                dq = 0 if q < 0 else d[q]
+                if dq < maxd:
+                    break
+            p.append(q)
+            d.append(dq + 1)
+        return p
+
+    c = ctx()
+    worst = 0.0
+    for it in range(24):
+        B = rng.choice([1, 2, 3])
+        Hk = rng.choice([1, 2])
+        Hv = Hk * rng.choice([1, 2, 3])
+        bias = rng.random() < 0.3
+        cases = []
+        for _ in range(2):
+            N = rng.choice([1, 2, 3, 17, 31, 32, 33, 63, 64])
+            parents = [rand_tree(N, rng.choice([2, 5, 9, 16])) for _ in range(B)]
+            Ns = N + rng.choice([0, 0, 7])
+            cases.append(W.make_case("f", parents, seed=rng.getrandbits(30), Hk=Hk, Hv=Hv, d=128, in_dtype="bf16", Ns=Ns,
+                                     permute_slots=Ns > N or rng.random() < 0.5, alpha_lo=rng.choice([0.5, 0.9]),
+                                     beta_uniform=rng.random() < 0.5, with_bias=bias))
+        P, C = cases
+        C.state_row, C.rows = P.state_row.copy(), P.rows
+        C.layers[0].state, C.layers[0].hist = P.layers[0].state.copy(), P.layers[0].hist.copy()
+        acc, ln = P.accepted.copy(), P.accepted_len.copy()
+        if rng.random() < 0.3:
+            ln[rng.randrange(B)] = 0
+        if rng.random() < 0.25 and P.N > 2:
+            acc[rng.randrange(B), 0] = P.N - 1            # (mostly) not a child of the pre-tree state
+        dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
+        dcP.verify()
+        layersC = _share_state(dcP, dcC)
+        dev = dcP.accepted.device
+        c.commit_verify(dcP.desc, dcP.layers, torch.from_numpy(acc).to(dev), torch.from_numpy(ln).to(dev), dcC.desc, layersC)
+        torch.cuda.synchronize()
+        st1, hist1, status, y, o_ref = _oracle(P, C, dcP, layersC, 0, acc, ln)
+        f = lambda t: t.to(torch.float64).cpu().numpy()
+        tc = layersC[0].tensors
+        hk = C.Hk * C.d
+        got = np.concatenate([f(tc["q"]).reshape(C.B, C.Ns, hk), f(tc["k"]).reshape(C.B, C.Ns, hk),
+                              f(tc["v"]).reshape(C.B, C.Ns, C.Hv * C.d)], axis=-1)
+        what = f"case {it}: nodes {P.N} -> {C.N}, batch {B}, heads {Hk}/{Hv}, lengths {ln.tolist()}"
+        worst = max(worst, assert_close(dcP.np("state"), st1, what=what + " state"),
+                    assert_close(f(tc["out"]), o_ref, what=what + " outputs"))
+        assert np.array_equal(dcP.np("conv_hist"), hist1), what
+        assert dcP.t("status").cpu().numpy().tolist() == status.tolist(), what
+        assert (got == y).mean() > 0.98, what
+    assert worst < 1e-4
