@@ -9,6 +9,11 @@
  *   commit      the same update for the accepted nodes in path order, published in place,
  *               plus the matching convolution history             (paper Algorithms 1 and 2)
  *
+ * Around these: lumo_gdn_commit_verify (the commit of the previous cycle folded into the next
+ * verify), lumo_tree_accept (device-resident acceptance walk between verify and commit),
+ * lumo_select_spine_top3 (fused draft selection upstream of the tree), lumo_gdn_tree_scan_static
+ * (the scan with library-internal static scratch) and small helpers.
+ *
  * Conventions
  *   - One GPU.  All tensor pointers are DEVICE pointers owned by the caller unless a
  *     comment says HOST; the library never frees or reallocates caller memory.
