@@ -112,15 +112,21 @@ const char* lumo_last_error(const lumo_ctx* ctx);
 int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx);
 
 /* Which scan kernel lumo_gdn_tree_verify uses: 0 = automatic (the tensor-core Gram form when the
- * shape allows it: d = 128, bf16 operands, N <= 64, depth <= 16, no snapshots; else rank-1),
- * 1 = always the rank-1 fp32 kernel, 2 = Gram form or LUMO_ERR_UNSUPPORTED. */
+ * shape allows it: d = 128, bf16 operands, tree depth <= 16, no snapshots; trees of more than 64
+ * nodes are cut into node groups on the host; else rank-1), 1 = always the rank-1 fp32 kernel,
+ * 2 = Gram form or LUMO_ERR_UNSUPPORTED. */
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo);
 
 /* Kernel overlap (default on): conv, scan and commit are launched with programmatic dependent launch,
  * so each kernel's set-up (and, for commit, its whole read phase) runs under the tail of the kernel
  * before it; each waits on the device before touching data its predecessor produces or still reads.
  * Applied only to small launches (n_layers * B * Hv <= 4 x SM count), where it measured faster.
- * Results are identical either way; 0 restores plain stream order. */
+ * Results are identical either way; 0 restores plain stream order.
+ * The commit (and a scan without convolution) reads part of its input ahead of that wait: the
+ * accepted path, the recorded operands, the state.  The library therefore overlaps it only when the
+ * previous call on this context was a verify; behind any other library call it runs in plain stream
+ * order.  A caller that fills accepted_dev / len_dev with a kernel of its own between verify and
+ * commit, on the same stream, switches overlap off. */
 int lumo_ctx_set_overlap(lumo_ctx* ctx, int on);
 
 /* Measurement aid.  While enabled, every kernel the library launches is bracketed by two CUDA
@@ -279,8 +285,14 @@ int lumo_gdn_tree_scan_static(lumo_ctx* ctx, const lumo_tree_desc* desc, const l
                               int n_layers, void* stream);
 int64_t lumo_static_stack_bytes(void);
 
+/* Diagnostic: how many entries of the visiting order one CTA of the tree convolution takes for this
+ * tree batch, head shape and layer count on this context's device (16, 8 or 4; the three are separate
+ * instantiations of the kernel, chosen so that the grid covers the GPU).  0 on a bad argument or a
+ * host-only context.  Lets a parity test state which instantiation it exercised. */
+int lumo_conv_rows_per_cta(const lumo_ctx* ctx, const lumo_tree_desc* desc, int Hk, int Hv, int d, int n_layers);
+
 /* Replays accepted_dev [B, lmax] (logical ids, root first; entries at or beyond len_dev[b] are
- * ignored) from the pre-tree state with the recorded operands and publishes state and
+ * ignored; 1 <= lmax <= 256, else LUMO_ERR_ARG and nothing is enqueued) from the pre-tree state with the recorded operands and publishes state and
  * convolution history in place (Algorithm 2, "Replay only the accepted path into native
  * recurrent state"; Algorithm 1, "Gather the convolution history for A into the native running
  * row").  len 0 leaves both bit-unchanged.  An invalid path sets status[b] and leaves the

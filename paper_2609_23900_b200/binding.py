@@ -37,7 +37,7 @@ EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_s
            "lumo_ctx_timing_enable", "lumo_ctx_timing_read", "lumo_ctx_set_scan_algo", "lumo_ctx_set_overlap",
            "lumo_tree_desc_create", "lumo_tree_desc_destroy", "lumo_tree_desc_get",
            "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit",
-           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_tree_accept", "lumo_select_spine_top3", "lumo_gdn_commit_verify"]
+           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_conv_rows_per_cta", "lumo_tree_accept", "lumo_select_spine_top3", "lumo_gdn_commit_verify"]
 
 
 class LumoError(RuntimeError):
@@ -106,6 +106,7 @@ _lib.lumo_gdn_tree_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.P
 _lib.lumo_gdn_tree_scan_static.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
                                            ctypes.c_void_p]
 _lib.lumo_static_stack_bytes.restype = ctypes.c_int64
+_lib.lumo_conv_rows_per_cta.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int]
 _lib.lumo_gdn_commit_verify.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
                                         ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
 _lib.lumo_select_spine_top3.argtypes = [ctypes.c_void_p, ctypes.POINTER(_SelectArgs), ctypes.c_void_p, ctypes.c_void_p,
@@ -204,6 +205,10 @@ class Context:
         ``static_stack_bytes()``.  Calls that overlap on the GPU race on the shared stack."""
         arr = layers if isinstance(layers, ctypes.Array) else self.pack(layers)
         self._check(_lib.lumo_gdn_tree_scan_static(self._h, desc._h, arr, len(arr), _stream(stream)))
+
+    def conv_rows_per_cta(self, desc: "TreeDesc", Hk: int, Hv: int, d: int, n_layers: int = 1) -> int:
+        """Which instantiation of the tree convolution (16, 8 or 4 entries per CTA) this shape launches."""
+        return int(_lib.lumo_conv_rows_per_cta(self._h, desc._h, int(Hk), int(Hv), int(d), int(n_layers)))
 
     @staticmethod
     def static_stack_bytes() -> int:

@@ -422,6 +422,7 @@ int lumo_tree_path_from_node(lumo_ctx* ctx, const lumo_tree_desc* desc, const in
     return launch_path_from_node(tree_view(desc, 0), desc->B, desc->N, node_dev, lmax, accepted_dev, len_dev,
                                  status_dev, st);
   });
+  ctx->last_call = lumo_ctx::kOther;
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "path_from_node launch");
 }
 
@@ -444,6 +445,7 @@ int lumo_tree_accept(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_accep
   v.uniforms = a->uniforms; v.noise = a->noise; v.work = a->work;
   cudaError_t e = launch_accept(tree_view(desc, 0), desc->B, desc->N, desc->Ns, v, lmax, accepted_dev, len_dev,
                                 next_token_dev, final_node_dev, (cudaStream_t)stream);
+  ctx->last_call = lumo_ctx::kOther;
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "accept launch");
 }
 
@@ -459,6 +461,7 @@ int lumo_select_spine_top3(lumo_ctx* ctx, const lumo_select_args* a, int32_t* sp
     return fail(ctx, LUMO_ERR_ARG, "split must be 0, 1, 2, 4, 8 or 16");
   DeviceGuard g(ctx->device);
   cudaError_t e = launch_select(a->logits, a->dtype, a->rows, a->V, sp, spine_dev, cand_dev, (cudaStream_t)stream);
+  ctx->last_call = lumo_ctx::kOther;
   if (e == cudaErrorInvalidConfiguration) {
     (void)cudaGetLastError();
     return fail(ctx, LUMO_ERR_UNSUPPORTED, "this device does not schedule clusters of that size");
@@ -479,13 +482,21 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
   const bool gram_ok = desc->d_tc_meta != nullptr && gram_supported(s, desc->max_depth);
   if (ctx->scan_algo == 2 && !gram_ok)
     return fail(ctx, LUMO_ERR_UNSUPPORTED, "the Gram-form scan needs d = 128, bf16 operands, depth <= 16, no snapshots");
+  // The Gram-form scan requests the pre-tree state ahead of its dependency wait.  Behind a convolution
+  // that is safe (the convolution waits first, so whatever wrote the state has completed); launched
+  // directly behind a call that rewrote the state it takes plain stream order instead.
+  const int prev_call = ctx->last_call;
+  ctx->last_call = lumo_ctx::kVerify;
   if (gram_ok && ctx->scan_algo != 1) {
     cudaError_t e = cudaSuccess;
     if (layers[0].x) {
       e = timed(ctx, LUMO_K_CONV, st, [&] { return launch_conv(s, t, lb, use_overlap(ctx, s), st); });
       if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
     }
-    e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram(s, t, lb, ctx->sm_count, use_overlap(ctx, s), st); });
+    const bool state_fresh = !layers[0].x && (prev_call == lumo_ctx::kCommit || prev_call == lumo_ctx::kCommitVerify);
+    e = timed(ctx, LUMO_K_SCAN, st, [&] {
+      return launch_scan_gram(s, t, lb, ctx->sm_count, use_overlap(ctx, s) && !state_fresh, st);
+    });
     return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "Gram-form scan launch");
   }
   int grid = 0;
@@ -517,6 +528,11 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
 
 int64_t lumo_static_stack_bytes(void) { return (int64_t)kStaticStackBytes; }
 
+int lumo_conv_rows_per_cta(const lumo_ctx* ctx, const lumo_tree_desc* desc, int Hk, int Hv, int d, int n_layers) {
+  if (!ctx || !desc || ctx->device < 0 || Hk < 1 || Hv < 1 || d < 1 || n_layers < 1) return 0;
+  return conv_rows_per_cta(2 * Hk * d + Hv * d, desc->Ns, desc->B * n_layers, ctx->sm_count);
+}
+
 int lumo_gdn_tree_scan_static(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers,
                               int n_layers, void* stream) {
   Shape s;
@@ -539,23 +555,30 @@ int lumo_gdn_tree_scan_static(lumo_ctx* ctx, const lumo_tree_desc* desc, const l
   e = static_stack_address(ctx->device, &stack);
   if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGetSymbolAddress(built-in scan stack)");
   e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan(s, t, lb, stack, grid, st); });
+  ctx->last_call = lumo_ctx::kVerify;
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "scan launch");
 }
 
 int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers,
                     const int32_t* accepted_dev, const int32_t* len_dev, int lmax, void* stream) {
+  // the kernel stages the whole path in arrays of kMaxNodes entries: refused here, before anything else
+  if (ctx && (lmax < 1 || lmax > kMaxNodes))
+    return fail(ctx, LUMO_ERR_ARG, "lmax must be in [1, " + std::to_string(kMaxNodes) + "] (a path holds each node at most once)");
   Shape s;
   LayerBatch lb;
   std::memset(&lb, 0, sizeof(lb));
   int rc = prepare(ctx, desc, layers, n_layers, false, &s, &lb);
   if (rc != LUMO_OK) return rc;
   if (!accepted_dev || !len_dev) return fail(ctx, LUMO_ERR_ARG, "accepted_dev and len_dev are required");
-  if (lmax < 1) return fail(ctx, LUMO_ERR_ARG, "lmax must be positive");
   DeviceGuard g(ctx->device);
   cudaStream_t st = (cudaStream_t)stream;
   const TreeDev t = tree_view(desc, 0);
+  // the commit reads the path, the operands and the state ahead of its dependency wait: overlap only
+  // right behind a verify call (see commit_kernel)
+  const bool pdl = use_overlap(ctx, s) && ctx->last_call == lumo_ctx::kVerify;
+  ctx->last_call = lumo_ctx::kCommit;
   cudaError_t e = timed(ctx, LUMO_K_COMMIT, st, [&] {
-    return launch_commit(s, t, lb, accepted_dev, len_dev, lmax, true, layers[0].x != nullptr, use_overlap(ctx, s), st);
+    return launch_commit(s, t, lb, accepted_dev, len_dev, lmax, true, layers[0].x != nullptr, pdl, st);
   });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "commit launch");
 }
@@ -563,6 +586,8 @@ int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_ar
 int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const lumo_gdn_args* prev_layers,
                            const int32_t* accepted_dev, const int32_t* len_dev, int lmax,
                            const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers, void* stream) {
+  if (ctx && (lmax < 1 || lmax > kMaxNodes))
+    return fail(ctx, LUMO_ERR_ARG, "lmax must be in [1, " + std::to_string(kMaxNodes) + "] (a path holds each node at most once)");
   Shape ps, s;
   LayerBatch lb;
   FusedPrev fp;
@@ -573,7 +598,6 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
   rc = prepare(ctx, desc, layers, n_layers, true, &s, &lb);
   if (rc != LUMO_OK) return rc;
   if (!accepted_dev || !len_dev) return fail(ctx, LUMO_ERR_ARG, "accepted_dev and len_dev are required");
-  if (lmax < 1) return fail(ctx, LUMO_ERR_ARG, "lmax must be positive");
   if (prev_desc->B != desc->B) return fail(ctx, LUMO_ERR_ARG, "both trees must cover the same batch");
   if (ps.Hk != s.Hk || ps.Hv != s.Hv || ps.d != s.d || ps.in_dtype != s.in_dtype || ps.gate_dtype != s.gate_dtype ||
       ps.l2norm != s.l2norm || ps.l2_eps != s.l2_eps || ps.gate_mode != s.gate_mode || ps.n_state_rows != s.n_state_rows)
@@ -596,6 +620,13 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
   }
   DeviceGuard g(ctx->device);
   cudaStream_t st = (cudaStream_t)stream;
+  // The convolution waits on its predecessor before it reads anything, so it may always overlap, and
+  // so may a scan launched behind it.  A fused scan (or the history launch) directly behind another
+  // call reads the path and the state ahead of its dependency wait: overlap then only behind a verify.
+  const bool pdl_conv = use_overlap(ctx, s);
+  const bool pdl = pdl_conv && ctx->last_call == lumo_ctx::kVerify;
+  const bool pdl_scan = pdl_conv && (layers[0].x != nullptr || ctx->last_call == lumo_ctx::kVerify);
+  ctx->last_call = lumo_ctx::kCommitVerify;
   const TreeDev pt = tree_view(prev_desc, 0);
   const TreeDev t = tree_view(desc, 0);
   fp.parent = pt.parent; fp.slot = pt.slot; fp.N = prev_desc->N; fp.Ns = prev_desc->Ns;
@@ -607,18 +638,17 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
   fp.hist_in_kernels = prev_layers[0].x != nullptr && layers[0].x != nullptr;
   if (prev_layers[0].x && !fp.hist_in_kernels) {
     e = timed(ctx, LUMO_K_COMMIT, st, [&] {
-      return launch_commit(ps, pt, fp.lb, accepted_dev, len_dev, lmax, false, true, use_overlap(ctx, s), st);
+      return launch_commit(ps, pt, fp.lb, accepted_dev, len_dev, lmax, false, true, pdl, st);
     });
     if (e != cudaSuccess) return cuda_fail(ctx, e, "history launch");
   }
   if (layers[0].x) {
     e = timed(ctx, LUMO_K_CONV, st, [&] {
-      return fp.hist_in_kernels ? launch_conv_fused(s, t, lb, fp, use_overlap(ctx, s), st)
-                                : launch_conv(s, t, lb, use_overlap(ctx, s), st);
+      return fp.hist_in_kernels ? launch_conv_fused(s, t, lb, fp, pdl_conv, st) : launch_conv(s, t, lb, pdl_conv, st);
     });
     if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
   }
-  e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, use_overlap(ctx, s), st); });
+  e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st); });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "fused scan launch");
 }
 

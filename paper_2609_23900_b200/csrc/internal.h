@@ -12,6 +12,7 @@ namespace lumo {
 constexpr int kMaxNodes = 256;
 constexpr int kMaxSlots = 1024;
 constexpr int kMaxLayers = 64;
+constexpr int kMaxDevices = 64;                    // per-device caches (kernel attributes, symbol addresses)
 constexpr size_t kStaticStackBytes = 64u << 20;   // capacity of the built-in scan stack
 
 // ---- scan schedule ------------------------------------------------------------------
@@ -48,6 +49,11 @@ struct lumo_ctx {
   // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
   int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form (tensor cores)
   bool overlap = true;          // programmatic dependent launch between conv -> scan -> commit
+  // Kind of the previous call that launched on this context.  Kernels that read some of their inputs
+  // ahead of their dependency wait (commit: path and state; scan without convolution: state) get the
+  // overlap attribute only when the call before them cannot have written those inputs.
+  enum Call { kNone = 0, kVerify, kCommit, kCommitVerify, kOther };
+  int last_call = kNone;
   bool timing = false;
   std::vector<cudaEvent_t> ev_start, ev_stop;
   std::vector<int> ev_kind;
@@ -239,6 +245,8 @@ cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t 
 
 // launchers (kernels.cu); all return cudaError_t and only enqueue
 cudaError_t launch_conv(const Shape& s, const TreeDev& t, const LayerBatch& lb, bool pdl, cudaStream_t st);
+// entries of the visiting order one CTA of the convolution takes (16, 8 or 4: fewer when the grid would not cover the GPU)
+int conv_rows_per_cta(int C, int Ns, int seqs, int sms);
 // same convolution reading the history the previous cycle's accepted path would commit (not yet in memory)
 cudaError_t launch_conv_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp, bool pdl,
                               cudaStream_t st);

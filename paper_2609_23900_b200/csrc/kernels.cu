@@ -511,9 +511,11 @@ commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ acc
   const int tid = threadIdx.x;
   const int row = L.state_row[b];
   const bool lead = blockIdx.x == 0 && tid == 0;
-  // Everything this kernel READS (state, operands, path) is complete once its predecessor passed its
-  // own dependency wait; what it WRITES (state, history, status) may still be read by the predecessor
-  // (the scan reads the pre-tree state), so every write sits behind pdl_wait().
+  // What this kernel WRITES (state, history, status) may still be read by its predecessor (the scan
+  // reads the pre-tree state), so every write sits behind pdl_wait().  What it READS ahead of that wait
+  // (state tile, path, operands) must be older than its predecessor: the host launches it with the
+  // overlap attribute only right after a verify call, whose own dependency wait orders everything
+  // before it; after any other call of the library it is launched in plain stream order.
   if (row < 0) { pdl_wait(); if (lead && L.status) L.status[b] = LUMO_SEQ_OK; return; }
   if (row >= s.n_state_rows) { pdl_wait(); if (lead && L.status) L.status[b] = LUMO_SEQ_BAD_ROW; return; }
   const int32_t* acc = accepted + (size_t)b * lmax;
@@ -535,8 +537,10 @@ commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ acc
     constexpr int kVec = 16 / (int)sizeof(T);
     const int c0 = ((blockIdx.x - n_state_ctas) * kScanThreads + tid) * kVec;
     __syncthreads();
-    if (c0 >= s.C || L.x == nullptr) return;
-    if (check_path_staged(s_acc, s_par, s.N, len, lmax) != LUMO_SEQ_OK || len == 0) return;
+    // every exit path passes the dependency wait: a CTA that left without it would let this grid complete
+    // (and its own dependent start) while the kernel before it is still running
+    if (c0 >= s.C || L.x == nullptr) { pdl_wait(); return; }
+    if (check_path_staged(s_acc, s_par, s.N, len, lmax) != LUMO_SEQ_OK || len == 0) { pdl_wait(); return; }
     T* hist = reinterpret_cast<T*>(L.conv_hist) + (size_t)row * 3 * s.C + c0;
     const T* x = reinterpret_cast<const T*>(L.x);
     uint4 v[3];
@@ -566,7 +570,7 @@ commit_kernel(Shape s, TreeDev t, LayerBatch lb, const int32_t* __restrict__ acc
   __syncthreads();
   const int st = check_path_staged(s_acc, s_par, s.N, len, lmax);
   if (lead && L.status) { pdl_wait(); L.status[b] = st; }
-  if (st != LUMO_SEQ_OK || len == 0) return;
+  if (st != LUMO_SEQ_OK || len == 0) { pdl_wait(); return; }
 
   const T* kg = reinterpret_cast<const T*>(L.k);
   const T* vg = reinterpret_cast<const T*>(L.v);
@@ -646,22 +650,30 @@ cudaError_t dispatch(int d, int in_dtype, F f) {
 // ---------------------------------------------------------------------------------------
 // sixteen entries per CTA amortise the window set-up; small launches take fewer so that the grid still
 // covers the GPU
+int conv_rows_per_cta(int C, int Ns, int seqs, int sms) {
+  const int slabs = (C / 4 + 255) / 256;
+  auto ctas = [&](int rows) { return (long long)slabs * ((Ns + rows - 1) / rows) * seqs; };
+  if (ctas(16) >= 2LL * sms) return 16;
+  if (ctas(8) >= 2LL * sms) return 8;
+  return 4;
+}
+
 template <typename T>
 static cudaError_t launch_conv_t(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev* fp, bool pdl,
                                  cudaStream_t st) {
   const int slabs = (s.C / 4 + 255) / 256, seqs = s.B * s.n_layers;
-  auto ctas = [&](int rows) { return (long long)slabs * ((s.Ns + rows - 1) / rows) * seqs; };
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int rows = conv_rows_per_cta(s.C, s.Ns, seqs, sms);
   auto go = [&](auto rows_c) {
     constexpr int kRowsPerCta = decltype(rows_c)::value;
     const dim3 grid(slabs, (s.Ns + kRowsPerCta - 1) / kRowsPerCta, seqs);
     if (fp) return launch_kernel(conv_fused_kernel<T, kRowsPerCta>, grid, dim3(256), 0, st, pdl, s, t, lb, *fp);
     return launch_kernel(conv_kernel<T, kRowsPerCta>, grid, dim3(256), 0, st, pdl, s, t, lb);
   };
-  if (ctas(16) >= 2LL * sms) return go(std::integral_constant<int, 16>{});
-  if (ctas(8) >= 2LL * sms) return go(std::integral_constant<int, 8>{});
+  if (rows == 16) return go(std::integral_constant<int, 16>{});
+  if (rows == 8) return go(std::integral_constant<int, 8>{});
   return go(std::integral_constant<int, 4>{});
 }
 
@@ -707,7 +719,6 @@ cudaError_t scan_plan(const Shape& s, const TreeDev& t, int sm_count, int* grid,
 __device__ __align__(256) static float g_static_stack[kStaticStackBytes / sizeof(float)];
 
 cudaError_t static_stack_address(int device, float** ptr) {
-  constexpr int kMaxDevices = 64;
   static float* cached[kMaxDevices] = {};
   static std::mutex mu;
   if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;

@@ -175,12 +175,6 @@ __device__ __forceinline__ void store_out(void* out, size_t idx, int dtype, floa
   if (dtype == LUMO_BF16) reinterpret_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16_rn(v);
   else reinterpret_cast<float*>(out)[idx] = v;
 }
-#ifdef LUMO_GRAM_PROFILE
-__device__ long long g_prof[32];
-#define PROF(i) do { if (blockIdx.x == 0 && tid == 0 && item == blockIdx.x) g_prof[i] = clock64(); } while (0)
-#else
-#define PROF(i) do {} while (0)
-#endif
 
 // fp32 x -> bf16 hi + lo of four values, written to the two swizzled operand tiles
 __device__ __forceinline__ void split_store(unsigned char* smem, uint32_t off, float4 x) {
@@ -252,6 +246,7 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     const size_t out_row_stride = (size_t)s.Hv * kD;
 
     if (row < 0 || row >= s.n_state_rows) {   // skipped sequence: zero outputs
+      pdl_wait();                             // every path through the kernel passes its dependency wait
       if (first_group) {
         for (int ps = grp; ps < s.Ns; ps += 2)
           store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + vrow, s.out_dtype, 0.f);
@@ -264,8 +259,6 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       continue;
     }
     if (first_group && L.status && hv == 0 && tid == 0) L.status[b] = LUMO_SEQ_OK;
-
-    PROF(0);
     int plen = 0;
     if constexpr (kFused) {
       // the accepted path of the previous cycle: entries, parents, physical rows (one level of dependent loads)
@@ -336,7 +329,6 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       }
       __syncthreads();
     }
-    PROF(1);
     // ---- b. gates (consumed much later); K and Q rows -> swizzled operand tile (cp.async) ---------
     // K, Q, V may still be in the making (the convolution runs right before this kernel): everything
     // above touched only the descriptor tables and the state.  The dependent kernel (commit) is let in
@@ -399,7 +391,6 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       }
       asm volatile("cp.async.commit_group;\n" ::: "memory");
     }
-    PROF(2);
     // ---- c. pre-tree state -> bf16 hi + lo operand tiles ------------------------------------------
     {
       const int kblock = lane >> 4, chunk = (lane & 15) >> 1, half = lane & 1;
@@ -451,13 +442,9 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       for (int ps = grp; ps < s.Ns; ps += 2)
         if (t.slot_inv[b * s.Ns + ps] < 0)
           store_out(L.out, ((size_t)b * s.Ns + ps) * out_row_stride + hv * kD + vrow, s.out_dtype, 0.f);
-    PROF(3);
-    PROF(4);
     asm volatile("cp.async.wait_group 0;\n" ::: "memory");
     fence_async_proxy();          // generic-proxy writes -> visible to the tensor core's async proxy
     __syncthreads();
-
-    PROF(5);
     // ---- e. MMAs: Gram = [K;Q] K^T, P = S0 [K|Q]^T (hi + lo); meanwhile |q|^2 when normalising ----
     if (tid == 0) {
       tc_fence_after();
@@ -494,7 +481,6 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       }
       sm.qq[vrow] = qq;
     }
-    PROF(6);
     // ---- f. wait for the tensor core (bounded) ---------------------------------------------------
     if (!mbar_wait(&sm.mbar, phase)) sm.timed_out = 1;
     phase ^= 1;
@@ -504,8 +490,6 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       if (L.status && tid == 0) L.status[b] = LUMO_SEQ_TIMEOUT;
       break;
     }
-
-    PROF(7);
     // ---- g. V rows -> shared (space of the dead S0 tiles); Gram rows out of tensor memory ----------
     {
       const __nv_bfloat16* vg = reinterpret_cast<const __nv_bfloat16*>(L.v);
@@ -523,12 +507,10 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     // both halves of the CTA read the Gram rows: 32 of the NT columns each (one half is enough for NT = 32)
     if (grp * 32 < NT) tmem_cols32_to_smem(tmem_lane + 128 + grp * 32, dump + vrow * kDumpStride + grp * 32, 1);
     __syncthreads();
-    PROF(8);
     // ---- h. normalisation factors ------------------------------------------------------------------
     if (tid < NT) sm.ks[tid] = s.l2norm ? rsqrtf(dump[tid * kDumpStride + tid] + s.l2_eps) : 1.f;
     else if (tid < 2 * NT) sm.qs[tid - NT] = s.l2norm ? s.scale * rsqrtf(sm.qq[tid - NT] + s.l2_eps) : s.scale;
     __syncthreads();
-    PROF(9);
     // ---- i. first half of the CTA: node records, one thread per (node, table); second half: the
     //         S0 q^ products move from tensor memory to shared memory [node][row] ---------------------
     if (grp == 0) {
@@ -583,8 +565,6 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     if (grp * 32 < N) tmem_cols32_to_smem(tmem_lane + grp * 32, dls + (grp * 32) * kD + vrow, kD);
     if (tid < kD) dls[kZeroRow + tid] = 0.f;
     __syncthreads();
-
-    PROF(10);
     // ---- j. forward substitution, level by level; one warp per node, lane l carries value rows
     //         4l .. 4l+3.  A node's record, v and S0 products are loaded before the barrier that
     //         publishes the previous level; only the ancestors' deltas are fetched after it ----------
@@ -657,13 +637,11 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
           }
         }
         lo = hi;
-        PROF(12 + d);
         if (lo >= N) break;                                        // uniform
         if (lo + warp < __shfl_sync(0xffffffffu, lvl_lane, d + 1)) load_ops(op, lo + warp);   // next level's first node
         __syncthreads();                                           // deltas of this level visible to the next
       }
     }
-    PROF(11);
     tc_fence_before();
     __syncthreads();      // tensor memory and the aliased shared memory are free for the next item
   }
@@ -693,13 +671,17 @@ bool gram_supported(const Shape& s, int max_depth) {
 cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
                              cudaStream_t st) {
   const int items = s.n_layers * t.n_groups * s.Hv;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kMaxDevices] = {};      // the attribute is a per-device setting
+  int dev = 0;
+  cudaError_t e0 = cudaGetDevice(&dev);
+  if (e0 != cudaSuccess) return e0;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(scan_gram_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(scan_gram_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[dev] = true;
   }
   // two CTAs per SM by construction: 102 KB of shared memory, 128 registers x 256 threads and 256
   // of the 512 tensor-memory columns each
@@ -712,24 +694,22 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
 cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
                                    int sm_count, bool pdl, cudaStream_t st) {
   const int items = s.n_layers * t.n_groups * s.Hv;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kMaxDevices] = {};      // the attribute is a per-device setting
+  int dev = 0;
+  cudaError_t e0 = cudaGetDevice(&dev);
+  if (e0 != cudaSuccess) return e0;
+  if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+  if (!configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(scan_gram_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesFused);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(scan_gram_fused_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesFused);
     if (e != cudaSuccess) return e;
-    configured = true;
+    configured[dev] = true;
   }
   const int grid = items < 2 * sm_count ? items : 2 * sm_count;
   if (t.max_group_nodes <= 32)
     return launch_kernel(scan_gram_fused_kernel<32>, dim3(grid), dim3(kThreads), kSmemBytesFused, st, pdl, s, t, lb, items, fp);
   return launch_kernel(scan_gram_fused_kernel<64>, dim3(grid), dim3(kThreads), kSmemBytesFused, st, pdl, s, t, lb, items, fp);
 }
-
-#ifdef LUMO_GRAM_PROFILE
-extern "C" int lumo_debug_gram_profile(long long* out32) {
-  return (int)cudaMemcpyFromSymbol(out32, g_prof, sizeof(long long) * 32);
-}
-#endif
 
 }  // namespace lumo

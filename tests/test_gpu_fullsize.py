@@ -13,6 +13,22 @@ from tests.harness import assert_close, ctx
 pytestmark = pytest.mark.gpu
 
 
+def check_conv_samples(dc, case, layer, seqs):
+    """The operands the convolution recorded for the sampled sequences, element by element against the
+    conv oracle (all channels, every row): the scan checks below read these same buffers on both sides,
+    so they alone would not notice a wrong convolution."""
+    L = case.layers[layer]
+    hk = case.Hk * case.d
+    for b in seqs:
+        sl = slice(b, b + 1)
+        y = O.conv(case.parent[sl], case.slot[sl], case.state_row[sl], L.x[sl], L.conv_w, L.conv_b, L.hist, case.Ns,
+                   out_dtype="none")
+        f = lambda name: dc.t(name, layer)[b].to(torch.float64).cpu().numpy()
+        got = np.concatenate([f("q").reshape(case.Ns, hk), f("k").reshape(case.Ns, hk),
+                              f("v").reshape(case.Ns, case.Hv * case.d)], axis=-1)
+        assert_close(got, y[0], bf16=True, what=f"{case.name} layer {layer} b={b} recorded operands")
+
+
 def check_samples(dc, case, layer, pairs):
     L = case.layers[layer]
     rep = case.Hv // case.Hk
@@ -47,6 +63,7 @@ def test_config4_full_size_sampled(shape):
     rs = np.random.default_rng(4)
     pairs = [(int(rs.integers(case.B)), int(rs.integers(case.Hv))) for _ in range(5)] + [(0, 0), (case.B - 1, case.Hv - 1)]
     check_samples(dc, case, 0, pairs)
+    check_conv_samples(dc, case, 0, sorted({b for b, _ in pairs})[:4])
     # properties that hold at any size: finite everywhere, rows of the pool that belong to nobody untouched
     assert torch.isfinite(dc.t("out").float()).all()
     other = sorted(set(range(case.rows)) - set(case.state_row.tolist()))
@@ -64,6 +81,7 @@ def test_config3_full_stack_sampled():
         assert dc.np("status", layer).tolist() == [0] * case.B
         pairs = [(int(rs.integers(case.B)), int(rs.integers(case.Hv))) for _ in range(4)]
         check_samples(dc, case, layer, pairs)
+        check_conv_samples(dc, case, layer, sorted({b for b, _ in pairs})[:2])
     for layer in range(48):
         assert torch.isfinite(dc.t("out", layer).float()).all()
 

@@ -77,26 +77,50 @@ def test_path_from_node_bit_exact(name):
 
 
 # ------------------------------------------------------------------ conv
-@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfgP_padded_permuted", "d64_bf16", "rand256_b2"])
+# The convolution kernel exists in three instantiations (16, 8 or 4 entries of the visiting order per
+# CTA, chosen from the grid size); each case names the one it must land on, so that every
+# instantiation a benchmark configuration launches is compared with the oracle element by element.
+CONV_CASES = {
+    "cfg0": (lambda: W.config0(), 4),
+    "cfg1": (lambda: W.config1(), 4),
+    "cfgP_padded_permuted": (lambda: W.config_paper(B=2), 4),
+    "d64_bf16": (CASES["d64_bf16"], 4),
+    "rand256_b2": (CASES["rand256_b2"], 4),
+    "cfg2_b8": (lambda: W.config2(), 8),                                  # what bench.py times at config 2
+    "cfg3_5layers": (lambda: W.config3(n_layers=5), 16),                  # config 3's instantiation
+    "cfg4_random_b3": (lambda: W.config4("random", B=3), 16),             # config 4's instantiation
+    "paper_b8_bias": (lambda: W.make_case("p", [W.tree_paper_geometry()] * 8, seed=31, Hk=16, Hv=32, d=128,
+                                          in_dtype="bf16", Ns=32, permute_slots=True, with_bias=True), 4),
+    "f32_8rows": (lambda: W.make_case("f8", rand_parents(11, 64, 8), seed=12, Hk=4, Hv=8, d=128, in_dtype="f32",
+                                      n_layers=3, with_bias=True), 8),
+    "f32_16rows": (lambda: W.make_case("f16", rand_parents(13, 61, 8), seed=14, Hk=4, Hv=8, d=128, in_dtype="f32",
+                                       n_layers=5, Ns=64, permute_slots=True), 16),
+}
+
+
+@pytest.mark.parametrize("name", list(CONV_CASES))
 def test_conv_recorded_operands(name):
-    c = CASES[name]()
+    make, rows = CONV_CASES[name]
+    c = make()
     dc = DeviceCase(ctx(), c)
-    for t in ("q", "k", "v"):
-        dc.t(t).fill_(777.0)     # must be overwritten everywhere, padding rows with zeros
+    assert ctx().conv_rows_per_cta(dc.desc, c.Hk, c.Hv, c.d, len(c.layers)) == rows, "case landed on another instantiation"
+    for l in range(len(c.layers)):
+        for t in ("q", "k", "v"):
+            dc.t(t, l).fill_(777.0)     # must be overwritten everywhere, padding rows with zeros
     dc.verify()
     torch.cuda.synchronize()
-    L = c.layers[0]
-    y = O.conv(c.parent, c.slot, c.state_row, L.x, L.conv_w, L.conv_b, L.hist, c.Ns, out_dtype="none")
     hk = c.Hk * c.d
-    got = np.concatenate([dc.np("q").reshape(c.B, c.Ns, hk), dc.np("k").reshape(c.B, c.Ns, hk),
-                          dc.np("v").reshape(c.B, c.Ns, c.Hv * c.d)], axis=-1)
-    assert_close(got, y, bf16=(c.in_dtype == "bf16"), what=f"{name} conv")
-    for b in range(c.B):
-        pad = sorted(set(range(c.Ns)) - set(c.slot[b].tolist()))
-        assert np.all(got[b, pad] == 0.0)
-    if c.in_dtype == "bf16":   # values are bf16 by construction; most must be the oracle's own rounding
-        y16 = O.conv(c.parent, c.slot, c.state_row, L.x, L.conv_w, L.conv_b, L.hist, c.Ns, out_dtype="bf16")
-        assert (got == y16).mean() > 0.98
+    for l, L in enumerate(c.layers):
+        y = O.conv(c.parent, c.slot, c.state_row, L.x, L.conv_w, L.conv_b, L.hist, c.Ns, out_dtype="none")
+        got = np.concatenate([dc.np("q", l).reshape(c.B, c.Ns, hk), dc.np("k", l).reshape(c.B, c.Ns, hk),
+                              dc.np("v", l).reshape(c.B, c.Ns, c.Hv * c.d)], axis=-1)
+        assert_close(got, y, bf16=(c.in_dtype == "bf16"), what=f"{name} conv, layer {l}")
+        for b in range(c.B):
+            pad = sorted(set(range(c.Ns)) - set(c.slot[b].tolist()))
+            assert np.all(got[b, pad] == 0.0)
+        if c.in_dtype == "bf16":   # values are bf16 by construction; most must be the oracle's own rounding
+            y16 = O.conv(c.parent, c.slot, c.state_row, L.x, L.conv_w, L.conv_b, L.hist, c.Ns, out_dtype="bf16")
+            assert (got == y16).mean() > 0.98
 
 
 # ------------------------------------------------------------------ scan
@@ -445,6 +469,43 @@ def test_kernel_overlap_changes_nothing(name):
     for i in (1, 2, 3):
         assert torch.equal(res[False][i], res[True][i])
     assert not torch.equal(res[True][0][0], res[True][0][1])      # the cycles really advanced the state
+
+
+def test_overlap_chain_survives_commits_that_have_nothing_to_do():
+    """No status words and every accepted length zero: every CTA of the commit leaves early.  It must
+    still pass its dependency wait, or the grid completes while the scan before it is running and the
+    next cycle's convolution overwrites the operand buffers that scan still reads.  Several cycles with
+    fresh inputs in the SAME operand buffers, bitwise against plain stream order and against the oracle."""
+    c = W.config2()
+    xs = [W.config2(seed=W.BASE_SEED + 500 + i).layers[0].x for i in range(3)]
+    res = {}
+    for on in (False, True):
+        cx = ctx("auto")
+        cx.set_overlap(on)
+        dc = DeviceCase(cx, c)
+        t = dict(dc.layers[0].tensors)
+        t["status"] = None
+        layers = [binding.GdnLayer(Hk=c.Hk, Hv=c.Hv, d=c.d, scale=dc.scale, qk_l2norm=dc.qk_l2norm, l2_eps=dc.l2_eps, **t)]
+        zero_len = torch.zeros_like(dc.accepted_len)
+        xdev = [torch.from_numpy(x).to(torch.bfloat16).to(dc.dev) for x in xs]
+        outs = []
+        for cycle in range(6):
+            dc.t("x").copy_(xdev[cycle % 3])
+            cx.verify(dc.desc, layers)
+            cx.commit(dc.desc, layers, dc.accepted, zero_len)
+            outs.append(dc.t("out").clone())
+        torch.cuda.synchronize()
+        res[on] = outs
+        if on:      # last cycle against the oracle (conv of the last x, scan from the untouched state)
+            L = c.layers[0]
+            o_ref, _, _ = oracle_scan_from_device(dc)
+            assert_close(dc.np("out"), o_ref, what="outputs of the last cycle")
+            y = O.conv(c.parent, c.slot, c.state_row, xs[5 % 3], L.conv_w, L.conv_b, L.hist, c.Ns, out_dtype="none")
+            assert_close(dc.np("k").reshape(c.B, c.Ns, -1), y[..., c.Hk * c.d:2 * c.Hk * c.d], bf16=True, what="recorded k")
+            assert torch.equal(dc.t("state").cpu(), torch.from_numpy(L.state))        # nothing was committed
+    ctx("auto").set_overlap(True)
+    for a, b in zip(res[False], res[True]):
+        assert torch.equal(a, b)
 
 
 def test_multi_layer_launch_and_snapshot_all():

@@ -157,6 +157,14 @@ def test_error_codes_and_no_cpu_fallback():
     assert rc == 4
     rc = binding._lib.lumo_gdn_tree_scan_static(ctx._h, desc._h, arr, 1, None)
     assert rc == 4
+    # a path bound beyond 256 nodes (the kernels stage the path in arrays of that size) or below 1 is
+    # refused on the host, before anything is looked at or enqueued
+    for bad_lmax in (0, -3, 257, 300, 1 << 20):
+        assert binding._lib.lumo_gdn_commit(ctx._h, desc._h, arr, 1, None, None, bad_lmax, None) == 1
+        assert b"lmax" in binding._lib.lumo_last_error(ctx._h)
+        assert binding._lib.lumo_gdn_commit_verify(ctx._h, desc._h, arr, None, None, bad_lmax, desc._h, arr, 1, None) == 1
+    assert binding._lib.lumo_gdn_commit(ctx._h, desc._h, arr, 1, None, None, 256, None) == 4
+    assert binding._lib.lumo_conv_rows_per_cta(ctx._h, desc._h, 16, 32, 128, 1) == 0     # host-only context
     import torch
     if not torch.cuda.is_available():
         with pytest.raises(binding.LumoError):

@@ -35,6 +35,29 @@ def rand_parents(seed, n, B=1):
     return [[int(rs.integers(-1, i)) for i in range(n)] for _ in range(B)]
 
 
+# ---------------------------------------------------------------- the sequential recurrence
+def test_chain_tree_equals_the_sequential_gated_delta_rule():
+    """A chain-shaped tree is an ordinary token sequence: the oracle must reproduce the sequential gated
+    delta rule in its matrix form S_t = alpha_t S_{t-1} (I - beta_t k_t k_t^T) + beta_t v_t k_t^T,
+    o_t = S_t q_t (Eq. 2-3 multiplied out), written here with library matrix products only."""
+    n, d = 9, 16
+    c = small_case([W.tree_chain(n)] * 2, seed=21, d=d, Hk=2, Hv=4, Ns=n + 3, permute=True)
+    L = c.layers[0]
+    o, snap, _ = run_scan(c, snap_nodes=all_nodes(c), mode="walk")
+    I = np.eye(d)
+    for b in range(c.B):
+        for h in range(c.Hv):
+            g = h // (c.Hv // c.Hk)
+            S = L.state[c.state_row[b], h].astype(np.float64)
+            for t in range(n):
+                r = c.slot[b, t]
+                k, q, v = (a.astype(np.float64) for a in (L.k[b, r, g], L.q[b, r, g], L.v[b, r, h]))
+                a_t, b_t = float(L.alpha[b, r, h]), float(L.beta[b, r, h])
+                S = a_t * S @ (I - b_t * np.outer(k, k)) + b_t * np.outer(v, k)
+                np.testing.assert_allclose(snap[b, t, h], S, rtol=1e-12, atol=1e-15)
+                np.testing.assert_allclose(o[b, r, h], S @ q, rtol=1e-11, atol=1e-15)
+
+
 # ---------------------------------------------------------------- closed forms
 def test_beta_zero_is_pure_decay():
     c = small_case(rand_parents(1, 12, B=2))
