@@ -256,6 +256,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2 twice)")
     ap.add_argument("--out-dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--scan-algo", default="auto", choices=["auto", "rank1", "gram", "solve"],
+                    help="which scan kernel verify uses (auto = the library's choice)")
     ap.add_argument("--fused-commit", action="store_true",
                     help="time lumo_gdn_commit_verify (the previous cycle's commit folded into the verify) instead of "
                          "verify + commit; every step still commits one accepted path and verifies one tree per sequence")
@@ -285,6 +287,7 @@ def main():
 
     ctx = binding.Context(local)
     ctx.set_overlap(not args.no_overlap)
+    ctx.set_scan_algo(args.scan_algo)
     # ---- buffer sets: distinct seeds per set and per rank, together larger than L2 -----------
     case0 = make_case(args.config, seed_offset=rank_seed_offset(rank))
     n_layers = len(case0.layers)

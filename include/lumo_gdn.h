@@ -111,11 +111,21 @@ const char* lumo_last_error(const lumo_ctx* ctx);
 /* Bytes of library-owned device scratch currently held (for reporting). */
 int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx);
 
-/* Which scan kernel lumo_gdn_tree_verify uses: 0 = automatic (the tensor-core Gram form when the
- * shape allows it: d = 128, bf16 operands, tree depth <= 16, no snapshots; trees of more than 64
- * nodes are cut into node groups on the host; else rank-1), 1 = always the rank-1 fp32 kernel,
- * 2 = Gram form or LUMO_ERR_UNSUPPORTED. */
+/* Which scan kernel lumo_gdn_tree_verify uses: 0 = automatic (the tensor-core kernel when the shape
+ * allows it: d = 128, bf16 operands, tree depth <= 16, no snapshots; trees of more than 64 nodes are
+ * cut into node groups on the host; else rank-1), 1 = always the rank-1 fp32 kernel, 2 = the Gram form
+ * with a forward substitution over value rows (what "automatic" picks: it measured faster), 3 = the
+ * solved Gram form (the triangular system is solved on scalars per head and the state enters a single
+ * product with "effective queries"); 2 and 3 return LUMO_ERR_UNSUPPORTED on other shapes. */
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo);
+
+/* Test aid for the failure path of the tensor-core scan.  That kernel waits for its tensor-core work
+ * on an mbarrier with a bounded number of polls; when the bound runs out it writes LUMO_SEQ_TIMEOUT
+ * into the status words, frees its tensor memory and returns.  With the drill on, the kernel issues
+ * no tensor-core work at all (so nothing asynchronous is in flight) and polls only 1024 times: the
+ * wait runs out by construction and the failure path executes, harmlessly.  Outputs of such a call are
+ * undefined.  Default off. */
+int lumo_ctx_set_timeout_drill(lumo_ctx* ctx, int on);
 
 /* Kernel overlap (default on): conv, scan and commit are launched with programmatic dependent launch,
  * so each kernel's set-up (and, for commit, its whole read phase) runs under the tail of the kernel

@@ -34,7 +34,7 @@ TABLES = ["depth", "n_child", "child_off", "child_list", "is_leaf", "leaves", "p
 KERNEL_KINDS = ["conv", "scan", "commit", "path"]
 
 EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_scratch_bytes",
-           "lumo_ctx_timing_enable", "lumo_ctx_timing_read", "lumo_ctx_set_scan_algo", "lumo_ctx_set_overlap",
+           "lumo_ctx_timing_enable", "lumo_ctx_timing_read", "lumo_ctx_set_scan_algo", "lumo_ctx_set_overlap", "lumo_ctx_set_timeout_drill",
            "lumo_tree_desc_create", "lumo_tree_desc_destroy", "lumo_tree_desc_get",
            "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit",
            "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_conv_rows_per_cta", "lumo_tree_accept", "lumo_select_spine_top3", "lumo_gdn_commit_verify"]
@@ -88,6 +88,7 @@ _lib.lumo_ctx_scratch_bytes.argtypes = [ctypes.c_void_p]
 _lib.lumo_ctx_scratch_bytes.restype = ctypes.c_int64
 _lib.lumo_ctx_set_scan_algo.argtypes = [ctypes.c_void_p, ctypes.c_int]
 _lib.lumo_ctx_set_overlap.argtypes = [ctypes.c_void_p, ctypes.c_int]
+_lib.lumo_ctx_set_timeout_drill.argtypes = [ctypes.c_void_p, ctypes.c_int]
 _lib.lumo_ctx_timing_enable.argtypes = [ctypes.c_void_p, ctypes.c_int]
 _lib.lumo_ctx_timing_read.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int,
                                       ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]
@@ -150,8 +151,12 @@ class Context:
         return _lib.lumo_ctx_scratch_bytes(self._h)
 
     def set_scan_algo(self, algo: str = "auto"):
-        """"auto" | "rank1" | "gram": which scan kernel verify uses."""
-        self._check(_lib.lumo_ctx_set_scan_algo(self._h, {"auto": 0, "rank1": 1, "gram": 2}[algo]))
+        """"auto" | "rank1" | "gram" | "solve": which scan kernel verify uses."""
+        self._check(_lib.lumo_ctx_set_scan_algo(self._h, {"auto": 0, "rank1": 1, "gram": 2, "solve": 3}[algo]))
+
+    def set_timeout_drill(self, on: bool):
+        """Test aid: the tensor-core scan issues no tensor-core work, so its bounded wait runs out."""
+        self._check(_lib.lumo_ctx_set_timeout_drill(self._h, int(on)))
 
     def set_overlap(self, on: bool = True):
         """Programmatic dependent launch between conv, scan and commit (default on)."""

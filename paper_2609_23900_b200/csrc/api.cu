@@ -61,6 +61,7 @@ int prepare(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* laye
   s->n_snap = a0.snapshot_mode == 2 ? desc->N : a0.n_snap;
   s->n_layers = n_layers;
   s->gate_mode = a0.gate_mode;
+  s->debug_skip_mma = ctx->timeout_drill ? 1 : 0;
   if (for_verify && a0.snapshot_mode == 1 && (a0.n_snap < 1 || a0.n_snap > kMaxNodes))
     return fail(ctx, LUMO_ERR_ARG, "n_snap must be in [1, 256] in snapshot list mode");
   for (int l = 0; l < n_layers; ++l) {
@@ -182,8 +183,15 @@ int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx) { return ctx ? (int64_t)ctx-
 
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo) {
   if (!ctx) return LUMO_ERR_ARG;
-  if (algo < 0 || algo > 2) return fail(ctx, LUMO_ERR_ARG, "scan algo must be 0 (auto), 1 (rank-1) or 2 (Gram form)");
+  if (algo < 0 || algo > 3)
+    return fail(ctx, LUMO_ERR_ARG, "scan algo must be 0 (auto), 1 (rank-1), 2 (Gram form, forward substitution) or 3 (solved Gram form)");
   ctx->scan_algo = algo;
+  return LUMO_OK;
+}
+
+int lumo_ctx_set_timeout_drill(lumo_ctx* ctx, int on) {
+  if (!ctx) return LUMO_ERR_ARG;
+  ctx->timeout_drill = on != 0;
   return LUMO_OK;
 }
 
@@ -367,6 +375,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
           const int dep = t.tab[LUMO_TAB_DEPTH][node];
           h[o_tc_meta + gi * 64 + pi] = h[o_slot + (size_t)b * N + node] | (dep << 16) | ((int)gr.emit[pi] << 24);
           int cur = parent[(size_t)b * N + node];
+          anc[pi * 16 + dep - 1] = (uint8_t)pi;
           for (int j = dep - 2; j >= 0; --j) { anc[pi * 16 + j] = (uint8_t)pos[cur]; cur = parent[(size_t)b * N + cur]; }
           for (int dd = dep; dd < 20; ++dd) lvl[dd] += 1;      // lvl[d] = members of depth <= d
         }
@@ -480,7 +489,7 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
   cudaStream_t st = (cudaStream_t)stream;
   const TreeDev t = tree_view(desc, s.snapshot_mode != 0 ? 1 : 0);
   const bool gram_ok = desc->d_tc_meta != nullptr && gram_supported(s, desc->max_depth);
-  if (ctx->scan_algo == 2 && !gram_ok)
+  if (ctx->scan_algo >= 2 && !gram_ok)
     return fail(ctx, LUMO_ERR_UNSUPPORTED, "the Gram-form scan needs d = 128, bf16 operands, depth <= 16, no snapshots");
   // The Gram-form scan requests the pre-tree state ahead of its dependency wait.  Behind a convolution
   // that is safe (the convolution waits first, so whatever wrote the state has completed); launched
@@ -495,7 +504,9 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
     }
     const bool state_fresh = !layers[0].x && (prev_call == lumo_ctx::kCommit || prev_call == lumo_ctx::kCommitVerify);
     e = timed(ctx, LUMO_K_SCAN, st, [&] {
-      return launch_scan_gram(s, t, lb, ctx->sm_count, use_overlap(ctx, s) && !state_fresh, st);
+      const bool pdl = use_overlap(ctx, s) && !state_fresh;
+      return ctx->scan_algo == 3 ? launch_scan_solve(s, t, lb, ctx->sm_count, pdl, st)
+                                 : launch_scan_gram(s, t, lb, ctx->sm_count, pdl, st);
     });
     return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "Gram-form scan launch");
   }
@@ -648,7 +659,10 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
     });
     if (e != cudaSuccess) return cuda_fail(ctx, e, "conv launch");
   }
-  e = timed(ctx, LUMO_K_SCAN, st, [&] { return launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st); });
+  e = timed(ctx, LUMO_K_SCAN, st, [&] {
+    return ctx->scan_algo == 3 ? launch_scan_solve_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st)
+                               : launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st);
+  });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "fused scan launch");
 }
 

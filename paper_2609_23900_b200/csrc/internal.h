@@ -47,7 +47,8 @@ struct lumo_ctx {
   void* scratch = nullptr;      // scan stack levels
   size_t scratch_bytes = 0;
   // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
-  int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form (tensor cores)
+  int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form with forward substitution, 3 solved Gram form
+  bool timeout_drill = false;   // test aid: the tensor-core scan skips its tensor-core work (lumo_ctx_set_timeout_drill)
   bool overlap = true;          // programmatic dependent launch between conv -> scan -> commit
   // Kind of the previous call that launched on this context.  Kernels that read some of their inputs
   // ahead of their dependency wait (commit: path and state; scan without convolution: state) get the
@@ -86,7 +87,7 @@ struct lumo_tree_desc {
   int max_group_nodes = 0;        // largest group (the scan picks a 32-node tile when every group fits it)
   int32_t* d_tc_group = nullptr;  // [G, 4]  sequence b, node count, first-group-of-b flag, 0
   int32_t* d_tc_meta = nullptr;   // [G, 64] physical row | depth << 16 | emit << 24 of the node at position pi
-  uint8_t* d_tc_anc = nullptr;    // [G, 64, 16] positions of the ancestors, root first
+  uint8_t* d_tc_anc = nullptr;    // [G, 64, 16] positions of the ancestors, root first, then the node's own position
   uint8_t* d_tc_lvl = nullptr;    // [G, 20] lvl[d] = number of group nodes of depth <= d (lvl[0] = 0)
 };
 
@@ -116,6 +117,7 @@ struct Shape {
   int snapshot_mode, n_snap;
   int n_layers;
   int gate_mode;
+  int debug_skip_mma;   // test aid of the tensor-core scan: issue no tensor-core work, let the bounded wait run out
 };
 
 // What the fused commit + verify scan needs of the previous cycle: its layers (recorded k, v, gates,
@@ -272,6 +274,11 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
 // same scan, first replaying the previous cycle's accepted path into the state it has just loaded
 cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
                                    int sm_count, bool pdl, cudaStream_t st);
+// solved Gram form on tcgen05 (scan_solve.cu): the triangular system solved on scalars, one state product
+cudaError_t launch_scan_solve(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
+                              cudaStream_t st);
+cudaError_t launch_scan_solve_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
+                                    int sm_count, bool pdl, cudaStream_t st);
 // device address of the built-in stack on `device` (which must be current); looked up once per device
 cudaError_t static_stack_address(int device, float** ptr);
 cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb, const int32_t* accepted,

@@ -101,6 +101,10 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)_
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* gmem) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(dst), "l"(gmem) : "memory");
 }
+// pull of the 128-byte line at `gmem` into L2 (a request without a destination register)
+__device__ __forceinline__ void prefetch_l2(const void* gmem) {
+  asm volatile("prefetch.global.L2 [%0];\n" ::"l"(gmem) : "memory");
+}
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
@@ -244,6 +248,21 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     const int g = hv / rep;
     const int row = L.state_row[b];
     const size_t out_row_stride = (size_t)s.Hv * kD;
+    // The item this CTA takes next: its state and operand rows are pulled into L2 while this item
+    // computes (requests issued behind the dependency wait below), so that its own loads find them there.
+    const int nxt = item + (int)gridDim.x;
+    // (trees cut into several groups re-read one state per group from L2 anyway: there it measured slower)
+    const bool has_next = !kFused && nxt < n_items && t.n_groups == s.B;
+    int n_hv = 0, n_layer = 0, n_b = 0, n_meta = -1, n_row = -1;
+    if (has_next) {
+      n_hv = nxt % s.Hv;
+      const int n_gi = (nxt / s.Hv) % t.n_groups;
+      n_layer = nxt / (s.Hv * t.n_groups);
+      const int4 gi4 = *reinterpret_cast<const int4*>(t.tc_group + n_gi * 4);
+      n_b = gi4.x;
+      if (tid < gi4.y) n_meta = t.tc_meta[n_gi * kNT + tid];
+      n_row = lb.l[n_layer].state_row[n_b];
+    }
 
     if (row < 0 || row >= s.n_state_rows) {   // skipped sequence: zero outputs
       pdl_wait();                             // every path through the kernel passes its dependency wait
@@ -337,6 +356,27 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     // A fused launch rewrites the state, which a dependent (a commit, the next scan) requests ahead of
     // its own wait: it lets nobody in before it has finished.
     if constexpr (!kFused) pdl_trigger();
+    if (has_next) {
+      if (n_meta >= 0) {      // a node's key, query and value rows (256 bytes = two lines each) and its gates
+        const LayerPtrs& NL = lb.l[n_layer];
+        const size_t pr = (size_t)n_b * s.Ns + (n_meta & 0xFFFF);
+        const int n_g = n_hv / rep;
+        const __nv_bfloat16* pk = reinterpret_cast<const __nv_bfloat16*>(NL.k) + (pr * s.Hk + n_g) * kD;
+        const __nv_bfloat16* pq = reinterpret_cast<const __nv_bfloat16*>(NL.q) + (pr * s.Hk + n_g) * kD;
+        const __nv_bfloat16* pv = reinterpret_cast<const __nv_bfloat16*>(NL.v) + (pr * s.Hv + n_hv) * kD;
+        prefetch_l2(pk); prefetch_l2(pk + 64);
+        prefetch_l2(pq); prefetch_l2(pq + 64);
+        prefetch_l2(pv); prefetch_l2(pv + 64);
+        const size_t gsz = s.gate_dtype == LUMO_BF16 ? 2 : 4;
+        prefetch_l2(reinterpret_cast<const unsigned char*>(NL.alpha) + (pr * s.Hv + n_hv) * gsz);
+        prefetch_l2(reinterpret_cast<const unsigned char*>(NL.beta) + (pr * s.Hv + n_hv) * gsz);
+      }
+      if (n_row >= 0 && n_row < s.n_state_rows) {      // the state: 64 KiB = 512 lines, two per thread
+        const float* ns0 = lb.l[n_layer].state + ((size_t)n_row * s.Hv + n_hv) * kD * kD;
+        prefetch_l2(ns0 + 32 * tid);
+        prefetch_l2(ns0 + 32 * (tid + kThreads));
+      }
+    }
     if constexpr (kFused) {
       // The convolution before this kernel read the committed history through the path; now that it has
       // finished, the history buffer itself is brought up to date: the value heads of a sequence share

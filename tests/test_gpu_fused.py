@@ -62,10 +62,17 @@ def _oracle(P, C, dcP, layersC, l, accepted, length):
     return st1, hist1, status, y, o_ref
 
 
+@pytest.fixture(params=["auto", "solve"])
+def algo(request):
+    """Both tensor-core scans have a fused variant; every fused test runs on each."""
+    yield request.param
+    ctx("auto")
+
+
 @pytest.mark.parametrize("kind", ["cfg2", "two_layers", "paper_then_cfg3", "fallback_many_groups"])
-def test_commit_verify_equals_commit_then_verify(kind):
+def test_commit_verify_equals_commit_then_verify(kind, algo):
     P, C = _cycles(kind)
-    c = ctx()
+    c = ctx(algo)
     dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
     dcP.verify()                                    # records the previous cycle's operands
     layersC = _share_state(dcP, dcC)
@@ -101,7 +108,7 @@ def test_commit_verify_equals_commit_then_verify(kind):
         assert np.abs(o1 - o2).max() <= 1e-4 * (1.0 + np.abs(o2).max())
 
 
-def test_commit_verify_rejects_a_bad_path_and_skips_empty_ones():
+def test_commit_verify_rejects_a_bad_path_and_skips_empty_ones(algo):
     P, C = _cycles("cfg2")
     acc, ln = P.accepted.copy(), P.accepted_len.copy()
     ln[1] = 0                                       # nothing accepted: state stays
@@ -109,7 +116,7 @@ def test_commit_verify_rejects_a_bad_path_and_skips_empty_ones():
     root = int(np.flatnonzero(P.parent[2] < 0)[0])
     acc[2, :2] = [root, next(i for i in range(P.N) if depth[i] == 3)]   # second entry is no child of the first
     ln[2] = 2
-    c = ctx()
+    c = ctx(algo)
     dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
     dcP.verify()
     layersC = _share_state(dcP, dcC)
@@ -127,7 +134,7 @@ def test_commit_verify_rejects_a_bad_path_and_skips_empty_ones():
     assert_close(layersC[0].tensors["out"].to(torch.float64).cpu().numpy(), o_ref, what="outputs")
 
 
-def test_commit_verify_every_mix_of_old_and_accepted_history_rows():
+def test_commit_verify_every_mix_of_old_and_accepted_history_rows(algo):
     """Accepted lengths 0, 1, 2, 3, 4 and 5 in one batch: the three history rows the new tree's
     convolution reads are then 3, 2, 1 and 0 old rows followed by 0, 1, 2 and 3 accepted inputs.  The
     recorded operands (every row, depth-1 rows read all three history taps), the committed state and
@@ -141,7 +148,7 @@ def test_commit_verify_every_mix_of_old_and_accepted_history_rows():
     assert P.accepted_len.tolist() == [0, 1, 2, 3, 4, 5]
     C.state_row, C.rows = P.state_row.copy(), P.rows
     C.layers[0].state, C.layers[0].hist = P.layers[0].state.copy(), P.layers[0].hist.copy()
-    c = ctx()
+    c = ctx(algo)
     dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
     dcP.verify()
     layersC = _share_state(dcP, dcC)
@@ -176,11 +183,11 @@ def test_commit_verify_argument_checks():
     assert e.value.code == 1
 
 
-def test_commit_verify_scan_only_cycle_updates_history_with_the_commit_kernel():
+def test_commit_verify_scan_only_cycle_updates_history_with_the_commit_kernel(algo):
     """The new cycle has no convolution (operands given): the history of the accepted path is then
     gathered by the commit kernel's history CTAs ahead of the fused scan."""
     P, C = _cycles("cfg2")
-    c = ctx()
+    c = ctx(algo)
     dcP, dcC = DeviceCase(c, P), DeviceCase(c, C, use_conv=False, qk_l2norm=True)
     dcP.verify()
     layersC = []
@@ -202,13 +209,13 @@ def test_commit_verify_scan_only_cycle_updates_history_with_the_commit_kernel():
     assert_close(f(tc["out"]), o_ref, what="outputs")
 
 
-def test_commit_after_commit_verify_sees_the_rewritten_state():
+def test_commit_after_commit_verify_sees_the_rewritten_state(algo):
     """A plain commit right after a fused call (the last cycle of a generation) under kernel overlap:
     it must start from the state the fused scan wrote, cycle after cycle, bitwise as without overlap."""
     P, C = _cycles("cfg2")
     res = {}
     for on in (False, True):
-        c = ctx()
+        c = ctx(algo)
         c.set_overlap(on)
         dcP, dcC = DeviceCase(c, P), DeviceCase(c, C)
         dcP.verify()

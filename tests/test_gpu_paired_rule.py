@@ -1,0 +1,51 @@
+"""The paper's recurrent component checks as tests (Sec. "Numerical and candidate-selection validation",
+Table "GDN component checks"): published states bit-equal to the native chain, and the paired error rule
+of the tree scan against the native sequential recurrence, both measured against the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_23900_b200 import workload as W
+from paper_2609_23900_b200.runtime import DeviceCase
+from tests.harness import ctx
+from tests.paired_rule import paired_rule
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name", ["paper_geometry", "cfg2_b2"])
+def test_verifier_node_states_equal_the_commit_chain_bit_for_bit(name):
+    """Every node's state as the sequential (rank-1) verifier holds it equals the state the commit kernel
+    publishes when it replays the path to that node from the pre-tree state: one per-token arithmetic on
+    both sides (the paper reports its published states bitwise equal to the native chain)."""
+    c = W.config_paper(B=2) if name == "paper_geometry" else W.config2(B=2)
+    cx = ctx("rank1")
+    dc = DeviceCase(cx, c, use_conv=False, qk_l2norm=False, snapshot_mode=2)
+    dc.verify()
+    torch.cuda.synchronize()
+    snap = dc.t("snap_out").clone()                                   # [B, N, Hv, d, d]
+    state = dc.t("state")
+    S0 = state.clone()
+    lmax = max(max(W.tree_depths(p.tolist())) for p in c.parent)
+    acc = torch.zeros((c.B, lmax), dtype=torch.int32, device=dc.dev)
+    ln = torch.zeros((c.B,), dtype=torch.int32, device=dc.dev)
+    rows = torch.from_numpy(c.state_row.astype(np.int64)).to(dc.dev)
+    for i in range(c.N):
+        cx.path_from_node(dc.desc, torch.full((c.B,), i, dtype=torch.int32, device=dc.dev), lmax, acc, ln)
+        state.copy_(S0)
+        cx.commit(dc.desc, dc.layers, acc, ln)
+        assert torch.equal(state[rows], snap[:, i]), f"node {i}"
+    ctx("auto")
+
+
+def test_paired_error_rule_counts():
+    """Against the sequential kernel as the native side the sequential kernel passes by construction; the
+    tensor-core kernels are counted and their error levels bounded (they sit four orders of magnitude
+    inside the 1e-3 (1 + |ref|) gate; the counts are reported by bench.py)."""
+    res = paired_rule(ctx(), W.config_paper(B=2))
+    k = res["kernels"]
+    assert k["rank1"]["passed_vs_sequential_kernel"] == res["cells"]
+    for algo in ("rank1", "gram", "solve"):
+        assert k[algo]["max_abs_error"] < 2e-6 and k[algo]["median_cell_rms_error"] < 2e-7
+    # the commit chain with a float64 output product is the more exact native side
+    assert res["native"]["commit_chain"]["median_cell_rms_error"] <= res["native"]["sequential_kernel"]["median_cell_rms_error"]

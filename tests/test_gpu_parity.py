@@ -126,12 +126,12 @@ def test_conv_recorded_operands(name):
 # ------------------------------------------------------------------ scan
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("use_conv", [False, True])
-@pytest.mark.parametrize("algo", ["rank1", "gram"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve"])
 def test_scan_outputs_match_oracle(name, use_conv, algo):
     c = CASES[name]()
-    if algo == "gram" and not gram_eligible(c):
+    if algo != "rank1" and not gram_eligible(c):
         with pytest.raises(binding.LumoError) as e:     # refused loudly, never a silent fallback
-            DeviceCase(ctx("gram"), c, use_conv=use_conv).verify()
+            DeviceCase(ctx(algo), c, use_conv=use_conv).verify()
         assert e.value.code == 4
         return
     dc = DeviceCase(ctx(algo), c, use_conv=use_conv)
@@ -154,7 +154,7 @@ def test_scan_outputs_match_oracle(name, use_conv, algo):
     assert_close(dc16.np("out"), o_ref, bf16=True, what=f"{name} scan bf16 out")
 
 
-@pytest.mark.parametrize("algo", ["rank1", "gram"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve"])
 def test_scan_twice_is_bitwise_reproducible(algo):
     c = CASES["cfg2"]()
     dc = DeviceCase(ctx(algo), c)
@@ -166,7 +166,7 @@ def test_scan_twice_is_bitwise_reproducible(algo):
     assert torch.equal(a, dc.t("out")) and torch.equal(qa, dc.t("q"))
 
 
-@pytest.mark.parametrize("algo", ["rank1", "gram"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve"])
 def test_l2norm_flag_scale_and_f32_gates(algo):
     c = small(rand_parents(4, 20, 2), d=128, dtype="bf16")
     rs = np.random.default_rng(1)
@@ -280,14 +280,15 @@ def test_commit_controls_len0_poisoned_tail_invalid_paths_skipped_rows():
     assert torch.all(dc2.t("out")[2] == 0) and torch.all(dc2.t("out")[3] == 0) and torch.all(dc2.t("q")[2] == 0)
 
 
-def test_gram_scan_skipped_rows_padding_and_depth_16():
+@pytest.mark.parametrize("tc", ["gram", "solve"])
+def test_gram_scan_skipped_rows_padding_and_depth_16(tc):
     # a 16-deep chain plus side leaves (depth limit of the Gram form), padded and permuted rows,
     # one skipped sequence and one row outside the pool
     parent = W.tree_chain(16) + [3, 3, 7, 11, 14]
     c = W.make_case("g16", [parent] * 4, seed=21, Hk=2, Hv=4, d=128, in_dtype="bf16", Ns=24, permute_slots=True,
                     alpha_lo=0.5, beta_uniform=True, extra_rows=2)
     assert gram_eligible(c)
-    dc = DeviceCase(ctx("gram"), c)
+    dc = DeviceCase(ctx(tc), c)
     dc.state_row[1] = -1
     dc.state_row[2] = c.rows + 3
     dc.t("out").fill_(float("nan"))
@@ -310,7 +311,8 @@ def test_gram_scan_skipped_rows_padding_and_depth_16():
     ctx("auto")
 
 
-def test_gram_groups_with_long_prefix_paths():
+@pytest.mark.parametrize("tc", ["gram", "solve"])
+def test_gram_groups_with_long_prefix_paths(tc):
     # caterpillar: a 10-node spine with 24 leaves under every spine node (250 nodes).  The tree is cut
     # into groups that each carry a prefix path of up to 10 recomputed nodes; every node must still be
     # written exactly once and match the oracle.
@@ -320,10 +322,10 @@ def test_gram_groups_with_long_prefix_paths():
         parent += [sp] * 24
     c = W.make_case("cat", [parent] * 2, seed=31, Hk=2, Hv=4, d=128, in_dtype="bf16", alpha_lo=0.5, beta_uniform=True)
     assert gram_eligible(c)
-    desc = ctx("gram").tree_desc(c.parent)
+    desc = ctx(tc).tree_desc(c.parent)
     tab = desc.table("gram_groups").tolist()
     assert tab[0] >= 5                                            # several groups
-    dc = DeviceCase(ctx("gram"), c)
+    dc = DeviceCase(ctx(tc), c)
     dc.t("out").fill_(float("nan"))
     dc.verify()
     torch.cuda.synchronize()
@@ -369,7 +371,7 @@ def test_randomized_shapes_both_kernels():
                         beta_uniform=rng.random() < 0.5, with_bias=rng.random() < 0.3)
         use_conv = rng.random() < 0.5
         ref = None
-        for algo in ("gram", "rank1"):
+        for algo in ("solve", "gram", "rank1"):
             dc = DeviceCase(ctx(algo), c, use_conv=use_conv)
             dc.t("out").fill_(float("nan"))
             dc.verify()
@@ -471,6 +473,33 @@ def test_kernel_overlap_changes_nothing(name):
     assert not torch.equal(res[True][0][0], res[True][0][1])      # the cycles really advanced the state
 
 
+def test_bounded_wait_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """The tensor-core scan waits for its tensor-core work on an mbarrier with a bounded number of polls.
+    With the drill on, the kernel issues no tensor-core work (nothing asynchronous is in flight) and polls
+    1024 times: the wait runs out, every CTA reports LUMO_SEQ_TIMEOUT for its sequence, frees its tensor
+    memory and returns.  The next ordinary call must be bitwise what it was before."""
+    c = CASES["cfg2"]()
+    cx = ctx("solve")
+    dc = DeviceCase(cx, c, use_conv=False, qk_l2norm=True)
+    dc.verify()
+    torch.cuda.synchronize()
+    ref = dc.t("out").clone()
+    assert dc.np("status").tolist() == [0] * c.B
+    cx.set_timeout_drill(True)
+    try:
+        dc.verify()
+        torch.cuda.synchronize()
+        assert dc.np("status").tolist() == [binding.SEQ_TIMEOUT] * c.B
+    finally:
+        cx.set_timeout_drill(False)
+    dc.t("out").fill_(float("nan"))
+    dc.verify()
+    torch.cuda.synchronize()
+    assert dc.np("status").tolist() == [0] * c.B
+    assert torch.equal(dc.t("out"), ref)
+    ctx("auto")
+
+
 def test_overlap_chain_survives_commits_that_have_nothing_to_do():
     """No status words and every accepted length zero: every CTA of the commit leaves early.  It must
     still pass its dependency wait, or the grid completes while the scan before it is running and the
@@ -558,8 +587,9 @@ def _raw_gates(c, seed):
     return out
 
 
-@pytest.mark.parametrize("name,algo", [("cfg0", "rank1"), ("cfg1", "rank1"), ("cfg1", "gram"), ("d64_bf16", "rank1"),
-                                       ("cfgP_padded_permuted", "rank1"), ("cfgP_padded_permuted", "gram")])
+@pytest.mark.parametrize("name,algo", [("cfg0", "rank1"), ("cfg1", "rank1"), ("cfg1", "gram"), ("cfg1", "solve"), ("d64_bf16", "rank1"),
+                                       ("cfgP_padded_permuted", "rank1"), ("cfgP_padded_permuted", "gram"),
+                                       ("cfgP_padded_permuted", "solve")])
 def test_raw_gate_inputs_verify_and_commit(name, algo):
     """Raw gate inputs activated inside the kernels: scan outputs and the committed state against the
     oracle fed with the fp64 activation of the same (rounded) inputs."""
