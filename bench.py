@@ -197,6 +197,24 @@ def run_oracle_steps(case, seconds: float, threads: int = 0):
     return case.B * case.N * n_layers * steps / dt, steps, used, dt
 
 
+def oracle_walk_mode():
+    """The oracle in its literal form (every node recomputed from the pre-tree state along its ancestry,
+    "walk" mode), scan only, on configs 0-2: nodes per second."""
+    from oracle import gdn_oracle as O
+    from paper_2609_23900_b200 import workload as W
+    out = {}
+    for name, case in (("cfg0", W.config0()), ("cfg1", W.config1()), ("cfg2", W.config2())):
+        L = case.layers[0]
+        best = None
+        for _ in range(3):
+            t0 = time.perf_counter()
+            O.scan(case.parent, case.slot, case.state_row, L.q, L.k, L.v, L.alpha, L.beta, L.state, mode="walk")
+            dt = time.perf_counter() - t0
+            best = dt if best is None else min(best, dt)
+        out[name] = case.B * case.N / best
+    return out
+
+
 def reference_arm(args, rank):
     """The oracle, as it stands, on the host cores (rank 0 only)."""
     if rank != 0:
@@ -224,6 +242,102 @@ def reference_arm(args, rank):
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
+
+
+def read_ncu_traffic(config_name):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one scan launch, from the ncu summary under
+    profiles/ -- used only when the kernel source is still the one that capture was taken from (the
+    summary records a hash of the source file); otherwise None."""
+    import hashlib
+    import re
+    path = os.path.join(ROOT, "profiles", "scan_gram_traffic.md")
+    src = os.path.join(ROOT, "paper_2609_23900_b200", "csrc", "scan_gram.cu")
+    if not (os.path.exists(path) and os.path.exists(src)):
+        return None
+    text = open(path).read()
+    sha = hashlib.sha256(open(src, "rb").read()).hexdigest()[:16]
+    m = re.search(r"source-sha256:\s*([0-9a-f]{16})", text)
+    t = re.search(r"traffic %s:\s*(\d+)" % re.escape(config_name), text)
+    if not (m and t) or m.group(1) != sha:
+        return None
+    return int(t.group(1))
+
+
+def measure_extra_config(ctx, name, out_dtype, peak_gbs, steps=20, warmup=3, snapshot_mode=0, n_sets=2):
+    """One more configuration of the benchmark spec in the same run: whole-step throughput, per-kernel device
+    time, the scan alone and the verify (conv + scan) alone from back-to-back launches, and the two
+    roofline fractions.  Fewer steps than the headline so that the whole run stays within minutes."""
+    import torch
+    from paper_2609_23900_b200 import binding
+    from paper_2609_23900_b200.runtime import DeviceCase
+    cases = [make_case(name, seed_offset=i) for i in range(n_sets)]
+    c0 = cases[0]
+    sets = [DeviceCase(ctx, c, out_dtype=out_dtype, snapshot_mode=snapshot_mode) for c in cases]
+    packed = [binding.Context.pack(s.layers) for s in sets]
+    n_layers = len(c0.layers)
+    nodes = c0.B * c0.N * n_layers
+    ab = algorithmic_bytes(c0, out_bytes=2 if out_dtype == "bf16" else 4)
+
+    def run_step(i):
+        s = sets[i % n_sets]
+        ctx.verify(s.desc, packed[i % n_sets])
+        ctx.commit(s.desc, packed[i % n_sets], s.accepted, s.accepted_len)
+
+    for i in range(max(warmup, n_sets)):
+        run_step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        run_step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_step = e0.elapsed_time(e1) / steps
+    ctx.timing_enable(True)
+    ctx.timing_read(reset=True)
+    for i in range(steps):
+        run_step(i)
+    torch.cuda.synchronize()
+    per_kernel = ctx.timing_read(reset=True)
+    ctx.timing_enable(False)
+    kern = {k: {"launches": n, "avg_us": 1e3 * ms / n} for k, (n, ms) in per_kernel.items() if n}
+
+    def back_to_back(arrs):
+        for i in range(warmup):
+            ctx.verify(sets[i % n_sets].desc, arrs[i % n_sets])
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(steps):
+            ctx.verify(sets[i % n_sets].desc, arrs[i % n_sets])
+        e1.record()
+        torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / steps
+
+    verify_us = back_to_back(packed)                  # conv + scan, launched as the library launches them
+    scan_only = []
+    for s_ in sets:
+        arr = binding.Context.pack(s_.layers)
+        for a in arr:
+            a.x = None
+        scan_only.append(arr)
+    scan_us = back_to_back(scan_only)
+    out = {"workload": WORKLOAD_TEXT[name], "value": nodes / (ms_step * 1e-3), "unit": UNIT, "ms_per_step": ms_step,
+           "steps": steps, "warmup": max(warmup, n_sets), "buffer_sets": n_sets,
+           "kernels": kern, "scan_us_back_to_back": scan_us, "verify_us_back_to_back": verify_us,
+           "scan_frac_of_hbm_peak": n_layers * ab["scan"] / (scan_us * 1e-6) / 1e9 / peak_gbs,
+           "verify_frac_of_hbm_peak": n_layers * ab["scan"] / (verify_us * 1e-6) / 1e9 / peak_gbs,
+           "algorithmic_bytes_verify": n_layers * ab["scan"],
+           "verify_nodes_per_s_per_layer": nodes / (verify_us * 1e-6),
+           "commit_us_per_layer": kern["commit"]["avg_us"] / n_layers if "commit" in kern else None}
+    if snapshot_mode == 2:
+        snap = c0.Hv * c0.d * c0.d * 4
+        out["snapshots"] = {"mode": "cached: every node state exported (snapshot_mode 2, sequential fp32 kernel)",
+                            "extra_state_bytes_per_node": snap,
+                            "extra_state_bytes_per_launch": snap * nodes,
+                            "algorithmic_bytes_per_node": n_layers * ab["scan"] / nodes}
+    del sets, packed, scan_only, cases
+    torch.cuda.empty_cache()
+    return out
 
 
 def fused_arm(args):
@@ -256,6 +370,10 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--sets", type=int, default=0, help="rotating buffer sets (0 = enough to exceed L2 twice)")
     ap.add_argument("--out-dtype", default="bf16", choices=["bf16", "f32"])
+    ap.add_argument("--extra-configs", dest="extra_configs", action="store_true", default=None,
+                    help="also measure configs 3 (recomputed and cached) and 4 (three shapes) in the same run "
+                         "(default: on for the default workload)")
+    ap.add_argument("--no-extra-configs", dest="extra_configs", action="store_false")
     ap.add_argument("--scan-algo", default="auto", choices=["auto", "rank1", "gram", "solve"],
                     help="which scan kernel verify uses (auto = the library's choice)")
     ap.add_argument("--fused-commit", action="store_true",
@@ -263,6 +381,8 @@ def main():
                          "verify + commit; every step still commits one accepted path and verifies one tree per sequence")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.extra_configs is None:
+        args.extra_configs = args.config == "cfg2" and not args.no_cpu_baseline
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -409,6 +529,16 @@ def main():
     torch.cuda.synchronize()
     kern["scan"]["avg_us_back_to_back"] = 1e3 * k0.elapsed_time(k1) / n_timed
     ctx.set_overlap(not args.no_overlap)
+    # the whole verify (conv + scan as the library launches them, kernel overlap included), back to back
+    for i in range(args.warmup):
+        ctx.verify(sets[i % n_sets].desc, packed[i % n_sets])
+    torch.cuda.synchronize()
+    k0.record()
+    for i in range(n_timed):
+        ctx.verify(sets[i % n_sets].desc, packed[i % n_sets])
+    k1.record()
+    torch.cuda.synchronize()
+    verify_b2b_us = 1e3 * k0.elapsed_time(k1) / n_timed
 
     # ---- end to end: inputs from pinned host memory, outputs back to the host --------------
     sampler.tag("e2e")
@@ -487,7 +617,9 @@ def main():
     fma = rank1_fma(case0) * n_layers
     sm_mhz = clocks["sm_mhz"] or 1965.0
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
-                "frac": achieved / peak_gbs, "peak_source": peak_src, "traffic": NCU_TRAFFIC.get(args.config),
+                "frac": achieved / peak_gbs, "peak_source": peak_src,
+                "traffic": read_ncu_traffic(args.config) if dominant == "scan" and args.scan_algo in ("auto", "gram") else None,
+                "traffic_source": "profiles/scan_gram_traffic.md (one ncu capture of this kernel source; null when the source changed since)",
                 "algorithmic_bytes_per_launch": n_layers * ab[dominant],
                 "avg_launch_us": dom_us,
                 "frac_of_8TBs_nominal": achieved / 8000.0,
@@ -499,6 +631,11 @@ def main():
                 if "scan" in kern else None}
     commit_us = kern["commit"]["avg_us"] / n_layers if "commit" in kern else None
     verify_us = sum(kern[k]["avg_us"] for k in ("conv", "scan") if k in kern)
+    # the metric's own unit: algorithmic bytes of the verify over the time of the whole verify (conv + scan)
+    verify_achieved = n_layers * ab["scan"] / (verify_b2b_us * 1e-6) / 1e9
+    roofline["verify_level"] = {"algorithmic_bytes": n_layers * ab["scan"], "us": verify_b2b_us, "achieved": verify_achieved,
+                                "frac": verify_achieved / peak_gbs, "unit": "GB/s",
+                                "timing": "K back-to-back lumo_gdn_tree_verify calls (conv + scan) between two CUDA events"}
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -518,8 +655,9 @@ def main():
             "gpu_launches": int(args.steps * sum(1 for k in ("conv", "scan", "commit") if k in kern)),
             "roofline": roofline,
             "kernels": kern,
-            "verify_nodes_per_s_per_layer": nodes_per_step / (verify_us * 1e-6),
-            "verify_us_per_layer": verify_us / n_layers, "commit_us_per_layer": commit_us,
+            "verify_nodes_per_s_per_layer": nodes_per_step / (verify_b2b_us * 1e-6),
+            "verify_us_per_layer": verify_b2b_us / n_layers, "verify_us_per_layer_event_bracketed": verify_us / n_layers,
+            "commit_us_per_layer": commit_us,
             "scratch_bytes": ctx.scratch_bytes}
 
     if world == 1 and not args.no_cpu_baseline:
@@ -530,19 +668,44 @@ def main():
             sample_case = copy.copy(case0)
             sample_case.layers = case0.layers[:2]
             sample += ", first 2 layers"
-        v, steps, cores, dt = run_oracle_steps(sample_case, args.cpu_seconds)
+        # best of three slices of the time budget (the oracle as it stands, memo mode)
+        runs = [run_oracle_steps(sample_case, args.cpu_seconds / 3.0) for _ in range(3)]
+        v, steps, cores, dt = max(runs, key=lambda r: r[0])
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                                "sample": f"{sample}; {steps} steps in {dt:.1f} s"}
+                                "sample": f"{sample}; best of 3 slices, {steps} steps in {dt:.1f} s",
+                                "walk_mode_scan_nodes_per_s": oracle_walk_mode()}
+        # the paper's paired error rule, counted for the tensor-core scans against the library's sequential
+        # recurrence (needs the fp64 oracle, hence in this leg); one layer of the headline workload
+        try:
+            from tests.paired_rule import paired_rule
+            pc = make_case(args.config, seed_offset=rank_seed_offset(rank))
+            if len(pc.layers) > 1:
+                pc.layers = pc.layers[:1]
+            line["paired_rule"] = paired_rule(ctx, pc, with_commit_chain=False)
+            line["paired_rule"]["rule"] = "E_tree <= 1.10 E_native + 2^-24 M_64 + 2^-149 per cell (sequence, node, value head), rms and max"
+        except Exception as e:      # an extra figure only
+            line["paired_rule"] = {"unavailable": f"{type(e).__name__}: {e}"[:200]}
     if world == 1 and not args.fused_commit and not args.no_cpu_baseline:
         line["fused_commit_verify"] = fused_arm(args)
+    if world == 1 and args.extra_configs and not args.fused_commit:
+        # the other configurations of the target in the same run (fewer steps each; configs 3 and 4)
+        extra = {}
+        plan = [("cfg3", "cfg3_recomputed", 0, 10, 2), ("cfg3", "cfg3_cached", 2, 4, 1),
+                ("cfg4_chains", "cfg4_chains", 0, 15, 2), ("cfg4_star", "cfg4_star", 0, 15, 2),
+                ("cfg4_random", "cfg4_random", 0, 15, 2)]
+        for name, key, snap, k_steps, k_sets in plan:
+            if name == args.config and snap == 0:
+                continue
+            try:
+                extra[key] = measure_extra_config(ctx, name, args.out_dtype, peak_gbs, steps=k_steps, snapshot_mode=snap,
+                                                  n_sets=k_sets)
+            except Exception as e:
+                extra[key] = {"unavailable": f"{type(e).__name__}: {e}"[:200]}
+        line["configs"] = extra
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
-
-# dram__bytes_read.sum + dram__bytes_write.sum of one scan launch, from the ncu captures
-# summarised under profiles/ (bytes per launch at the bench's launch configuration)
-NCU_TRAFFIC = {"cfg2": 25_297_152, "cfg4_star": 255_584_768}
 
 if __name__ == "__main__":
     main()
