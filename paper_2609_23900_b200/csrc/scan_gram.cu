@@ -96,6 +96,28 @@ struct PrevStage {
 constexpr int kOffPrev = kOffSmall + (((int)sizeof(Small) + 15) / 16) * 16;
 constexpr int kSmemBytesFused = kOffPrev + (int)sizeof(PrevStage) + 1024;
 
+// Layout of one CTA.  Compact (trees of at most 32 nodes, not fused): the state crosses shared memory
+// one 64-column half at a time (hi + lo of one k-block, 32 KB), the aliased areas shrink with the node
+// count, and a CTA needs 68 KB of shared memory and 128 tensor-memory columns: three CTAs per SM
+// instead of two (and 80 registers per thread instead of 128).
+template <bool C>
+struct GL {
+  static constexpr int kNodes = C ? 32 : kNT;
+  static constexpr int kAhi = 0, kAlo = C ? 16384 : 32768;
+  static constexpr int kKQ = C ? 32768 : kOffKQ;
+  static constexpr int kSmall = C ? 65536 : kOffSmall;
+  static constexpr int kStride = C ? 33 : kDumpStride;         // floats per dumped Gram row
+  static constexpr int kRec = C ? 128 * 33 * 4 : kOffRec;      // records behind the Gram dump / the deltas
+  static constexpr int kV = kRec + kNodes * (int)sizeof(NodeRec);
+  static constexpr int kZero = kNodes * kD;                    // element offset of the all-zero delta row
+  static constexpr int kTmem = C ? 128 : kTmemCols;
+  static constexpr int kGramCol = C ? 64 : 128;                // first tensor-memory column of the Gram block
+  static constexpr int kBytes = kSmall + (int)sizeof(Small) + 1024;
+};
+static_assert((GL<true>::kNodes + 1) * kD * 4 <= GL<true>::kRec, "delta array overflows the dump area");
+static_assert(GL<true>::kV + GL<true>::kNodes * kD * 2 <= GL<true>::kKQ, "aliased region overflows the state tiles");
+static_assert(3 * (GL<true>::kBytes + 1024) <= 228 * 1024, "three compact CTAs must share an SM");
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* gmem) {
@@ -181,13 +203,14 @@ __device__ __forceinline__ void store_out(void* out, size_t idx, int dtype, floa
 }
 
 // fp32 x -> bf16 hi + lo of four values, written to the two swizzled operand tiles
+template <int kHi = kOffAhi, int kLo = kOffAlo>
 __device__ __forceinline__ void split_store(unsigned char* smem, uint32_t off, float4 x) {
   __nv_bfloat162 h01 = __floats2bfloat162_rn(x.x, x.y), h23 = __floats2bfloat162_rn(x.z, x.w);
   const float2 f01 = __bfloat1622float2(h01), f23 = __bfloat1622float2(h23);
   __nv_bfloat162 l01 = __floats2bfloat162_rn(x.x - f01.x, x.y - f01.y);
   __nv_bfloat162 l23 = __floats2bfloat162_rn(x.z - f23.x, x.w - f23.y);
-  *reinterpret_cast<uint2*>(smem + kOffAhi + off) = make_uint2(*reinterpret_cast<uint32_t*>(&h01), *reinterpret_cast<uint32_t*>(&h23));
-  *reinterpret_cast<uint2*>(smem + kOffAlo + off) = make_uint2(*reinterpret_cast<uint32_t*>(&l01), *reinterpret_cast<uint32_t*>(&l23));
+  *reinterpret_cast<uint2*>(smem + kHi + off) = make_uint2(*reinterpret_cast<uint32_t*>(&h01), *reinterpret_cast<uint32_t*>(&h23));
+  *reinterpret_cast<uint2*>(smem + kLo + off) = make_uint2(*reinterpret_cast<uint32_t*>(&l01), *reinterpret_cast<uint32_t*>(&l23));
 }
 
 // what a warp needs for one node besides its ancestors' deltas
@@ -205,7 +228,7 @@ struct NodeOps {
 // kFused: before anything else the previous cycle's accepted path is replayed into the state rows as
 // they pass through the registers (same per-token update as the commit kernel), and the rows are
 // written back in place; the scan then runs from the updated state.  One group per sequence only.
-template <int NT, bool kFused>
+template <int NT, bool kFused, bool kCompact = false>
 __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t, const LayerBatch& lb, int n_items,
                                                const FusedPrev* fp) {
   extern __shared__ unsigned char smem_raw[];
@@ -213,12 +236,14 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
   // array keeps the pointers in the shared address space
   unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t sbase = smem_u32(smem);
-  Small& sm = *reinterpret_cast<Small*>(smem + kOffSmall);
+  static_assert(!kCompact || (NT == 32 && !kFused), "the compact layout serves the 32-node tile of the plain scan");
+  using LY = GL<kCompact>;
+  Small& sm = *reinterpret_cast<Small*>(smem + LY::kSmall);
   float* dump = reinterpret_cast<float*>(smem + kOffDump);
-  float* dls = reinterpret_cast<float*>(smem + kOffDump);     // [65][128]; row 64 stays zero
-  float* Pq = reinterpret_cast<float*>(smem + kOffPq);
-  NodeRec* recs = reinterpret_cast<NodeRec*>(smem + kOffRec);
-  const __nv_bfloat16* Vs = reinterpret_cast<const __nv_bfloat16*>(smem + kOffV);
+  float* dls = reinterpret_cast<float*>(smem + kOffDump);     // [nodes + 1][128]; the last row stays zero
+  float* Pq = reinterpret_cast<float*>(smem + LY::kKQ);
+  NodeRec* recs = reinterpret_cast<NodeRec*>(smem + LY::kRec);
+  const __nv_bfloat16* Vs = reinterpret_cast<const __nv_bfloat16*>(smem + LY::kV);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int grp = tid >> 7;            // half of the CTA: 0 or 1
@@ -226,7 +251,7 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
   const int rep = s.Hv / s.Hk;
 
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&sm.tmem_base)), "r"(LY::kTmem) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   if (tid == 0) { mbar_init(&sm.mbar, 1); sm.timed_out = 0; }
@@ -236,6 +261,10 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
   const uint32_t tmem = sm.tmem_base;
   const uint32_t tmem_lane = tmem + ((uint32_t)((warp & 3) * 32) << 16);   // this warp's 32 lanes
   uint32_t phase = 0;
+  // compact mode: state rows of this thread r = 16 u + 2 warp + (lane >> 4), four floats at column
+  // 4 (lane & 15) of the current 64-column half
+  const int srow0 = 2 * warp + (lane >> 4), c4 = lane & 15;
+  const uint32_t s0_off0 = sw128_offset(srow0, c4 >> 1) + (c4 & 1) * 8;   // rows 16 u on: + 2048 u
 
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {   // bounded: n_items
     const int hv = item % s.Hv;
@@ -299,7 +328,9 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     const float* S0 = L.state + ((size_t)row * s.Hv + hv) * kD * kD;
     float4 x[8];
 #pragma unroll
-    for (int u = 0; u < 8; ++u) x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * u) * kD + lane * 4);
+    for (int u = 0; u < 8; ++u)
+      x[u] = kCompact ? *reinterpret_cast<const float4*>(S0 + (size_t)(16 * u + srow0) * kD + 4 * c4)
+                      : *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * u) * kD + lane * 4);
     // ---- a. per-node tables (the addresses of everything else depend on them) -------------------
     if (tid < kNT) {
       sm.meta[tid] = tid < N ? t.tc_meta[gi * kNT + tid] : 0;
@@ -425,7 +456,7 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       for (int i = 0; i < kCopies; ++i) {
         const int idx = i * kThreads + tid;
         const int R = idx >> 4, c = idx & 15;
-        const uint32_t dst = sbase + kOffKQ + (c >> 3) * 16384 + sw128_offset(R, c & 7);
+        const uint32_t dst = sbase + LY::kKQ + (c >> 3) * 16384 + sw128_offset(R, c & 7);
         if (src[i]) cp_async16(dst, src[i]);
         else asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};\n" ::"r"(dst), "r"(0u) : "memory");
       }
@@ -465,16 +496,26 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
           for (int u = 0; u < 8; ++u) *reinterpret_cast<float4*>(Sw + (size_t)(r0 + 8 * u) * kD + lane * 4) = x[u];
         }
       };
-      replay_rows(warp);
+      if constexpr (kCompact) {
+        // first 64-column half -> tiles; the second half is requested at once and converted after the
+        // products of the first
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        split_store(smem, kblock * 16384 + sw128_offset(warp + 8 * u, chunk) + half * 8, x[u]);
-        x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * (8 + u)) * kD + lane * 4);   // second half
+        for (int u = 0; u < 8; ++u) {
+          split_store<LY::kAhi, LY::kAlo>(smem, s0_off0 + 2048 * u, x[u]);
+          x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(16 * u + srow0) * kD + 64 + 4 * c4);
+        }
+      } else {
+        replay_rows(warp);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          split_store(smem, kblock * 16384 + sw128_offset(warp + 8 * u, chunk) + half * 8, x[u]);
+          x[u] = *reinterpret_cast<const float4*>(S0 + (size_t)(warp + 8 * (8 + u)) * kD + lane * 4);   // second half
+        }
+        replay_rows(warp + 64);
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          split_store(smem, kblock * 16384 + sw128_offset(warp + 8 * (8 + u), chunk) + half * 8, x[u]);
       }
-      replay_rows(warp + 64);
-#pragma unroll
-      for (int u = 0; u < 8; ++u)
-        split_store(smem, kblock * 16384 + sw128_offset(warp + 8 * (8 + u), chunk) + half * 8, x[u]);
     }
     if (tid < kNT) { sm.alpha[tid] = gate_a; sm.beta[tid] = gate_b; }
     // padding rows: zero outputs
@@ -489,21 +530,31 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     if (tid == 0) {
       tc_fence_after();
       constexpr uint32_t idesc_p = umma_idesc(128, 2 * NT), idesc_g = umma_idesc(128, NT);
-      const uint64_t d_kq = umma_desc(sbase + kOffKQ), d_hi = umma_desc(sbase + kOffAhi), d_lo = umma_desc(sbase + kOffAlo);
+      const uint64_t d_kq = umma_desc(sbase + LY::kKQ), d_hi = umma_desc(sbase + LY::kAhi), d_lo = umma_desc(sbase + LY::kAlo);
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-        umma(tmem + 128, d_kq + koff, d_kq + koff, idesc_g, ks ? 1u : 0u);
+        umma(tmem + LY::kGramCol, d_kq + koff, d_kq + koff, idesc_g, ks ? 1u : 0u);
       }
+      if constexpr (kCompact) {
+        // the state tiles hold the first 64-column half only: its four contraction steps now
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-        umma(tmem, d_hi + koff, d_kq + koff, idesc_p, ks ? 1u : 0u);
-      }
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint64_t koff = (uint64_t)((ks * 32) >> 4);
+          umma(tmem, d_hi + koff, d_kq + koff, idesc_p, ks ? 1u : 0u);
+          umma(tmem, d_lo + koff, d_kq + koff, idesc_p, 1u);
+        }
+      } else {
 #pragma unroll
-      for (int ks = 0; ks < 8; ++ks) {
-        const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
-        umma(tmem, d_lo + koff, d_kq + koff, idesc_p, 1u);
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+          umma(tmem, d_hi + koff, d_kq + koff, idesc_p, ks ? 1u : 0u);
+        }
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint64_t koff = (uint64_t)(((ks >> 2) * 16384 + (ks & 3) * 32) >> 4);
+          umma(tmem, d_lo + koff, d_kq + koff, idesc_p, 1u);
+        }
       }
       umma_commit(&sm.mbar);
     } else if (grp == 1 && s.l2norm && vrow < NT) {
@@ -511,7 +562,7 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       float qq = 0.f;
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
-        const uint4 w = *reinterpret_cast<const uint4*>(smem + kOffKQ + (c >> 3) * 16384 + sw128_offset(R, c & 7));
+        const uint4 w = *reinterpret_cast<const uint4*>(smem + LY::kKQ + (c >> 3) * 16384 + sw128_offset(R, c & 7));
         const uint32_t ws[4] = {w.x, w.y, w.z, w.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -530,6 +581,33 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       if (L.status && tid == 0) L.status[b] = LUMO_SEQ_TIMEOUT;
       break;
     }
+    if constexpr (kCompact) {
+      // second 64-column half of the state through the same tiles, accumulated onto the first
+#pragma unroll
+      for (int u = 0; u < 8; ++u) split_store<LY::kAhi, LY::kAlo>(smem, s0_off0 + 2048 * u, x[u]);
+      fence_async_proxy();
+      __syncthreads();
+      if (tid == 0) {
+        tc_fence_after();
+        constexpr uint32_t idesc_p = umma_idesc(128, 2 * NT);
+        const uint64_t d_kq = umma_desc(sbase + LY::kKQ + 16384), d_hi = umma_desc(sbase + LY::kAhi), d_lo = umma_desc(sbase + LY::kAlo);
+#pragma unroll
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint64_t koff = (uint64_t)((ks * 32) >> 4);
+          umma(tmem, d_hi + koff, d_kq + koff, idesc_p, 1u);
+          umma(tmem, d_lo + koff, d_kq + koff, idesc_p, 1u);
+        }
+        umma_commit(&sm.mbar);
+      }
+      if (!mbar_wait(&sm.mbar, phase)) sm.timed_out = 1;
+      phase ^= 1;
+      tc_fence_after();
+      __syncthreads();
+      if (sm.timed_out) {
+        if (L.status && tid == 0) L.status[b] = LUMO_SEQ_TIMEOUT;
+        break;
+      }
+    }
     // ---- g. V rows -> shared (space of the dead S0 tiles); Gram rows out of tensor memory ----------
     {
       const __nv_bfloat16* vg = reinterpret_cast<const __nv_bfloat16*>(L.v);
@@ -539,16 +617,16 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
         const int pi = idx >> 4, c = idx & 15;
         if (pi < N) {
           const size_t pr = (size_t)b * s.Ns + (sm.meta[pi] & 0xFFFF);
-          cp_async16(sbase + kOffV + pi * 256 + c * 16, vg + (pr * s.Hv + hv) * kD + c * 8);
+          cp_async16(sbase + LY::kV + pi * 256 + c * 16, vg + (pr * s.Hv + hv) * kD + c * 8);
         }
       }
       asm volatile("cp.async.commit_group;\n" ::: "memory");
     }
     // both halves of the CTA read the Gram rows: 32 of the NT columns each (one half is enough for NT = 32)
-    if (grp * 32 < NT) tmem_cols32_to_smem(tmem_lane + 128 + grp * 32, dump + vrow * kDumpStride + grp * 32, 1);
+    if (grp * 32 < NT) tmem_cols32_to_smem(tmem_lane + LY::kGramCol + grp * 32, dump + vrow * LY::kStride + grp * 32, 1);
     __syncthreads();
     // ---- h. normalisation factors ------------------------------------------------------------------
-    if (tid < NT) sm.ks[tid] = s.l2norm ? rsqrtf(dump[tid * kDumpStride + tid] + s.l2_eps) : 1.f;
+    if (tid < NT) sm.ks[tid] = s.l2norm ? rsqrtf(dump[tid * LY::kStride + tid] + s.l2_eps) : 1.f;
     else if (tid < 2 * NT) sm.qs[tid - NT] = s.l2norm ? s.scale * rsqrtf(sm.qq[tid - NT] + s.l2_eps) : s.scale;
     __syncthreads();
     // ---- i. first half of the CTA: node records, one thread per (node, table); second half: the
@@ -562,14 +640,14 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       const int D = pi < N ? ((meta >> 16) & 0xFF) : 0;          // depth, 1..16
       const float a_t = sm.alpha[pi], b_t = sm.beta[pi];
       const float self = is_q ? sm.qs[pi] : -b_t * sm.ks[pi];    // factor of the node itself (k side negated)
-      const float* grow = dump + (is_q ? NT + pi : pi) * kDumpStride;
+      const float* grow = dump + (is_q ? NT + pi : pi) * LY::kStride;
       float G = a_t;
       float w[16];
       uint32_t ao[8];
 #pragma unroll
       for (int j = 15; j >= 0; --j) {                            // bounded: 16 depth slots
         float val = 0.f;
-        uint32_t off = kZeroRow;
+        uint32_t off = LY::kZero;
         if (j <= D - 2) {
           const int sidx = sm.anc[pi][j];
           val = self * G * sm.ks[sidx] * grow[sidx];
@@ -603,7 +681,7 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     __syncthreads();      // records, V and Pq are in place; the Gram dump is dead from here on
     // the S0 k^ products take the place of the dump; each delta later overwrites its own product
     if (grp * 32 < N) tmem_cols32_to_smem(tmem_lane + grp * 32, dls + (grp * 32) * kD + vrow, kD);
-    if (tid < kD) dls[kZeroRow + tid] = 0.f;
+    if (tid < kD) dls[LY::kZero + tid] = 0.f;
     __syncthreads();
     // ---- j. forward substitution, level by level; one warp per node, lane l carries value rows
     //         4l .. 4l+3.  A node's record, v and S0 products are loaded before the barrier that
@@ -687,13 +765,19 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
   }
 
   __syncthreads();
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(LY::kTmem) : "memory");
 }
 
 template <int NT>
 __global__ void __launch_bounds__(kThreads, 2)
 scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
   scan_gram_body<NT, false>(s, t, lb, n_items, nullptr);
+}
+
+// trees of at most 32 nodes, launches of several waves: three smaller CTAs per SM
+__global__ void __launch_bounds__(kThreads, 3)
+scan_gram_compact_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
+  scan_gram_body<32, false, true>(s, t, lb, n_items, nullptr);
 }
 
 template <int NT>
@@ -721,10 +805,17 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(scan_gram_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(scan_gram_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GL<true>::kBytes);
+    if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   // two CTAs per SM by construction: 102 KB of shared memory, 128 registers x 256 threads and 256
   // of the 512 tensor-memory columns each
+  // Compact CTAs (68 KB, 80 registers, 128 tensor-memory columns: three per SM) pay one more tensor-core
+  // round trip per item: they win when a launch has several waves of items (the 48-layer stack: 205 ->
+  // 190 us) and lose on a single wave (batch 1: 9.3 -> 10.5 us).
+  if (t.max_group_nodes <= 32 && items >= 4 * sm_count)
+    return launch_kernel(scan_gram_compact_kernel, dim3(3 * sm_count), dim3(kThreads), GL<true>::kBytes, st, pdl, s, t, lb, items);
   const int grid = items < 2 * sm_count ? items : 2 * sm_count;
   if (t.max_group_nodes <= 32)
     return launch_kernel(scan_gram_kernel<32>, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);

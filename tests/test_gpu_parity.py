@@ -473,6 +473,36 @@ def test_kernel_overlap_changes_nothing(name):
     assert not torch.equal(res[True][0][0], res[True][0][1])      # the cycles really advanced the state
 
 
+@pytest.mark.parametrize("name", ["cfg3_5layers", "paper_geometry_5layers"])
+def test_compact_three_cta_scan_matches_oracle(name):
+    """Launches with several waves of items over trees of at most 32 nodes take the compact variant of the
+    Gram scan (the state crosses shared memory in two 64-column halves, three CTAs per SM).  Every layer,
+    every output, element by element against the oracle; padded and permuted rows in the second case."""
+    c = W.config3(n_layers=5) if name == "cfg3_5layers" else W.config_paper(B=4, n_layers=5)
+    assert len(c.layers) * c.B * c.Hv >= 4 * 148          # enough items for the compact kernel to be chosen
+    dc = DeviceCase(ctx("gram"), c)
+    for l in range(len(c.layers)):
+        dc.t("out", l).fill_(float("nan"))
+    dc.verify()
+    torch.cuda.synchronize()
+    worst = 0.0
+    for l in range(len(c.layers)):
+        assert dc.np("status", l).tolist() == [0] * c.B
+        o_ref, _, _ = oracle_scan_from_device(dc, layer=l)
+        got = dc.np("out", l)
+        worst = max(worst, assert_close(got, o_ref, what=f"{name} layer {l}"))
+        for b in range(c.B):
+            pad = sorted(set(range(c.Ns)) - set(c.slot[b].tolist()))
+            assert np.all(got[b, pad] == 0.0)
+    assert worst < 1e-4
+    # same bits on a second run, and the sequential kernel agrees
+    first = [dc.t("out", l).clone() for l in range(len(c.layers))]
+    dc.verify()
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, dc.t("out", l)) for l, a in enumerate(first))
+    ctx("auto")
+
+
 def test_bounded_wait_runs_out_reports_timeout_and_leaves_the_context_usable():
     """The tensor-core scan waits for its tensor-core work on an mbarrier with a bounded number of polls.
     With the drill on, the kernel issues no tensor-core work (nothing asynchronous is in flight) and polls
