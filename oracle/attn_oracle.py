@@ -15,6 +15,8 @@ the recurrent path; Algorithm 1, "remap KV"):
     order is kept: q and out are indexed by logical node).
   * Node i sees every context position and the entries of its ancestors and of itself, nothing else
     (padding slots and other branches are invisible).  Query head h reads KV head h // (Hq / Hkv).
+  * The tree's own entries reach the cache through the same map: kv_write puts the key / value of node i
+    at position ctx_len[b] + slot[b][i] before attention runs.
   * logits = scale * q . k;  lse = log sum exp(logits);  out = sum softmax(logits) v.
     Keys are taken in logical order (context ascending, then the ancestry root first, the node last), so
     the result does not depend on the slot map bit for bit.
@@ -29,7 +31,8 @@ the number of split-K partitions are kernel schedule, not semantics (the oracle 
 Pins (tests/test_oracle_attn.py): a chain tree equals causal attention by
 torch.nn.functional.scaled_dot_product_attention; visibility by poisoning invisible entries; slot
 permutation invariance bit for bit; single-key and uniform-logit closed forms; the split merge identity;
-the grouped-head map; publication by hand-worked tables and by "attention over the published cache equals
+the grouped-head map; the write by a hand-worked table and by "write, attend, publish" against plain
+causal attention over the appended path; publication by hand-worked tables and by "attention over the published cache equals
 tree attention at the accepted node".
 """
 from __future__ import annotations
@@ -80,6 +83,19 @@ def tree_attention(parent, slot, q, k_cache, v_cache, ctx_len, cache_row, scale)
                 g = h // (Hq // Hkv)
                 out[b, i, h], lse[b, i, h] = attend(q[b, i, h], k_cache[row, pos, g], v_cache[row, pos, g], scale)
     return out, lse
+
+
+def kv_write(slot, k_new, v_new, k_cache, v_cache, ctx_len, cache_row):
+    """Places the tree's entries: k_new / v_new [B, N, Hkv, dh] (logical node order) go to position
+    ctx_len[b] + slot[b][i] of row cache_row[b].  Returns new caches; inputs untouched."""
+    k2, v2 = np.array(k_cache, copy=True), np.array(v_cache, copy=True)
+    B, N = np.asarray(slot).shape
+    for b in range(B):
+        for i in range(N):
+            p = int(ctx_len[b]) + int(slot[b][i])
+            k2[int(cache_row[b]), p] = k_new[b][i]
+            v2[int(cache_row[b]), p] = v_new[b][i]
+    return k2, v2
 
 
 def merge_partials(outs, lses):

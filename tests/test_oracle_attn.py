@@ -174,3 +174,38 @@ def test_attention_over_the_published_cache_equals_tree_attention_at_the_accepte
         for h in range(4):
             o, l = A.attend(c["q"][b, last, h], k2[row, :T, h // 2], v2[row, :T, h // 2], c["scale"])
             assert np.array_equal(o, out[b, last, h]) and l == lse[b, last, h]
+
+
+def test_write_attend_publish_equals_plain_causal_attention_over_the_appended_path():
+    """The three steps under one slot map: the tree's entries are written through the map, attention reads
+    them through it, publication moves the accepted ones; the result is what a sequential decoder that
+    appended the accepted tokens one by one would hold and compute (library attention, explicit lists)."""
+    rs = np.random.default_rng(11)
+    parent = np.array([[-1, 0, 0, 1, 1, 2, 4]], dtype=np.int32)
+    slot = np.array([[0, 4, 1, 6, 2, 5, 3]], dtype=np.int32)            # spine 0 -> 1 -> 4 -> 6 is NOT contiguous here
+    ctx, Hkv, Hq, dh, N = 6, 2, 4, 8, 7
+    k_cache, v_cache = rs.standard_normal((2, 16, Hkv, dh)), rs.standard_normal((2, 16, Hkv, dh))
+    k_new, v_new, q = rs.standard_normal((1, N, Hkv, dh)), rs.standard_normal((1, N, Hkv, dh)), rs.standard_normal((1, N, Hq, dh))
+    ctx_len, row = np.array([ctx]), np.array([1])
+    k1, v1 = A.kv_write(slot, k_new, v_new, k_cache, v_cache, ctx_len, row)
+    # hand table: position ctx + s holds node slot^-1(s)
+    inv = {int(s): i for i, s in enumerate(slot[0])}
+    for s_, i in inv.items():
+        assert np.array_equal(k1[1, ctx + s_], k_new[0, i]) and np.array_equal(v1[1, ctx + s_], v_new[0, i])
+    assert np.array_equal(k1[0], k_cache[0]) and np.array_equal(k1[1, :ctx], k_cache[1, :ctx]) and np.array_equal(k1[1, ctx + N:], k_cache[1, ctx + N:])
+    out, _ = A.tree_attention(parent, slot, q, k1, v1, ctx_len, row, 0.5)
+    path = [0, 1, 4, 6]
+    acc = np.array([path], dtype=np.int32)
+    k2, v2, ctx2, st = A.kv_publish(parent, slot, k1, v1, ctx_len, row, acc, np.array([4]))
+    assert st.tolist() == [0] and ctx2.tolist() == [ctx + 4]
+    # the sequential decoder's cache: old context followed by the accepted tokens' entries
+    Kseq = np.concatenate([k_cache[1, :ctx], k_new[0, path]], 0)
+    Vseq = np.concatenate([v_cache[1, :ctx], v_new[0, path]], 0)
+    assert np.array_equal(k2[1, :ctx + 4], Kseq) and np.array_equal(v2[1, :ctx + 4], Vseq)
+    for t, node in enumerate(path):
+        T = ctx + t + 1
+        qq = torch.from_numpy(q[0, node])[:, None, :]                                    # [Hq, 1, dh]
+        kk = torch.from_numpy(Kseq[:T]).permute(1, 0, 2).repeat_interleave(2, dim=0)
+        vv = torch.from_numpy(Vseq[:T]).permute(1, 0, 2).repeat_interleave(2, dim=0)
+        ref = torch.nn.functional.scaled_dot_product_attention(qq, kk, vv, scale=0.5)[:, 0]
+        np.testing.assert_allclose(out[0, node], ref.numpy(), rtol=1e-12, atol=1e-14)
