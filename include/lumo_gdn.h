@@ -62,7 +62,8 @@ typedef enum {
   LUMO_SEQ_BAD_ROOT = 3,  /* first accepted entry is not a child of the pre-tree state */
   LUMO_SEQ_BAD_LINK = 4,  /* accepted entry t is not a child of entry t-1 */
   LUMO_SEQ_BAD_ROW = 5,   /* state_row[b] >= n_state_rows */
-  LUMO_SEQ_TIMEOUT = 6    /* a bounded device-side wait ran out; outputs of the call are invalid */
+  LUMO_SEQ_TIMEOUT = 6,   /* a bounded device-side wait ran out; outputs of the call are invalid */
+  LUMO_SEQ_BAD_CTX = 7    /* attention calls: ctx_len[b] < 0 or ctx_len[b] + Ns > max_positions */
 } lumo_seq_status;
 
 /* Integer tables of one tree (lumo_tree_desc_get).  The paper's tree descriptor holds parent
@@ -96,7 +97,10 @@ typedef enum {
                                   group: n, n node ids ordered by (depth, index), n emit flags].  A group
                                   holds at most 64 nodes and every ancestor of each member; each node is
                                   emitted by exactly one group */
-  LUMO_TAB_COUNT = 18
+  LUMO_TAB_ATTN_VIS = 18,      /* [N, ceil(Ns/32)] attention visibility over the physical suffix: bit s of word s/32
+                                  of node i is set when slot s holds i or an ancestor of i (32-bit patterns stored
+                                  as int32); empty when Ns > 256, and then the attention calls are refused */
+  LUMO_TAB_COUNT = 19
 } lumo_table;
 
 /* ---- context ------------------------------------------------------------------------- */
@@ -145,7 +149,8 @@ int lumo_ctx_set_overlap(lumo_ctx* ctx, int on);
  * device time of kernels of `kind` (lumo_kernel_kind) and, with reset != 0, forgets all
  * records.  Enabling allocates the event pool; do not enable inside a stream capture. */
 typedef enum { LUMO_K_CONV = 0, LUMO_K_SCAN = 1, LUMO_K_COMMIT = 2, LUMO_K_PATH = 3,
-               LUMO_K_COUNT = 4 } lumo_kernel_kind;
+               LUMO_K_ATTN = 4, LUMO_K_ATTN_MERGE = 5, LUMO_K_KV_WRITE = 6, LUMO_K_KV_PUBLISH = 7,
+               LUMO_K_COUNT = 8 } lumo_kernel_kind;
 int lumo_ctx_timing_enable(lumo_ctx* ctx, int enable);
 int lumo_ctx_timing_read(lumo_ctx* ctx, int kind, int reset, int64_t* launches, double* total_ms);
 
@@ -327,6 +332,75 @@ int lumo_gdn_commit(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_ar
 int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const lumo_gdn_args* prev_layers,
                            const int32_t* accepted_dev, const int32_t* len_dev, int lmax,
                            const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers, void* stream);
+
+/* ---- attention half of the verifier ------------------------------------------------------
+ * The hybrid model's full-attention layers see the same tree through the same slot map (Sec. "One
+ * slot map governs attention and publication"; Sec. "State and the execution boundary": the
+ * attention visibility relation selects the same logical prefix and ancestry as the recurrent path;
+ * Algorithm 1, "Remap the accepted KV entries using the same logical-to-physical slot map").
+ *
+ * KV cache of one layer: k_cache, v_cache [n_cache_rows, max_positions, Hkv, dh] bf16.  Sequence b
+ * owns row cache_row[b]; positions [0, ctx_len[b]) hold the committed context, and the entry of tree
+ * node i lives at position ctx_len[b] + slot[b][i] (the candidates occupy the physical suffix in slot
+ * order; a spine-first slot map makes the principal chain contiguous there).  Queries and outputs
+ * keep LOGICAL node order.  Node i attends to every context position and to the entries of its
+ * ancestors and of itself; padding slots, other branches and anything beyond the suffix are never
+ * read arithmetically (their bytes may be anything, NaN patterns included).  Query head h reads KV
+ * head h / (Hq / Hkv).
+ *
+ * ctx_len and cache_row are DEVICE arrays [B] shared by all layers.  A sequence with
+ * cache_row[b] outside [0, n_cache_rows) gets LUMO_SEQ_BAD_ROW, one with ctx_len[b] < 0 or
+ * ctx_len[b] + Ns > max_positions LUMO_SEQ_BAD_CTX; such a sequence is skipped (write, publish) or
+ * gets zero outputs and lse (attention).  Supported: dh = 128, Ns <= 256, 1 <= Hq / Hkv, n_layers <= 32.
+ */
+typedef struct {
+  int32_t Hq, Hkv, dh;
+  float scale;              /* logits = scale * q . k (the paper prints none: a parameter) */
+  int32_t n_cache_rows, max_positions;
+  void* k_cache;            /* [n_cache_rows, max_positions, Hkv, dh] bf16 */
+  void* v_cache;
+  const int32_t* ctx_len;   /* [B] */
+  const int32_t* cache_row; /* [B] */
+  const void* q;            /* [B, N, Hq, dh] bf16, logical node order (tree attention) */
+  const void* k_new;        /* [B, N, Hkv, dh] bf16, logical node order (write) */
+  const void* v_new;
+  float* out;               /* [B, N, Hq, dh] fp32 (tree attention) */
+  float* lse;               /* [B, N, Hq] fp32 natural-log sum of exp of the logits; may be NULL */
+  int32_t n_splits;         /* partitions of the key range per (sequence, KV head): 0 = chosen to fill the GPU,
+                               else 1..32 (Sec. "Evaluation Setup": the paper's deployment used 4) */
+  int32_t* status;          /* [B] lumo_seq_status; may be NULL */
+} lumo_attn_args;
+
+/* Writes the tree's keys and values through the slot map: entry of node i of sequence b goes to
+ * position ctx_len[b] + slot[b][i] of row cache_row[b] (Sec. "One slot map governs attention and
+ * publication": the same permutation is applied to KV write slots and to the mask's key columns).
+ * A pure scatter, bit-exact.  `layers` is a HOST array; all layers share shapes, ctx_len and cache_row. */
+int lumo_kv_write_tree(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers,
+                       void* stream);
+
+/* Ancestry-masked decode attention of every tree node over [context ; tree entries]:
+ *   out[b,i,h,:] = sum_p softmax_p(scale q[b,i,h] . k[p]) v[p],  p over the visible positions,
+ * on tcgen05 tensor cores: the query rows of all heads that share a KV head form one 128-row tile
+ * (rows = (h mod G) * N + i, G = Hq / Hkv; further tiles when G N > 128), so a staged key/value tile
+ * is read once for the whole group (Sec. "One slot map governs attention and publication": grouped
+ * query heads share staged KV tiles); the key range of a sequence is cut into n_splits partitions
+ * handled by different CTAs, combined by the log-sum-exp rule (same section: split-K context
+ * partitions).  Probabilities enter the second product rounded to bf16; all sums are fp32.
+ * The result for a given n_splits is bitwise reproducible; different n_splits differ by rounding.
+ * Needs max_positions * Hkv * dh * 2 bytes < 2^40 per cache row.  Enqueues only; library scratch for
+ * the partial results grows on the first call with a shape. */
+int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers,
+                        void* stream);
+
+/* Publication of the accepted path in the KV cache (Algorithm 1, "remap KV"): for t < len[b] the entry
+ * at ctx_len[b] + slot[b][accepted[b][t]] moves to position ctx_len[b] + t, all reads before any write;
+ * entries already in place move no bytes (a spine-first slot map makes publication of the principal
+ * chain free).  ctx_len_out[b] = ctx_len[b] + len[b] (ctx_len_out may be NULL; it must not alias
+ * ctx_len).  Same path rules, lmax bound and status codes as lumo_gdn_commit; an invalid path leaves
+ * the row untouched and ctx_len_out[b] = ctx_len[b].  Bit-exact. */
+int lumo_kv_publish(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers,
+                    const int32_t* accepted_dev, const int32_t* len_dev, int lmax, int32_t* ctx_len_out,
+                    void* stream);
 
 #ifdef __cplusplus
 }

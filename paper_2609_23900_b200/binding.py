@@ -25,19 +25,20 @@ _lib = ctypes.CDLL(LIB_PATH)
 LUMO_F32, LUMO_BF16 = 0, 1
 _DTYPE = {torch.float32: LUMO_F32, torch.bfloat16: LUMO_BF16}
 
-SEQ_OK, SEQ_BAD_LEN, SEQ_BAD_NODE, SEQ_BAD_ROOT, SEQ_BAD_LINK, SEQ_BAD_ROW, SEQ_TIMEOUT = range(7)
+SEQ_OK, SEQ_BAD_LEN, SEQ_BAD_NODE, SEQ_BAD_ROOT, SEQ_BAD_LINK, SEQ_BAD_ROW, SEQ_TIMEOUT, SEQ_BAD_CTX = range(8)
 
 TABLES = ["depth", "n_child", "child_off", "child_list", "is_leaf", "leaves", "path_off", "path_nodes",
           "anc_win", "slot_inv", "chain_head", "chain_off", "chain_nodes", "chain_level", "cut_nodes",
-          "schedule", "schedule_full", "gram_groups"]
+          "schedule", "schedule_full", "gram_groups", "attn_vis"]
 
-KERNEL_KINDS = ["conv", "scan", "commit", "path"]
+KERNEL_KINDS = ["conv", "scan", "commit", "path", "attn", "attn_merge", "kv_write", "kv_publish"]
 
 EXPORTS = ["lumo_ctx_create", "lumo_ctx_destroy", "lumo_last_error", "lumo_ctx_scratch_bytes",
            "lumo_ctx_timing_enable", "lumo_ctx_timing_read", "lumo_ctx_set_scan_algo", "lumo_ctx_set_overlap", "lumo_ctx_set_timeout_drill",
            "lumo_tree_desc_create", "lumo_tree_desc_destroy", "lumo_tree_desc_get",
            "lumo_tree_path_from_node", "lumo_gdn_tree_verify", "lumo_gdn_commit",
-           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_conv_rows_per_cta", "lumo_tree_accept", "lumo_select_spine_top3", "lumo_gdn_commit_verify"]
+           "lumo_gdn_tree_scan_static", "lumo_static_stack_bytes", "lumo_conv_rows_per_cta", "lumo_tree_accept", "lumo_select_spine_top3", "lumo_gdn_commit_verify",
+           "lumo_kv_write_tree", "lumo_tree_attention", "lumo_kv_publish"]
 
 
 class LumoError(RuntimeError):
@@ -79,6 +80,17 @@ class _SelectArgs(ctypes.Structure):
                 ("logits", ctypes.c_void_p)]
 
 
+class _AttnArgs(ctypes.Structure):
+    """Mirror of lumo_attn_args."""
+    _fields_ = [("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("dh", ctypes.c_int32), ("scale", ctypes.c_float),
+                ("n_cache_rows", ctypes.c_int32), ("max_positions", ctypes.c_int32),
+                ("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
+                ("ctx_len", ctypes.c_void_p), ("cache_row", ctypes.c_void_p),
+                ("q", ctypes.c_void_p), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
+                ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p),
+                ("n_splits", ctypes.c_int32), ("status", ctypes.c_void_p)]
+
+
 _lib.lumo_ctx_create.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
 _lib.lumo_ctx_destroy.argtypes = [ctypes.c_void_p]
 _lib.lumo_ctx_destroy.restype = None
@@ -116,6 +128,12 @@ _lib.lumo_tree_accept.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINT
                                   ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
 _lib.lumo_gdn_commit.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_Args), ctypes.c_int,
                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p]
+
+
+_lib.lumo_kv_write_tree.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_AttnArgs), ctypes.c_int, ctypes.c_void_p]
+_lib.lumo_tree_attention.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_AttnArgs), ctypes.c_int, ctypes.c_void_p]
+_lib.lumo_kv_publish.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.POINTER(_AttnArgs), ctypes.c_int,
+                                 ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
@@ -254,6 +272,26 @@ class Context:
                                          int(accepted.shape[1]), _stream(stream)))
 
 
+    # ---- attention half ----
+    @staticmethod
+    def pack_attn(layers: Sequence["AttnLayer"]):
+        return (_AttnArgs * len(layers))(*[l.args for l in layers])
+
+    def kv_write_tree(self, desc: "TreeDesc", layers, stream=None):
+        arr = layers if isinstance(layers, ctypes.Array) else self.pack_attn(layers)
+        self._check(_lib.lumo_kv_write_tree(self._h, desc._h, arr, len(arr), _stream(stream)))
+
+    def tree_attention(self, desc: "TreeDesc", layers, stream=None):
+        arr = layers if isinstance(layers, ctypes.Array) else self.pack_attn(layers)
+        self._check(_lib.lumo_tree_attention(self._h, desc._h, arr, len(arr), _stream(stream)))
+
+    def kv_publish(self, desc: "TreeDesc", layers, accepted: torch.Tensor, length: torch.Tensor,
+                   ctx_len_out: Optional[torch.Tensor] = None, stream=None):
+        arr = layers if isinstance(layers, ctypes.Array) else self.pack_attn(layers)
+        self._check(_lib.lumo_kv_publish(self._h, desc._h, arr, len(arr), _ptr(accepted), _ptr(length),
+                                         int(accepted.shape[1]), _ptr(ctx_len_out), _stream(stream)))
+
+
 class TreeDesc:
     """lumo_tree_desc built from host arrays parent [B, N] (and optional slot, depth)."""
 
@@ -335,5 +373,37 @@ class GdnLayer:
         a.gate_mode = 0 if a_log is None else 1
         for name in ("q", "k", "v", "alpha", "beta", "x", "conv_w", "conv_b", "conv_hist", "state",
                      "state_row", "out", "snap_nodes", "snap_out", "status", "a_log", "dt_bias"):
+            setattr(a, name, _ptr(self.tensors[name]))
+        self.args = a
+
+
+class AttnLayer:
+    """lumo_attn_args for one full-attention layer; keeps the tensors alive."""
+
+    def __init__(self, *, Hq: int, Hkv: int, k_cache, v_cache, ctx_len, cache_row, scale: float, q=None, k_new=None,
+                 v_new=None, out=None, lse=None, n_splits: int = 0, status=None):
+        self.tensors = dict(k_cache=k_cache, v_cache=v_cache, ctx_len=ctx_len, cache_row=cache_row, q=q, k_new=k_new,
+                            v_new=v_new, out=out, lse=lse, status=status)
+        if k_cache.dtype != torch.bfloat16 or v_cache.dtype != torch.bfloat16 or k_cache.shape != v_cache.shape:
+            raise ValueError("k_cache and v_cache must be bfloat16 tensors of one shape [rows, positions, Hkv, dh]")
+        if k_cache.dim() != 4 or k_cache.shape[2] != Hkv:
+            raise ValueError("cache shape must be [rows, positions, Hkv, dh]")
+        for name in ("q", "k_new", "v_new"):
+            t = self.tensors[name]
+            if t is not None and t.dtype != torch.bfloat16:
+                raise ValueError(f"{name} must be bfloat16")
+        for name in ("out", "lse"):
+            t = self.tensors[name]
+            if t is not None and t.dtype != torch.float32:
+                raise ValueError(f"{name} must be float32")
+        for name in ("ctx_len", "cache_row", "status"):
+            t = self.tensors[name]
+            if t is not None and t.dtype != torch.int32:
+                raise ValueError(f"{name} must be int32")
+        a = _AttnArgs()
+        a.Hq, a.Hkv, a.dh, a.scale = int(Hq), int(Hkv), int(k_cache.shape[3]), float(scale)
+        a.n_cache_rows, a.max_positions = int(k_cache.shape[0]), int(k_cache.shape[1])
+        a.n_splits = int(n_splits)
+        for name in self.tensors:
             setattr(a, name, _ptr(self.tensors[name]))
         self.args = a

@@ -171,6 +171,7 @@ void lumo_ctx_destroy(lumo_ctx* ctx) {
   if (ctx->device >= 0) {
     DeviceGuard g(ctx->device);
     if (ctx->scratch) cudaFree(ctx->scratch);
+    if (ctx->attn_scratch) cudaFree(ctx->attn_scratch);
     for (cudaEvent_t e : ctx->ev_start) cudaEventDestroy(e);
     for (cudaEvent_t e : ctx->ev_stop) cudaEventDestroy(e);
   }
@@ -179,7 +180,9 @@ void lumo_ctx_destroy(lumo_ctx* ctx) {
 
 const char* lumo_last_error(const lumo_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_err.c_str(); }
 
-int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx) { return ctx ? (int64_t)ctx->scratch_bytes : 0; }
+int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx) {
+  return ctx ? (int64_t)(ctx->scratch_bytes + ctx->attn_scratch_bytes) : 0;
+}
 
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo) {
   if (!ctx) return LUMO_ERR_ARG;
@@ -298,9 +301,20 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   const size_t G = (size_t)d->n_groups;
   const size_t o_tc_group = tc ? reserve(G * 4) : 0, o_tc_meta = tc ? reserve(G * 64) : 0;
   const size_t o_tc_anc = tc ? reserve(G * 64 * 4) : 0, o_tc_lvl = tc ? reserve(G * 5) : 0;
+  const bool attn = Ns <= kMaxAttnSlots;
+  const size_t o_vis = attn ? reserve((size_t)B * N * 8) : 0, o_used = attn ? reserve((size_t)B * 8) : 0;
   size_t gi = 0;
   for (int b = 0; b < B; ++b) {
     const HostTree& t = d->trees[b];
+    if (attn) {
+      const int W = (Ns + 31) / 32;
+      for (int i = 0; i < N; ++i)
+        for (int w = 0; w < W; ++w) {
+          const int32_t m = t.tab[LUMO_TAB_ATTN_VIS][(size_t)i * W + w];
+          h[o_vis + ((size_t)b * N + i) * 8 + w] = m;
+          h[o_used + (size_t)b * 8 + w] |= m;       // every node sees its own slot
+        }
+    }
     for (int i = 0; i < N; ++i) {
       h[o_parent + (size_t)b * N + i] = parent[(size_t)b * N + i];
       h[o_depth + (size_t)b * N + i] = t.tab[LUMO_TAB_DEPTH][i];
@@ -397,6 +411,10 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
     d->d_tc_meta = d->dev + o_tc_meta;
     d->d_tc_anc = reinterpret_cast<uint8_t*>(d->dev + o_tc_anc);
     d->d_tc_lvl = reinterpret_cast<uint8_t*>(d->dev + o_tc_lvl);
+  }
+  if (attn) {
+    d->d_vis = reinterpret_cast<uint32_t*>(d->dev + o_vis);
+    d->d_slot_used = reinterpret_cast<uint32_t*>(d->dev + o_used);
   }
   *out = d;
   return LUMO_OK;
@@ -664,6 +682,148 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
                                : launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st);
   });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "fused scan launch");
+}
+
+// ---- attention half ---------------------------------------------------------------------
+namespace {
+
+// Common checks of the three attention-side calls; fills the shape shared by all layers.
+int prepare_attn(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers, AttnShape* s) {
+  if (!ctx || !desc || !layers) return fail(ctx, LUMO_ERR_ARG, "null ctx, desc or layers");
+  if (desc->ctx != ctx) return fail(ctx, LUMO_ERR_ARG, "descriptor belongs to another context");
+  if (ctx->device < 0) return fail(ctx, LUMO_ERR_UNSUPPORTED, "host-only context cannot launch");
+  if (n_layers < 1 || n_layers > kMaxAttnLayers)
+    return fail(ctx, LUMO_ERR_ARG, "n_layers must be in [1, " + std::to_string(kMaxAttnLayers) + "]");
+  if (!desc->d_vis) return fail(ctx, LUMO_ERR_UNSUPPORTED, "the attention calls take at most 256 physical slots");
+  const lumo_attn_args& a0 = layers[0];
+  if (a0.dh != 128) return fail(ctx, LUMO_ERR_UNSUPPORTED, "dh must be 128");
+  if (a0.Hq < 1 || a0.Hkv < 1 || a0.Hq % a0.Hkv != 0) return fail(ctx, LUMO_ERR_UNSUPPORTED, "Hq must be a positive multiple of Hkv");
+  if (a0.Hkv > 32767) return fail(ctx, LUMO_ERR_UNSUPPORTED, "at most 32767 KV heads");
+  if (!(a0.scale > 0.f)) return fail(ctx, LUMO_ERR_ARG, "scale must be positive");
+  if (a0.n_cache_rows < 1 || a0.max_positions < desc->Ns)
+    return fail(ctx, LUMO_ERR_ARG, "need n_cache_rows >= 1 and max_positions >= n_slots");
+  if ((long long)a0.max_positions * a0.Hkv * a0.dh * 2 >= (1LL << 40))
+    return fail(ctx, LUMO_ERR_UNSUPPORTED, "a cache row must span less than 2^40 bytes");
+  if (!a0.ctx_len || !a0.cache_row) return fail(ctx, LUMO_ERR_ARG, "ctx_len and cache_row are required");
+  if (a0.n_splits < 0 || a0.n_splits > 32) return fail(ctx, LUMO_ERR_ARG, "n_splits must be 0 (automatic) or in [1, 32]");
+  for (int l = 0; l < n_layers; ++l) {
+    const lumo_attn_args& a = layers[l];
+    const std::string at = " (layer " + std::to_string(l) + ")";
+    if (a.Hq != a0.Hq || a.Hkv != a0.Hkv || a.dh != a0.dh || a.scale != a0.scale || a.n_cache_rows != a0.n_cache_rows ||
+        a.max_positions != a0.max_positions || a.ctx_len != a0.ctx_len || a.cache_row != a0.cache_row ||
+        a.n_splits != a0.n_splits)
+      return fail(ctx, LUMO_ERR_ARG, "all layers must share shapes, options, ctx_len and cache_row" + at);
+    if (!a.k_cache || !a.v_cache) return fail(ctx, LUMO_ERR_ARG, "k_cache and v_cache are required" + at);
+    for (const void* p : {(const void*)a.k_cache, (const void*)a.v_cache, a.q, a.k_new, a.v_new, (const void*)a.out})
+      if (p && !aligned16(p)) return fail(ctx, LUMO_ERR_ARG, "tensor pointers must be 16-byte aligned" + at);
+  }
+  s->B = desc->B; s->N = desc->N; s->Ns = desc->Ns; s->Hq = a0.Hq; s->Hkv = a0.Hkv;
+  s->n_rows = a0.n_cache_rows; s->max_pos = a0.max_positions; s->scale = a0.scale;
+  s->ctx_len = a0.ctx_len; s->cache_row = a0.cache_row;
+  const int ctas = desc->B * a0.Hkv * attn_row_tiles(a0.Hq / a0.Hkv, desc->N);
+  s->S = a0.n_splits ? a0.n_splits : std::min(32, std::max(1, (2 * ctx->sm_count + ctas - 1) / ctas));
+  return LUMO_OK;
+}
+
+void kv_views(const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers, const AttnShape& s, KvLayers* L, KvShape* k) {
+  std::memset(L, 0, sizeof(*L));
+  for (int l = 0; l < n_layers; ++l) {
+    L->k[l] = layers[l].k_cache; L->v[l] = layers[l].v_cache;
+    L->kn[l] = layers[l].k_new; L->vn[l] = layers[l].v_new;
+    L->status[l] = layers[l].status;
+  }
+  k->B = s.B; k->N = s.N; k->Ns = s.Ns; k->Hkv = s.Hkv; k->n_rows = s.n_rows; k->max_pos = s.max_pos;
+  k->ctx_len = s.ctx_len; k->cache_row = s.cache_row; k->parent = desc->d_parent; k->slot = desc->d_slot;
+}
+
+}  // namespace
+
+int lumo_kv_write_tree(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers, void* stream) {
+  AttnShape s;
+  int rc = prepare_attn(ctx, desc, layers, n_layers, &s);
+  if (rc != LUMO_OK) return rc;
+  for (int l = 0; l < n_layers; ++l)
+    if (!layers[l].k_new || !layers[l].v_new) return fail(ctx, LUMO_ERR_ARG, "k_new and v_new are required");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  KvLayers L;
+  KvShape k;
+  kv_views(desc, layers, n_layers, s, &L, &k);
+  cudaError_t e = cudaSuccess;
+  for (int l = 0; l < n_layers && e == cudaSuccess; ++l)
+    if (layers[l].status) e = cudaMemsetAsync(layers[l].status, 0, (size_t)s.B * sizeof(int32_t), st);
+  if (e == cudaSuccess) e = timed(ctx, LUMO_K_KV_WRITE, st, [&] { return launch_kv_write(L, k, n_layers, st); });
+  ctx->last_call = lumo_ctx::kOther;
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "kv write launch");
+}
+
+int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers, void* stream) {
+  AttnShape s;
+  int rc = prepare_attn(ctx, desc, layers, n_layers, &s);
+  if (rc != LUMO_OK) return rc;
+  for (int l = 0; l < n_layers; ++l)
+    if (!layers[l].q || !layers[l].out) return fail(ctx, LUMO_ERR_ARG, "q and out are required");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t need = attn_scratch_bytes(s);
+  if (need > ctx->attn_scratch_bytes) {
+    // first call with this shape: grow the scratch (synchronises; later calls allocate nothing)
+    cudaError_t e = cudaSuccess;
+    if (ctx->attn_scratch) {
+      e = cudaDeviceSynchronize();
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaDeviceSynchronize");
+      cudaFree(ctx->attn_scratch);
+      ctx->attn_scratch = nullptr;
+      ctx->attn_scratch_bytes = 0;
+    }
+    e = cudaMalloc(&ctx->attn_scratch, need);
+    if (e != cudaSuccess) return fail(ctx, LUMO_ERR_NOMEM, std::string("scratch allocation failed: ") + cudaGetErrorString(e));
+    ctx->attn_scratch_bytes = need;
+  }
+  ctx->last_call = lumo_ctx::kOther;
+  // the layers of a model are not adjacent in time: one launch (and one pair of tensor maps) per layer;
+  // they share the scratch, which stream order makes safe
+  for (int l = 0; l < n_layers; ++l) {
+    AttnLayerPtrs p;
+    p.k_cache = layers[l].k_cache; p.v_cache = layers[l].v_cache; p.q = layers[l].q;
+    p.out = layers[l].out; p.lse = layers[l].lse; p.status = layers[l].status;
+    AttnPlan plan;
+    std::string err;
+    cudaError_t e = attn_plan(s, p, desc->d_vis, desc->d_slot_used, reinterpret_cast<float*>(ctx->attn_scratch), &plan, &err);
+    if (e != cudaSuccess) return err.empty() ? cuda_fail(ctx, e, "attention set-up") : fail(ctx, LUMO_ERR_CUDA, err);
+    if (p.status) {   // the kernels write failures only
+      e = cudaMemsetAsync(p.status, 0, (size_t)s.B * sizeof(int32_t), st);
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemsetAsync(status)");
+    }
+    e = timed(ctx, LUMO_K_ATTN, st, [&] { return launch_attn(plan, st); });
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
+    if (s.S > 1) {
+      e = timed(ctx, LUMO_K_ATTN_MERGE, st, [&] { return launch_attn_merge(plan, st); });
+      if (e != cudaSuccess) return cuda_fail(ctx, e, "attention merge launch");
+    }
+  }
+  return LUMO_OK;
+}
+
+int lumo_kv_publish(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers,
+                    const int32_t* accepted_dev, const int32_t* len_dev, int lmax, int32_t* ctx_len_out, void* stream) {
+  if (ctx && (lmax < 1 || lmax > kMaxNodes))
+    return fail(ctx, LUMO_ERR_ARG, "lmax must be in [1, " + std::to_string(kMaxNodes) + "] (a path holds each node at most once)");
+  AttnShape s;
+  int rc = prepare_attn(ctx, desc, layers, n_layers, &s);
+  if (rc != LUMO_OK) return rc;
+  if (!accepted_dev || !len_dev) return fail(ctx, LUMO_ERR_ARG, "accepted_dev and len_dev are required");
+  if (ctx_len_out == s.ctx_len) return fail(ctx, LUMO_ERR_ARG, "ctx_len_out must not alias ctx_len");
+  DeviceGuard g(ctx->device);
+  cudaStream_t st = (cudaStream_t)stream;
+  KvLayers L;
+  KvShape k;
+  kv_views(desc, layers, n_layers, s, &L, &k);
+  cudaError_t e = timed(ctx, LUMO_K_KV_PUBLISH, st, [&] {
+    return launch_kv_publish(L, k, n_layers, accepted_dev, len_dev, lmax, ctx_len_out, st);
+  });
+  ctx->last_call = lumo_ctx::kOther;
+  return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "kv publish launch");
 }
 
 }  // extern "C"

@@ -1,5 +1,6 @@
 // Internal declarations shared by the host side and the kernels of liblumo_gdn.
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <cstdint>
 #include <string>
@@ -12,6 +13,8 @@ namespace lumo {
 constexpr int kMaxNodes = 256;
 constexpr int kMaxSlots = 1024;
 constexpr int kMaxLayers = 64;
+constexpr int kMaxAttnSlots = 256;                 // physical suffix the attention kernels take (8 mask words per node)
+constexpr int kMaxAttnLayers = 32;
 constexpr int kMaxDevices = 64;                    // per-device caches (kernel attributes, symbol addresses)
 constexpr size_t kStaticStackBytes = 64u << 20;   // capacity of the built-in scan stack
 
@@ -46,6 +49,8 @@ struct lumo_ctx {
   std::string err;
   void* scratch = nullptr;      // scan stack levels
   size_t scratch_bytes = 0;
+  void* attn_scratch = nullptr; // partial results of the attention partitions
+  size_t attn_scratch_bytes = 0;
   // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
   int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form with forward substitution, 3 solved Gram form
   bool timeout_drill = false;   // test aid: the tensor-core scan skips its tensor-core work (lumo_ctx_set_timeout_drill)
@@ -89,6 +94,8 @@ struct lumo_tree_desc {
   int32_t* d_tc_meta = nullptr;   // [G, 64] physical row | depth << 16 | emit << 24 of the node at position pi
   uint8_t* d_tc_anc = nullptr;    // [G, 64, 16] positions of the ancestors, root first, then the node's own position
   uint8_t* d_tc_lvl = nullptr;    // [G, 20] lvl[d] = number of group nodes of depth <= d (lvl[0] = 0)
+  uint32_t* d_vis = nullptr;      // [B, N, 8] attention visibility over physical slots (present when Ns <= 256)
+  uint32_t* d_slot_used = nullptr;// [B, 8] slots that hold a node
 };
 
 namespace lumo {
@@ -285,5 +292,52 @@ cudaError_t launch_commit(const Shape& s, const TreeDev& t, const LayerBatch& lb
                           const int32_t* len, int lmax, bool with_state, bool with_hist, bool pdl, cudaStream_t st);
 cudaError_t launch_path_from_node(const TreeDev& t, int B, int N, const int32_t* node, int lmax,
                                   int32_t* accepted, int32_t* len, int32_t* status, cudaStream_t st);
+
+// ---- attention half (attn.cu) ------------------------------------------------------------
+struct AttnShape {
+  int B, N, Ns, Hq, Hkv, S, n_rows, max_pos;
+  float scale;
+  const int32_t* ctx_len; const int32_t* cache_row;
+};
+struct AttnLayerPtrs {
+  void* k_cache; void* v_cache; const void* q; float* out; float* lse; int32_t* status;
+};
+struct AttnArgs {
+  const void* q;
+  float* out; float* lse;
+  float* part_o; float* part_lse;
+  const int32_t* ctx_len; const int32_t* cache_row;
+  const uint32_t* vis; const uint32_t* used;
+  int32_t* status;
+  int B, N, Ns, Hq, Hkv, G, RT, S, n_rows, max_pos;
+  float scale_log2;
+};
+// one attention launch: the tensor maps of the layer's two caches, the kernel arguments and the grid
+struct AttnPlan {
+  CUtensorMap tk, tv;
+  AttnArgs a;
+  dim3 grid;
+};
+struct KvLayers {
+  void* k[kMaxAttnLayers]; void* v[kMaxAttnLayers];
+  const void* kn[kMaxAttnLayers]; const void* vn[kMaxAttnLayers];
+  int32_t* status[kMaxAttnLayers];
+};
+struct KvShape {
+  int B, N, Ns, Hkv, n_rows, max_pos;
+  const int32_t* ctx_len; const int32_t* cache_row;
+  const int32_t* parent; const int32_t* slot;
+};
+
+int attn_row_tiles(int G, int N);
+// scratch for the partitions' partial results (0 with a single partition)
+size_t attn_scratch_bytes(const AttnShape& s);
+cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t* vis, const uint32_t* used, float* scratch,
+                      AttnPlan* plan, std::string* err);
+cudaError_t launch_attn(const AttnPlan& plan, cudaStream_t st);
+cudaError_t launch_attn_merge(const AttnPlan& plan, cudaStream_t st);
+cudaError_t launch_kv_write(const KvLayers& L, const KvShape& s, int n_layers, cudaStream_t st);
+cudaError_t launch_kv_publish(const KvLayers& L, const KvShape& s, int n_layers, const int32_t* accepted, const int32_t* len,
+                              int lmax, int32_t* ctx_len_out, cudaStream_t st);
 
 }  // namespace lumo

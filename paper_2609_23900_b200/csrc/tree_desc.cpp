@@ -127,6 +127,19 @@ bool build_tree(const int32_t* parent, const int32_t* slot, int N, int Ns, HostT
     slot_inv[s] = i;
   }
 
+  // attention visibility over the physical suffix: a node sees its own slot and what its parent sees
+  if (Ns <= kMaxAttnSlots) {
+    auto& vis = t->tab[LUMO_TAB_ATTN_VIS];
+    const int W = (Ns + 31) / 32;
+    vis.assign((size_t)N * W, 0);
+    for (int i = 0; i < N; ++i) {
+      if (parent[i] >= 0)
+        for (int w = 0; w < W; ++w) vis[(size_t)i * W + w] = vis[(size_t)parent[i] * W + w];
+      const int s = slot ? slot[i] : i;
+      vis[(size_t)i * W + (s >> 5)] = (int32_t)((uint32_t)vis[(size_t)i * W + (s >> 5)] | (1u << (s & 31)));
+    }
+  }
+
   // chain decomposition: principal child = lowest index
   auto& c_head = t->tab[LUMO_TAB_CHAIN_HEAD];
   auto& c_off = t->tab[LUMO_TAB_CHAIN_OFF];

@@ -83,3 +83,47 @@ class DeviceCase:
         if t.dtype in (torch.float32, torch.bfloat16):
             return t.to(torch.float64).cpu().numpy()
         return t.cpu().numpy()
+
+
+class DeviceAttnCase:
+    """Device-side holder of one ``workload.AttnCase`` (one or more identical-shape layers that share the
+    inputs of layer 0 unless ``cases`` lists one case per layer).  Marshalling only."""
+
+    def __init__(self, ctx: binding.Context, case, *, n_splits: int = 0, cases=None, with_lse: bool = True,
+                 device: Optional[torch.device] = None):
+        self.ctx, self.case = ctx, case
+        self.cases = list(cases) if cases is not None else [case]
+        dev = device or torch.device("cuda", ctx.device)
+        self.dev = dev
+        self.desc = ctx.tree_desc(case.parent, slot=case.slot, n_slots=case.Ns)
+        up16 = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).to(dev)
+        self.ctx_len = torch.from_numpy(case.ctx_len.copy()).to(dev)
+        self.ctx_len_out = torch.full_like(self.ctx_len, -1)
+        self.cache_row = torch.from_numpy(case.cache_row.copy()).to(dev)
+        self.accepted = torch.from_numpy(case.accepted.copy()).to(dev)
+        self.accepted_len = torch.from_numpy(case.accepted_len.copy()).to(dev)
+        self.layers: List[binding.AttnLayer] = []
+        for c in self.cases:
+            self.layers.append(binding.AttnLayer(
+                Hq=c.Hq, Hkv=c.Hkv, k_cache=up16(c.k_cache), v_cache=up16(c.v_cache), ctx_len=self.ctx_len,
+                cache_row=self.cache_row, scale=c.scale, q=up16(c.q), k_new=up16(c.k_new), v_new=up16(c.v_new),
+                out=torch.full((c.B, c.N, c.Hq, c.dh), float("nan"), dtype=torch.float32, device=dev),
+                lse=torch.full((c.B, c.N, c.Hq), float("nan"), dtype=torch.float32, device=dev) if with_lse else None,
+                n_splits=n_splits, status=torch.full((c.B,), -1, dtype=torch.int32, device=dev)))
+        self.packed = ctx.pack_attn(self.layers)
+
+    def t(self, name: str, layer: int = 0):
+        return self.layers[layer].tensors[name]
+
+    def np(self, name: str, layer: int = 0) -> np.ndarray:
+        t = self.t(name, layer)
+        return t.to(torch.float64).cpu().numpy() if t.is_floating_point() else t.cpu().numpy()
+
+    def write(self, stream=None):
+        self.ctx.kv_write_tree(self.desc, self.packed, stream)
+
+    def attend(self, stream=None):
+        self.ctx.tree_attention(self.desc, self.packed, stream)
+
+    def publish(self, stream=None):
+        self.ctx.kv_publish(self.desc, self.packed, self.accepted, self.accepted_len, self.ctx_len_out, stream)

@@ -414,3 +414,99 @@ def config_paper(seed: int = BASE_SEED + 5, B: int = 1, n_layers: int = 1) -> Ca
     """The paper's evaluated geometry: 28 active rows padded to 32, slots permuted."""
     return make_case("cfgP_28of32", [tree_paper_geometry() for _ in range(B)], seed=seed, Hk=16,
                      Hv=32, d=128, in_dtype="bf16", n_layers=n_layers, Ns=32, permute_slots=True)
+
+
+# ---------------------------------------------------------------------------
+# attention half: KV cache, tree queries and entries
+# ---------------------------------------------------------------------------
+def spine_first_slots(parent: Sequence[int]) -> List[int]:
+    """Slot map that places the principal spine (from the first child of the pre-tree state, always the
+    lowest-index child) in slots 0, 1, ... and the remaining nodes after it in logical order (the layout
+    of Sec. "One slot map governs attention and publication")."""
+    ch = _children(parent)
+    spine, cur = [], -1
+    while ch[cur]:
+        cur = ch[cur][0]
+        spine.append(cur)
+    on = set(spine)
+    order = spine + [i for i in range(len(parent)) if i not in on]
+    slot = [0] * len(parent)
+    for s, i in enumerate(order):
+        slot[i] = s
+    return slot
+
+
+@dataclasses.dataclass
+class AttnCase:
+    """Inputs of one full-attention layer; float arrays are float32 holding bf16 values exactly."""
+    name: str
+    B: int
+    N: int
+    Ns: int
+    Hq: int
+    Hkv: int
+    dh: int
+    scale: float
+    parent: np.ndarray      # int32 [B, N]
+    slot: np.ndarray        # int32 [B, N]
+    ctx_len: np.ndarray     # int32 [B]
+    cache_row: np.ndarray   # int32 [B]
+    q: np.ndarray           # [B, N, Hq, dh]
+    k_new: np.ndarray       # [B, N, Hkv, dh]
+    v_new: np.ndarray
+    k_cache: np.ndarray     # [rows, S, Hkv, dh]; the suffix holds unrelated values until the tree is written
+    v_cache: np.ndarray
+    accepted: np.ndarray    # int32 [B, lmax], -1 padded
+    accepted_len: np.ndarray
+    lmax: int
+
+
+def make_attn_case(name: str, parents: Sequence[Sequence[int]], ctx_len: Sequence[int], *, seed: int, Hq: int, Hkv: int,
+                   dh: int = 128, Ns: Optional[int] = None, layout: str = "identity", max_positions: Optional[int] = None,
+                   extra_rows: int = 1, layer: int = 0) -> AttnCase:
+    """layout: "identity", "spine" (spine_first_slots) or "permuted" (seeded injective map into Ns slots).
+    q, k, v ~ N(0, 1); scale = dh^-1/2, so logits are ~N(0, 1) like trained attention at moderate temperature."""
+    B, N = len(parents), len(parents[0])
+    Ns = N if Ns is None else Ns
+    parent = np.asarray(parents, dtype=np.int32).reshape(B, N)
+    slot = np.tile(np.arange(N, dtype=np.int32), (B, 1))
+    for b in range(B):
+        if layout == "spine":
+            slot[b] = np.asarray(spine_first_slots(parents[b]), dtype=np.int32)
+        elif layout == "permuted":
+            rs = IntStream(stream_key(seed, _T["slot"], b, 77))
+            perm = list(range(Ns))
+            for i in range(Ns - 1, 0, -1):
+                j = rs.randint(0, i)
+                perm[i], perm[j] = perm[j], perm[i]
+            slot[b] = np.asarray(perm[:N], dtype=np.int32)
+        elif layout != "identity":
+            raise ValueError(layout)
+    ctx = np.asarray(ctx_len, dtype=np.int32).reshape(B)
+    S = int(ctx.max()) + Ns if max_positions is None else int(max_positions)
+    rows = B + extra_rows
+    rows_perm = list(range(rows))
+    rs = IntStream(stream_key(seed, _T["rows"], 77))
+    for i in range(rows - 1, 0, -1):
+        j = rs.randint(0, i)
+        rows_perm[i], rows_perm[j] = rows_perm[j], rows_perm[i]
+    cache_row = np.asarray(rows_perm[:B], dtype=np.int32)
+
+    def draw(tid: int, shape) -> np.ndarray:
+        n = int(np.prod(shape))
+        return round_to(normals(stream_key(seed, tid, layer, 77), n).reshape(shape), "bf16")
+
+    q = draw(_T["q"], (B, N, Hq, dh))
+    k_new = draw(_T["k"], (B, N, Hkv, dh))
+    v_new = draw(_T["v"], (B, N, Hkv, dh))
+    k_cache = draw(_T["state"], (rows, S, Hkv, dh))
+    v_cache = draw(_T["hist"], (rows, S, Hkv, dh))
+    acc_lists = [draw_accepted(IntStream(stream_key(seed, _T["accept"], b, 77)), parents[b]) for b in range(B)]
+    lmax = max(max(tree_depths(p)) for p in parents)
+    acc = np.full((B, lmax), -1, dtype=np.int32)
+    ln = np.zeros(B, dtype=np.int32)
+    for b, a in enumerate(acc_lists):
+        acc[b, :len(a)] = a
+        ln[b] = len(a)
+    return AttnCase(name, B, N, Ns, Hq, Hkv, dh, float(dh) ** -0.5, parent, slot, ctx, cache_row, q, k_new, v_new,
+                    k_cache, v_cache, acc, ln, lmax)

@@ -169,3 +169,32 @@ def test_error_codes_and_no_cpu_fallback():
     if not torch.cuda.is_available():
         with pytest.raises(binding.LumoError):
             binding.Context(0)
+
+
+def test_attention_visibility_table_matches_the_oracle_bit_for_bit():
+    """The mask rows the attention kernel reads (bit s of node i = slot s holds i or an ancestor) against
+    the oracle's visible positions, on permuted slot maps with padding."""
+    from oracle import attn_oracle as A
+    ctx = binding.Context(-1)
+    for seed, N, Ns in ((1, 7, 7), (2, 28, 32), (3, 100, 131), (4, 256, 256)):
+        parents = [W.tree_random(W.IntStream(W.stream_key(seed, b)), N, 9) for b in range(2)]
+        c = W.make_attn_case("vis", parents, [0, 0], seed=seed, Hq=1, Hkv=1, dh=8, Ns=Ns, layout="permuted")
+        desc = ctx.tree_desc(c.parent, slot=c.slot, n_slots=Ns)
+        Wd = (Ns + 31) // 32
+        for b in range(2):
+            tab = desc.table("attn_vis", b).view(np.uint32).reshape(N, Wd)
+            for i in range(N):
+                want = np.zeros(Wd, dtype=np.uint32)
+                for p in A.visible_positions(c.parent[b], c.slot[b], 0, i):
+                    want[p >> 5] |= np.uint32(1 << (p & 31))
+                assert np.array_equal(tab[i], want), (seed, b, i)
+    wide = ctx.tree_desc(np.array([[-1, 0]], dtype=np.int32), n_slots=300)
+    assert wide.table("attn_vis").size == 0          # beyond 256 slots the attention calls are refused
+
+
+def test_spine_first_slot_map_is_contiguous_on_the_principal_chain():
+    p = W.tree_paper_geometry()
+    s = W.spine_first_slots(p)
+    assert sorted(s) == list(range(len(p)))
+    spine = [0, 1, 4, 7, 10, 13, 16, 17, 18, 19, 20, 21]
+    assert [s[i] for i in spine] == list(range(12))
