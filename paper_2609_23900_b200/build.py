@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblumo_gdn.so")
-SOURCES = ["api.cu", "kernels.cu", "scan_gram.cu", "scan_solve.cu", "attn.cu", "accept.cu", "select.cu", "tree_desc.cpp"]
+SOURCES = ["api.cu", "kernels.cu", "scan_gram.cu", "scan_solve.cu", "attn.cu", "kv_cache.cu", "accept.cu", "select.cu", "tree_desc.cpp"]
 HEADERS = [os.path.join(CSRC, "internal.h"), os.path.join(ROOT, "include", "lumo_gdn.h")]
 
 NVCC_FLAGS = [

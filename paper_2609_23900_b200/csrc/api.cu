@@ -720,8 +720,7 @@ int prepare_attn(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args
   s->B = desc->B; s->N = desc->N; s->Ns = desc->Ns; s->Hq = a0.Hq; s->Hkv = a0.Hkv;
   s->n_rows = a0.n_cache_rows; s->max_pos = a0.max_positions; s->scale = a0.scale;
   s->ctx_len = a0.ctx_len; s->cache_row = a0.cache_row;
-  const int ctas = desc->B * a0.Hkv * attn_row_tiles(a0.Hq / a0.Hkv, desc->N);
-  s->S = a0.n_splits ? a0.n_splits : std::min(32, std::max(1, (2 * ctx->sm_count + ctas - 1) / ctas));
+  s->S = a0.n_splits;
   return LUMO_OK;
 }
 
@@ -765,7 +764,7 @@ int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_at
     if (!layers[l].q || !layers[l].out) return fail(ctx, LUMO_ERR_ARG, "q and out are required");
   DeviceGuard g(ctx->device);
   cudaStream_t st = (cudaStream_t)stream;
-  const size_t need = attn_scratch_bytes(s);
+  const size_t need = attn_scratch_bytes(s, ctx->sm_count);
   if (need > ctx->attn_scratch_bytes) {
     // first call with this shape: grow the scratch (synchronises; later calls allocate nothing)
     cudaError_t e = cudaSuccess;
@@ -789,7 +788,8 @@ int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_at
     p.out = layers[l].out; p.lse = layers[l].lse; p.status = layers[l].status;
     AttnPlan plan;
     std::string err;
-    cudaError_t e = attn_plan(s, p, desc->d_vis, desc->d_slot_used, reinterpret_cast<float*>(ctx->attn_scratch), &plan, &err);
+    cudaError_t e = attn_plan(s, p, desc->d_vis, desc->d_slot_used, reinterpret_cast<float*>(ctx->attn_scratch),
+                              ctx->sm_count, &plan, &err);
     if (e != cudaSuccess) return err.empty() ? cuda_fail(ctx, e, "attention set-up") : fail(ctx, LUMO_ERR_CUDA, err);
     if (p.status) {   // the kernels write failures only
       e = cudaMemsetAsync(p.status, 0, (size_t)s.B * sizeof(int32_t), st);
@@ -797,10 +797,8 @@ int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_at
     }
     e = timed(ctx, LUMO_K_ATTN, st, [&] { return launch_attn(plan, st); });
     if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
-    if (s.S > 1) {
-      e = timed(ctx, LUMO_K_ATTN_MERGE, st, [&] { return launch_attn_merge(plan, st); });
-      if (e != cudaSuccess) return cuda_fail(ctx, e, "attention merge launch");
-    }
+    e = timed(ctx, LUMO_K_ATTN_MERGE, st, [&] { return launch_attn_merge(plan, st); });
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "attention merge launch");
   }
   return LUMO_OK;
 }

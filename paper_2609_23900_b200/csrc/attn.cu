@@ -1,31 +1,37 @@
-// Attention half of the tree verifier (sm_100a): ancestry-masked decode attention on tcgen05 with
-// TMA-staged key/value tiles, the write of the tree's entries through the slot map, and the
-// re-linearisation of the accepted path at publication (paper Sec. "One slot map governs attention
-// and publication"; Algorithm 1, "remap KV").
+// Ancestry-masked decode attention of the tree verifier on tcgen05 (sm_100a): paper Sec. "One slot map
+// governs attention and publication" (grouped query heads share staged KV tiles; split-K context
+// partitions) and Sec. "State and the execution boundary" (the visibility relation).
 //
-// tree_attn_kernel.  One CTA (256 threads) takes one (sequence, KV head, 128-row query tile, key-range
-// partition).  The query rows of all heads that share the KV head sit in one tile (row = head-in-group
-// * N + node), so each staged key/value tile serves the whole group.  Per tile of 64 keys:
+// tree_attn_kernel: persistent, warp-specialised, one CTA per SM.  The work is the list of 64-key tiles
+// of all (sequence, KV head, 128-row query tile) units in order; a CTA takes a contiguous share of that
+// list (or, with an explicit partition count, one partition of one unit), and every maximal piece of
+// its share that lies in one unit is a SEGMENT: one flash-attention pass whose normalised output and
+// base-2 log-sum-exp go to a scratch slot; attn_merge_kernel combines the slots of a unit in order.
+// The query rows of all heads that share the KV head sit in one tile (row = head-in-group * N + node),
+// so a staged key/value tile serves the whole group.
 //
-//   TMA       K tile [64 keys x 128] and V tile, 128-byte swizzle, two stages, one mbarrier per stage
-//   tcgen05   S = Q K^T           (M 128, N 64, K 128; fp32 in tensor memory columns 0..63)
-//   threads   row = tensor-memory lane; a row is shared by two threads (warps w and w+4): both read the
-//             whole row for the running maximum, each turns its 32 keys into probabilities (exp2 in
-//             fp32, visibility applied by selection, never by arithmetic on the masked logit), rounds
-//             them to bf16 and stores them as the next A operand
-//   tcgen05   O_tile = P V        (M 128, N 2 x 64, K 64; V is the MN-major B operand as it lies in
-//             memory; fp32 in tensor memory columns 64..191)
-//   threads   each adds its 64 of the 128 output columns to fp32 registers, rescaled when the running
-//             maximum moved.  The next tile's S product is issued together with this tile's O product.
+//   warp 0     producer: TMA loads of K and V tiles (4-d tensor maps, 128-byte swizzle) into a ring of
+//              four stages, one mbarrier pair (full / empty) per stage
+//   warp 1     tensor-core issuer: S = Q K^T into one of two S buffers in tensor memory (M 128, N 64,
+//              K 128), and O += P V (M 128, N 2 x 64, K 64; V is the MN-major B operand as it lies in
+//              memory) into a 128-column accumulator that stays in tensor memory for the whole segment;
+//              the next tile's S product is issued before this tile's P is awaited
+//   warps 2-5  softmax: thread = query row = tensor-memory lane.  Reads the 64 logits, applies visibility
+//              by selection (never by arithmetic on a masked logit), exponentiates against a REFERENCE
+//              maximum m, rounds to bf16 and stores P as the next A operand.  m is the row maximum of
+//              the first tile and moves only when a later maximum exceeds it by more than 2^16; only
+//              then is the accumulator rescaled in tensor memory (probabilities up to 2^16 are exact
+//              enough in bf16/fp32: the exponent range is that of fp32).  At the end of a segment the
+//              same threads read O, divide by the row sum and write the slot.
 //
 // Only tiles that reach past the committed context need a mask; the mask of node i over the physical
 // suffix is a bit row built with the tree descriptor.  Value rows of positions nobody may read (padding
-// slots, beyond the suffix) are zeroed in shared memory before the product, so that bytes outside the
-// visible set cannot reach any output (0 x NaN).  A partition writes normalised partial outputs and
-// base-2 log-sum-exps to scratch; attn_merge_kernel combines them in partition order.
+// slots, beyond the suffix) are zeroed in the staged tile before the product, so that bytes outside the
+// visible set cannot reach any output (0 x NaN).
 //
-// Every wait is bounded; a wait that runs out marks the sequence LUMO_SEQ_TIMEOUT and the CTA leaves
-// through the normal exit (barriers stay uniform, tensor memory is freed).
+// Every wait is bounded; a wait that runs out marks the sequence LUMO_SEQ_TIMEOUT, later waits of that
+// thread are skipped, and every role still runs its (bounded) loops to the common exit, where tensor
+// memory is freed.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -37,33 +43,36 @@ namespace lumo {
 namespace {
 
 constexpr int kDh = 128;
-constexpr int kRows = 128;            // query rows per CTA = tensor-memory lanes
+constexpr int kRows = 128;            // query rows per unit = tensor-memory lanes
 constexpr int kKeys = 64;             // keys per tile
-constexpr int kThreads = 256;
-constexpr int kStages = 2;
-constexpr int kTmemCols = 256;        // S: columns 0..63, O tile: 64..191 (power-of-two allocation)
-constexpr int kColO = 64;
+constexpr int kThreads = 192;         // producer warp, issuer warp, four softmax warps
+constexpr int kSoftmaxThreads = 128;
+constexpr int kStages = 4;
+constexpr int kTmemCols = 256;        // S buffers: columns 0..63 and 64..127, O: 128..255
+constexpr int kColO = 128;
+constexpr int kMinTilesPerCta = 8;    // automatic mode: do not cut the work finer than this
+constexpr float kRescaleStep = 16.f;  // the reference maximum moves when exceeded by more than this (log2 units)
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
 // shared memory map; the dynamic segment starts at offset 0 of the CTA's window (no static shared
-// variables in this file), which the 128-byte swizzle needs 1024-aligned; checked at run time
+// variables in this kernel), which the 128-byte swizzle needs 1024-aligned; checked at run time
 constexpr int kOffQ = 0;              // 2 halves of dh x [128 rows x 128 B]
-constexpr int kOffP = 32768;          // [128 rows x 128 B] probabilities, bf16
-constexpr int kOffKV = 49152;         // per stage: K 2 halves x [64 keys x 128 B], then V the same
+constexpr int kOffP = 32768;          // 2 buffers x [128 rows x 128 B] probabilities, bf16
+constexpr int kOffKV = 65536;         // per stage: K 2 halves x [64 keys x 128 B], then V the same
 constexpr int kStageBytes = 32768;
-constexpr int kOffSmall = kOffKV + kStages * kStageBytes;   // 114688
+constexpr int kOffSmall = kOffKV + kStages * kStageBytes;   // 196608
 struct Small {
-  unsigned long long full[kStages];
-  unsigned long long bar_qk, bar_pv;
+  unsigned long long kv_full[kStages], kv_empty[kStages];
+  unsigned long long s_full[2], p_full[2], p_empty[2];
+  unsigned long long q_full, o_free;
   uint32_t tmem_base;
   uint32_t timed_out;
 };
-constexpr int kSmemBytes = kOffSmall + 64;
-static_assert(sizeof(Small) <= 64, "small block");
-static_assert(2 * (kSmemBytes + 1024) <= 228 * 1024, "two CTAs must share an SM");
-
+constexpr int kSmemBytes = kOffSmall + 256;
+static_assert(sizeof(Small) <= 256, "small block");
+static_assert(kSmemBytes + 1024 <= 227 * 1024, "one CTA per SM");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
@@ -146,270 +155,395 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   return *reinterpret_cast<const uint32_t*>(&t);
 }
 
-__device__ __forceinline__ int seq_check(int ctx, int crow, int Ns, int n_rows, int max_pos) {
-  if (crow < 0 || crow >= n_rows) return LUMO_SEQ_BAD_ROW;
-  if (ctx < 0 || ctx > max_pos - Ns) return LUMO_SEQ_BAD_CTX;
-  return LUMO_SEQ_OK;
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(smem_u32(bar)) : "memory");
 }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+      "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+        "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+        "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
 
-__global__ void __launch_bounds__(kThreads, 2)
+// ---- work decomposition ----------------------------------------------------------------
+// Units are numbered u = (b * Hkv + hkv) * RT + rt; unit u owns nt(b) tiles (0 for a sequence that fails
+// its check).  Automatic mode: CTA c owns the global tiles [c * per, (c + 1) * per) and the slot of a
+// segment is u + c (strictly increasing along the tile list, so unique).  Fixed mode (S partitions):
+// CTA c owns partition c mod S of unit c / S, slot c.
+struct Segment {
+  int b, hkv, rt;     // unit
+  int t0, n;          // first tile within the unit, tile count (n = 0 possible in fixed mode)
+  int slot;
+  int ctx, crow;
+};
+
+struct Work {
+  const AttnArgs& a;
+  int b, q;           // current sequence, unit within the sequence
+  long long g, g_end; // next global tile, end of this CTA's share
+  long long g_unit;   // global tile at which the current unit starts
+  int nt;             // tiles per unit of the current sequence
+  bool fixed_done;
+
+  __device__ int tiles_of(int bb, int* ctx, int* crow) const {
+    *ctx = a.ctx_len[bb];
+    *crow = a.cache_row[bb];
+    if (seq_check(*ctx, *crow, a.Ns, a.n_rows, a.max_pos) != LUMO_SEQ_OK) return 0;
+    return (*ctx + a.Ns + kKeys - 1) / kKeys;
+  }
+
+  __device__ explicit Work(const AttnArgs& args) : a(args), b(0), q(0), g(0), g_end(0), g_unit(0), nt(0), fixed_done(false) {
+    if (a.S > 0) return;
+    const int upb = a.Hkv * a.RT;       // units per sequence
+    long long total = 0;
+    int cx, cr;
+    for (int bb = 0; bb < a.B; ++bb) total += (long long)tiles_of(bb, &cx, &cr) * upb;
+    long long per = (total + gridDim.x - 1) / gridDim.x;
+    if (per < kMinTilesPerCta) per = kMinTilesPerCta;
+    g = (long long)blockIdx.x * per;
+    g_end = g + per < total ? g + per : total;
+    // position on the unit that holds tile g
+    long long acc = 0;
+    for (b = 0; b < a.B; ++b) {
+      nt = tiles_of(b, &cx, &cr);
+      const long long span = (long long)nt * upb;
+      if (g < acc + span) { q = (int)((g - acc) / nt); g_unit = acc + (long long)q * nt; break; }
+      acc += span;
+    }
+  }
+
+  // next segment of this CTA; false when the share is exhausted
+  __device__ bool next(Segment* s) {
+    const int upb = a.Hkv * a.RT;
+    if (a.S > 0) {
+      if (fixed_done) return false;
+      fixed_done = true;
+      const int u = blockIdx.x / a.S, part = blockIdx.x - u * a.S;
+      s->b = u / upb;
+      const int r = u - s->b * upb;
+      s->hkv = r / a.RT; s->rt = r - s->hkv * a.RT;
+      const int n_all = tiles_of(s->b, &s->ctx, &s->crow);
+      s->t0 = (int)(((long long)part * n_all) / a.S);
+      s->n = (int)(((long long)(part + 1) * n_all) / a.S) - s->t0;
+      s->slot = blockIdx.x;
+      return n_all > 0;
+    }
+    while (g < g_end && b < a.B) {
+      if (nt == 0 || g >= g_unit + nt) {     // move to the next unit (skipping sequences without tiles)
+        if (nt > 0) g_unit += nt;
+        if (nt == 0 || ++q == upb) {
+          q = 0;
+          int cx, cr;
+          do { ++b; nt = b < a.B ? tiles_of(b, &cx, &cr) : 0; } while (b < a.B && nt == 0);
+        }
+        continue;
+      }
+      const int u = b * upb + q;
+      s->b = b; s->hkv = q / a.RT; s->rt = q - s->hkv * a.RT;
+      tiles_of(b, &s->ctx, &s->crow);
+      s->t0 = (int)(g - g_unit);
+      const long long end = g_unit + nt < g_end ? g_unit + nt : g_end;
+      s->n = (int)(end - g);
+      s->slot = u + blockIdx.x;
+      g = end;
+      return true;
+    }
+    return false;
+  }
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
 tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, const AttnArgs a) {
   extern __shared__ __align__(1024) unsigned char smem[];
   Small& sm = *reinterpret_cast<Small*>(smem + kOffSmall);
   const uint32_t sbase = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int split = blockIdx.x, hkv = blockIdx.y / a.RT, rt = blockIdx.y % a.RT, b = blockIdx.z;
-  const int row = 32 * (warp & 3) + lane;   // tensor-memory lane = query row of the tile
-  const int half = warp >> 2;               // key half in the softmax, dh half in the accumulation
-  const int GN = a.G * a.N;
-  const int rg = rt * kRows + row;          // row within the (sequence, KV head) group
-  const bool row_ok = rg < GN;
-  const int hl = row_ok ? rg / a.N : 0, node = row_ok ? rg - hl * a.N : 0;
+  const bool aligned = (sbase & 1023u) == 0;   // cannot fail with this file's layout; refuse rather than mis-swizzle
 
-  const int ctx = a.ctx_len[b], crow = a.cache_row[b];
-  int bad = seq_check(ctx, crow, a.Ns, a.n_rows, a.max_pos);
-  if ((sbase & 1023u) != 0) bad = LUMO_SEQ_TIMEOUT;   // cannot happen with this file's layout; refuse rather than mis-swizzle
-  const size_t out_row = (((size_t)b * a.N + node) * a.Hq + (size_t)hkv * a.G + hl);
-  const size_t part_row = ((((size_t)b * a.Hkv + hkv) * a.RT + rt) * a.S + split) * kRows + row;
-  if (bad != LUMO_SEQ_OK) {                 // uniform over the CTA: nothing was allocated or issued yet
-    if (a.status && split == 0 && blockIdx.y == 0 && tid == 0) a.status[b] = bad;
-    if (row_ok && split == 0) {
-      float4* o = reinterpret_cast<float4*>(a.out + out_row * kDh + half * 64);
-      for (int e = 0; e < 16; ++e) o[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (a.lse && half == 0) a.lse[out_row] = 0.f;
-    }
-    return;
-  }
-
-  // key tiles of this partition
-  const int T = ctx + a.Ns;
-  const int nt = (T + kKeys - 1) / kKeys;
-  const int t0 = (int)(((long long)split * nt) / a.S), t1 = (int)(((long long)(split + 1) * nt) / a.S);
-  const int n = t1 - t0;
-
-  if (warp == 0) {
+  if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(&sm.full[s], 1);
-    mbar_init(&sm.bar_qk, 1);
-    mbar_init(&sm.bar_pv, 1);
+    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sm.s_full[s], 1);
+      mbar_init(&sm.p_full[s], kSoftmaxThreads);
+      mbar_init(&sm.p_empty[s], 1);
+    }
+    mbar_init(&sm.q_full, kSoftmaxThreads);
+    mbar_init(&sm.o_free, kSoftmaxThreads);
     sm.timed_out = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
-  // query tile: 128 rows x 16 chunks of 16 bytes, zero rows beyond the group
-  for (int c = tid; c < kRows * 16; c += kThreads) {
-    const int r = c >> 4, ch = c & 15;
-    const int g = rt * kRows + r;
-    uint4 val = make_uint4(0u, 0u, 0u, 0u);
-    if (g < GN) {
-      const int h = g / a.N, i = g - h * a.N;
-      val = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) + ((((size_t)b * a.N + i) * a.Hq + (size_t)hkv * a.G + h) * kDh + ch * 8)));
-    }
-    *reinterpret_cast<uint4*>(smem + kOffQ + (ch >> 3) * 16384 + sw128(r, ch & 7)) = val;
-  }
-  fence_async_proxy();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
-  const uint32_t tmem_lane = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
 
-  // thread 0 is the producer (TMA) and the tensor-core issuer
-  auto issue_tile = [&](int tile, int st) {
-    mbar_expect_tx(&sm.full[st], kStageBytes);
-    const uint32_t dst = sbase + kOffKV + st * kStageBytes;
-    tma_load_4d(dst, &tm_k, &sm.full[st], 0, hkv, tile * kKeys, crow);
-    tma_load_4d(dst + 8192, &tm_k, &sm.full[st], 64, hkv, tile * kKeys, crow);
-    tma_load_4d(dst + 16384, &tm_v, &sm.full[st], 0, hkv, tile * kKeys, crow);
-    tma_load_4d(dst + 24576, &tm_v, &sm.full[st], 64, hkv, tile * kKeys, crow);
-  };
-  auto issue_qk = [&](int st) {
-    constexpr uint32_t id = umma_idesc(kRows, kKeys, 0, 0);
-    const uint32_t kb = sbase + kOffKV + st * kStageBytes;
-#pragma unroll
-    for (int ks = 0; ks < 8; ++ks)
-      umma(tmem, umma_desc(sbase + kOffQ + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-           umma_desc(kb + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id, ks ? 1u : 0u);
-    umma_commit(&sm.bar_qk);
-  };
-  auto issue_pv = [&](int st) {
-    constexpr uint32_t id = umma_idesc(kRows, 64, 0, 1);
-    const uint32_t vb = sbase + kOffKV + st * kStageBytes + 16384;
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-      for (int ks = 0; ks < 4; ++ks)
-        umma(tmem + kColO + hh * 64, umma_desc(sbase + kOffP + ks * 32, 16, 1024),
-             umma_desc(vb + hh * 8192 + ks * 2048, 8192, 1024), id, ks ? 1u : 0u);
-    umma_commit(&sm.bar_pv);
-  };
+  Work work(a);
+  Segment sg;
+  bool ok = aligned;
+  uint32_t it = 0;        // tiles this CTA has started, over all segments: ring stage, S / P buffer and phases
+  uint32_t nseg = 0;      // segments with tiles so far: phases of q_full and o_free
 
-  bool ok = true;
-  int issued = 0;                           // tiles whose loads thread 0 has issued
-  if (tid == 0) {
-    for (; issued < n && issued < kStages; ++issued) issue_tile(t0 + issued, issued);
-    if (n > 0) {
-      ok = mbar_wait(&sm.full[0], 0);
-      tc_fence_after();
-      issue_qk(0);
-    }
-  }
-
-  const uint32_t* visw = a.vis + ((size_t)b * a.N + node) * 8;
-  const uint32_t* usedw = a.used + (size_t)b * 8;
-  const float sl2 = a.scale_log2;
-  float m = -INFINITY, l = 0.f;
-  float o[64];
-#pragma unroll
-  for (int e = 0; e < 64; ++e) o[e] = 0.f;
-  uint32_t ph_qk = 0, ph_pv = 0;
-
-  for (int jj = 0; jj < n; ++jj) {
-    const int st = jj & 1;
-    const int kpos0 = (t0 + jj) * kKeys;
-    const bool tail = kpos0 + kKeys > ctx;   // uniform: the tile reaches past the committed context
-    // visibility of this row over the tile's 64 keys
-    unsigned long long vm = row_ok ? ~0ull : 0ull;
-    if (tail && row_ok) {
-      vm = 0ull;
-      for (int c = 0; c < kKeys; ++c) {
-        const int p = kpos0 + c;
-        bool v = p < ctx;
-        if (!v) {
-          const int s = p - ctx;
-          if (s < a.Ns) v = (__ldg(visw + (s >> 5)) >> (s & 31)) & 1u;
-        }
-        vm |= (unsigned long long)v << c;
-      }
-    }
-    if (ok) ok = mbar_wait(&sm.bar_qk, ph_qk);
-    ph_qk ^= 1u;
-    tc_fence_after();
-    __syncwarp();                            // the tensor-memory loads below are warp-collective
-
-    // pass 1: running maximum over the whole row
-    float mx = -INFINITY;
-#pragma unroll
-    for (int c4 = 0; c4 < 4; ++c4) {
-      uint32_t r[16];
-      tmem_ld16(tmem_lane + c4 * 16, r);
-      const uint32_t bits = (uint32_t)(vm >> (c4 * 16));
-#pragma unroll
-      for (int e = 0; e < 16; ++e) {
-        const float s = __uint_as_float(r[e]);
-        mx = fmaxf(mx, ((bits >> e) & 1u) ? s : -INFINITY);
-      }
-    }
-    const float m_new = fmaxf(m, mx * sl2);
-    const float m_use = m_new == -INFINITY ? 0.f : m_new;
-    const float corr = ex2(m - m_use);       // m = -inf: 0
-    m = m_new;
-    l *= corr;
-#pragma unroll
-    for (int e = 0; e < 64; ++e) o[e] *= corr;
-    // pass 2: this thread's 32 keys -> probabilities, bf16, A operand of the second product
-    float lsum = 0.f;
-#pragma unroll
-    for (int c2 = 0; c2 < 2; ++c2) {
-      uint32_t r[16];
-      tmem_ld16(tmem_lane + half * 32 + c2 * 16, r);
-      const uint32_t bits = (uint32_t)(vm >> (half * 32 + c2 * 16));
-      uint32_t pk[8];
-#pragma unroll
-      for (int e = 0; e < 16; e += 2) {
-        const float p0 = ((bits >> e) & 1u) ? ex2(fmaf(__uint_as_float(r[e]), sl2, -m_use)) : 0.f;
-        const float p1 = ((bits >> (e + 1)) & 1u) ? ex2(fmaf(__uint_as_float(r[e + 1]), sl2, -m_use)) : 0.f;
-        lsum += p0 + p1;
-        pk[e >> 1] = pack_bf16(p0, p1);
-      }
-      const int chunk = half * 4 + c2 * 2;
-      *reinterpret_cast<uint4*>(smem + kOffP + sw128(row, chunk)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-      *reinterpret_cast<uint4*>(smem + kOffP + sw128(row, chunk + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-    }
-    l += lsum;
-
-    if (tail) {
-      // value rows nobody may read: zero them in the staged tile (two 128-byte rows per key)
-      if (ok) ok = mbar_wait(&sm.full[st], (uint32_t)(jj >> 1) & 1u);
-      if (tid < 2 * kKeys) {
-        const int c = tid >> 1, hh = tid & 1;
-        const int p = kpos0 + c;
-        bool dead = false;
-        if (p >= ctx) {
-          const int s = p - ctx;
-          dead = s >= a.Ns || !((__ldg(usedw + (s >> 5)) >> (s & 31)) & 1u);
-        }
-        if (dead) {
-          uint4* vrow = reinterpret_cast<uint4*>(smem + kOffKV + st * kStageBytes + 16384 + hh * 8192 + c * 128);
-#pragma unroll
-          for (int e = 0; e < 8; ++e) vrow[e] = make_uint4(0u, 0u, 0u, 0u);
+  if (warp == 0) {
+    // ---------------- producer ----------------
+    if (lane == 0) {
+      while (work.next(&sg)) {
+        for (int j = 0; j < sg.n; ++j, ++it) {
+          const uint32_t st = it % kStages, use = it / kStages;
+          if (use > 0 && ok) ok = mbar_wait(&sm.kv_empty[st], (use - 1) & 1u);
+          if (!ok) continue;
+          mbar_expect_tx(&sm.kv_full[st], kStageBytes);
+          const uint32_t dst = sbase + kOffKV + st * kStageBytes;
+          const int pos = (sg.t0 + j) * kKeys;
+          tma_load_4d(dst, &tm_k, &sm.kv_full[st], 0, sg.hkv, pos, sg.crow);
+          tma_load_4d(dst + 8192, &tm_k, &sm.kv_full[st], 64, sg.hkv, pos, sg.crow);
+          tma_load_4d(dst + 16384, &tm_v, &sm.kv_full[st], 0, sg.hkv, pos, sg.crow);
+          tma_load_4d(dst + 24576, &tm_v, &sm.kv_full[st], 64, sg.hkv, pos, sg.crow);
         }
       }
+      if (!ok) sm.timed_out = 1u;
     }
-    fence_async_proxy();
-    tc_fence_before();
-    __syncthreads();
-    if (tid == 0) {
-      tc_fence_after();
-      issue_pv(st);
-      if (jj + 1 < n) {                      // next tile's logits run under this tile's accumulation
-        if (ok) ok = mbar_wait(&sm.full[st ^ 1], (uint32_t)((jj + 1) >> 1) & 1u);
+  } else if (warp == 1) {
+    // ---------------- tensor-core issuer ----------------
+    if (lane == 0) {
+      auto issue_qk = [&](uint32_t t) {
+        constexpr uint32_t id = umma_idesc(kRows, kKeys, 0, 0);
+        const uint32_t kb = sbase + kOffKV + (t % kStages) * kStageBytes;
+        const uint32_t d = tmem + (t & 1u) * 64;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks)
+          umma(d, umma_desc(sbase + kOffQ + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
+               umma_desc(kb + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id, ks ? 1u : 0u);
+        umma_commit(&sm.s_full[t & 1u]);
+      };
+      auto issue_pv = [&](uint32_t t, bool first) {
+        constexpr uint32_t id = umma_idesc(kRows, 64, 0, 1);
+        const uint32_t vb = sbase + kOffKV + (t % kStages) * kStageBytes + 16384;
+        const uint32_t pb = sbase + kOffP + (t & 1u) * 16384;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks)
+            umma(tmem + kColO + hh * 64, umma_desc(pb + ks * 32, 16, 1024), umma_desc(vb + hh * 8192 + ks * 2048, 8192, 1024),
+                 id, (first && ks == 0) ? 0u : 1u);
+        umma_commit(&sm.kv_empty[t % kStages]);
+        umma_commit(&sm.p_empty[t & 1u]);
+      };
+      while (work.next(&sg)) {
+        if (sg.n == 0) continue;
+        if (ok) ok = mbar_wait(&sm.q_full, nseg & 1u);
+        for (int j = 0; j < sg.n; ++j, ++it) {
+          if (j == 0) {
+            if (ok) ok = mbar_wait(&sm.kv_full[it % kStages], (it / kStages) & 1u);
+            tc_fence_after();
+            if (ok) issue_qk(it);
+          }
+          if (j + 1 < sg.n) {        // the next tile's logits run while the softmax warps work on this tile
+            if (ok) ok = mbar_wait(&sm.kv_full[(it + 1) % kStages], ((it + 1) / kStages) & 1u);
+            tc_fence_after();
+            if (ok) issue_qk(it + 1);
+          }
+          if (ok) ok = mbar_wait(&sm.p_full[it & 1u], (it >> 1) & 1u);
+          if (j == 0 && nseg > 0 && ok) ok = mbar_wait(&sm.o_free, (nseg - 1) & 1u);
+          tc_fence_after();
+          if (ok) issue_pv(it, j == 0);
+        }
+        ++nseg;
+      }
+      if (!ok) sm.timed_out = 1u;
+    }
+  } else {
+    // ---------------- softmax warps ----------------
+    const int row = 32 * (warp & 3) + lane;      // tensor-memory lane this warp may touch
+    const int sthread = tid - 64;                // 0..127
+    const uint32_t tmem_lane = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+    const float sl2 = a.scale_log2;
+    const int GN = a.G * a.N;
+    while (work.next(&sg)) {
+      const int rg = sg.rt * kRows + row;
+      const bool row_ok = rg < GN;
+      const int hl = row_ok ? rg / a.N : 0, node = row_ok ? rg - hl * a.N : 0;
+      float* slot_o = a.part_o + ((size_t)sg.slot * kRows + row) * kDh;
+      float* slot_l = a.part_lse + (size_t)sg.slot * kRows + row;
+      if (sg.n == 0) {                           // empty partition (fixed mode): an empty slot
+        if (row_ok) {
+          for (int e = 0; e < kDh / 4; ++e) reinterpret_cast<float4*>(slot_o)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+          *slot_l = -INFINITY;
+        }
+        continue;
+      }
+      // query tile: 128 rows x 16 chunks of 16 bytes, zero rows beyond the group.  The previous segment's
+      // S products have all completed (their s_full phases were awaited), so the tile may be replaced.
+      for (int c = sthread; c < kRows * 16; c += kSoftmaxThreads) {
+        const int r = c >> 4, ch = c & 15;
+        const int g = sg.rt * kRows + r;
+        uint4 val = make_uint4(0u, 0u, 0u, 0u);
+        if (g < GN) {
+          const int h = g / a.N, i = g - h * a.N;
+          val = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
+                                                      ((((size_t)sg.b * a.N + i) * a.Hq + (size_t)sg.hkv * a.G + h) * kDh + ch * 8)));
+        }
+        *reinterpret_cast<uint4*>(smem + kOffQ + (ch >> 3) * 16384 + sw128(r, ch & 7)) = val;
+      }
+      fence_async_proxy();
+      mbar_arrive(&sm.q_full);
+
+      const uint32_t* visw = a.vis + ((size_t)sg.b * a.N + node) * 8;
+      const uint32_t* usedw = a.used + (size_t)sg.b * 8;
+      float m = -INFINITY, l = 0.f;              // reference maximum (log2 units), row sum against it
+      for (int j = 0; j < sg.n; ++j, ++it) {
+        const uint32_t buf = it & 1u;
+        const int kpos0 = (sg.t0 + j) * kKeys;
+        const bool tail = kpos0 + kKeys > sg.ctx;    // uniform: the tile reaches past the committed context
+        unsigned long long vm = ~0ull;
+        if (tail) {
+          vm = 0ull;
+          for (int c = 0; c < kKeys; ++c) {
+            const int p = kpos0 + c;
+            bool v = p < sg.ctx;
+            if (!v) {
+              const int s = p - sg.ctx;
+              if (s < a.Ns) v = (__ldg(visw + (s >> 5)) >> (s & 31)) & 1u;
+            }
+            vm |= (unsigned long long)v << c;
+          }
+        }
+        if (ok) ok = mbar_wait(&sm.s_full[buf], (it >> 1) & 1u);
         tc_fence_after();
-        issue_qk(st ^ 1);
+        __syncwarp();
+        uint32_t sr[64];
+        tmem_ld32(tmem_lane + buf * 64, sr);
+        tmem_ld32(tmem_lane + buf * 64 + 32, sr + 32);
+        tmem_ld_wait();
+        float mx = -INFINITY;
+        if (!tail) {
+#pragma unroll
+          for (int e = 0; e < 64; ++e) mx = fmaxf(mx, __uint_as_float(sr[e]));
+        } else {
+#pragma unroll
+          for (int e = 0; e < 64; ++e) mx = fmaxf(mx, ((vm >> e) & 1ull) ? __uint_as_float(sr[e]) : -INFINITY);
+        }
+        mx *= sl2;
+        // reference maximum: set by the first tile that shows the row a key; moved (with a rescale of the
+        // accumulator) only when exceeded by more than kRescaleStep
+        float corr = 1.f;
+        if (m == -INFINITY) m = mx;
+        else if (mx > m + kRescaleStep) { corr = ex2(m - mx); m = mx; }
+        if (__any_sync(0xffffffffu, corr != 1.f)) {
+          // O still holds the products up to the previous tile: wait for them, then scale this warp's rows
+          if (ok) ok = mbar_wait(&sm.p_empty[(it - 1) & 1u], ((it - 1) >> 1) & 1u);
+          tc_fence_after();
+          __syncwarp();
+#pragma unroll 1
+          for (int c = 0; c < kDh; c += 32) {
+            uint32_t orr[32];
+            tmem_ld32(tmem_lane + kColO + c, orr);
+            tmem_ld_wait();
+#pragma unroll
+            for (int e = 0; e < 32; ++e) orr[e] = __float_as_uint(__uint_as_float(orr[e]) * corr);
+            tmem_st32(tmem_lane + kColO + c, orr);
+          }
+          tmem_st_wait();
+          l *= corr;
+        }
+        const float mu = m == -INFINITY ? 0.f : m;
+        // P buffer `buf` was last read by the O product of tile it - 2
+        if (it >= 2 && ok) ok = mbar_wait(&sm.p_empty[buf], ((it - 2) >> 1) & 1u);
+        unsigned char* prow = smem + kOffP + buf * 16384;
+        float lsum = 0.f;
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) {
+          uint32_t pk[4];
+#pragma unroll
+          for (int e = 0; e < 8; e += 2) {
+            const int c = ch * 8 + e;
+            float p0 = ex2(fmaf(__uint_as_float(sr[c]), sl2, -mu));
+            float p1 = ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -mu));
+            if (tail) {
+              p0 = ((vm >> c) & 1ull) ? p0 : 0.f;
+              p1 = ((vm >> (c + 1)) & 1ull) ? p1 : 0.f;
+            }
+            lsum += p0 + p1;
+            pk[e >> 1] = pack_bf16(p0, p1);
+          }
+          *reinterpret_cast<uint4*>(prow + sw128(row, ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+        l += lsum;
+        if (tail) {
+          // value rows nobody may read: zero them in the staged tile (two 128-byte rows per key)
+          const uint32_t st = it % kStages;
+          if (ok) ok = mbar_wait(&sm.kv_full[st], (it / kStages) & 1u);
+          const int c = sthread >> 1, hh = sthread & 1;
+          const int p = kpos0 + c;
+          bool dead = false;
+          if (p >= sg.ctx) {
+            const int s = p - sg.ctx;
+            dead = s >= a.Ns || !((__ldg(usedw + (s >> 5)) >> (s & 31)) & 1u);
+          }
+          if (dead) {
+            uint4* vrow = reinterpret_cast<uint4*>(smem + kOffKV + st * kStageBytes + 16384 + hh * 8192 + c * 128);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) vrow[e] = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+        fence_async_proxy();
+        tc_fence_before();
+        mbar_arrive(&sm.p_full[buf]);
       }
-    }
-    if (ok) ok = mbar_wait(&sm.bar_pv, ph_pv);
-    ph_pv ^= 1u;
-    tc_fence_after();
-    if (tid == 0 && issued < n) {            // both products of this stage have completed: refill it
-      issue_tile(t0 + issued, st);
-      ++issued;
-    }
-    __syncwarp();
+      // end of the segment: the last O product, then normalise and write the slot
+      if (ok) ok = mbar_wait(&sm.p_empty[(it - 1) & 1u], ((it - 1) >> 1) & 1u);
+      tc_fence_after();
+      __syncwarp();
+      const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll 1
+      for (int c = 0; c < kDh; c += 32) {
+        uint32_t orr[32];
+        tmem_ld32(tmem_lane + kColO + c, orr);
+        tmem_ld_wait();
+        if (row_ok) {
 #pragma unroll
-    for (int c4 = 0; c4 < 4; ++c4) {
-      uint32_t r[16];
-      tmem_ld16(tmem_lane + kColO + half * 64 + c4 * 16, r);
-#pragma unroll
-      for (int e = 0; e < 16; ++e) o[c4 * 16 + e] += __uint_as_float(r[e]);
+          for (int e = 0; e < 32; e += 4)
+            *reinterpret_cast<float4*>(slot_o + c + e) =
+                make_float4(__uint_as_float(orr[e]) * inv, __uint_as_float(orr[e + 1]) * inv,
+                            __uint_as_float(orr[e + 2]) * inv, __uint_as_float(orr[e + 3]) * inv);
+        }
+      }
+      if (row_ok) *slot_l = l > 0.f ? m + log2f(l) : -INFINITY;
+      tc_fence_before();
+      mbar_arrive(&sm.o_free);
+      ++nseg;
     }
+    if (!ok) sm.timed_out = 1u;
   }
 
-  // after a wait that ran out, loads may still be in flight: give them a bounded chance to land
-  if (tid == 0 && !ok)
-    for (int t = 0; t < issued; ++t) (void)mbar_wait(&sm.full[t & 1], (uint32_t)(t >> 1) & 1u);
-  if (!ok) sm.timed_out = 1u;
   tc_fence_before();
   __syncthreads();
-  // the two halves of a row hold partial sums of the same scale (same running maximum)
-  float* lbuf = reinterpret_cast<float*>(smem + kOffP);
-  lbuf[half * kRows + row] = l;
-  __syncthreads();
-  const float lt = lbuf[row] + lbuf[kRows + row];
-  const float inv = lt > 0.f ? 1.f / lt : 0.f;
-  const float lse2 = lt > 0.f ? m + log2f(lt) : -INFINITY;
-  if (row_ok) {
-    float4* dst = a.S == 1 ? reinterpret_cast<float4*>(a.out + out_row * kDh + half * 64)
-                           : reinterpret_cast<float4*>(a.part_o + part_row * kDh + half * 64);
-#pragma unroll
-    for (int e = 0; e < 16; ++e)
-      dst[e] = make_float4(o[4 * e] * inv, o[4 * e + 1] * inv, o[4 * e + 2] * inv, o[4 * e + 3] * inv);
-    if (half == 0) {
-      if (a.S == 1) { if (a.lse) a.lse[out_row] = lse2 * kLn2; }
-      else a.part_lse[part_row] = lse2;
-    }
-  }
-  if (a.status && tid == 0) {
-    if (sm.timed_out) a.status[b] = LUMO_SEQ_TIMEOUT;
-    else if (split == 0 && blockIdx.y == 0) a.status[b] = LUMO_SEQ_OK;
-  }
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  if (sm.timed_out && a.status && tid == 0)      // the outputs of the whole call are suspect
+    for (int b = 0; b < a.B; ++b) a.status[b] = LUMO_SEQ_TIMEOUT;
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
-// Combination of the partitions' results: one warp per output row, partitions in index order (so the
-// result for a given partition count is reproducible), weights exp2(lse_s - max lse).
+// Combination of a unit's slots: one warp per output row, slots in order (so the result for a given
+// decomposition is reproducible), weights exp2(lse_s - max lse).
 __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int GN = a.G * a.N;
@@ -422,17 +556,44 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   const int hl = rg / a.N, node = rg - hl * a.N;
   const size_t out_row = (((size_t)b * a.N + node) * a.Hq + (size_t)hkv * a.G + hl);
   float4* dst = reinterpret_cast<float4*>(a.out + out_row * kDh) + lane;
-  if (seq_check(a.ctx_len[b], a.cache_row[b], a.Ns, a.n_rows, a.max_pos) != LUMO_SEQ_OK) {
+  const int upb = a.Hkv * a.RT;
+  const int u = b * upb + hkv * a.RT + rt;
+  // this unit's slots
+  int slot0 = 0, nslot = 0;
+  {
+    long long total = 0, before = 0;
+    int nt_b = 0;
+    for (int bb = 0; bb < a.B; ++bb) {
+      const int ok = seq_check(a.ctx_len[bb], a.cache_row[bb], a.Ns, a.n_rows, a.max_pos) == LUMO_SEQ_OK;
+      const int nt = ok ? (a.ctx_len[bb] + a.Ns + kKeys - 1) / kKeys : 0;
+      if (bb < b) before += (long long)nt * upb;
+      if (bb == b) nt_b = nt;
+      total += (long long)nt * upb;
+    }
+    if (nt_b > 0) {
+      if (a.S > 0) { slot0 = u * a.S; nslot = a.S; }
+      else {
+        long long per = (total + a.C - 1) / a.C;
+        if (per < kMinTilesPerCta) per = kMinTilesPerCta;
+        const long long g0 = before + (long long)(hkv * a.RT + rt) * nt_b;
+        const int c0 = (int)(g0 / per), c1 = (int)((g0 + nt_b - 1) / per);
+        slot0 = u + c0; nslot = c1 - c0 + 1;
+      }
+    }
+  }
+  if (nslot == 0) {                          // the sequence failed its check (it owns no tiles): zeros and its status
     *dst = make_float4(0.f, 0.f, 0.f, 0.f);
     if (a.lse && lane == 0) a.lse[out_row] = 0.f;
+    if (a.status && lane == 0 && hkv == 0 && rg == 0)
+      a.status[b] = seq_check(a.ctx_len[b], a.cache_row[b], a.Ns, a.n_rows, a.max_pos);
     return;
   }
-  const size_t base = ((((size_t)b * a.Hkv + hkv) * a.RT + rt) * a.S) * kRows + r;
+  const size_t base = (size_t)slot0 * kRows + r;
   float mx = -INFINITY;
-  for (int s = 0; s < a.S; ++s) mx = fmaxf(mx, a.part_lse[base + (size_t)s * kRows]);
+  for (int s = 0; s < nslot; ++s) mx = fmaxf(mx, a.part_lse[base + (size_t)s * kRows]);
   float den = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s = 0; s < a.S; ++s) {
+  for (int s = 0; s < nslot; ++s) {
     const float ls = a.part_lse[base + (size_t)s * kRows];
     if (ls == -INFINITY) continue;
     const float wgt = ex2(ls - mx);
@@ -444,78 +605,6 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   const float inv = den > 0.f ? 1.f / den : 0.f;
   *dst = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
   if (a.lse && lane == 0) a.lse[out_row] = den > 0.f ? (mx + log2f(den)) * kLn2 : -INFINITY;
-}
-
-
-// Scatter of the tree's entries: grid (node, sequence, layer); a CTA copies the Hkv x 128 keys and
-// values of one node to position ctx + slot[node].
-__global__ void __launch_bounds__(128) kv_write_kernel(const KvLayers L, const KvShape s) {
-  const int i = blockIdx.x, b = blockIdx.y, l = blockIdx.z;
-  const int ctx = s.ctx_len[b], crow = s.cache_row[b];
-  const int bad = seq_check(ctx, crow, s.Ns, s.n_rows, s.max_pos);
-  if (bad != LUMO_SEQ_OK) {
-    if (L.status[l] && i == 0 && threadIdx.x == 0) L.status[l][b] = bad;
-    return;
-  }
-  const int chunks = s.Hkv * kDh / 8;      // 16-byte chunks per entry
-  const size_t src = ((size_t)b * s.N + i) * chunks;
-  const size_t dst = ((size_t)crow * s.max_pos + ctx + s.slot[(size_t)b * s.N + i]) * chunks;
-  const uint4* kn = reinterpret_cast<const uint4*>(L.kn[l]) + src;
-  const uint4* vn = reinterpret_cast<const uint4*>(L.vn[l]) + src;
-  uint4* kc = reinterpret_cast<uint4*>(L.k[l]) + dst;
-  uint4* vc = reinterpret_cast<uint4*>(L.v[l]) + dst;
-  for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
-    kc[c] = __ldg(kn + c);
-    vc[c] = __ldg(vn + c);
-  }
-}
-
-// Publication: grid (KV head x {K, V}, sequence, layer).  A CTA stages the 256-byte pieces of all
-// accepted entries that have to move (source != destination) in shared memory, then writes them: all
-// reads come before any write, and pieces of different heads never overlap.
-__global__ void __launch_bounds__(256) kv_publish_kernel(const KvLayers L, const KvShape s, const int32_t* __restrict__ accepted,
-                                                         const int32_t* __restrict__ len, int lmax, int32_t* ctx_len_out) {
-  extern __shared__ __align__(16) unsigned char stage[];     // [lmax][256 B]
-  __shared__ int acc_s[kMaxNodes], par_s[kMaxNodes], src_s[kMaxNodes];
-  __shared__ int st_s;
-  const int hkv = blockIdx.x >> 1, which = blockIdx.x & 1, b = blockIdx.y, l = blockIdx.z;
-  const int tid = threadIdx.x;
-  const int ctx = s.ctx_len[b], crow = s.cache_row[b];
-  const int n = len[b];
-  const int nn = n < 0 ? 0 : (n > lmax ? lmax : n);
-  for (int t = tid; t < nn; t += blockDim.x) {
-    const int a = accepted[(size_t)b * lmax + t];
-    acc_s[t] = a;
-    const bool in = a >= 0 && a < s.N;
-    par_s[t] = in ? s.parent[(size_t)b * s.N + a] : -2;
-    src_s[t] = in ? s.slot[(size_t)b * s.N + a] : 0;
-  }
-  __syncthreads();
-  if (tid == 0) {
-    int st = seq_check(ctx, crow, s.Ns, s.n_rows, s.max_pos);
-    if (st == LUMO_SEQ_OK) st = check_path_staged(acc_s, par_s, s.N, n, lmax);
-    st_s = st;
-    const bool lead = blockIdx.x == 0;
-    if (lead && L.status[l]) L.status[l][b] = st;
-    if (lead && l == 0 && ctx_len_out) ctx_len_out[b] = st == LUMO_SEQ_OK ? ctx + n : ctx;
-  }
-  __syncthreads();
-  if (st_s != LUMO_SEQ_OK) return;
-  unsigned char* cache = reinterpret_cast<unsigned char*>(which ? L.v[l] : L.k[l]);
-  const size_t pos_bytes = (size_t)s.Hkv * kDh * 2;
-  unsigned char* rowp = cache + ((size_t)crow * s.max_pos + ctx) * pos_bytes + (size_t)hkv * kDh * 2;
-  // 16 chunks of 16 bytes per entry
-  for (int c = tid; c < nn * 16; c += blockDim.x) {
-    const int t = c >> 4, ch = c & 15;
-    if (src_s[t] != t)
-      reinterpret_cast<uint4*>(stage)[c] = *reinterpret_cast<const uint4*>(rowp + (size_t)src_s[t] * pos_bytes + ch * 16);
-  }
-  __syncthreads();
-  for (int c = tid; c < nn * 16; c += blockDim.x) {
-    const int t = c >> 4, ch = c & 15;
-    if (src_s[t] != t)
-      *reinterpret_cast<uint4*>(rowp + (size_t)t * pos_bytes + ch * 16) = reinterpret_cast<const uint4*>(stage)[c];
-  }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -548,13 +637,18 @@ cudaError_t encode_cache_map(void* cache, int Hkv, int max_pos, int n_rows, CUte
 
 int attn_row_tiles(int G, int N) { return (G * N + kRows - 1) / kRows; }
 
-size_t attn_scratch_bytes(const AttnShape& s) {
-  if (s.S <= 1) return 0;
-  return (size_t)s.B * s.Hkv * attn_row_tiles(s.Hq / s.Hkv, s.N) * s.S * kRows * (kDh + 1) * sizeof(float);
+// slots of partial results: automatic mode needs at most units + CTAs - 1, fixed mode units x partitions
+static size_t attn_slots(const AttnShape& s, int ctas) {
+  const size_t units = (size_t)s.B * s.Hkv * attn_row_tiles(s.Hq / s.Hkv, s.N);
+  return s.S > 0 ? units * s.S : units + ctas;
+}
+
+size_t attn_scratch_bytes(const AttnShape& s, int sm_count) {
+  return attn_slots(s, sm_count) * kRows * (kDh + 1) * sizeof(float);
 }
 
 cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t* vis, const uint32_t* used, float* scratch,
-                      AttnPlan* plan, std::string* err) {
+                      int sm_count, AttnPlan* plan, std::string* err) {
   static bool configured[kMaxDevices] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -572,12 +666,14 @@ cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t
   a.q = p.q;
   a.out = p.out; a.lse = p.lse;
   a.G = s.Hq / s.Hkv; a.RT = attn_row_tiles(a.G, s.N); a.S = s.S;
+  const size_t units = (size_t)s.B * s.Hkv * a.RT;
+  a.C = s.S > 0 ? (int)(units * s.S) : sm_count;
   a.part_o = scratch;
-  a.part_lse = scratch ? scratch + (size_t)s.B * s.Hkv * a.RT * s.S * kRows * kDh : nullptr;
+  a.part_lse = scratch + attn_slots(s, sm_count) * kRows * kDh;
   a.ctx_len = s.ctx_len; a.cache_row = s.cache_row; a.vis = vis; a.used = used; a.status = p.status;
   a.B = s.B; a.N = s.N; a.Ns = s.Ns; a.Hq = s.Hq; a.Hkv = s.Hkv; a.n_rows = s.n_rows; a.max_pos = s.max_pos;
   a.scale_log2 = s.scale * kLog2e;
-  plan->grid = dim3(s.S, s.Hkv * a.RT, s.B);
+  plan->grid = dim3(a.C, 1, 1);
   return cudaSuccess;
 }
 
@@ -589,26 +685,6 @@ cudaError_t launch_attn(const AttnPlan& plan, cudaStream_t st) {
 cudaError_t launch_attn_merge(const AttnPlan& plan, cudaStream_t st) {
   const long long rows = (long long)plan.a.B * plan.a.Hkv * plan.a.G * plan.a.N;
   attn_merge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(plan.a);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_kv_write(const KvLayers& L, const KvShape& s, int n_layers, cudaStream_t st) {
-  kv_write_kernel<<<dim3(s.N, s.B, n_layers), 128, 0, st>>>(L, s);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_kv_publish(const KvLayers& L, const KvShape& s, int n_layers, const int32_t* accepted, const int32_t* len,
-                              int lmax, int32_t* ctx_len_out, cudaStream_t st) {
-  static bool configured[kMaxDevices] = {};
-  int dev = 0;
-  cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  if (dev >= 0 && dev < kMaxDevices && !configured[dev]) {
-    e = cudaFuncSetAttribute(kv_publish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxNodes * 256);
-    if (e != cudaSuccess) return e;
-    configured[dev] = true;
-  }
-  kv_publish_kernel<<<dim3(2 * s.Hkv, s.B, n_layers), 256, (size_t)lmax * 256, st>>>(L, s, accepted, len, lmax, ctx_len_out);
   return cudaGetLastError();
 }
 

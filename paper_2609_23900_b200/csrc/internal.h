@@ -192,6 +192,13 @@ __device__ __forceinline__ int check_path_staged(const int* acc, const int* par,
   return LUMO_SEQ_OK;
 }
 
+// attention-side sequence check: the cache row exists and context plus suffix fit the row
+__device__ __forceinline__ int seq_check(int ctx, int crow, int Ns, int n_rows, int max_pos) {
+  if (crow < 0 || crow >= n_rows) return LUMO_SEQ_BAD_ROW;
+  if (ctx < 0 || ctx > max_pos - Ns) return LUMO_SEQ_BAD_CTX;
+  return LUMO_SEQ_OK;
+}
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;\n" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory"); }
 
@@ -309,7 +316,9 @@ struct AttnArgs {
   const int32_t* ctx_len; const int32_t* cache_row;
   const uint32_t* vis; const uint32_t* used;
   int32_t* status;
-  int B, N, Ns, Hq, Hkv, G, RT, S, n_rows, max_pos;
+  int B, N, Ns, Hq, Hkv, G, RT, n_rows, max_pos;
+  int S;   // partitions per unit; 0: the CTAs share the tile list evenly
+  int C;   // CTAs of the attention launch
   float scale_log2;
 };
 // one attention launch: the tensor maps of the layer's two caches, the kernel arguments and the grid
@@ -330,10 +339,10 @@ struct KvShape {
 };
 
 int attn_row_tiles(int G, int N);
-// scratch for the partitions' partial results (0 with a single partition)
-size_t attn_scratch_bytes(const AttnShape& s);
+// scratch for the segments' partial results
+size_t attn_scratch_bytes(const AttnShape& s, int sm_count);
 cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t* vis, const uint32_t* used, float* scratch,
-                      AttnPlan* plan, std::string* err);
+                      int sm_count, AttnPlan* plan, std::string* err);
 cudaError_t launch_attn(const AttnPlan& plan, cudaStream_t st);
 cudaError_t launch_attn_merge(const AttnPlan& plan, cudaStream_t st);
 cudaError_t launch_kv_write(const KvLayers& L, const KvShape& s, int n_layers, cudaStream_t st);
