@@ -2,7 +2,7 @@
 // governs attention and publication" (grouped query heads share staged KV tiles; split-K context
 // partitions) and Sec. "State and the execution boundary" (the visibility relation).
 //
-// tree_attn_kernel: persistent, warp-specialised, one CTA per SM.  The work is the list of 64-key tiles
+// tree_attn_kernel: persistent, warp-specialised, one CTA per SM.  The work is the list of 128-key tiles
 // of all (sequence, KV head, 128-row query tile) units in order; a CTA takes a contiguous share of that
 // list (or, with an explicit partition count, one partition of one unit), and every maximal piece of
 // its share that lies in one unit is a SEGMENT: one flash-attention pass whose normalised output and
@@ -11,18 +11,22 @@
 // so a staged key/value tile serves the whole group.
 //
 //   warp 0     producer: TMA loads of K and V tiles (4-d tensor maps, 128-byte swizzle) into a ring of
-//              four stages, one mbarrier pair (full / empty) per stage
-//   warp 1     tensor-core issuer: S = Q K^T into one of two S buffers in tensor memory (M 128, N 64,
-//              K 128), and O += P V (M 128, N 2 x 64, K 64; V is the MN-major B operand as it lies in
+//              three 64 KB stages, one mbarrier pair (full / empty) per stage
+//   warp 1     tensor-core issuer: S = Q K^T into one of two S buffers in tensor memory (M 128, N 128,
+//              K 128), and O += P V (M 128, N 128, K 128; V is the MN-major B operand as it lies in
 //              memory) into a 128-column accumulator that stays in tensor memory for the whole segment;
-//              the next tile's S product is issued before this tile's P is awaited
-//   warps 2-5  softmax: thread = query row = tensor-memory lane.  Reads the 64 logits, applies visibility
-//              by selection (never by arithmetic on a masked logit), exponentiates against a REFERENCE
-//              maximum m, rounds to bf16 and stores P as the next A operand.  m is the row maximum of
-//              the first tile and moves only when a later maximum exceeds it by more than 2^16; only
-//              then is the accumulator rescaled in tensor memory (probabilities up to 2^16 are exact
-//              enough in bf16/fp32: the exponent range is that of fp32).  At the end of a segment the
-//              same threads read O, divide by the row sum and write the slot.
+//              the next tile's S product is issued before this tile's P is awaited.  Both A operands (Q and
+//              P) live in tensor memory, so shared memory carries only the staged K and V tiles.  (Measured:
+//              an N = 128 product issues at the tensor core's full rate, an N = 64 one at 70 % of it.)
+//   warps 2-9  softmax: a query row (= tensor-memory lane) is shared by two threads (warps w and w + 4),
+//              64 keys each.  A thread reads its logits, applies visibility by selection (never by
+//              arithmetic on a masked logit), exponentiates against a REFERENCE maximum m, rounds to bf16
+//              and stores P over the S buffer as the next A operand.  m is the row maximum of the first
+//              tile and moves only when a later maximum exceeds it by more than 2^16; only then is the
+//              accumulator rescaled in tensor memory (probabilities up to 2^16 are harmless: bf16 and fp32
+//              share their exponent range).  The two threads of a row exchange their tile maxima through
+//              shared memory and a 64-thread named barrier, so both take the same decision.  At the end of
+//              a segment each reads its 64 columns of O, divides by the row sum and writes the slot.
 //
 // Only tiles that reach past the committed context need a mask; the mask of node i over the physical
 // suffix is a bit row built with the tree descriptor.  Value rows of positions nobody may read (padding
@@ -44,13 +48,15 @@ namespace {
 
 constexpr int kDh = 128;
 constexpr int kRows = 128;            // query rows per unit = tensor-memory lanes
-constexpr int kKeys = 64;             // keys per tile
-constexpr int kThreads = 192;         // producer warp, issuer warp, four softmax warps
-constexpr int kSoftmaxThreads = 128;
-constexpr int kStages = 4;
-constexpr int kTmemCols = 256;        // S buffers: columns 0..63 and 64..127, O: 128..255
-constexpr int kColO = 128;
-constexpr int kMinTilesPerCta = 8;    // automatic mode: do not cut the work finer than this
+constexpr int kKeys = 128;            // keys per tile
+constexpr int kSoftmaxWarps = 8;
+constexpr int kThreads = 64 + 32 * kSoftmaxWarps;   // producer warp, issuer warp, eight softmax warps
+constexpr int kStages = 3;
+constexpr int kTmemCols = 512;        // S buffers: columns 0..127 and 128..255 (P overwrites the first 64 columns of its S
+                                      // buffer), O: 256..383, Q (bf16 pairs): 384..447; power-of-two allocation
+constexpr int kColO = 256;
+constexpr int kColQ = 384;
+constexpr int kMinTilesPerCta = 4;    // automatic mode: do not cut the work finer than this
 constexpr float kRescaleStep = 16.f;  // the reference maximum moves when exceeded by more than this (log2 units)
 constexpr uint32_t kSpinLimit = 1u << 24;
 constexpr float kLog2e = 1.4426950408889634f;
@@ -58,20 +64,20 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 // shared memory map; the dynamic segment starts at offset 0 of the CTA's window (no static shared
 // variables in this kernel), which the 128-byte swizzle needs 1024-aligned; checked at run time
-constexpr int kOffQ = 0;              // 2 halves of dh x [128 rows x 128 B]
-constexpr int kOffP = 32768;          // 2 buffers x [128 rows x 128 B] probabilities, bf16
-constexpr int kOffKV = 65536;         // per stage: K 2 halves x [64 keys x 128 B], then V the same
-constexpr int kStageBytes = 32768;
+constexpr int kOffKV = 0;             // per stage: K as 2 halves of dh x [128 keys x 128 B], then V the same
+constexpr int kHalfBytes = 16384;
+constexpr int kStageBytes = 4 * kHalfBytes;
 constexpr int kOffSmall = kOffKV + kStages * kStageBytes;   // 196608
 struct Small {
   unsigned long long kv_full[kStages], kv_empty[kStages];
-  unsigned long long s_full[2], p_full[2], p_empty[2];
+  unsigned long long s_full[2], p_full[2];
   unsigned long long q_full, o_free;
   uint32_t tmem_base;
   uint32_t timed_out;
+  float xchg[2][2][kRows];           // [tile parity][key half][row]: row maxima (and row sums at a segment's end)
 };
-constexpr int kSmemBytes = kOffSmall + 256;
-static_assert(sizeof(Small) <= 256, "small block");
+constexpr int kSmemBytes = kOffSmall + 2560;
+static_assert(sizeof(Small) <= 2560, "small block");
 static_assert(kSmemBytes + 1024 <= 227 * 1024, "one CTA per SM");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -130,6 +136,13 @@ __device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a, uint64_t b, ui
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
       ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
 }
+// same product with the A operand in tensor memory (row = lane, two bf16 per 32-bit column, K-major)
+__device__ __forceinline__ void umma_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}\n"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -145,10 +158,6 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
   return y;
-}
-// byte offset of 16-byte chunk `chunk` (0..7) of row `row` in a 128-byte-swizzled tile of 128-byte rows
-__device__ __forceinline__ uint32_t sw128(int row, int chunk) {
-  return (uint32_t)((row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
@@ -284,11 +293,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     for (int s = 0; s < kStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sm.s_full[s], 1);
-      mbar_init(&sm.p_full[s], kSoftmaxThreads);
-      mbar_init(&sm.p_empty[s], 1);
+      mbar_init(&sm.p_full[s], kSoftmaxWarps);   // one arrival per softmax warp
     }
-    mbar_init(&sm.q_full, kSoftmaxThreads);
-    mbar_init(&sm.o_free, kSoftmaxThreads);
+    mbar_init(&sm.q_full, kSoftmaxWarps);
+    mbar_init(&sm.o_free, kSoftmaxWarps);
     sm.timed_out = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
@@ -300,7 +308,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   Work work(a);
   Segment sg;
   bool ok = aligned;
-  uint32_t it = 0;        // tiles this CTA has started, over all segments: ring stage, S / P buffer and phases
+  uint32_t it = 0;        // tiles this CTA has started, over all segments: ring stage, S buffer and phases
   uint32_t nseg = 0;      // segments with tiles so far: phases of q_full and o_free
 
   if (warp == 0) {
@@ -315,9 +323,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           const uint32_t dst = sbase + kOffKV + st * kStageBytes;
           const int pos = (sg.t0 + j) * kKeys;
           tma_load_4d(dst, &tm_k, &sm.kv_full[st], 0, sg.hkv, pos, sg.crow);
-          tma_load_4d(dst + 8192, &tm_k, &sm.kv_full[st], 64, sg.hkv, pos, sg.crow);
-          tma_load_4d(dst + 16384, &tm_v, &sm.kv_full[st], 0, sg.hkv, pos, sg.crow);
-          tma_load_4d(dst + 24576, &tm_v, &sm.kv_full[st], 64, sg.hkv, pos, sg.crow);
+          tma_load_4d(dst + kHalfBytes, &tm_k, &sm.kv_full[st], 64, sg.hkv, pos, sg.crow);
+          tma_load_4d(dst + 2 * kHalfBytes, &tm_v, &sm.kv_full[st], 0, sg.hkv, pos, sg.crow);
+          tma_load_4d(dst + 3 * kHalfBytes, &tm_v, &sm.kv_full[st], 64, sg.hkv, pos, sg.crow);
         }
       }
       if (!ok) sm.timed_out = 1u;
@@ -325,28 +333,26 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   } else if (warp == 1) {
     // ---------------- tensor-core issuer ----------------
     if (lane == 0) {
+      // S = Q K^T: A = Q in tensor memory, B = K tile (K-major: 128 key rows of 128 B per dh half)
       auto issue_qk = [&](uint32_t t) {
         constexpr uint32_t id = umma_idesc(kRows, kKeys, 0, 0);
         const uint32_t kb = sbase + kOffKV + (t % kStages) * kStageBytes;
-        const uint32_t d = tmem + (t & 1u) * 64;
+        const uint32_t d = tmem + (t & 1u) * kKeys;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma(d, umma_desc(sbase + kOffQ + (ks >> 2) * 16384 + (ks & 3) * 32, 16, 1024),
-               umma_desc(kb + (ks >> 2) * 8192 + (ks & 3) * 32, 16, 1024), id, ks ? 1u : 0u);
+        for (int ks = 0; ks < kDh / 16; ++ks)
+          umma_ta(d, tmem + kColQ + ks * 8, umma_desc(kb + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024), id, ks ? 1u : 0u);
         umma_commit(&sm.s_full[t & 1u]);
       };
+      // O += P V: A = P in tensor memory (over the S buffer), B = V tile as it lies in memory (MN-major:
+      // 128 B of dh per key row, the two dh halves kHalfBytes apart, 16 keys = 2048 B per K step)
       auto issue_pv = [&](uint32_t t, bool first) {
-        constexpr uint32_t id = umma_idesc(kRows, 64, 0, 1);
-        const uint32_t vb = sbase + kOffKV + (t % kStages) * kStageBytes + 16384;
-        const uint32_t pb = sbase + kOffP + (t & 1u) * 16384;
+        constexpr uint32_t id = umma_idesc(kRows, kDh, 0, 1);
+        const uint32_t vb = sbase + kOffKV + (t % kStages) * kStageBytes + 2 * kHalfBytes;
+        const uint32_t pa = tmem + (t & 1u) * kKeys;
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh)
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks)
-            umma(tmem + kColO + hh * 64, umma_desc(pb + ks * 32, 16, 1024), umma_desc(vb + hh * 8192 + ks * 2048, 8192, 1024),
-                 id, (first && ks == 0) ? 0u : 1u);
-        umma_commit(&sm.kv_empty[t % kStages]);
-        umma_commit(&sm.p_empty[t & 1u]);
+        for (int ks = 0; ks < kKeys / 16; ++ks)
+          umma_ta(tmem + kColO, pa + ks * 8, umma_desc(vb + ks * 2048, kHalfBytes, 1024), id, (first && ks == 0) ? 0u : 1u);
+        umma_commit(&sm.kv_empty[t % kStages]);   // also "this tile's O product has completed" for the softmax warps
       };
       while (work.next(&sg)) {
         if (sg.n == 0) continue;
@@ -373,51 +379,58 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     }
   } else {
     // ---------------- softmax warps ----------------
+    // Warps w and w + 4 share the 32 rows of one lane quarter; the first takes keys 0..63 of every tile
+    // and output columns 0..63, the second the other halves.
+    const int sw = warp - 2;                     // 0..7
+    const int half = sw >> 2;
     const int row = 32 * (warp & 3) + lane;      // tensor-memory lane this warp may touch
-    const int sthread = tid - 64;                // 0..127
+    const int sthread = tid - 64;                // 0..255
     const uint32_t tmem_lane = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
+    const int pair_bar = 1 + (warp & 3);         // named barrier of the two warps of a lane quarter
     const float sl2 = a.scale_log2;
     const int GN = a.G * a.N;
     while (work.next(&sg)) {
       const int rg = sg.rt * kRows + row;
       const bool row_ok = rg < GN;
       const int hl = row_ok ? rg / a.N : 0, node = row_ok ? rg - hl * a.N : 0;
-      float* slot_o = a.part_o + ((size_t)sg.slot * kRows + row) * kDh;
+      float* slot_o = a.part_o + ((size_t)sg.slot * kRows + row) * kDh + half * 64;
       float* slot_l = a.part_lse + (size_t)sg.slot * kRows + row;
       if (sg.n == 0) {                           // empty partition (fixed mode): an empty slot
         if (row_ok) {
-          for (int e = 0; e < kDh / 4; ++e) reinterpret_cast<float4*>(slot_o)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-          *slot_l = -INFINITY;
+          for (int e = 0; e < 16; ++e) reinterpret_cast<float4*>(slot_o)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (half == 0) *slot_l = -INFINITY;
         }
         continue;
       }
-      // query tile: 128 rows x 16 chunks of 16 bytes, zero rows beyond the group.  The previous segment's
-      // S products have all completed (their s_full phases were awaited), so the tile may be replaced.
-      for (int c = sthread; c < kRows * 16; c += kSoftmaxThreads) {
-        const int r = c >> 4, ch = c & 15;
-        const int g = sg.rt * kRows + r;
-        uint4 val = make_uint4(0u, 0u, 0u, 0u);
-        if (g < GN) {
-          const int h = g / a.N, i = g - h * a.N;
-          val = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
-                                                      ((((size_t)sg.b * a.N + i) * a.Hq + (size_t)sg.hkv * a.G + h) * kDh + ch * 8)));
+      // query tile into tensor memory: this thread's half of its row, two bf16 per column (zeros beyond the
+      // group).  The previous segment's S products have all completed (their s_full phases were awaited).
+      {
+        const uint4* qrow = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
+                                                           (((size_t)sg.b * a.N + node) * a.Hq + (size_t)sg.hkv * a.G + hl) * kDh);
+        uint32_t qr[32];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const uint4 v = row_ok ? __ldg(qrow + half * 8 + c) : make_uint4(0u, 0u, 0u, 0u);
+          qr[4 * c] = v.x; qr[4 * c + 1] = v.y; qr[4 * c + 2] = v.z; qr[4 * c + 3] = v.w;
         }
-        *reinterpret_cast<uint4*>(smem + kOffQ + (ch >> 3) * 16384 + sw128(r, ch & 7)) = val;
+        tmem_st32(tmem_lane + kColQ + half * 32, qr);
+        tmem_st_wait();
       }
-      fence_async_proxy();
-      mbar_arrive(&sm.q_full);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.q_full);
 
       const uint32_t* visw = a.vis + ((size_t)sg.b * a.N + node) * 8;
       const uint32_t* usedw = a.used + (size_t)sg.b * 8;
-      float m = -INFINITY, l = 0.f;              // reference maximum (log2 units), row sum against it
+      float m = -INFINITY, l = 0.f;              // reference maximum (log2 units), this thread's part of the row sum
       for (int j = 0; j < sg.n; ++j, ++it) {
         const uint32_t buf = it & 1u;
-        const int kpos0 = (sg.t0 + j) * kKeys;
-        const bool tail = kpos0 + kKeys > sg.ctx;    // uniform: the tile reaches past the committed context
+        const int kpos0 = (sg.t0 + j) * kKeys + half * 64;   // first key of this thread's 64
+        const bool tail = (sg.t0 + j + 1) * kKeys > sg.ctx;  // uniform: the tile reaches past the committed context
         unsigned long long vm = ~0ull;
         if (tail) {
           vm = 0ull;
-          for (int c = 0; c < kKeys; ++c) {
+          for (int c = 0; c < 64; ++c) {
             const int p = kpos0 + c;
             bool v = p < sg.ctx;
             if (!v) {
@@ -431,93 +444,97 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         tc_fence_after();
         __syncwarp();
         uint32_t sr[64];
-        tmem_ld32(tmem_lane + buf * 64, sr);
-        tmem_ld32(tmem_lane + buf * 64 + 32, sr + 32);
+        tmem_ld32(tmem_lane + buf * kKeys + half * 64, sr);
+        tmem_ld32(tmem_lane + buf * kKeys + half * 64 + 32, sr + 32);
         tmem_ld_wait();
-        float mx = -INFINITY;
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         if (!tail) {
 #pragma unroll
-          for (int e = 0; e < 64; ++e) mx = fmaxf(mx, __uint_as_float(sr[e]));
+          for (int e = 0; e < 64; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(sr[e]));
         } else {
 #pragma unroll
-          for (int e = 0; e < 64; ++e) mx = fmaxf(mx, ((vm >> e) & 1ull) ? __uint_as_float(sr[e]) : -INFINITY);
+          for (int e = 0; e < 64; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], ((vm >> e) & 1ull) ? __uint_as_float(sr[e]) : -INFINITY);
         }
-        mx *= sl2;
+        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;
+        // the row maximum of the tile: exchange with the thread that holds the other 64 keys
+        sm.xchg[buf][half][row] = mx;
+        asm volatile("bar.sync %0, 64;\n" ::"r"(pair_bar) : "memory");
+        mx = fmaxf(mx, sm.xchg[buf][half ^ 1][row]);
         // reference maximum: set by the first tile that shows the row a key; moved (with a rescale of the
-        // accumulator) only when exceeded by more than kRescaleStep
+        // accumulator) only when exceeded by more than kRescaleStep.  Both threads of a row decide alike.
         float corr = 1.f;
         if (m == -INFINITY) m = mx;
         else if (mx > m + kRescaleStep) { corr = ex2(m - mx); m = mx; }
         if (__any_sync(0xffffffffu, corr != 1.f)) {
-          // O still holds the products up to the previous tile: wait for them, then scale this warp's rows
-          if (ok) ok = mbar_wait(&sm.p_empty[(it - 1) & 1u], ((it - 1) >> 1) & 1u);
+          // O still holds the products up to the previous tile: wait for them, then scale this thread's columns
+          if (ok) ok = mbar_wait(&sm.kv_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
           tc_fence_after();
           __syncwarp();
 #pragma unroll 1
-          for (int c = 0; c < kDh; c += 32) {
+          for (int c = 0; c < 64; c += 32) {
             uint32_t orr[32];
-            tmem_ld32(tmem_lane + kColO + c, orr);
+            tmem_ld32(tmem_lane + kColO + half * 64 + c, orr);
             tmem_ld_wait();
 #pragma unroll
             for (int e = 0; e < 32; ++e) orr[e] = __float_as_uint(__uint_as_float(orr[e]) * corr);
-            tmem_st32(tmem_lane + kColO + c, orr);
+            tmem_st32(tmem_lane + kColO + half * 64 + c, orr);
           }
           tmem_st_wait();
           l *= corr;
         }
         const float mu = m == -INFINITY ? 0.f : m;
-        // P buffer `buf` was last read by the O product of tile it - 2
-        if (it >= 2 && ok) ok = mbar_wait(&sm.p_empty[buf], ((it - 2) >> 1) & 1u);
-        unsigned char* prow = smem + kOffP + buf * 16384;
-        float lsum = 0.f;
+        // P goes over the first 64 columns of this S buffer, 32 per thread.  The second thread's share lies in
+        // columns the first thread read its logits from: it has finished (its loads completed before the pair
+        // barrier above).  The S product of tile it + 2 is issued behind the O product that reads P.
+        uint32_t pk[32];
+        float ls4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int ch = 0; ch < 8; ++ch) {
-          uint32_t pk[4];
-#pragma unroll
-          for (int e = 0; e < 8; e += 2) {
-            const int c = ch * 8 + e;
-            float p0 = ex2(fmaf(__uint_as_float(sr[c]), sl2, -mu));
-            float p1 = ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -mu));
-            if (tail) {
-              p0 = ((vm >> c) & 1ull) ? p0 : 0.f;
-              p1 = ((vm >> (c + 1)) & 1ull) ? p1 : 0.f;
-            }
-            lsum += p0 + p1;
-            pk[e >> 1] = pack_bf16(p0, p1);
+        for (int c = 0; c < 64; c += 2) {
+          float p0 = ex2(fmaf(__uint_as_float(sr[c]), sl2, -mu));
+          float p1 = ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -mu));
+          if (tail) {
+            p0 = ((vm >> c) & 1ull) ? p0 : 0.f;
+            p1 = ((vm >> (c + 1)) & 1ull) ? p1 : 0.f;
           }
-          *reinterpret_cast<uint4*>(prow + sw128(row, ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          ls4[(c >> 1) & 3] += p0 + p1;
+          pk[c >> 1] = pack_bf16(p0, p1);
         }
-        l += lsum;
+        l += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
+        tmem_st32(tmem_lane + buf * kKeys + half * 32, pk);
         if (tail) {
           // value rows nobody may read: zero them in the staged tile (two 128-byte rows per key)
           const uint32_t st = it % kStages;
           if (ok) ok = mbar_wait(&sm.kv_full[st], (it / kStages) & 1u);
           const int c = sthread >> 1, hh = sthread & 1;
-          const int p = kpos0 + c;
+          const int p = (sg.t0 + j) * kKeys + c;
           bool dead = false;
           if (p >= sg.ctx) {
             const int s = p - sg.ctx;
             dead = s >= a.Ns || !((__ldg(usedw + (s >> 5)) >> (s & 31)) & 1u);
           }
           if (dead) {
-            uint4* vrow = reinterpret_cast<uint4*>(smem + kOffKV + st * kStageBytes + 16384 + hh * 8192 + c * 128);
+            uint4* vrow = reinterpret_cast<uint4*>(smem + kOffKV + st * kStageBytes + (2 + hh) * kHalfBytes + c * 128);
 #pragma unroll
             for (int e = 0; e < 8; ++e) vrow[e] = make_uint4(0u, 0u, 0u, 0u);
           }
+          fence_async_proxy();                   // for the tensor core's reads
         }
-        fence_async_proxy();
+        tmem_st_wait();
         tc_fence_before();
-        mbar_arrive(&sm.p_full[buf]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.p_full[buf]);
       }
       // end of the segment: the last O product, then normalise and write the slot
-      if (ok) ok = mbar_wait(&sm.p_empty[(it - 1) & 1u], ((it - 1) >> 1) & 1u);
+      if (ok) ok = mbar_wait(&sm.kv_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
       tc_fence_after();
-      __syncwarp();
-      const float inv = l > 0.f ? 1.f / l : 0.f;
+      sm.xchg[0][half][row] = l;
+      asm volatile("bar.sync %0, 64;\n" ::"r"(pair_bar) : "memory");
+      const float lt = sm.xchg[0][0][row] + sm.xchg[0][1][row];
+      const float inv = lt > 0.f ? 1.f / lt : 0.f;
 #pragma unroll 1
-      for (int c = 0; c < kDh; c += 32) {
+      for (int c = 0; c < 64; c += 32) {
         uint32_t orr[32];
-        tmem_ld32(tmem_lane + kColO + c, orr);
+        tmem_ld32(tmem_lane + kColO + half * 64 + c, orr);
         tmem_ld_wait();
         if (row_ok) {
 #pragma unroll
@@ -527,9 +544,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                             __uint_as_float(orr[e + 2]) * inv, __uint_as_float(orr[e + 3]) * inv);
         }
       }
-      if (row_ok) *slot_l = l > 0.f ? m + log2f(l) : -INFINITY;
+      if (row_ok && half == 0) *slot_l = lt > 0.f ? m + log2f(lt) : -INFINITY;
       tc_fence_before();
-      mbar_arrive(&sm.o_free);
+      asm volatile("bar.sync %0, 64;\n" ::"r"(pair_bar) : "memory");   // the partner has read xchg[0] before the next segment writes it
+      if (lane == 0) mbar_arrive(&sm.o_free);
       ++nseg;
     }
     if (!ok) sm.timed_out = 1u;
@@ -625,7 +643,7 @@ cudaError_t encode_cache_map(void* cache, int Hkv, int max_pos, int n_rows, CUte
   }
   const cuuint64_t dims[4] = {(cuuint64_t)kDh, (cuuint64_t)Hkv, (cuuint64_t)max_pos, (cuuint64_t)n_rows};
   const cuuint64_t strides[3] = {(cuuint64_t)kDh * 2, (cuuint64_t)Hkv * kDh * 2, (cuuint64_t)max_pos * Hkv * kDh * 2};
-  const cuuint32_t box[4] = {64, 1, (cuuint32_t)kKeys, 1};
+  const cuuint32_t box[4] = {64, 1, (cuuint32_t)kKeys, 1};   // 16 KB
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
