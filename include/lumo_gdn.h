@@ -339,7 +339,8 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
  * attention visibility relation selects the same logical prefix and ancestry as the recurrent path;
  * Algorithm 1, "Remap the accepted KV entries using the same logical-to-physical slot map").
  *
- * KV cache of one layer: k_cache, v_cache [n_cache_rows, max_positions, Hkv, dh] bf16.  Sequence b
+ * KV cache of one layer: k_cache, v_cache [n_cache_rows, max_positions, Hkv, dh] bf16 (or with the
+ * head and position axes swapped, see kv_layout).  Sequence b
  * owns row cache_row[b]; positions [0, ctx_len[b]) hold the committed context, and the entry of tree
  * node i lives at position ctx_len[b] + slot[b][i] (the candidates occupy the physical suffix in slot
  * order; a spine-first slot map makes the principal chain contiguous there).  Queries and outputs
@@ -366,6 +367,9 @@ typedef struct {
   const void* v_new;
   float* out;               /* [B, N, Hq, dh] fp32 (tree attention) */
   float* lse;               /* [B, N, Hq] fp32 natural-log sum of exp of the logits; may be NULL */
+  int32_t kv_layout;        /* 0: caches are [n_cache_rows, max_positions, Hkv, dh] (a position's heads adjacent);
+                               1: [n_cache_rows, Hkv, max_positions, dh] (a head's positions adjacent: a tile of keys is
+                               one contiguous 32 KB run, which the attention kernel reads at a higher HBM efficiency) */
   int32_t n_splits;         /* partitions of the key range per (sequence, KV head): 0 = chosen to fill the GPU,
                                else 1..32 (Sec. "Evaluation Setup": the paper's deployment used 4) */
   int32_t* status;          /* [B] lumo_seq_status; may be NULL */

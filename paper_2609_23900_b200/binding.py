@@ -88,7 +88,7 @@ class _AttnArgs(ctypes.Structure):
                 ("ctx_len", ctypes.c_void_p), ("cache_row", ctypes.c_void_p),
                 ("q", ctypes.c_void_p), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
                 ("out", ctypes.c_void_p), ("lse", ctypes.c_void_p),
-                ("n_splits", ctypes.c_int32), ("status", ctypes.c_void_p)]
+                ("kv_layout", ctypes.c_int32), ("n_splits", ctypes.c_int32), ("status", ctypes.c_void_p)]
 
 
 _lib.lumo_ctx_create.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
@@ -381,13 +381,14 @@ class AttnLayer:
     """lumo_attn_args for one full-attention layer; keeps the tensors alive."""
 
     def __init__(self, *, Hq: int, Hkv: int, k_cache, v_cache, ctx_len, cache_row, scale: float, q=None, k_new=None,
-                 v_new=None, out=None, lse=None, n_splits: int = 0, status=None):
+                 v_new=None, out=None, lse=None, n_splits: int = 0, status=None, kv_layout: int = 0):
+        """kv_layout 0: caches are [rows, positions, Hkv, dh]; 1: [rows, Hkv, positions, dh]."""
         self.tensors = dict(k_cache=k_cache, v_cache=v_cache, ctx_len=ctx_len, cache_row=cache_row, q=q, k_new=k_new,
                             v_new=v_new, out=out, lse=lse, status=status)
         if k_cache.dtype != torch.bfloat16 or v_cache.dtype != torch.bfloat16 or k_cache.shape != v_cache.shape:
             raise ValueError("k_cache and v_cache must be bfloat16 tensors of one shape [rows, positions, Hkv, dh]")
-        if k_cache.dim() != 4 or k_cache.shape[2] != Hkv:
-            raise ValueError("cache shape must be [rows, positions, Hkv, dh]")
+        if k_cache.dim() != 4 or k_cache.shape[1 if kv_layout else 2] != Hkv:
+            raise ValueError("cache shape must be [rows, positions, Hkv, dh] (layout 0) or [rows, Hkv, positions, dh] (layout 1)")
         for name in ("q", "k_new", "v_new"):
             t = self.tensors[name]
             if t is not None and t.dtype != torch.bfloat16:
@@ -402,8 +403,9 @@ class AttnLayer:
                 raise ValueError(f"{name} must be int32")
         a = _AttnArgs()
         a.Hq, a.Hkv, a.dh, a.scale = int(Hq), int(Hkv), int(k_cache.shape[3]), float(scale)
-        a.n_cache_rows, a.max_positions = int(k_cache.shape[0]), int(k_cache.shape[1])
+        a.n_cache_rows, a.max_positions = int(k_cache.shape[0]), int(k_cache.shape[2 if kv_layout else 1])
         a.n_splits = int(n_splits)
+        a.kv_layout = int(kv_layout)
         for name in self.tensors:
             setattr(a, name, _ptr(self.tensors[name]))
         self.args = a

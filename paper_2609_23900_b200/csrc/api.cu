@@ -705,13 +705,17 @@ int prepare_attn(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args
   if ((long long)a0.max_positions * a0.Hkv * a0.dh * 2 >= (1LL << 40))
     return fail(ctx, LUMO_ERR_UNSUPPORTED, "a cache row must span less than 2^40 bytes");
   if (!a0.ctx_len || !a0.cache_row) return fail(ctx, LUMO_ERR_ARG, "ctx_len and cache_row are required");
+  // the kernels count key tiles of all (sequence, KV head, row tile) units in 32 bits
+  if ((double)desc->B * a0.Hkv * attn_row_tiles(a0.Hq / a0.Hkv, desc->N) * ((double)a0.max_positions / 128 + 1) >= 2147483648.0)
+    return fail(ctx, LUMO_ERR_UNSUPPORTED, "batch x KV heads x positions too large for one call");
+  if (a0.kv_layout != 0 && a0.kv_layout != 1) return fail(ctx, LUMO_ERR_ARG, "kv_layout must be 0 or 1");
   if (a0.n_splits < 0 || a0.n_splits > 32) return fail(ctx, LUMO_ERR_ARG, "n_splits must be 0 (automatic) or in [1, 32]");
   for (int l = 0; l < n_layers; ++l) {
     const lumo_attn_args& a = layers[l];
     const std::string at = " (layer " + std::to_string(l) + ")";
     if (a.Hq != a0.Hq || a.Hkv != a0.Hkv || a.dh != a0.dh || a.scale != a0.scale || a.n_cache_rows != a0.n_cache_rows ||
         a.max_positions != a0.max_positions || a.ctx_len != a0.ctx_len || a.cache_row != a0.cache_row ||
-        a.n_splits != a0.n_splits)
+        a.n_splits != a0.n_splits || a.kv_layout != a0.kv_layout)
       return fail(ctx, LUMO_ERR_ARG, "all layers must share shapes, options, ctx_len and cache_row" + at);
     if (!a.k_cache || !a.v_cache) return fail(ctx, LUMO_ERR_ARG, "k_cache and v_cache are required" + at);
     for (const void* p : {(const void*)a.k_cache, (const void*)a.v_cache, a.q, a.k_new, a.v_new, (const void*)a.out})
@@ -721,6 +725,7 @@ int prepare_attn(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args
   s->n_rows = a0.n_cache_rows; s->max_pos = a0.max_positions; s->scale = a0.scale;
   s->ctx_len = a0.ctx_len; s->cache_row = a0.cache_row;
   s->S = a0.n_splits;
+  s->layout = a0.kv_layout;
   return LUMO_OK;
 }
 
@@ -731,7 +736,7 @@ void kv_views(const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_la
     L->kn[l] = layers[l].k_new; L->vn[l] = layers[l].v_new;
     L->status[l] = layers[l].status;
   }
-  k->B = s.B; k->N = s.N; k->Ns = s.Ns; k->Hkv = s.Hkv; k->n_rows = s.n_rows; k->max_pos = s.max_pos;
+  k->B = s.B; k->N = s.N; k->Ns = s.Ns; k->Hkv = s.Hkv; k->n_rows = s.n_rows; k->max_pos = s.max_pos; k->layout = s.layout;
   k->ctx_len = s.ctx_len; k->cache_row = s.cache_row; k->parent = desc->d_parent; k->slot = desc->d_slot;
 }
 

@@ -10,18 +10,19 @@
 // The query rows of all heads that share the KV head sit in one tile (row = head-in-group * N + node),
 // so a staged key/value tile serves the whole group.
 //
-//   warp 0     producer: TMA loads of K and V tiles (4-d tensor maps, 128-byte swizzle) into a ring of
-//              three 64 KB stages, one mbarrier pair (full / empty) per stage
-//   warp 1     tensor-core issuer: S = Q K^T into one of two S buffers in tensor memory (M 128, N 128,
+//   warps 0-1  producers: TMA loads (4-d tensor maps, 128-byte swizzle) of K tiles into one ring of three
+//              32 KB stages and of V tiles into another, one mbarrier pair (full / empty) per stage; a K
+//              stage is free as soon as its S product has completed, long before the V stage of that tile
+//   warp 2     tensor-core issuer: S = Q K^T into one of two S buffers in tensor memory (M 128, N 128,
 //              K 128), and O += P V (M 128, N 128, K 128; V is the MN-major B operand as it lies in
 //              memory) into a 128-column accumulator that stays in tensor memory for the whole segment;
-//              the next tile's S product is issued before this tile's P is awaited.  Both A operands (Q and
-//              P) live in tensor memory, so shared memory carries only the staged K and V tiles.  (Measured:
+//              the S products run two tiles ahead of the O products, so the softmax warps never wait for
+//              logits.  Both A operands (Q and P) live in tensor memory, so shared memory carries only the staged K and V tiles.  (Measured:
 //              an N = 128 product issues at the tensor core's full rate, an N = 64 one at 70 % of it.)
-//   warps 2-9  softmax: a query row (= tensor-memory lane) is shared by two threads (warps w and w + 4),
+//   warps 3-10 softmax: a query row (= tensor-memory lane) is shared by two threads (warps w and w + 4),
 //              64 keys each.  A thread reads its logits, applies visibility by selection (never by
 //              arithmetic on a masked logit), exponentiates against a REFERENCE maximum m, rounds to bf16
-//              and stores P over the S buffer as the next A operand.  m is the row maximum of the first
+//              and stores P as the next A operand.  m is the row maximum of the first
 //              tile and moves only when a later maximum exceeds it by more than 2^16; only then is the
 //              accumulator rescaled in tensor memory (probabilities up to 2^16 are harmless: bf16 and fp32
 //              share their exponent range).  The two threads of a row exchange their tile maxima through
@@ -50,12 +51,14 @@ constexpr int kDh = 128;
 constexpr int kRows = 128;            // query rows per unit = tensor-memory lanes
 constexpr int kKeys = 128;            // keys per tile
 constexpr int kSoftmaxWarps = 8;
-constexpr int kThreads = 64 + 32 * kSoftmaxWarps;   // producer warp, issuer warp, eight softmax warps
-constexpr int kStages = 3;
-constexpr int kTmemCols = 512;        // S buffers: columns 0..127 and 128..255 (P overwrites the first 64 columns of its S
-                                      // buffer), O: 256..383, Q (bf16 pairs): 384..447; power-of-two allocation
+constexpr int kFirstSoftmaxWarp = 3;
+constexpr int kThreads = 32 * (kFirstSoftmaxWarp + kSoftmaxWarps);   // K producer, V producer, issuer, eight softmax warps
+constexpr int kStages = 3;            // per ring (K tiles and V tiles have a ring each)
+constexpr int kTmemCols = 512;        // S buffers: columns 0..127 and 128..255, O: 256..383, Q (bf16 pairs): 384..447,
+                                      // P (bf16 pairs): 448..511
 constexpr int kColO = 256;
 constexpr int kColQ = 384;
+constexpr int kColP = 448;
 constexpr int kMinTilesPerCta = 4;    // automatic mode: do not cut the work finer than this
 constexpr float kRescaleStep = 16.f;  // the reference maximum moves when exceeded by more than this (log2 units)
 constexpr uint32_t kSpinLimit = 1u << 24;
@@ -64,13 +67,14 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 // shared memory map; the dynamic segment starts at offset 0 of the CTA's window (no static shared
 // variables in this kernel), which the 128-byte swizzle needs 1024-aligned; checked at run time
-constexpr int kOffKV = 0;             // per stage: K as 2 halves of dh x [128 keys x 128 B], then V the same
-constexpr int kHalfBytes = 16384;
-constexpr int kStageBytes = 4 * kHalfBytes;
-constexpr int kOffSmall = kOffKV + kStages * kStageBytes;   // 196608
+constexpr int kHalfBytes = 16384;     // one dh half of a tile: [128 keys x 128 B]
+constexpr int kTileBytes = 2 * kHalfBytes;
+constexpr int kOffK = 0;              // K ring
+constexpr int kOffV = kStages * kTileBytes;
+constexpr int kOffSmall = 2 * kStages * kTileBytes;   // 196608
 struct Small {
-  unsigned long long kv_full[kStages], kv_empty[kStages];
-  unsigned long long s_full[2], p_full[2];
+  unsigned long long k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
+  unsigned long long s_full[2], p_full;
   unsigned long long q_full, o_free;
   uint32_t tmem_base;
   uint32_t timed_out;
@@ -104,6 +108,17 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
     if (done) return true;
   }
   return false;
+}
+
+// single poll
+__device__ __forceinline__ bool mbar_test(unsigned long long* bar, uint32_t parity) {
+  uint32_t done;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}\n"
+      : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return done != 0;
 }
 
 // One box of a 4-d tiled tensor map (dh, KV head, position, cache row) into shared memory; completion
@@ -205,40 +220,43 @@ struct Segment {
 struct Work {
   const AttnArgs& a;
   int b, q;           // current sequence, unit within the sequence
-  long long g, g_end; // next global tile, end of this CTA's share
-  long long g_unit;   // global tile at which the current unit starts
+  int g, g_end;       // next global tile, end of this CTA's share (the host bounds the tile count below 2^31)
+  int g_unit;         // global tile at which the current unit starts
   int nt;             // tiles per unit of the current sequence
   bool fixed_done;
 
-  __device__ int tiles_of(int bb, int* ctx, int* crow) const {
+  static __device__ __forceinline__ int tiles_of(const AttnArgs& a, int bb, int* ctx, int* crow) {
     *ctx = a.ctx_len[bb];
     *crow = a.cache_row[bb];
     if (seq_check(*ctx, *crow, a.Ns, a.n_rows, a.max_pos) != LUMO_SEQ_OK) return 0;
     return (*ctx + a.Ns + kKeys - 1) / kKeys;
   }
 
-  __device__ explicit Work(const AttnArgs& args) : a(args), b(0), q(0), g(0), g_end(0), g_unit(0), nt(0), fixed_done(false) {
+  __device__ __forceinline__ void init() {
+    b = 0; q = 0; g = 0; g_end = 0; g_unit = 0; nt = 0; fixed_done = false;
     if (a.S > 0) return;
     const int upb = a.Hkv * a.RT;       // units per sequence
-    long long total = 0;
+    int total = 0;
     int cx, cr;
-    for (int bb = 0; bb < a.B; ++bb) total += (long long)tiles_of(bb, &cx, &cr) * upb;
-    long long per = (total + gridDim.x - 1) / gridDim.x;
+    for (int bb = 0; bb < a.B; ++bb) total += tiles_of(a, bb, &cx, &cr) * upb;
+    int per = (total + (int)gridDim.x - 1) / (int)gridDim.x;
     if (per < kMinTilesPerCta) per = kMinTilesPerCta;
-    g = (long long)blockIdx.x * per;
+    g = (int)blockIdx.x * per;
     g_end = g + per < total ? g + per : total;
     // position on the unit that holds tile g
-    long long acc = 0;
+    int acc = 0;
     for (b = 0; b < a.B; ++b) {
-      nt = tiles_of(b, &cx, &cr);
-      const long long span = (long long)nt * upb;
-      if (g < acc + span) { q = (int)((g - acc) / nt); g_unit = acc + (long long)q * nt; break; }
+      nt = tiles_of(a, b, &cx, &cr);
+      const int span = nt * upb;
+      if (g < acc + span) { q = (g - acc) / nt; g_unit = acc + q * nt; break; }
       acc += span;
     }
   }
 
+  __device__ explicit Work(const AttnArgs& args) : a(args) { init(); }
+
   // next segment of this CTA; false when the share is exhausted
-  __device__ bool next(Segment* s) {
+  __device__ __forceinline__ bool next(Segment* s) {
     const int upb = a.Hkv * a.RT;
     if (a.S > 0) {
       if (fixed_done) return false;
@@ -247,7 +265,7 @@ struct Work {
       s->b = u / upb;
       const int r = u - s->b * upb;
       s->hkv = r / a.RT; s->rt = r - s->hkv * a.RT;
-      const int n_all = tiles_of(s->b, &s->ctx, &s->crow);
+      const int n_all = tiles_of(a, s->b, &s->ctx, &s->crow);
       s->t0 = (int)(((long long)part * n_all) / a.S);
       s->n = (int)(((long long)(part + 1) * n_all) / a.S) - s->t0;
       s->slot = blockIdx.x;
@@ -259,16 +277,16 @@ struct Work {
         if (nt == 0 || ++q == upb) {
           q = 0;
           int cx, cr;
-          do { ++b; nt = b < a.B ? tiles_of(b, &cx, &cr) : 0; } while (b < a.B && nt == 0);
+          do { ++b; nt = b < a.B ? tiles_of(a, b, &cx, &cr) : 0; } while (b < a.B && nt == 0);
         }
         continue;
       }
       const int u = b * upb + q;
       s->b = b; s->hkv = q / a.RT; s->rt = q - s->hkv * a.RT;
-      tiles_of(b, &s->ctx, &s->crow);
-      s->t0 = (int)(g - g_unit);
-      const long long end = g_unit + nt < g_end ? g_unit + nt : g_end;
-      s->n = (int)(end - g);
+      tiles_of(a, b, &s->ctx, &s->crow);
+      s->t0 = g - g_unit;
+      const int end = g_unit + nt < g_end ? g_unit + nt : g_end;
+      s->n = end - g;
       s->slot = u + blockIdx.x;
       g = end;
       return true;
@@ -285,16 +303,18 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const bool aligned = (sbase & 1023u) == 0;   // cannot fail with this file's layout; refuse rather than mis-swizzle
 
-  if (warp == 1) {
+  if (warp == 2) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
   }
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&sm.kv_full[s], 1); mbar_init(&sm.kv_empty[s], 1); }
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&sm.s_full[s], 1);
-      mbar_init(&sm.p_full[s], kSoftmaxWarps);   // one arrival per softmax warp
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sm.k_full[s], 1); mbar_init(&sm.k_empty[s], 1);
+      mbar_init(&sm.v_full[s], 1); mbar_init(&sm.v_empty[s], 1);
     }
+    mbar_init(&sm.s_full[0], 1);
+    mbar_init(&sm.s_full[1], 1);
+    mbar_init(&sm.p_full, kSoftmaxWarps);        // one arrival per softmax warp
     mbar_init(&sm.q_full, kSoftmaxWarps);
     mbar_init(&sm.o_free, kSoftmaxWarps);
     sm.timed_out = 0;
@@ -311,67 +331,78 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   uint32_t it = 0;        // tiles this CTA has started, over all segments: ring stage, S buffer and phases
   uint32_t nseg = 0;      // segments with tiles so far: phases of q_full and o_free
 
-  if (warp == 0) {
-    // ---------------- producer ----------------
+  if (warp < 2) {
+    // ---------------- producers: warp 0 feeds the K ring, warp 1 the V ring ----------------
     if (lane == 0) {
+      const bool is_v = warp == 1;
+      const CUtensorMap* map = is_v ? &tm_v : &tm_k;
+      unsigned long long* full = is_v ? sm.v_full : sm.k_full;
+      unsigned long long* empty = is_v ? sm.v_empty : sm.k_empty;
+      const uint32_t ring = sbase + (is_v ? kOffV : kOffK);
       while (work.next(&sg)) {
         for (int j = 0; j < sg.n; ++j, ++it) {
           const uint32_t st = it % kStages, use = it / kStages;
-          if (use > 0 && ok) ok = mbar_wait(&sm.kv_empty[st], (use - 1) & 1u);
+          if (use > 0 && ok) ok = mbar_wait(&empty[st], (use - 1) & 1u);
           if (!ok) continue;
-          mbar_expect_tx(&sm.kv_full[st], kStageBytes);
-          const uint32_t dst = sbase + kOffKV + st * kStageBytes;
+          mbar_expect_tx(&full[st], kTileBytes);
+          const uint32_t dst = ring + st * kTileBytes;
           const int pos = (sg.t0 + j) * kKeys;
-          tma_load_4d(dst, &tm_k, &sm.kv_full[st], 0, sg.hkv, pos, sg.crow);
-          tma_load_4d(dst + kHalfBytes, &tm_k, &sm.kv_full[st], 64, sg.hkv, pos, sg.crow);
-          tma_load_4d(dst + 2 * kHalfBytes, &tm_v, &sm.kv_full[st], 0, sg.hkv, pos, sg.crow);
-          tma_load_4d(dst + 3 * kHalfBytes, &tm_v, &sm.kv_full[st], 64, sg.hkv, pos, sg.crow);
+          // tensor-map dimensions ascend in stride: (dh, head, position, row) or (dh, position, head, row)
+          const int c1 = a.layout ? pos : sg.hkv, c2 = a.layout ? sg.hkv : pos;
+          tma_load_4d(dst, map, &full[st], 0, c1, c2, sg.crow);
+          tma_load_4d(dst + kHalfBytes, map, &full[st], 64, c1, c2, sg.crow);
         }
       }
       if (!ok) sm.timed_out = 1u;
     }
-  } else if (warp == 1) {
+  } else if (warp == 2) {
     // ---------------- tensor-core issuer ----------------
     if (lane == 0) {
-      // S = Q K^T: A = Q in tensor memory, B = K tile (K-major: 128 key rows of 128 B per dh half)
+      // S = Q K^T: A = Q in tensor memory, B = K tile (K-major: 128 key rows of 128 B per dh half).  Its
+      // completion frees the K stage.
       auto issue_qk = [&](uint32_t t) {
         constexpr uint32_t id = umma_idesc(kRows, kKeys, 0, 0);
-        const uint32_t kb = sbase + kOffKV + (t % kStages) * kStageBytes;
+        const uint32_t kb = sbase + kOffK + (t % kStages) * kTileBytes;
         const uint32_t d = tmem + (t & 1u) * kKeys;
 #pragma unroll
         for (int ks = 0; ks < kDh / 16; ++ks)
           umma_ta(d, tmem + kColQ + ks * 8, umma_desc(kb + (ks >> 2) * kHalfBytes + (ks & 3) * 32, 16, 1024), id, ks ? 1u : 0u);
         umma_commit(&sm.s_full[t & 1u]);
+        umma_commit(&sm.k_empty[t % kStages]);
       };
-      // O += P V: A = P in tensor memory (over the S buffer), B = V tile as it lies in memory (MN-major:
-      // 128 B of dh per key row, the two dh halves kHalfBytes apart, 16 keys = 2048 B per K step)
+      // O += P V: A = P in tensor memory, B = V tile as it lies in memory (MN-major: 128 B of dh per key
+      // row, the two dh halves kHalfBytes apart, 16 keys = 2048 B per K step).  Its completion frees the
+      // V stage and the P columns.
       auto issue_pv = [&](uint32_t t, bool first) {
         constexpr uint32_t id = umma_idesc(kRows, kDh, 0, 1);
-        const uint32_t vb = sbase + kOffKV + (t % kStages) * kStageBytes + 2 * kHalfBytes;
-        const uint32_t pa = tmem + (t & 1u) * kKeys;
+        const uint32_t vb = sbase + kOffV + (t % kStages) * kTileBytes;
 #pragma unroll
         for (int ks = 0; ks < kKeys / 16; ++ks)
-          umma_ta(tmem + kColO, pa + ks * 8, umma_desc(vb + ks * 2048, kHalfBytes, 1024), id, (first && ks == 0) ? 0u : 1u);
-        umma_commit(&sm.kv_empty[t % kStages]);   // also "this tile's O product has completed" for the softmax warps
+          umma_ta(tmem + kColO, tmem + kColP + ks * 8, umma_desc(vb + ks * 2048, kHalfBytes, 1024), id, (first && ks == 0) ? 0u : 1u);
+        umma_commit(&sm.v_empty[t % kStages]);
+      };
+      auto qk_when_ready = [&](uint32_t t) {
+        if (ok) ok = mbar_wait(&sm.k_full[t % kStages], (t / kStages) & 1u);
+        tc_fence_after();
+        if (ok) issue_qk(t);
       };
       while (work.next(&sg)) {
         if (sg.n == 0) continue;
         if (ok) ok = mbar_wait(&sm.q_full, nseg & 1u);
+        // the logits run two tiles ahead of the O products: S buffer t & 1 is free once the softmax warps
+        // have turned tile t - 2 into P (their p_full arrival, awaited below)
+        qk_when_ready(it);
+        if (sg.n > 1) qk_when_ready(it + 1);
         for (int j = 0; j < sg.n; ++j, ++it) {
-          if (j == 0) {
-            if (ok) ok = mbar_wait(&sm.kv_full[it % kStages], (it / kStages) & 1u);
-            tc_fence_after();
-            if (ok) issue_qk(it);
-          }
-          if (j + 1 < sg.n) {        // the next tile's logits run while the softmax warps work on this tile
-            if (ok) ok = mbar_wait(&sm.kv_full[(it + 1) % kStages], ((it + 1) / kStages) & 1u);
-            tc_fence_after();
-            if (ok) issue_qk(it + 1);
-          }
-          if (ok) ok = mbar_wait(&sm.p_full[it & 1u], (it >> 1) & 1u);
+          if (ok) ok = mbar_wait(&sm.p_full, it & 1u);
           if (j == 0 && nseg > 0 && ok) ok = mbar_wait(&sm.o_free, (nseg - 1) & 1u);
           tc_fence_after();
+          // One wait per tile: an mbarrier wait between tensor-core instructions costs this thread a few
+          // hundred cycles (measured), so the first softmax warp also awaits the V tile of this product and the
+          // K tile of the next logits before it arrives on p_full.  The O product first (its completion frees
+          // the P columns for the next tile), then the logits of tile it + 2 into the S buffer tile it has left.
           if (ok) issue_pv(it, j == 0);
+          if (j + 2 < sg.n && ok) issue_qk(it + 2);
         }
         ++nseg;
       }
@@ -381,10 +412,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     // ---------------- softmax warps ----------------
     // Warps w and w + 4 share the 32 rows of one lane quarter; the first takes keys 0..63 of every tile
     // and output columns 0..63, the second the other halves.
-    const int sw = warp - 2;                     // 0..7
+    const int sw = warp - kFirstSoftmaxWarp;     // 0..7
     const int half = sw >> 2;
     const int row = 32 * (warp & 3) + lane;      // tensor-memory lane this warp may touch
-    const int sthread = tid - 64;                // 0..255
+    const int sthread = tid - 32 * kFirstSoftmaxWarp;   // 0..255
     const uint32_t tmem_lane = tmem + ((uint32_t)(32 * (warp & 3)) << 16);
     const int pair_bar = 1 + (warp & 3);         // named barrier of the two warps of a lane quarter
     const float sl2 = a.scale_log2;
@@ -467,7 +498,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         else if (mx > m + kRescaleStep) { corr = ex2(m - mx); m = mx; }
         if (__any_sync(0xffffffffu, corr != 1.f)) {
           // O still holds the products up to the previous tile: wait for them, then scale this thread's columns
-          if (ok) ok = mbar_wait(&sm.kv_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
+          if (ok) ok = mbar_wait(&sm.v_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
           tc_fence_after();
           __syncwarp();
 #pragma unroll 1
@@ -483,28 +514,34 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           l *= corr;
         }
         const float mu = m == -INFINITY ? 0.f : m;
-        // P goes over the first 64 columns of this S buffer, 32 per thread.  The second thread's share lies in
-        // columns the first thread read its logits from: it has finished (its loads completed before the pair
-        // barrier above).  The S product of tile it + 2 is issued behind the O product that reads P.
+        // P has columns of its own (32 per thread), free once the previous tile's O product has completed
         uint32_t pk[32];
         float ls4[4] = {0.f, 0.f, 0.f, 0.f};
+        if (!tail) {
 #pragma unroll
-        for (int c = 0; c < 64; c += 2) {
-          float p0 = ex2(fmaf(__uint_as_float(sr[c]), sl2, -mu));
-          float p1 = ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -mu));
-          if (tail) {
-            p0 = ((vm >> c) & 1ull) ? p0 : 0.f;
-            p1 = ((vm >> (c + 1)) & 1ull) ? p1 : 0.f;
+          for (int c = 0; c < 64; c += 2) {
+            const float p0 = ex2(fmaf(__uint_as_float(sr[c]), sl2, -mu));
+            const float p1 = ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -mu));
+            ls4[(c >> 1) & 3] += p0 + p1;
+            pk[c >> 1] = pack_bf16(p0, p1);
           }
-          ls4[(c >> 1) & 3] += p0 + p1;
-          pk[c >> 1] = pack_bf16(p0, p1);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 64; c += 2) {
+            const float p0 = ((vm >> c) & 1ull) ? ex2(fmaf(__uint_as_float(sr[c]), sl2, -mu)) : 0.f;
+            const float p1 = ((vm >> (c + 1)) & 1ull) ? ex2(fmaf(__uint_as_float(sr[c + 1]), sl2, -mu)) : 0.f;
+            ls4[(c >> 1) & 3] += p0 + p1;
+            pk[c >> 1] = pack_bf16(p0, p1);
+          }
         }
         l += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-        tmem_st32(tmem_lane + buf * kKeys + half * 32, pk);
+        if (it > 0 && ok) ok = mbar_wait(&sm.v_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
+        tc_fence_after();
+        tmem_st32(tmem_lane + kColP + half * 32, pk);
         if (tail) {
           // value rows nobody may read: zero them in the staged tile (two 128-byte rows per key)
           const uint32_t st = it % kStages;
-          if (ok) ok = mbar_wait(&sm.kv_full[st], (it / kStages) & 1u);
+          if (ok) ok = mbar_wait(&sm.v_full[st], (it / kStages) & 1u);
           const int c = sthread >> 1, hh = sthread & 1;
           const int p = (sg.t0 + j) * kKeys + c;
           bool dead = false;
@@ -513,7 +550,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             dead = s >= a.Ns || !((__ldg(usedw + (s >> 5)) >> (s & 31)) & 1u);
           }
           if (dead) {
-            uint4* vrow = reinterpret_cast<uint4*>(smem + kOffKV + st * kStageBytes + (2 + hh) * kHalfBytes + c * 128);
+            uint4* vrow = reinterpret_cast<uint4*>(smem + kOffV + st * kTileBytes + hh * kHalfBytes + c * 128);
 #pragma unroll
             for (int e = 0; e < 8; ++e) vrow[e] = make_uint4(0u, 0u, 0u, 0u);
           }
@@ -522,10 +559,16 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         tmem_st_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.p_full[buf]);
+        if (lane == 0) {
+          if (sw == 0) {     // on behalf of the issuer: the tiles its next two products read have landed
+            if (ok) ok = mbar_wait(&sm.v_full[it % kStages], (it / kStages) & 1u);
+            if (j + 2 < sg.n && ok) ok = mbar_wait(&sm.k_full[(it + 2) % kStages], ((it + 2) / kStages) & 1u);
+          }
+          mbar_arrive(&sm.p_full);
+        }
       }
       // end of the segment: the last O product, then normalise and write the slot
-      if (ok) ok = mbar_wait(&sm.kv_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
+      if (ok) ok = mbar_wait(&sm.v_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
       tc_fence_after();
       sm.xchg[0][half][row] = l;
       asm volatile("bar.sync %0, 64;\n" ::"r"(pair_bar) : "memory");
@@ -557,7 +600,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   __syncthreads();
   if (sm.timed_out && a.status && tid == 0)      // the outputs of the whole call are suspect
     for (int b = 0; b < a.B; ++b) a.status[b] = LUMO_SEQ_TIMEOUT;
-  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
 // Combination of a unit's slots: one warp per output row, slots in order (so the result for a given
@@ -579,22 +622,22 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   // this unit's slots
   int slot0 = 0, nslot = 0;
   {
-    long long total = 0, before = 0;
+    int total = 0, before = 0;
     int nt_b = 0;
     for (int bb = 0; bb < a.B; ++bb) {
       const int ok = seq_check(a.ctx_len[bb], a.cache_row[bb], a.Ns, a.n_rows, a.max_pos) == LUMO_SEQ_OK;
       const int nt = ok ? (a.ctx_len[bb] + a.Ns + kKeys - 1) / kKeys : 0;
-      if (bb < b) before += (long long)nt * upb;
+      if (bb < b) before += nt * upb;
       if (bb == b) nt_b = nt;
-      total += (long long)nt * upb;
+      total += nt * upb;
     }
     if (nt_b > 0) {
       if (a.S > 0) { slot0 = u * a.S; nslot = a.S; }
       else {
-        long long per = (total + a.C - 1) / a.C;
+        int per = (total + a.C - 1) / a.C;
         if (per < kMinTilesPerCta) per = kMinTilesPerCta;
-        const long long g0 = before + (long long)(hkv * a.RT + rt) * nt_b;
-        const int c0 = (int)(g0 / per), c1 = (int)((g0 + nt_b - 1) / per);
+        const int g0 = before + (hkv * a.RT + rt) * nt_b;
+        const int c0 = g0 / per, c1 = (g0 + nt_b - 1) / per;
         slot0 = u + c0; nslot = c1 - c0 + 1;
       }
     }
@@ -631,7 +674,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 // Tensor map of one cache: dims (dh, KV head, position, row), box 64 x 1 x 64 x 1, 128-byte swizzle;
 // positions beyond max_positions read as zeros.
-cudaError_t encode_cache_map(void* cache, int Hkv, int max_pos, int n_rows, CUtensorMap* map, std::string* err) {
+cudaError_t encode_cache_map(void* cache, int Hkv, int max_pos, int n_rows, int layout, CUtensorMap* map, std::string* err) {
   static EncodeTiledFn fn = nullptr;
   if (!fn) {
     void* p = nullptr;
@@ -641,9 +684,15 @@ cudaError_t encode_cache_map(void* cache, int Hkv, int max_pos, int n_rows, CUte
     if (q != cudaDriverEntryPointSuccess || !p) { *err = "the driver does not export cuTensorMapEncodeTiled"; return cudaErrorNotSupported; }
     fn = reinterpret_cast<EncodeTiledFn>(p);
   }
-  const cuuint64_t dims[4] = {(cuuint64_t)kDh, (cuuint64_t)Hkv, (cuuint64_t)max_pos, (cuuint64_t)n_rows};
-  const cuuint64_t strides[3] = {(cuuint64_t)kDh * 2, (cuuint64_t)Hkv * kDh * 2, (cuuint64_t)max_pos * Hkv * kDh * 2};
-  const cuuint32_t box[4] = {64, 1, (cuuint32_t)kKeys, 1};   // 16 KB
+  const cuuint64_t row_bytes = (cuuint64_t)max_pos * Hkv * kDh * 2;
+  cuuint64_t dims[4] = {(cuuint64_t)kDh, (cuuint64_t)Hkv, (cuuint64_t)max_pos, (cuuint64_t)n_rows};
+  cuuint64_t strides[3] = {(cuuint64_t)kDh * 2, (cuuint64_t)Hkv * kDh * 2, row_bytes};
+  cuuint32_t box[4] = {64, 1, (cuuint32_t)kKeys, 1};   // 16 KB
+  if (layout == 1) {   // a head's positions adjacent
+    dims[1] = (cuuint64_t)max_pos; dims[2] = (cuuint64_t)Hkv;
+    strides[1] = (cuuint64_t)max_pos * kDh * 2;
+    box[1] = (cuuint32_t)kKeys; box[2] = 1;
+  }
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, cache, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -676,9 +725,9 @@ cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
-  e = encode_cache_map(p.k_cache, s.Hkv, s.max_pos, s.n_rows, &plan->tk, err);
+  e = encode_cache_map(p.k_cache, s.Hkv, s.max_pos, s.n_rows, s.layout, &plan->tk, err);
   if (e != cudaSuccess) return e;
-  e = encode_cache_map(p.v_cache, s.Hkv, s.max_pos, s.n_rows, &plan->tv, err);
+  e = encode_cache_map(p.v_cache, s.Hkv, s.max_pos, s.n_rows, s.layout, &plan->tv, err);
   if (e != cudaSuccess) return e;
   AttnArgs& a = plan->a;
   a.q = p.q;
@@ -691,6 +740,7 @@ cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t
   a.ctx_len = s.ctx_len; a.cache_row = s.cache_row; a.vis = vis; a.used = used; a.status = p.status;
   a.B = s.B; a.N = s.N; a.Ns = s.Ns; a.Hq = s.Hq; a.Hkv = s.Hkv; a.n_rows = s.n_rows; a.max_pos = s.max_pos;
   a.scale_log2 = s.scale * kLog2e;
+  a.layout = s.layout;
   plan->grid = dim3(a.C, 1, 1);
   return cudaSuccess;
 }

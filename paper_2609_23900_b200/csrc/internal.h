@@ -302,7 +302,7 @@ cudaError_t launch_path_from_node(const TreeDev& t, int B, int N, const int32_t*
 
 // ---- attention half (attn.cu) ------------------------------------------------------------
 struct AttnShape {
-  int B, N, Ns, Hq, Hkv, S, n_rows, max_pos;
+  int B, N, Ns, Hq, Hkv, S, n_rows, max_pos, layout;
   float scale;
   const int32_t* ctx_len; const int32_t* cache_row;
 };
@@ -319,6 +319,7 @@ struct AttnArgs {
   int B, N, Ns, Hq, Hkv, G, RT, n_rows, max_pos;
   int S;   // partitions per unit; 0: the CTAs share the tile list evenly
   int C;   // CTAs of the attention launch
+  int layout;   // 0: cache [row, position, head, dh]; 1: [row, head, position, dh]
   float scale_log2;
 };
 // one attention launch: the tensor maps of the layer's two caches, the kernel arguments and the grid
@@ -333,7 +334,7 @@ struct KvLayers {
   int32_t* status[kMaxAttnLayers];
 };
 struct KvShape {
-  int B, N, Ns, Hkv, n_rows, max_pos;
+  int B, N, Ns, Hkv, n_rows, max_pos, layout;
   const int32_t* ctx_len; const int32_t* cache_row;
   const int32_t* parent; const int32_t* slot;
 };

@@ -21,16 +21,19 @@ __global__ void __launch_bounds__(128) kv_write_kernel(const KvLayers L, const K
     if (L.status[l] && i == 0 && threadIdx.x == 0) L.status[l][b] = bad;
     return;
   }
-  const int chunks = s.Hkv * kDh / 8;      // 16-byte chunks per entry
+  const int chunks = s.Hkv * kDh / 8;      // 16-byte chunks per entry (16 per head)
   const size_t src = ((size_t)b * s.N + i) * chunks;
-  const size_t dst = ((size_t)crow * s.max_pos + ctx + s.slot[(size_t)b * s.N + i]) * chunks;
   const uint4* kn = reinterpret_cast<const uint4*>(L.kn[l]) + src;
   const uint4* vn = reinterpret_cast<const uint4*>(L.vn[l]) + src;
+  // chunk strides of the cache: position and head
+  const size_t pos_st = s.layout ? 16 : (size_t)s.Hkv * 16, head_st = s.layout ? (size_t)s.max_pos * 16 : 16;
+  const size_t dst = (size_t)crow * s.max_pos * chunks + (size_t)(ctx + s.slot[(size_t)b * s.N + i]) * pos_st;
   uint4* kc = reinterpret_cast<uint4*>(L.k[l]) + dst;
   uint4* vc = reinterpret_cast<uint4*>(L.v[l]) + dst;
   for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
-    kc[c] = __ldg(kn + c);
-    vc[c] = __ldg(vn + c);
+    const size_t o = (size_t)(c >> 4) * head_st + (c & 15);
+    kc[o] = __ldg(kn + c);
+    vc[o] = __ldg(vn + c);
   }
 }
 
@@ -66,8 +69,9 @@ __global__ void __launch_bounds__(256) kv_publish_kernel(const KvLayers L, const
   __syncthreads();
   if (st_s != LUMO_SEQ_OK) return;
   unsigned char* cache = reinterpret_cast<unsigned char*>(which ? L.v[l] : L.k[l]);
-  const size_t pos_bytes = (size_t)s.Hkv * kDh * 2;
-  unsigned char* rowp = cache + ((size_t)crow * s.max_pos + ctx) * pos_bytes + (size_t)hkv * kDh * 2;
+  const size_t pos_bytes = s.layout ? (size_t)kDh * 2 : (size_t)s.Hkv * kDh * 2;
+  const size_t head_bytes = s.layout ? (size_t)s.max_pos * kDh * 2 : (size_t)kDh * 2;
+  unsigned char* rowp = cache + (size_t)crow * s.max_pos * s.Hkv * kDh * 2 + (size_t)ctx * pos_bytes + (size_t)hkv * head_bytes;
   // 16 chunks of 16 bytes per entry
   for (int c = tid; c < nn * 16; c += blockDim.x) {
     const int t = c >> 4, ch = c & 15;

@@ -90,13 +90,16 @@ class DeviceAttnCase:
     inputs of layer 0 unless ``cases`` lists one case per layer).  Marshalling only."""
 
     def __init__(self, ctx: binding.Context, case, *, n_splits: int = 0, cases=None, with_lse: bool = True,
-                 device: Optional[torch.device] = None):
+                 device: Optional[torch.device] = None, kv_layout: int = 0):
         self.ctx, self.case = ctx, case
         self.cases = list(cases) if cases is not None else [case]
         dev = device or torch.device("cuda", ctx.device)
         self.dev = dev
         self.desc = ctx.tree_desc(case.parent, slot=case.slot, n_slots=case.Ns)
         up16 = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).to(dev)
+        self.kv_layout = kv_layout
+        # the case holds caches as [rows, positions, Hkv, dh]; layout 1 stores them head-major
+        upc = lambda a: up16(a).permute(0, 2, 1, 3).contiguous() if kv_layout else up16(a)
         self.ctx_len = torch.from_numpy(case.ctx_len.copy()).to(dev)
         self.ctx_len_out = torch.full_like(self.ctx_len, -1)
         self.cache_row = torch.from_numpy(case.cache_row.copy()).to(dev)
@@ -105,7 +108,7 @@ class DeviceAttnCase:
         self.layers: List[binding.AttnLayer] = []
         for c in self.cases:
             self.layers.append(binding.AttnLayer(
-                Hq=c.Hq, Hkv=c.Hkv, k_cache=up16(c.k_cache), v_cache=up16(c.v_cache), ctx_len=self.ctx_len,
+                Hq=c.Hq, Hkv=c.Hkv, k_cache=upc(c.k_cache), v_cache=upc(c.v_cache), kv_layout=kv_layout, ctx_len=self.ctx_len,
                 cache_row=self.cache_row, scale=c.scale, q=up16(c.q), k_new=up16(c.k_new), v_new=up16(c.v_new),
                 out=torch.full((c.B, c.N, c.Hq, c.dh), float("nan"), dtype=torch.float32, device=dev),
                 lse=torch.full((c.B, c.N, c.Hq), float("nan"), dtype=torch.float32, device=dev) if with_lse else None,
@@ -116,7 +119,10 @@ class DeviceAttnCase:
         return self.layers[layer].tensors[name]
 
     def np(self, name: str, layer: int = 0) -> np.ndarray:
+        """Host copy in float64; caches always as [rows, positions, Hkv, dh], whatever the device layout."""
         t = self.t(name, layer)
+        if self.kv_layout and name in ("k_cache", "v_cache"):
+            t = t.permute(0, 2, 1, 3)
         return t.to(torch.float64).cpu().numpy() if t.is_floating_point() else t.cpu().numpy()
 
     def write(self, stream=None):

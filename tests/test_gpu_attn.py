@@ -64,10 +64,11 @@ CASES = [
 ]
 
 
+@pytest.mark.parametrize("kv_layout", [0, 1], ids=["pos_major", "head_major"])
 @pytest.mark.parametrize("name,kind,B,N,Ns,Hq,Hkv,ctxs,layout,splits", CASES, ids=[c[0] for c in CASES])
-def test_write_attend_publish_match_the_oracle(name, kind, B, N, Ns, Hq, Hkv, ctxs, layout, splits):
+def test_write_attend_publish_match_the_oracle(name, kind, B, N, Ns, Hq, Hkv, ctxs, layout, splits, kv_layout):
     c = W.make_attn_case(name, trees(kind, B, N, 900), ctxs, seed=W.BASE_SEED + 40, Hq=Hq, Hkv=Hkv, Ns=Ns, layout=layout)
-    dc = DeviceAttnCase(ctx(), c, n_splits=splits)
+    dc = DeviceAttnCase(ctx(), c, n_splits=splits, kv_layout=kv_layout)
     dc.write()
     k1, v1 = oracle_caches(c)
     torch.cuda.synchronize()
