@@ -340,6 +340,97 @@ def measure_extra_config(ctx, name, out_dtype, peak_gbs, steps=20, warmup=3, sna
     return out
 
 
+def measure_attention(ctx, peak_gbs, steps=30, warmup=4, B=8, context=16384, Hq=32, Hkv=8, n_sets=2):
+    """The attention half of the verifier on the paper's tree geometry (28 candidates + root padded to 32
+    rows, spine-first slots): tree KV write, ancestry-masked decode attention and KV publication of one
+    full-attention layer, timed back to back over rotating cache sets larger than L2.  The paper states no
+    head counts or context lengths for its model: 32 query / 8 KV heads of 128 and a 16k-token context per
+    sequence stand in for a coding-agent request (the design doc gives the recipe).  Inputs are drawn on the
+    device; parity with the oracle is the tests' business."""
+    import numpy as np
+    import torch
+    from paper_2609_23900_b200 import binding
+    from paper_2609_23900_b200 import workload as W
+    dev = torch.device("cuda", ctx.device)
+    tree = W.tree_paper_geometry()
+    N, Ns, dh = len(tree), 32, 128
+    parent = np.asarray([tree] * B, dtype=np.int32)
+    slot = np.asarray([W.spine_first_slots(tree)] * B, dtype=np.int32)
+    desc = ctx.tree_desc(parent, slot=slot, n_slots=Ns)
+    S = context + Ns
+    ctx_len = torch.full((B,), context, dtype=torch.int32, device=dev)
+    ctx_out = torch.zeros((B,), dtype=torch.int32, device=dev)
+    rows = torch.arange(B, dtype=torch.int32, device=dev)
+    spine = [i for i in range(N) if slot[0][i] < 6][:6]                 # six accepted spine nodes: already in place
+    branch = []
+    i = N - 1                                                           # and a rescue branch for the odd sequences
+    while i >= 0:
+        branch.append(i)
+        i = tree[i]
+    branch = branch[::-1]
+    lmax = max(len(spine), len(branch))
+    acc = np.full((B, lmax), -1, dtype=np.int32)
+    ln = np.zeros(B, dtype=np.int32)
+    for b in range(B):
+        path = spine if b % 2 == 0 else branch
+        acc[b, :len(path)] = path
+        ln[b] = len(path)
+    acc_d, ln_d = torch.from_numpy(acc).to(dev), torch.from_numpy(ln).to(dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(20260923)
+    rnd = lambda *shape: torch.randn(*shape, device=dev, dtype=torch.float32, generator=gen).to(torch.bfloat16)
+    layers, packs = [], []
+    for _ in range(n_sets):
+        L = binding.AttnLayer(Hq=Hq, Hkv=Hkv, k_cache=rnd(B, S, Hkv, dh), v_cache=rnd(B, S, Hkv, dh), ctx_len=ctx_len,
+                              cache_row=rows, scale=dh ** -0.5, q=rnd(B, N, Hq, dh), k_new=rnd(B, N, Hkv, dh),
+                              v_new=rnd(B, N, Hkv, dh), out=torch.empty(B, N, Hq, dh, device=dev),
+                              lse=torch.empty(B, N, Hq, device=dev), status=torch.zeros(B, dtype=torch.int32, device=dev))
+        layers.append(L)
+        packs.append(ctx.pack_attn([L]))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn):
+        for i in range(warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / steps
+
+    attn_us = timed(lambda i: ctx.tree_attention(desc, packs[i % n_sets]))
+    write_us = timed(lambda i: ctx.kv_write_tree(desc, packs[i % n_sets]))
+    publish_us = timed(lambda i: ctx.kv_publish(desc, packs[i % n_sets], acc_d, ln_d, ctx_out))
+    cycle_us = timed(lambda i: (ctx.kv_write_tree(desc, packs[i % n_sets]), ctx.tree_attention(desc, packs[i % n_sets]),
+                                ctx.kv_publish(desc, packs[i % n_sets], acc_d, ln_d, ctx_out)))
+    ctx.timing_enable(True)
+    ctx.timing_read(reset=True)
+    for i in range(steps):
+        ctx.tree_attention(desc, packs[i % n_sets])
+    torch.cuda.synchronize()
+    per_kernel = ctx.timing_read(reset=True)
+    ctx.timing_enable(False)
+    ok = all(int(L.tensors["status"].abs().sum()) == 0 for L in layers) and all(bool(torch.isfinite(L.tensors["out"]).all()) for L in layers)
+    # algorithmic bytes of one attention launch: every key and value of context and suffix once, queries, outputs
+    kv = 2 * B * S * Hkv * dh * 2
+    alg = kv + B * N * Hq * dh * (2 + 4) + B * N * Hq * 4
+    out = {"workload": f"one full-attention layer: batch {B}, {Hq}/{Hkv} heads of {dh}, {context}-token context per sequence, "
+                       f"paper tree ({N} nodes in {Ns} rows, spine-first slots), bf16 cache",
+           "attention_us": attn_us, "kv_write_us": write_us, "kv_publish_us": publish_us, "write_attend_publish_us": cycle_us,
+           "kernels": {k: {"launches": n, "avg_us": 1e3 * ms / n} for k, (n, ms) in per_kernel.items() if n},
+           "algorithmic_bytes": alg, "achieved_gbs": alg / (attn_us * 1e-6) / 1e9,
+           "frac_of_hbm_peak": alg / (attn_us * 1e-6) / 1e9 / peak_gbs,
+           "tree_nodes_per_s_per_layer": B * N / (attn_us * 1e-6),
+           "timing": f"{steps} back-to-back calls between two CUDA events, {n_sets} cache sets of {kv // 2 ** 20} MiB each rotated (larger than L2)",
+           "accepted": "even sequences accept six spine nodes (in place under the spine-first map: no bytes move), odd ones a rescue branch",
+           "status_ok_and_finite": ok}
+    del layers, packs
+    torch.cuda.empty_cache()
+    return out
+
+
 def fused_arm(args):
     """The same workload through lumo_gdn_commit_verify (the previous cycle's commit folded into the
     verify), timed by a run of this script of its own; reported beside the headline, never as it."""
@@ -702,6 +793,10 @@ def main():
             except Exception as e:
                 extra[key] = {"unavailable": f"{type(e).__name__}: {e}"[:200]}
         line["configs"] = extra
+        try:
+            line["attention"] = measure_attention(ctx, peak_gbs)
+        except Exception as e:
+            line["attention"] = {"unavailable": f"{type(e).__name__}: {e}"[:200]}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -110,16 +110,6 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
   return false;
 }
 
-// single poll
-__device__ __forceinline__ bool mbar_test(unsigned long long* bar, uint32_t parity) {
-  uint32_t done;
-  asm volatile(
-      "{\n.reg .pred p;\n"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-      "selp.u32 %0, 1, 0, p;\n}\n"
-      : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return done != 0;
-}
 
 // One box of a 4-d tiled tensor map (dh, KV head, position, cache row) into shared memory; completion
 // is counted in bytes on `bar`.  c0 is 0 or 64 elements: a multiple of 16 bytes.
@@ -145,12 +135,6 @@ __host__ __device__ constexpr uint32_t umma_idesc(int M, int N, int a_mn, int b_
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn << 15) | ((uint32_t)b_mn << 16) |
          ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
-__device__ __forceinline__ void umma(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
-      ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
-}
 // same product with the A operand in tensor memory (row = lane, two bf16 per 32-bit column, K-major)
 __device__ __forceinline__ void umma_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -160,14 +144,6 @@ __device__ __forceinline__ void umma_ta(uint32_t d_tmem, uint32_t a_tmem, uint64
 }
 __device__ __forceinline__ void umma_commit(unsigned long long* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr) : "memory");
-  asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory");
 }
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -214,6 +190,7 @@ struct Segment {
   int b, hkv, rt;     // unit
   int t0, n;          // first tile within the unit, tile count (n = 0 possible in fixed mode)
   int slot;
+  int unit, slot0, nslots;   // the unit, and the slots all its segments write (ascending along the key range)
   int ctx, crow;
 };
 
@@ -223,6 +200,7 @@ struct Work {
   int g, g_end;       // next global tile, end of this CTA's share (the host bounds the tile count below 2^31)
   int g_unit;         // global tile at which the current unit starts
   int nt;             // tiles per unit of the current sequence
+  int per;            // automatic mode: tiles per CTA
   bool fixed_done;
 
   static __device__ __forceinline__ int tiles_of(const AttnArgs& a, int bb, int* ctx, int* crow) {
@@ -233,13 +211,13 @@ struct Work {
   }
 
   __device__ __forceinline__ void init() {
-    b = 0; q = 0; g = 0; g_end = 0; g_unit = 0; nt = 0; fixed_done = false;
+    b = 0; q = 0; g = 0; g_end = 0; g_unit = 0; nt = 0; per = 1; fixed_done = false;
     if (a.S > 0) return;
     const int upb = a.Hkv * a.RT;       // units per sequence
     int total = 0;
     int cx, cr;
     for (int bb = 0; bb < a.B; ++bb) total += tiles_of(a, bb, &cx, &cr) * upb;
-    int per = (total + (int)gridDim.x - 1) / (int)gridDim.x;
+    per = (total + (int)gridDim.x - 1) / (int)gridDim.x;
     if (per < kMinTilesPerCta) per = kMinTilesPerCta;
     g = (int)blockIdx.x * per;
     g_end = g + per < total ? g + per : total;
@@ -269,6 +247,7 @@ struct Work {
       s->t0 = (int)(((long long)part * n_all) / a.S);
       s->n = (int)(((long long)(part + 1) * n_all) / a.S) - s->t0;
       s->slot = blockIdx.x;
+      s->unit = u; s->slot0 = u * a.S; s->nslots = a.S;
       return n_all > 0;
     }
     while (g < g_end && b < a.B) {
@@ -288,6 +267,9 @@ struct Work {
       const int end = g_unit + nt < g_end ? g_unit + nt : g_end;
       s->n = end - g;
       s->slot = u + blockIdx.x;
+      s->unit = u;
+      s->slot0 = u + g_unit / per;
+      s->nslots = (g_unit + nt - 1) / per - g_unit / per + 1;
       g = end;
       return true;
     }
@@ -426,6 +408,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const int hl = row_ok ? rg / a.N : 0, node = row_ok ? rg - hl * a.N : 0;
       float* slot_o = a.part_o + ((size_t)sg.slot * kRows + row) * kDh + half * 64;
       float* slot_l = a.part_lse + (size_t)sg.slot * kRows + row;
+      if (sthread == 0) a.unit_slots[sg.unit] = make_int2(sg.slot0, sg.nslots);   // for the merge (same pair from every writer)
       if (sg.n == 0) {                           // empty partition (fixed mode): an empty slot
         if (row_ok) {
           for (int e = 0; e < 16; ++e) reinterpret_cast<float4*>(slot_o)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -606,6 +589,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 // Combination of a unit's slots: one warp per output row, slots in order (so the result for a given
 // decomposition is reproducible), weights exp2(lse_s - max lse).
 __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
+  pdl_wait();          // launched as a programmatic dependent of the attention kernel: its slots are complete from here on
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int GN = a.G * a.N;
   const long long w = (long long)blockIdx.x * 8 + warp;
@@ -619,28 +603,11 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   float4* dst = reinterpret_cast<float4*>(a.out + out_row * kDh) + lane;
   const int upb = a.Hkv * a.RT;
   const int u = b * upb + hkv * a.RT + rt;
-  // this unit's slots
+  // this unit's slots, as the attention kernel recorded them; a sequence that fails its check owns none
   int slot0 = 0, nslot = 0;
-  {
-    int total = 0, before = 0;
-    int nt_b = 0;
-    for (int bb = 0; bb < a.B; ++bb) {
-      const int ok = seq_check(a.ctx_len[bb], a.cache_row[bb], a.Ns, a.n_rows, a.max_pos) == LUMO_SEQ_OK;
-      const int nt = ok ? (a.ctx_len[bb] + a.Ns + kKeys - 1) / kKeys : 0;
-      if (bb < b) before += nt * upb;
-      if (bb == b) nt_b = nt;
-      total += nt * upb;
-    }
-    if (nt_b > 0) {
-      if (a.S > 0) { slot0 = u * a.S; nslot = a.S; }
-      else {
-        int per = (total + a.C - 1) / a.C;
-        if (per < kMinTilesPerCta) per = kMinTilesPerCta;
-        const int g0 = before + (hkv * a.RT + rt) * nt_b;
-        const int c0 = g0 / per, c1 = (g0 + nt_b - 1) / per;
-        slot0 = u + c0; nslot = c1 - c0 + 1;
-      }
-    }
+  if (seq_check(a.ctx_len[b], a.cache_row[b], a.Ns, a.n_rows, a.max_pos) == LUMO_SEQ_OK) {
+    const int2 t = a.unit_slots[u];
+    slot0 = t.x; nslot = t.y;
   }
   if (nslot == 0) {                          // the sequence failed its check (it owns no tiles): zeros and its status
     *dst = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -705,13 +672,16 @@ cudaError_t encode_cache_map(void* cache, int Hkv, int max_pos, int n_rows, int 
 int attn_row_tiles(int G, int N) { return (G * N + kRows - 1) / kRows; }
 
 // slots of partial results: automatic mode needs at most units + CTAs - 1, fixed mode units x partitions
+size_t attn_units(const AttnShape& s) { return (size_t)s.B * s.Hkv * attn_row_tiles(s.Hq / s.Hkv, s.N); }
+
 static size_t attn_slots(const AttnShape& s, int ctas) {
   const size_t units = (size_t)s.B * s.Hkv * attn_row_tiles(s.Hq / s.Hkv, s.N);
   return s.S > 0 ? units * s.S : units + ctas;
 }
 
+// partial results [slots][128][128], their log-sum-exps [slots][128], the slot range of every unit [units][2]
 size_t attn_scratch_bytes(const AttnShape& s, int sm_count) {
-  return attn_slots(s, sm_count) * kRows * (kDh + 1) * sizeof(float);
+  return attn_slots(s, sm_count) * kRows * (kDh + 1) * sizeof(float) + attn_units(s) * sizeof(int2);
 }
 
 cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t* vis, const uint32_t* used, float* scratch,
@@ -737,6 +707,7 @@ cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t
   a.C = s.S > 0 ? (int)(units * s.S) : sm_count;
   a.part_o = scratch;
   a.part_lse = scratch + attn_slots(s, sm_count) * kRows * kDh;
+  a.unit_slots = reinterpret_cast<int2*>(a.part_lse + attn_slots(s, sm_count) * kRows);
   a.ctx_len = s.ctx_len; a.cache_row = s.cache_row; a.vis = vis; a.used = used; a.status = p.status;
   a.B = s.B; a.N = s.N; a.Ns = s.Ns; a.Hq = s.Hq; a.Hkv = s.Hkv; a.n_rows = s.n_rows; a.max_pos = s.max_pos;
   a.scale_log2 = s.scale * kLog2e;
@@ -752,8 +723,8 @@ cudaError_t launch_attn(const AttnPlan& plan, cudaStream_t st) {
 
 cudaError_t launch_attn_merge(const AttnPlan& plan, cudaStream_t st) {
   const long long rows = (long long)plan.a.B * plan.a.Hkv * plan.a.G * plan.a.N;
-  attn_merge_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(plan.a);
-  return cudaGetLastError();
+  // dependent launch: the CTAs are staged while the attention kernel drains and wait on the device for its end
+  return launch_kernel(attn_merge_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, st, true, plan.a);
 }
 
 }  // namespace lumo

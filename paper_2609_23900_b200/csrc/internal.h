@@ -313,6 +313,7 @@ struct AttnArgs {
   const void* q;
   float* out; float* lse;
   float* part_o; float* part_lse;
+  int2* unit_slots;   // per unit: first slot and slot count of its segments, written by the attention kernel
   const int32_t* ctx_len; const int32_t* cache_row;
   const uint32_t* vis; const uint32_t* used;
   int32_t* status;

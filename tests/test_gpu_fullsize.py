@@ -119,3 +119,56 @@ def test_config3_fused_commit_verify_matches_the_separate_calls():
         of, ou = lf[l].tensors["out"].float(), lu[l].tensors["out"].float()
         assert bool(((of - ou).abs() <= 2.0 ** -7 * ou.abs() + 1e-3).all())   # bf16 outputs: one ulp apart at most
         assert torch.equal(lf[l].tensors["k"], lu[l].tensors["k"]) and torch.equal(lf[l].tensors["v"], lu[l].tensors["v"])
+
+
+def test_attention_at_the_bench_shape_sampled():
+    """The attention launch bench.py times (batch 8, 32/8 heads, 16k-token contexts, paper tree, spine-first
+    slots, automatic decomposition over all SMs): inputs drawn on the device by a seeded generator, the
+    oracle run on sampled (sequence, query head) pairs from copies of those inputs, every node of the pair."""
+    from oracle import attn_oracle as A
+    from paper_2609_23900_b200 import binding
+    c = ctx()
+    dev = torch.device("cuda", c.device)
+    B, context, Hq, Hkv, dh = 8, 16384, 32, 8, 128
+    tree = W.tree_paper_geometry()
+    N, Ns = len(tree), 32
+    parent = np.asarray([tree] * B, dtype=np.int32)
+    slot = np.asarray([W.spine_first_slots(tree)] * B, dtype=np.int32)
+    desc = c.tree_desc(parent, slot=slot, n_slots=Ns)
+    S = context + Ns
+    ctx_host = np.asarray([context - 37 * b for b in range(B)], dtype=np.int32)        # ragged tile edges
+    ctx_len = torch.from_numpy(ctx_host).to(dev)
+    rows = torch.arange(B - 1, -1, -1, dtype=torch.int32, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(99)
+    rnd = lambda *shape: torch.randn(*shape, device=dev, dtype=torch.float32, generator=gen).to(torch.bfloat16)
+    L = binding.AttnLayer(Hq=Hq, Hkv=Hkv, k_cache=rnd(B, S, Hkv, dh), v_cache=rnd(B, S, Hkv, dh), ctx_len=ctx_len, cache_row=rows,
+                          scale=dh ** -0.5, q=rnd(B, N, Hq, dh), k_new=rnd(B, N, Hkv, dh), v_new=rnd(B, N, Hkv, dh),
+                          out=torch.empty(B, N, Hq, dh, device=dev), lse=torch.empty(B, N, Hq, device=dev),
+                          status=torch.full((B,), -1, dtype=torch.int32, device=dev))
+    pk = c.pack_attn([L])
+    k0 = {b: L.tensors["k_cache"][int(rows[b])].to(torch.float64).cpu().numpy() for b in (0, 3, 7)}     # before the write
+    v0 = {b: L.tensors["v_cache"][int(rows[b])].to(torch.float64).cpu().numpy() for b in (0, 3, 7)}
+    c.kv_write_tree(desc, pk)
+    c.tree_attention(desc, pk)
+    torch.cuda.synchronize()
+    assert L.tensors["status"].tolist() == [0] * B
+    out, lse = L.tensors["out"].to(torch.float64).cpu().numpy(), L.tensors["lse"].to(torch.float64).cpu().numpy()
+    q = L.tensors["q"].to(torch.float64).cpu().numpy()
+    kn, vn = L.tensors["k_new"].to(torch.float64).cpu().numpy(), L.tensors["v_new"].to(torch.float64).cpu().numpy()
+    worst = 0.0
+    for b in (0, 3, 7):
+        one = lambda a: a[b:b + 1]
+        k1, v1 = A.kv_write(one(slot), one(kn), one(vn), k0[b][None], v0[b][None], ctx_host[b:b + 1], np.zeros(1, np.int32))
+        for h in (0, 13, 31):
+            g = h // (Hq // Hkv)
+            qq = q[b:b + 1, :, h:h + 1]
+            kk, vv = k1[:, :, g:g + 1], v1[:, :, g:g + 1]
+            ref, rl = A.tree_attention(one(parent), one(slot), qq, kk, vv, ctx_host[b:b + 1], np.zeros(1, np.int32), dh ** -0.5)
+            bound, _ = A.tree_attention(one(parent), one(slot), qq, kk, np.abs(vv), ctx_host[b:b + 1], np.zeros(1, np.int32), dh ** -0.5)
+            err = np.abs(out[b, :, h] - ref[0, :, 0])
+            tol = 1.05 * 2.0 ** -8 * bound[0, :, 0] + 2e-5 * (1.0 + np.abs(ref[0, :, 0]))
+            assert (err <= tol).all(), f"b={b} h={h}: worst ratio {(err / tol).max():.2f}"
+            assert (np.abs(lse[b, :, h] - rl[0, :, 0]) <= 2e-5 * (1.0 + np.abs(rl[0, :, 0]))).all(), f"b={b} h={h}: lse"
+            worst = max(worst, float((err / tol).max()))
+    assert worst > 0.0
