@@ -16,8 +16,8 @@
 //   warp 2     tensor-core issuer: S = Q K^T into one of two S buffers in tensor memory (M 128, N 128,
 //              K 128), and O += P V (M 128, N 128, K 128; V is the MN-major B operand as it lies in
 //              memory) into a 128-column accumulator that stays in tensor memory for the whole segment;
-//              the S products run two tiles ahead of the O products, so the softmax warps never wait for
-//              logits.  Both A operands (Q and P) live in tensor memory, so shared memory carries only the staged K and V tiles.  (Measured:
+//              the S products run two tiles ahead of the O products (a buffer is refilled as soon as the
+//              softmax warps hold its logits in registers), so the softmax warps never wait for logits.  Both A operands (Q and P) live in tensor memory, so shared memory carries only the staged K and V tiles.  (Measured:
 //              an N = 128 product issues at the tensor core's full rate, an N = 64 one at 70 % of it.)
 //   warps 3-10 softmax: a query row (= tensor-memory lane) is shared by two threads (warps w and w + 4),
 //              64 keys each.  A thread reads its logits, applies visibility by selection (never by
@@ -74,7 +74,7 @@ constexpr int kOffV = kStages * kTileBytes;
 constexpr int kOffSmall = 2 * kStages * kTileBytes;   // 196608
 struct Small {
   unsigned long long k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
-  unsigned long long s_full[2], p_full;
+  unsigned long long s_full[2], s_read[2], p_full;
   unsigned long long q_full, o_free;
   uint32_t tmem_base;
   uint32_t timed_out;
@@ -110,6 +110,23 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
   return false;
 }
 
+
+// Same bounded wait without acquire semantics: for waits that are followed by tensor-memory accesses only,
+// which tcgen05.fence::after_thread_sync orders (the default acquire form measured ~200 cycles even on a
+// completed phase).
+__device__ __forceinline__ bool mbar_wait_relaxed(unsigned long long* bar, uint32_t parity) {
+  const uint32_t addr = smem_u32(bar);
+  for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+    uint32_t done;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.relaxed.cta.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}\n"
+        : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+    if (done) return true;
+  }
+  return false;
+}
 
 // One box of a 4-d tiled tensor map (dh, KV head, position, cache row) into shared memory; completion
 // is counted in bytes on `bar`.  c0 is 0 or 64 elements: a multiple of 16 bytes.
@@ -296,6 +313,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     }
     mbar_init(&sm.s_full[0], 1);
     mbar_init(&sm.s_full[1], 1);
+    mbar_init(&sm.s_read[0], kSoftmaxWarps);
+    mbar_init(&sm.s_read[1], kSoftmaxWarps);
     mbar_init(&sm.p_full, kSoftmaxWarps);        // one arrival per softmax warp
     mbar_init(&sm.q_full, kSoftmaxWarps);
     mbar_init(&sm.o_free, kSoftmaxWarps);
@@ -376,15 +395,19 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         qk_when_ready(it);
         if (sg.n > 1) qk_when_ready(it + 1);
         for (int j = 0; j < sg.n; ++j, ++it) {
+          // Two waits per tile, each followed by one product.  (An mbarrier wait between tensor-core
+          // instructions costs this thread a few hundred cycles, measured; the waits for the TMA tiles are
+          // therefore done by the first softmax warp before it arrives on these two barriers.)
+          if (j + 2 < sg.n) {
+            // the softmax warps hold tile it's logits in registers: its S buffer takes the logits of tile it + 2
+            if (ok) ok = mbar_wait(&sm.s_read[it & 1u], (it >> 1) & 1u);
+            tc_fence_after();
+            if (ok) issue_qk(it + 2);
+          }
           if (ok) ok = mbar_wait(&sm.p_full, it & 1u);
           if (j == 0 && nseg > 0 && ok) ok = mbar_wait(&sm.o_free, (nseg - 1) & 1u);
           tc_fence_after();
-          // One wait per tile: an mbarrier wait between tensor-core instructions costs this thread a few
-          // hundred cycles (measured), so the first softmax warp also awaits the V tile of this product and the
-          // K tile of the next logits before it arrives on p_full.  The O product first (its completion frees
-          // the P columns for the next tile), then the logits of tile it + 2 into the S buffer tile it has left.
           if (ok) issue_pv(it, j == 0);
-          if (j + 2 < sg.n && ok) issue_qk(it + 2);
         }
         ++nseg;
       }
@@ -454,13 +477,20 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             vm |= (unsigned long long)v << c;
           }
         }
-        if (ok) ok = mbar_wait(&sm.s_full[buf], (it >> 1) & 1u);
+        if (ok) ok = mbar_wait_relaxed(&sm.s_full[buf], (it >> 1) & 1u);
         tc_fence_after();
         __syncwarp();
         uint32_t sr[64];
         tmem_ld32(tmem_lane + buf * kKeys + half * 64, sr);
         tmem_ld32(tmem_lane + buf * kKeys + half * 64 + 32, sr + 32);
         tmem_ld_wait();
+        // the logits are in registers: the S buffer may take the logits of tile it + 2 (whose keys must have landed)
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (sw == 0 && j + 2 < sg.n && ok) ok = mbar_wait(&sm.k_full[(it + 2) % kStages], ((it + 2) / kStages) & 1u);
+          mbar_arrive(&sm.s_read[buf]);
+        }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
         if (!tail) {
 #pragma unroll
@@ -518,7 +548,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           }
         }
         l += (ls4[0] + ls4[1]) + (ls4[2] + ls4[3]);
-        if (it > 0 && ok) ok = mbar_wait(&sm.v_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
+        if (it > 0 && ok) ok = mbar_wait_relaxed(&sm.v_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
         tc_fence_after();
         tmem_st32(tmem_lane + kColP + half * 32, pk);
         if (tail) {
@@ -543,10 +573,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         tc_fence_before();
         __syncwarp();
         if (lane == 0) {
-          if (sw == 0) {     // on behalf of the issuer: the tiles its next two products read have landed
-            if (ok) ok = mbar_wait(&sm.v_full[it % kStages], (it / kStages) & 1u);
-            if (j + 2 < sg.n && ok) ok = mbar_wait(&sm.k_full[(it + 2) % kStages], ((it + 2) / kStages) & 1u);
-          }
+          if (sw == 0 && ok) ok = mbar_wait(&sm.v_full[it % kStages], (it / kStages) & 1u);   // on behalf of the issuer
           mbar_arrive(&sm.p_full);
         }
       }
