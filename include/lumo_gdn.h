@@ -370,8 +370,9 @@ typedef struct {
   int32_t kv_layout;        /* 0: caches are [n_cache_rows, max_positions, Hkv, dh] (a position's heads adjacent);
                                1: [n_cache_rows, Hkv, max_positions, dh] (a head's positions adjacent: a tile of keys is
                                one contiguous 32 KB run, which the attention kernel reads at a higher HBM efficiency) */
-  int32_t n_splits;         /* partitions of the key range per (sequence, KV head): 0 = chosen to fill the GPU,
-                               else 1..32 (Sec. "Evaluation Setup": the paper's deployment used 4) */
+  int32_t n_splits;         /* partitions of the key range per (sequence, KV head, row tile): 0 = the key tiles of the
+                               whole call are dealt out evenly over the SMs (a unit is cut wherever a share ends),
+                               else 1..32 equal partitions (Sec. "Evaluation Setup": the paper's deployment used 4) */
   int32_t* status;          /* [B] lumo_seq_status; may be NULL */
 } lumo_attn_args;
 
@@ -387,10 +388,11 @@ int lumo_kv_write_tree(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_att
  * on tcgen05 tensor cores: the query rows of all heads that share a KV head form one 128-row tile
  * (rows = (h mod G) * N + i, G = Hq / Hkv; further tiles when G N > 128), so a staged key/value tile
  * is read once for the whole group (Sec. "One slot map governs attention and publication": grouped
- * query heads share staged KV tiles); the key range of a sequence is cut into n_splits partitions
- * handled by different CTAs, combined by the log-sum-exp rule (same section: split-K context
+ * query heads share staged KV tiles); the key range of a unit is cut into partitions handled by
+ * different CTAs, combined in key order by the log-sum-exp rule (same section: split-K context
  * partitions).  Probabilities enter the second product rounded to bf16; all sums are fp32.
- * The result for a given n_splits is bitwise reproducible; different n_splits differ by rounding.
+ * The result is bitwise reproducible for a given device, shape and n_splits; other partitionings differ
+ * by rounding.
  * Needs max_positions * Hkv * dh * 2 bytes < 2^40 per cache row.  Enqueues only; library scratch for
  * the partial results grows on the first call with a shape. */
 int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers,
