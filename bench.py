@@ -467,6 +467,10 @@ def main():
     ap.add_argument("--no-extra-configs", dest="extra_configs", action="store_false")
     ap.add_argument("--scan-algo", default="auto", choices=["auto", "rank1", "gram", "solve"],
                     help="which scan kernel verify uses (auto = the library's choice)")
+    ap.add_argument("--attention-only", action="store_true",
+                    help="time only the attention layer (the 'attention' block of the default line) and print it as its own JSON line")
+    ap.add_argument("--attn-batch", type=int, default=8)
+    ap.add_argument("--attn-context", type=int, default=16384)
     ap.add_argument("--fused-commit", action="store_true",
                     help="time lumo_gdn_commit_verify (the previous cycle's commit folded into the verify) instead of "
                          "verify + commit; every step still commits one accepted path and verifies one tree per sequence")
@@ -499,6 +503,16 @@ def main():
     ctx = binding.Context(local)
     ctx.set_overlap(not args.no_overlap)
     ctx.set_scan_algo(args.scan_algo)
+    if args.attention_only:
+        # the attention layer alone (used for profiling that kernel); not the headline metric
+        if is_reporting_rank(rank):
+            peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+            peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else 6650.0
+            print(json.dumps({"attention": measure_attention(ctx, peak, steps=args.steps, warmup=args.warmup, B=args.attn_batch,
+                                                             context=args.attn_context)}), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     # ---- buffer sets: distinct seeds per set and per rank, together larger than L2 -----------
     case0 = make_case(args.config, seed_offset=rank_seed_offset(rank))
     n_layers = len(case0.layers)
