@@ -224,3 +224,70 @@ def test_attention_after_publication_continues_the_accepted_path():
     torch.cuda.synchronize()
     k3, v3 = oracle_caches(c2)
     check_attention(dc2, c2, k3, v3, "second cycle")
+
+
+def test_several_layers_in_one_call_and_optional_outputs():
+    """Two layers with different inputs through one call each of write, attend and publish; the second
+    layer without lse and without status words."""
+    parents = trees("random", 2, 14, 5)
+    cs = [W.make_attn_case("multi", parents, [90, 310], seed=W.BASE_SEED + 47, Hq=4, Hkv=2, Ns=16, layout="spine", layer=l,
+                           max_positions=340) for l in range(2)]
+    dc = DeviceAttnCase(ctx(), cs[0], cases=cs, n_splits=0)
+    L1 = dc.layers[1]
+    L1.tensors["lse"], L1.tensors["status"] = None, None
+    L1.args.lse, L1.args.status = None, None
+    dc.packed = ctx().pack_attn(dc.layers)
+    dc.write(); dc.attend()
+    torch.cuda.synchronize()
+    for l, c in enumerate(cs):
+        k1, v1 = oracle_caches(c)
+        ref, _ = A.tree_attention(c.parent, c.slot, c.q, k1, v1, c.ctx_len, c.cache_row, c.scale)
+        bound, _ = A.tree_attention(c.parent, c.slot, c.q, k1, np.abs(v1), c.ctx_len, c.cache_row, c.scale)
+        err = np.abs(dc.np("out", l) - ref)
+        assert (err <= 1.05 * 2.0 ** -8 * bound + 2e-5 * (1.0 + np.abs(ref))).all(), f"layer {l}"
+    dc.publish()
+    torch.cuda.synchronize()
+    for l, c in enumerate(cs):
+        k1, v1 = oracle_caches(c)
+        k2, v2, ctx2, _ = A.kv_publish(c.parent, c.slot, k1, v1, c.ctx_len, c.cache_row, c.accepted, c.accepted_len)
+        assert np.array_equal(dc.np("k_cache", l), k2) and np.array_equal(dc.np("v_cache", l), v2), f"layer {l} publication"
+    assert dc.ctx_len_out.tolist() == ctx2.tolist()
+
+
+def test_host_side_refusals_enqueue_nothing():
+    c = W.make_attn_case("refuse", trees("random", 1, 6, 1), [10], seed=1, Hq=4, Hkv=2, Ns=8, layout="identity")
+    cx = ctx()
+    dc = DeviceAttnCase(cx, c)
+    out0 = dc.t("out").clone()
+
+    def refused(mutate, call=None, code=None):
+        L = dc.layers[0]
+        saved = {f[0]: getattr(L.args, f[0]) for f in L.args._fields_}
+        mutate(L.args)
+        try:
+            with pytest.raises(binding.LumoError) as e:
+                (call or (lambda: cx.tree_attention(dc.desc, cx.pack_attn([L]))))()
+            if code is not None:
+                assert e.value.code == code
+        finally:
+            for k, v in saved.items():
+                setattr(L.args, k, v)
+
+    refused(lambda a: setattr(a, "dh", 64), code=4)
+    refused(lambda a: setattr(a, "Hq", 5), code=4)
+    refused(lambda a: setattr(a, "scale", 0.0), code=1)
+    refused(lambda a: setattr(a, "n_splits", 33), code=1)
+    refused(lambda a: setattr(a, "kv_layout", 2), code=1)
+    refused(lambda a: setattr(a, "max_positions", 4), code=1)          # fewer positions than slots
+    refused(lambda a: setattr(a, "q", None), code=1)
+    refused(lambda a: setattr(a, "k_new", None), call=lambda: cx.kv_write_tree(dc.desc, cx.pack_attn([dc.layers[0]])), code=1)
+    refused(lambda a: None, call=lambda: cx.kv_publish(dc.desc, dc.packed, dc.accepted, dc.accepted_len, dc.ctx_len), code=1)  # alias
+    wide = cx.tree_desc(np.array([[-1, 0]], dtype=np.int32), n_slots=300)
+    with pytest.raises(binding.LumoError) as e:
+        cx.tree_attention(wide, dc.packed)
+    assert e.value.code == 4
+    torch.cuda.synchronize()
+    assert torch.equal(dc.t("out"), out0) or (torch.isnan(dc.t("out")) & torch.isnan(out0)).all()
+    dc.write(); dc.attend()                                             # the context is still usable
+    torch.cuda.synchronize()
+    assert dc.t("status").tolist() == [0]

@@ -198,3 +198,14 @@ def test_spine_first_slot_map_is_contiguous_on_the_principal_chain():
     assert sorted(s) == list(range(len(p)))
     spine = [0, 1, 4, 7, 10, 13, 16, 17, 18, 19, 20, 21]
     assert [s[i] for i in spine] == list(range(12))
+
+
+def test_attention_calls_refuse_to_launch_on_a_host_only_context():
+    import ctypes as C
+    ctx = binding.Context(-1)
+    desc = ctx.tree_desc(np.array([[-1, 0, 1]], dtype=np.int32))
+    arr = (binding._AttnArgs * 1)()
+    for fn in (binding._lib.lumo_kv_write_tree, binding._lib.lumo_tree_attention):
+        assert fn(ctx._h, desc._h, arr, 1, None) == 4            # LUMO_ERR_UNSUPPORTED: there is no CPU path
+    assert binding._lib.lumo_kv_publish(ctx._h, desc._h, arr, 1, None, None, 4, None, None) == 4
+    assert b"host-only" in binding._lib.lumo_last_error(ctx._h)
