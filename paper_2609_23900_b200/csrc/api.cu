@@ -783,6 +783,8 @@ int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_at
     e = cudaMalloc(&ctx->attn_scratch, need);
     if (e != cudaSuccess) return fail(ctx, LUMO_ERR_NOMEM, std::string("scratch allocation failed: ") + cudaGetErrorString(e));
     ctx->attn_scratch_bytes = need;
+    e = cudaMemset(ctx->attn_scratch, 0, 256);   // the failure flag in the first bytes: launch numbers are never 0
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemset(attention scratch)");
   }
   ctx->last_call = lumo_ctx::kOther;
   // the layers of a model are not adjacent in time: one launch (and one pair of tensor maps) per layer;
@@ -793,13 +795,11 @@ int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_at
     p.out = layers[l].out; p.lse = layers[l].lse; p.status = layers[l].status;
     AttnPlan plan;
     std::string err;
+    if (++ctx->attn_launch_id == 0) ctx->attn_launch_id = 1;
+    const uint32_t launch_id = ctx->attn_launch_id;
     cudaError_t e = attn_plan(s, p, desc->d_vis, desc->d_slot_used, reinterpret_cast<float*>(ctx->attn_scratch),
-                              ctx->sm_count, &plan, &err);
+                              ctx->sm_count, launch_id, &plan, &err);
     if (e != cudaSuccess) return err.empty() ? cuda_fail(ctx, e, "attention set-up") : fail(ctx, LUMO_ERR_CUDA, err);
-    if (p.status) {   // the kernels write failures only
-      e = cudaMemsetAsync(p.status, 0, (size_t)s.B * sizeof(int32_t), st);
-      if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemsetAsync(status)");
-    }
     e = timed(ctx, LUMO_K_ATTN, st, [&] { return launch_attn(plan, st); });
     if (e != cudaSuccess) return cuda_fail(ctx, e, "attention launch");
     e = timed(ctx, LUMO_K_ATTN_MERGE, st, [&] { return launch_attn_merge(plan, st); });

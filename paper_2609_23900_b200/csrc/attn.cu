@@ -608,8 +608,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
   tc_fence_before();
   __syncthreads();
-  if (sm.timed_out && a.status && tid == 0)      // the outputs of the whole call are suspect
-    for (int b = 0; b < a.B; ++b) a.status[b] = LUMO_SEQ_TIMEOUT;
+  if (sm.timed_out && tid == 0) *a.fail_flag = a.launch_id;   // the merge kernel turns this into status words
   if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
@@ -636,11 +635,15 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
     const int2 t = a.unit_slots[u];
     slot0 = t.x; nslot = t.y;
   }
-  if (nslot == 0) {                          // the sequence failed its check (it owns no tiles): zeros and its status
+  // status word of the sequence: its check, else whether any wait of this launch's attention kernel ran out
+  // (then the outputs of the whole call are suspect)
+  if (a.status && lane == 0 && hkv == 0 && rg == 0) {
+    const int st = seq_check(a.ctx_len[b], a.cache_row[b], a.Ns, a.n_rows, a.max_pos);
+    a.status[b] = st != LUMO_SEQ_OK ? st : (*a.fail_flag == a.launch_id ? (int)LUMO_SEQ_TIMEOUT : (int)LUMO_SEQ_OK);
+  }
+  if (nslot == 0) {                          // the sequence failed its check (it owns no tiles): zeros
     *dst = make_float4(0.f, 0.f, 0.f, 0.f);
     if (a.lse && lane == 0) a.lse[out_row] = 0.f;
-    if (a.status && lane == 0 && hkv == 0 && rg == 0)
-      a.status[b] = seq_check(a.ctx_len[b], a.cache_row[b], a.Ns, a.n_rows, a.max_pos);
     return;
   }
   const size_t base = (size_t)slot0 * kRows + r;
@@ -706,13 +709,14 @@ static size_t attn_slots(const AttnShape& s, int ctas) {
   return s.S > 0 ? units * s.S : units + ctas;
 }
 
+// 256 bytes whose first word says "a wait ran out in launch number ..." (at a fixed place, zero at allocation), then
 // partial results [slots][128][128], their log-sum-exps [slots][128], the slot range of every unit [units][2]
 size_t attn_scratch_bytes(const AttnShape& s, int sm_count) {
-  return attn_slots(s, sm_count) * kRows * (kDh + 1) * sizeof(float) + attn_units(s) * sizeof(int2);
+  return 256 + attn_slots(s, sm_count) * kRows * (kDh + 1) * sizeof(float) + attn_units(s) * sizeof(int2);
 }
 
 cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t* vis, const uint32_t* used, float* scratch,
-                      int sm_count, AttnPlan* plan, std::string* err) {
+                      int sm_count, uint32_t launch_id, AttnPlan* plan, std::string* err) {
   static bool configured[kMaxDevices] = {};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
@@ -732,9 +736,12 @@ cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t
   a.G = s.Hq / s.Hkv; a.RT = attn_row_tiles(a.G, s.N); a.S = s.S;
   const size_t units = (size_t)s.B * s.Hkv * a.RT;
   a.C = s.S > 0 ? (int)(units * s.S) : sm_count;
+  a.fail_flag = reinterpret_cast<uint32_t*>(scratch);
+  scratch += 64;
   a.part_o = scratch;
   a.part_lse = scratch + attn_slots(s, sm_count) * kRows * kDh;
   a.unit_slots = reinterpret_cast<int2*>(a.part_lse + attn_slots(s, sm_count) * kRows);
+  a.launch_id = launch_id;
   a.ctx_len = s.ctx_len; a.cache_row = s.cache_row; a.vis = vis; a.used = used; a.status = p.status;
   a.B = s.B; a.N = s.N; a.Ns = s.Ns; a.Hq = s.Hq; a.Hkv = s.Hkv; a.n_rows = s.n_rows; a.max_pos = s.max_pos;
   a.scale_log2 = s.scale * kLog2e;

@@ -51,6 +51,7 @@ struct lumo_ctx {
   size_t scratch_bytes = 0;
   void* attn_scratch = nullptr; // partial results of the attention partitions
   size_t attn_scratch_bytes = 0;
+  uint32_t attn_launch_id = 0;
   // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
   int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form with forward substitution, 3 solved Gram form
   bool timeout_drill = false;   // test aid: the tensor-core scan skips its tensor-core work (lumo_ctx_set_timeout_drill)
@@ -314,6 +315,8 @@ struct AttnArgs {
   float* out; float* lse;
   float* part_o; float* part_lse;
   int2* unit_slots;   // per unit: first slot and slot count of its segments, written by the attention kernel
+  uint32_t* fail_flag;   // set to launch_id by an attention CTA whose bounded wait ran out
+  uint32_t launch_id;    // distinct per launch (never 0), so that the flag needs no clearing
   const int32_t* ctx_len; const int32_t* cache_row;
   const uint32_t* vis; const uint32_t* used;
   int32_t* status;
@@ -344,7 +347,7 @@ int attn_row_tiles(int G, int N);
 // scratch for the segments' partial results
 size_t attn_scratch_bytes(const AttnShape& s, int sm_count);
 cudaError_t attn_plan(const AttnShape& s, const AttnLayerPtrs& p, const uint32_t* vis, const uint32_t* used, float* scratch,
-                      int sm_count, AttnPlan* plan, std::string* err);
+                      int sm_count, uint32_t launch_id, AttnPlan* plan, std::string* err);
 cudaError_t launch_attn(const AttnPlan& plan, cudaStream_t st);
 cudaError_t launch_attn_merge(const AttnPlan& plan, cudaStream_t st);
 cudaError_t launch_kv_write(const KvLayers& L, const KvShape& s, int n_layers, cudaStream_t st);
