@@ -59,6 +59,7 @@ constexpr int kTmemCols = 512;        // S buffers: columns 0..127 and 128..255,
 constexpr int kColO = 256;
 constexpr int kColQ = 384;
 constexpr int kColP = 448;
+constexpr int kSeqCache = 64;         // sequences whose context length, cache row and tile count are kept in shared memory
 constexpr int kMinTilesPerCta = 4;    // automatic mode: do not cut the work finer than this
 constexpr float kRescaleStep = 16.f;  // the reference maximum moves when exceeded by more than this (log2 units)
 constexpr uint32_t kSpinLimit = 1u << 24;
@@ -78,10 +79,11 @@ struct Small {
   unsigned long long q_full, o_free;
   uint32_t tmem_base;
   uint32_t timed_out;
+  int seq_ctx[kSeqCache], seq_row[kSeqCache], seq_nt[kSeqCache];   // ctx_len, cache_row and tile count of the first sequences
   float xchg[2][2][kRows];           // [tile parity][key half][row]: row maxima (and row sums at a segment's end)
 };
-constexpr int kSmemBytes = kOffSmall + 2560;
-static_assert(sizeof(Small) <= 2560, "small block");
+constexpr int kSmemBytes = kOffSmall + 3584;
+static_assert(sizeof(Small) <= 3584, "small block");
 static_assert(kSmemBytes + 1024 <= 227 * 1024, "one CTA per SM");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -130,11 +132,18 @@ __device__ __forceinline__ bool mbar_wait_relaxed(unsigned long long* bar, uint3
 
 // One box of a 4-d tiled tensor map (dh, KV head, position, cache row) into shared memory; completion
 // is counted in bytes on `bar`.  c0 is 0 or 64 elements: a multiple of 16 bytes.
+// The keys and values stream through once: they carry an evict-first L2 policy, so that what is reused across
+// tiles and launches (queries, partial results, tables, the kernel's own instructions) stays in L2.
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, unsigned long long* bar, int c0, int c1,
-                                            int c2, int c3) {
+                                            int c2, int c3, uint64_t policy) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
-      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5, %6}], [%2], %7;\n"
+      ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;\n" : "=l"(p));
+  return p;
 }
 
 // shared-memory matrix descriptor, 128-byte swizzle
@@ -213,6 +222,7 @@ struct Segment {
 
 struct Work {
   const AttnArgs& a;
+  const Small& sm;
   int b, q;           // current sequence, unit within the sequence
   int g, g_end;       // next global tile, end of this CTA's share (the host bounds the tile count below 2^31)
   int g_unit;         // global tile at which the current unit starts
@@ -220,7 +230,8 @@ struct Work {
   int per;            // automatic mode: tiles per CTA
   bool fixed_done;
 
-  static __device__ __forceinline__ int tiles_of(const AttnArgs& a, int bb, int* ctx, int* crow) {
+  __device__ __forceinline__ int tiles_of(const AttnArgs& a, int bb, int* ctx, int* crow) const {
+    if (bb < kSeqCache) { *ctx = sm.seq_ctx[bb]; *crow = sm.seq_row[bb]; return sm.seq_nt[bb]; }
     *ctx = a.ctx_len[bb];
     *crow = a.cache_row[bb];
     if (seq_check(*ctx, *crow, a.Ns, a.n_rows, a.max_pos) != LUMO_SEQ_OK) return 0;
@@ -248,7 +259,7 @@ struct Work {
     }
   }
 
-  __device__ explicit Work(const AttnArgs& args) : a(args) { init(); }
+  __device__ Work(const AttnArgs& args, const Small& small) : a(args), sm(small) { init(); }
 
   // next segment of this CTA; false when the share is exhausted
   __device__ __forceinline__ bool next(Segment* s) {
@@ -321,12 +332,17 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     sm.timed_out = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
   }
+  if (tid < kSeqCache && tid < a.B) {          // the work iterator of every role reads these instead of global memory
+    const int cx = a.ctx_len[tid], cr = a.cache_row[tid];
+    sm.seq_ctx[tid] = cx; sm.seq_row[tid] = cr;
+    sm.seq_nt[tid] = seq_check(cx, cr, a.Ns, a.n_rows, a.max_pos) == LUMO_SEQ_OK ? (cx + a.Ns + kKeys - 1) / kKeys : 0;
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
-  Work work(a);
+  Work work(a, sm);
   Segment sg;
   bool ok = aligned;
   uint32_t it = 0;        // tiles this CTA has started, over all segments: ring stage, S buffer and phases
@@ -340,18 +356,23 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       unsigned long long* full = is_v ? sm.v_full : sm.k_full;
       unsigned long long* empty = is_v ? sm.v_empty : sm.k_empty;
       const uint32_t ring = sbase + (is_v ? kOffV : kOffK);
+      const uint64_t stream_policy = l2_evict_first_policy();
       while (work.next(&sg)) {
         for (int j = 0; j < sg.n; ++j, ++it) {
           const uint32_t st = it % kStages, use = it / kStages;
           if (use > 0 && ok) ok = mbar_wait(&empty[st], (use - 1) & 1u);
+          // Start-up: the rings of all CTAs fill at once (28 MB in flight) and the first segment's query rows
+          // would queue behind them (measured: 3.4 us for 256 bytes per thread).  Only the first K tile goes
+          // ahead of the queries; everything else waits for their arrival in tensor memory.
+          if (it == (is_v ? 0u : 1u) && ok) ok = mbar_wait(&sm.q_full, 0);
           if (!ok) continue;
           mbar_expect_tx(&full[st], kTileBytes);
           const uint32_t dst = ring + st * kTileBytes;
           const int pos = (sg.t0 + j) * kKeys;
           // tensor-map dimensions ascend in stride: (dh, head, position, row) or (dh, position, head, row)
           const int c1 = a.layout ? pos : sg.hkv, c2 = a.layout ? sg.hkv : pos;
-          tma_load_4d(dst, map, &full[st], 0, c1, c2, sg.crow);
-          tma_load_4d(dst + kHalfBytes, map, &full[st], 64, c1, c2, sg.crow);
+          tma_load_4d(dst, map, &full[st], 0, c1, c2, sg.crow, stream_policy);
+          tma_load_4d(dst + kHalfBytes, map, &full[st], 64, c1, c2, sg.crow, stream_policy);
         }
       }
       if (!ok) sm.timed_out = 1u;
@@ -425,7 +446,33 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const int pair_bar = 1 + (warp & 3);         // named barrier of the two warps of a lane quarter
     const float sl2 = a.scale_log2;
     const int GN = a.G * a.N;
-    while (work.next(&sg)) {
+    // Query tile of a segment into tensor memory: this thread's half of its row, two bf16 per column (zeros
+    // beyond the group); then one arrival per warp on q_full.  Called when the S products of the segment before
+    // have all completed (every thread awaited their s_full phases): for the first segment at once, for the
+    // others right after the last tile's probabilities have been handed over, BEFORE that segment's read-out,
+    // so that the next logits are computed while the accumulator is being written out.
+    auto store_q = [&](const Segment& g) {
+      const int rgq = g.rt * kRows + row;
+      const bool okq = rgq < GN;
+      const int hq = okq ? rgq / a.N : 0, nq = okq ? rgq - hq * a.N : 0;
+      const uint4* qrow = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
+                                                         (((size_t)g.b * a.N + nq) * a.Hq + (size_t)g.hkv * a.G + hq) * kDh);
+      uint32_t qr[32];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 v = okq ? __ldg(qrow + half * 8 + c) : make_uint4(0u, 0u, 0u, 0u);
+        qr[4 * c] = v.x; qr[4 * c + 1] = v.y; qr[4 * c + 2] = v.z; qr[4 * c + 3] = v.w;
+      }
+      tmem_st32(tmem_lane + kColQ + half * 32, qr);
+      tmem_st_wait();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.q_full);
+    };
+    Segment sgn;
+    bool have = work.next(&sg);
+    if (have && sg.n > 0) store_q(sg);
+    for (; have; sg = sgn) {
       const int rg = sg.rt * kRows + row;
       const bool row_ok = rg < GN;
       const int hl = row_ok ? rg / a.N : 0, node = row_ok ? rg - hl * a.N : 0;
@@ -437,26 +484,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           for (int e = 0; e < 16; ++e) reinterpret_cast<float4*>(slot_o)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
           if (half == 0) *slot_l = -INFINITY;
         }
+        have = work.next(&sgn);                  // (an empty partition is a CTA's only segment)
+        if (have && sgn.n > 0) store_q(sgn);
         continue;
       }
-      // query tile into tensor memory: this thread's half of its row, two bf16 per column (zeros beyond the
-      // group).  The previous segment's S products have all completed (their s_full phases were awaited).
-      {
-        const uint4* qrow = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.q) +
-                                                           (((size_t)sg.b * a.N + node) * a.Hq + (size_t)sg.hkv * a.G + hl) * kDh);
-        uint32_t qr[32];
-#pragma unroll
-        for (int c = 0; c < 8; ++c) {
-          const uint4 v = row_ok ? __ldg(qrow + half * 8 + c) : make_uint4(0u, 0u, 0u, 0u);
-          qr[4 * c] = v.x; qr[4 * c + 1] = v.y; qr[4 * c + 2] = v.z; qr[4 * c + 3] = v.w;
-        }
-        tmem_st32(tmem_lane + kColQ + half * 32, qr);
-        tmem_st_wait();
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.q_full);
-
       const uint32_t* visw = a.vis + ((size_t)sg.b * a.N + node) * 8;
       const uint32_t* usedw = a.used + (size_t)sg.b * 8;
       float m = -INFINITY, l = 0.f;              // reference maximum (log2 units), this thread's part of the row sum
@@ -577,7 +608,10 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           mbar_arrive(&sm.p_full);
         }
       }
-      // end of the segment: the last O product, then normalise and write the slot
+      // end of the segment.  First the next segment's queries (its logits then run under this read-out) ...
+      have = work.next(&sgn);
+      if (have && sgn.n > 0) store_q(sgn);
+      // ... then the last O product, normalise and write the slot
       if (ok) ok = mbar_wait(&sm.v_empty[(it - 1) % kStages], ((it - 1) / kStages) & 1u);
       tc_fence_after();
       sm.xchg[0][half][row] = l;
