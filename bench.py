@@ -37,7 +37,7 @@ L2_BYTES = 126 * 2 ** 20
 
 
 def make_case(name: str, seed_offset: int = 0):
-    from paper_2609_23900_b200 import workload as W
+    from synthetic import workload as W
     if name == "cfg1":
         return W.config1(seed=W.BASE_SEED + 1 + 1000 * seed_offset)
     if name == "cfg2":
@@ -201,7 +201,7 @@ def oracle_walk_mode():
     """The oracle in its literal form (every node recomputed from the pre-tree state along its ancestry,
     "walk" mode), scan only, on configs 0-2: nodes per second."""
     from oracle import gdn_oracle as O
-    from paper_2609_23900_b200 import workload as W
+    from synthetic import workload as W
     out = {}
     for name, case in (("cfg0", W.config0()), ("cfg1", W.config1()), ("cfg2", W.config2())):
         L = case.layers[0]
@@ -269,7 +269,7 @@ def measure_extra_config(ctx, name, out_dtype, peak_gbs, steps=20, warmup=3, sna
     roofline fractions.  Fewer steps than the headline so that the whole run stays within minutes."""
     import torch
     from paper_2609_23900_b200 import binding
-    from paper_2609_23900_b200.runtime import DeviceCase
+    from synthetic.device_case import DeviceCase
     cases = [make_case(name, seed_offset=i) for i in range(n_sets)]
     c0 = cases[0]
     sets = [DeviceCase(ctx, c, out_dtype=out_dtype, snapshot_mode=snapshot_mode) for c in cases]
@@ -350,7 +350,7 @@ def measure_attention(ctx, peak_gbs, steps=30, warmup=4, B=8, context=16384, Hq=
     import numpy as np
     import torch
     from paper_2609_23900_b200 import binding
-    from paper_2609_23900_b200 import workload as W
+    from synthetic import workload as W
     dev = torch.device("cuda", ctx.device)
     tree = W.tree_paper_geometry()
     N, Ns, dh = len(tree), 32, 128
@@ -490,7 +490,7 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2609_23900_b200 import binding
-    from paper_2609_23900_b200.runtime import DeviceCase
+    from synthetic.device_case import DeviceCase
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the GDN tree verifier has no CPU fallback")

@@ -7,7 +7,7 @@ from typing import List, Optional
 import numpy as np
 import torch
 
-from . import binding
+from paper_2609_23900_b200 import binding
 from .workload import Case
 
 _TORCH_DT = {"f32": torch.float32, "bf16": torch.bfloat16}

@@ -18,7 +18,7 @@ sys.path.insert(0, ROOT)
 
 from oracle import gdn_oracle as O          # noqa: E402
 from oracle import tree_tables as T         # noqa: E402
-from paper_2609_23900_b200 import workload as W   # noqa: E402
+from synthetic import workload as W   # noqa: E402
 
 
 def compute():

@@ -5,7 +5,7 @@ import torch
 
 from oracle import gdn_oracle as O
 from paper_2609_23900_b200 import binding
-from paper_2609_23900_b200.runtime import DeviceCase
+from synthetic.device_case import DeviceCase
 
 _ctx = None
 
@@ -21,7 +21,7 @@ def ctx(algo="auto"):
 
 def gram_eligible(c) -> bool:
     """Shapes the tensor-core Gram-form scan takes: d = 128, bf16 operands, depth <= 16."""
-    from paper_2609_23900_b200 import workload as W
+    from synthetic import workload as W
     depth = max(max(W.tree_depths(p.tolist())) for p in c.parent)
     return c.d == 128 and c.in_dtype == "bf16" and depth <= 16
 

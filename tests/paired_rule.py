@@ -26,8 +26,8 @@ import numpy as np
 import torch
 
 from oracle import gdn_oracle as O
-from paper_2609_23900_b200 import workload as W
-from paper_2609_23900_b200.runtime import DeviceCase
+from synthetic import workload as W
+from synthetic.device_case import DeviceCase
 
 
 def native_chain_outputs(ctx, dc, layer=0):

@@ -30,8 +30,8 @@ def test_oracle_reproduces_stored_values():
 @pytest.mark.gpu
 def test_cuda_path_matches_stored_values():
     import torch
-    from paper_2609_23900_b200 import workload as W
-    from paper_2609_23900_b200.runtime import DeviceCase
+    from synthetic import workload as W
+    from synthetic.device_case import DeviceCase
     from tests.harness import ctx
     c = W.config0()
     dc = DeviceCase(ctx("auto"), c, use_conv=False, snapshot_mode=1, snap_nodes=[[6]])

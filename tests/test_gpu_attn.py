@@ -15,8 +15,8 @@ import torch
 
 from oracle import attn_oracle as A
 from paper_2609_23900_b200 import binding
-from paper_2609_23900_b200 import workload as W
-from paper_2609_23900_b200.runtime import DeviceAttnCase
+from synthetic import workload as W
+from synthetic.device_case import DeviceAttnCase
 from tests.harness import ctx
 
 pytestmark = pytest.mark.gpu

@@ -6,8 +6,8 @@ import pytest
 import torch
 
 from oracle import gdn_oracle as O
-from paper_2609_23900_b200 import workload as W
-from paper_2609_23900_b200.runtime import DeviceCase
+from synthetic import workload as W
+from synthetic.device_case import DeviceCase
 from tests.harness import assert_close, ctx
 
 pytestmark = pytest.mark.gpu

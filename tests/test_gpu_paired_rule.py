@@ -5,8 +5,8 @@ import numpy as np
 import pytest
 import torch
 
-from paper_2609_23900_b200 import workload as W
-from paper_2609_23900_b200.runtime import DeviceCase
+from synthetic import workload as W
+from synthetic.device_case import DeviceCase
 from tests.harness import ctx
 from tests.paired_rule import paired_rule
 

@@ -12,8 +12,8 @@ import torch
 from oracle import gdn_oracle as O
 from oracle import tree_tables as T
 from paper_2609_23900_b200 import binding
-from paper_2609_23900_b200 import workload as W
-from paper_2609_23900_b200.runtime import DeviceCase
+from synthetic import workload as W
+from synthetic.device_case import DeviceCase
 from tests.harness import assert_close, ctx, gram_eligible, oracle_commit_from_device, oracle_scan_from_device
 
 pytestmark = pytest.mark.gpu

@@ -13,8 +13,8 @@ import pytest
 import torch
 
 from paper_2609_23900_b200 import binding
-from paper_2609_23900_b200 import workload as W
-from paper_2609_23900_b200.runtime import DeviceCase
+from synthetic import workload as W
+from synthetic.device_case import DeviceCase
 from tests.harness import ctx, oracle_commit_from_device, oracle_scan_from_device
 
 pytestmark = pytest.mark.gpu
@@ -25,8 +25,9 @@ _CHILD = r"""
 import hashlib, sys
 sys.path.insert(0, %r)
 import torch
-from paper_2609_23900_b200 import binding, workload as W
-from paper_2609_23900_b200.runtime import DeviceCase
+from paper_2609_23900_b200 import binding
+from synthetic import workload as W
+from synthetic.device_case import DeviceCase
 ctx = binding.Context(0)
 h = hashlib.sha256()
 for algo in ("gram", "solve", "rank1"):

@@ -15,7 +15,7 @@ entry.build()
 
 from oracle import tree_tables as T                      # noqa: E402
 from paper_2609_23900_b200 import binding               # noqa: E402
-from paper_2609_23900_b200 import workload as W         # noqa: E402
+from synthetic import workload as W         # noqa: E402
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 

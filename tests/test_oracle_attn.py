@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from oracle import attn_oracle as A
-from paper_2609_23900_b200 import workload as W
+from synthetic import workload as W
 
 
 def make(parents, *, seed=0, Hq=4, Hkv=2, dh=16, ctx=(5, 9), Ns=None, permute=False, S=None):

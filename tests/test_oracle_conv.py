@@ -10,7 +10,7 @@ import torch
 import torch.nn.functional as F
 
 from oracle import gdn_oracle as O
-from paper_2609_23900_b200 import workload as W
+from synthetic import workload as W
 
 TINY = [-1, -1, 0, 0, 1, 1, 2]
 

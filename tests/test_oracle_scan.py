@@ -11,7 +11,7 @@ import scipy.linalg
 
 from oracle import gdn_oracle as O
 from oracle import tree_tables as T
-from paper_2609_23900_b200 import workload as W
+from synthetic import workload as W
 
 TINY = [-1, -1, 0, 0, 1, 1, 2]
 

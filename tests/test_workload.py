@@ -2,7 +2,7 @@
 import numpy as np
 import torch
 
-from paper_2609_23900_b200 import workload as W
+from synthetic import workload as W
 
 
 def test_streams_are_counter_based_and_reproducible():

@@ -11,8 +11,8 @@ import pytest
 import torch
 
 from paper_2609_23900_b200 import binding
-from paper_2609_23900_b200 import workload as W
-from paper_2609_23900_b200.runtime import DeviceCase
+from synthetic import workload as W
+from synthetic.device_case import DeviceCase
 
 pytestmark = pytest.mark.gpu
 
