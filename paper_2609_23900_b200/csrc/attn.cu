@@ -663,36 +663,51 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   float4* dst = reinterpret_cast<float4*>(a.out + out_row * kDh) + lane;
   const int upb = a.Hkv * a.RT;
   const int u = b * upb + hkv * a.RT + rt;
-  // this unit's slots, as the attention kernel recorded them; a sequence that fails its check owns none
-  int slot0 = 0, nslot = 0;
-  if (seq_check(a.ctx_len[b], a.cache_row[b], a.Ns, a.n_rows, a.max_pos) == LUMO_SEQ_OK) {
-    const int2 t = a.unit_slots[u];
-    slot0 = t.x; nslot = t.y;
-  }
+  // Three independent loads first (one round trip): the sequence's context length and cache row, and the slot
+  // range the attention kernel recorded for this unit (meaningless for a sequence that fails its check).
+  const int cx = a.ctx_len[b], cr = a.cache_row[b];
+  const int2 t = a.unit_slots[u];
+  const int st = seq_check(cx, cr, a.Ns, a.n_rows, a.max_pos);
   // status word of the sequence: its check, else whether any wait of this launch's attention kernel ran out
   // (then the outputs of the whole call are suspect)
-  if (a.status && lane == 0 && hkv == 0 && rg == 0) {
-    const int st = seq_check(a.ctx_len[b], a.cache_row[b], a.Ns, a.n_rows, a.max_pos);
+  if (a.status && lane == 0 && hkv == 0 && rg == 0)
     a.status[b] = st != LUMO_SEQ_OK ? st : (*a.fail_flag == a.launch_id ? (int)LUMO_SEQ_TIMEOUT : (int)LUMO_SEQ_OK);
-  }
-  if (nslot == 0) {                          // the sequence failed its check (it owns no tiles): zeros
+  if (st != LUMO_SEQ_OK) {                   // the sequence owns no tiles: zeros
     *dst = make_float4(0.f, 0.f, 0.f, 0.f);
     if (a.lse && lane == 0) a.lse[out_row] = 0.f;
     return;
   }
+  const int slot0 = t.x, nslot = t.y;
   const size_t base = (size_t)slot0 * kRows + r;
+  // Second round trip: four slots at a time, their log-sum-exps (one per lane) and their rows together; the
+  // combination itself runs in slot order against the maximum of all log-sum-exps.
   float mx = -INFINITY;
-  for (int s = 0; s < nslot; ++s) mx = fmaxf(mx, a.part_lse[base + (size_t)s * kRows]);
+  for (int s0 = 0; s0 < nslot; s0 += 32) {
+    const float ls = (s0 + lane < nslot) ? a.part_lse[base + (size_t)(s0 + lane) * kRows] : -INFINITY;
+    mx = fmaxf(mx, ls);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   float den = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s = 0; s < nslot; ++s) {
-    const float ls = a.part_lse[base + (size_t)s * kRows];
-    if (ls == -INFINITY) continue;
-    const float wgt = ex2(ls - mx);
-    const float4 v = reinterpret_cast<const float4*>(a.part_o + (base + (size_t)s * kRows) * kDh)[lane];
-    den += wgt;
-    acc.x = fmaf(wgt, v.x, acc.x); acc.y = fmaf(wgt, v.y, acc.y);
-    acc.z = fmaf(wgt, v.z, acc.z); acc.w = fmaf(wgt, v.w, acc.w);
+  for (int s0 = 0; s0 < nslot; s0 += 4) {
+    float ls[4];
+    float4 v[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const bool in = s0 + k < nslot;
+      ls[k] = in ? a.part_lse[base + (size_t)(s0 + k) * kRows] : -INFINITY;
+      v[k] = in ? reinterpret_cast<const float4*>(a.part_o + (base + (size_t)(s0 + k) * kRows) * kDh)[lane]
+                : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (ls[k] == -INFINITY) continue;      // an empty slot (or none)
+      const float wgt = ex2(ls[k] - mx);
+      den += wgt;
+      acc.x = fmaf(wgt, v[k].x, acc.x); acc.y = fmaf(wgt, v[k].y, acc.y);
+      acc.z = fmaf(wgt, v[k].z, acc.z); acc.w = fmaf(wgt, v[k].w, acc.w);
+    }
   }
   const float inv = den > 0.f ? 1.f / den : 0.f;
   *dst = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
