@@ -706,7 +706,7 @@ int prepare_attn(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args
     return fail(ctx, LUMO_ERR_UNSUPPORTED, "a cache row must span less than 2^40 bytes");
   if (!a0.ctx_len || !a0.cache_row) return fail(ctx, LUMO_ERR_ARG, "ctx_len and cache_row are required");
   // the kernels count key tiles of all (sequence, KV head, row tile) units in 32 bits
-  if ((double)desc->B * a0.Hkv * attn_row_tiles(a0.Hq / a0.Hkv, desc->N) * ((double)a0.max_positions / 128 + 1) >= 2147483648.0)
+  if ((double)desc->B * a0.Hkv * attn_row_tiles(a0.Hq / a0.Hkv, desc->N) * ((double)a0.max_positions / 128 + 8) >= 2147483648.0)
     return fail(ctx, LUMO_ERR_UNSUPPORTED, "batch x KV heads x positions too large for one call");
   if (a0.kv_layout != 0 && a0.kv_layout != 1) return fail(ctx, LUMO_ERR_ARG, "kv_layout must be 0 or 1");
   if (a0.n_splits < 0 || a0.n_splits > 32) return fail(ctx, LUMO_ERR_ARG, "n_splits must be 0 (automatic) or in [1, 32]");

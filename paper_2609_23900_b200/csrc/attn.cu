@@ -60,6 +60,8 @@ constexpr int kColO = 256;
 constexpr int kColQ = 384;
 constexpr int kColP = 448;
 constexpr int kSeqCache = 64;         // sequences whose context length, cache row and tile count are kept in shared memory
+constexpr int kUnitCost = 5;          // what starting a unit costs a CTA (read-out of the one before, new queries, refill of
+                                      // the pipeline: ~8 us measured), in tiles: the shares are evened out in these terms
 constexpr int kMinTilesPerCta = 4;    // automatic mode: do not cut the work finer than this
 constexpr float kRescaleStep = 16.f;  // the reference maximum moves when exceeded by more than this (log2 units)
 constexpr uint32_t kSpinLimit = 1u << 24;
@@ -209,8 +211,9 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 
 // ---- work decomposition ----------------------------------------------------------------
 // Units are numbered u = (b * Hkv + hkv) * RT + rt; unit u owns nt(b) tiles (0 for a sequence that fails
-// its check).  Automatic mode: CTA c owns the global tiles [c * per, (c + 1) * per) and the slot of a
-// segment is u + c (strictly increasing along the tile list, so unique).  Fixed mode (S partitions):
+// its check).  Automatic mode: the units are laid end to end on a line, each preceded by kUnitCost idle
+// positions (the price of starting it); CTA c owns the positions [c * per, (c + 1) * per), works on the tiles
+// among them, and the slot of a segment is u + c (strictly increasing along the line, so unique).  Fixed mode (S partitions):
 // CTA c owns partition c mod S of unit c / S, slot c.
 struct Segment {
   int b, hkv, rt;     // unit
@@ -224,10 +227,10 @@ struct Work {
   const AttnArgs& a;
   const Small& sm;
   int b, q;           // current sequence, unit within the sequence
-  int g, g_end;       // next global tile, end of this CTA's share (the host bounds the tile count below 2^31)
-  int g_unit;         // global tile at which the current unit starts
+  int g, g_end;       // next position on the line, end of this CTA's share (the host bounds the line below 2^31)
+  int g_unit;         // position at which the current unit's stretch (idle prefix, then its tiles) starts
   int nt;             // tiles per unit of the current sequence
-  int per;            // automatic mode: tiles per CTA
+  int per;            // automatic mode: positions per CTA
   bool fixed_done;
 
   __device__ __forceinline__ int tiles_of(const AttnArgs& a, int bb, int* ctx, int* crow) const {
@@ -244,17 +247,20 @@ struct Work {
     const int upb = a.Hkv * a.RT;       // units per sequence
     int total = 0;
     int cx, cr;
-    for (int bb = 0; bb < a.B; ++bb) total += tiles_of(a, bb, &cx, &cr) * upb;
+    for (int bb = 0; bb < a.B; ++bb) {
+      const int n = tiles_of(a, bb, &cx, &cr);
+      if (n > 0) total += (n + kUnitCost) * upb;
+    }
     per = (total + (int)gridDim.x - 1) / (int)gridDim.x;
     if (per < kMinTilesPerCta) per = kMinTilesPerCta;
     g = (int)blockIdx.x * per;
     g_end = g + per < total ? g + per : total;
-    // position on the unit that holds tile g
+    // the unit whose stretch holds position g
     int acc = 0;
     for (b = 0; b < a.B; ++b) {
       nt = tiles_of(a, b, &cx, &cr);
-      const int span = nt * upb;
-      if (g < acc + span) { q = (g - acc) / nt; g_unit = acc + q * nt; break; }
+      const int span = nt > 0 ? (nt + kUnitCost) * upb : 0;
+      if (g < acc + span) { q = (g - acc) / (nt + kUnitCost); g_unit = acc + q * (nt + kUnitCost); break; }
       acc += span;
     }
   }
@@ -279,8 +285,8 @@ struct Work {
       return n_all > 0;
     }
     while (g < g_end && b < a.B) {
-      if (nt == 0 || g >= g_unit + nt) {     // move to the next unit (skipping sequences without tiles)
-        if (nt > 0) g_unit += nt;
+      if (nt == 0 || g >= g_unit + nt + kUnitCost) {     // move to the next unit (skipping sequences without tiles)
+        if (nt > 0) g_unit += nt + kUnitCost;
         if (nt == 0 || ++q == upb) {
           q = 0;
           int cx, cr;
@@ -288,17 +294,20 @@ struct Work {
         }
         continue;
       }
+      const int first = g_unit + kUnitCost;              // position of the unit's tile 0
+      const int lo = g > first ? g : first;
+      const int hi = first + nt < g_end ? first + nt : g_end;
+      g = g_unit + nt + kUnitCost < g_end ? g_unit + nt + kUnitCost : g_end;
+      if (lo >= hi) continue;                            // only idle positions of this unit fall into the share
       const int u = b * upb + q;
       s->b = b; s->hkv = q / a.RT; s->rt = q - s->hkv * a.RT;
       tiles_of(a, b, &s->ctx, &s->crow);
-      s->t0 = g - g_unit;
-      const int end = g_unit + nt < g_end ? g_unit + nt : g_end;
-      s->n = end - g;
+      s->t0 = lo - first;
+      s->n = hi - lo;
       s->slot = u + blockIdx.x;
       s->unit = u;
-      s->slot0 = u + g_unit / per;
-      s->nslots = (g_unit + nt - 1) / per - g_unit / per + 1;
-      g = end;
+      s->slot0 = u + first / per;
+      s->nslots = (first + nt - 1) / per - first / per + 1;
       return true;
     }
     return false;
