@@ -12,7 +12,9 @@
  * Around these: lumo_gdn_commit_verify (the commit of the previous cycle folded into the next
  * verify), lumo_tree_accept (device-resident acceptance walk between verify and commit),
  * lumo_select_spine_top3 (fused draft selection upstream of the tree), lumo_gdn_tree_scan_static
- * (the scan with library-internal static scratch) and small helpers.
+ * (the scan with library-internal static scratch), the attention half of the same cycle
+ * (lumo_kv_write_tree, lumo_tree_attention, lumo_kv_publish: the tree's KV entries written, read and
+ * re-linearised through the same slot map) and small helpers.
  *
  * Conventions
  *   - One GPU.  All tensor pointers are DEVICE pointers owned by the caller unless a
