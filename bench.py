@@ -345,7 +345,7 @@ def measure_attention(ctx, peak_gbs, steps=30, warmup=4, B=8, context=16384, Hq=
     rows, spine-first slots): tree KV write, ancestry-masked decode attention and KV publication of one
     full-attention layer, timed back to back over rotating cache sets larger than L2.  The paper states no
     head counts or context lengths for its model: 32 query / 8 KV heads of 128 and a 16k-token context per
-    sequence stand in for a coding-agent request (the design doc gives the recipe).  Inputs are drawn on the
+    sequence stand in for a coding-agent request.  Inputs are drawn on the
     device; parity with the oracle is the tests' business."""
     import numpy as np
     import torch
