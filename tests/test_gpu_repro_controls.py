@@ -14,7 +14,7 @@ import torch
 
 from paper_2609_23900_b200 import binding
 from synthetic import workload as W
-from synthetic.device_case import DeviceCase
+from synthetic.device_case import DeviceAttnCase, DeviceCase
 from tests.harness import ctx, oracle_commit_from_device, oracle_scan_from_device
 
 pytestmark = pytest.mark.gpu
@@ -27,7 +27,7 @@ sys.path.insert(0, %r)
 import torch
 from paper_2609_23900_b200 import binding
 from synthetic import workload as W
-from synthetic.device_case import DeviceCase
+from synthetic.device_case import DeviceAttnCase, DeviceCase
 ctx = binding.Context(0)
 h = hashlib.sha256()
 for algo in ("gram", "solve", "rank1"):
@@ -153,3 +153,55 @@ def test_stale_publication_metadata_is_detected_or_refused():
     dc.commit()
     torch.cuda.synchronize()
     assert torch.equal(dc.t("state"), clean)
+
+
+_ATTN_CHILD = r"""
+import hashlib, sys
+sys.path.insert(0, %r)
+import torch
+from paper_2609_23900_b200 import binding
+from synthetic import workload as W
+from synthetic.device_case import DeviceAttnCase
+ctx = binding.Context(0)
+cases = []
+for k, (ctxs, splits, layout) in enumerate([([700, 45], 0, "spine"), ([700, 45], 4, "spine"), ([1999, 64, 3], 0, "permuted"),
+                                            ([129, 128], 1, "identity"), ([5000], 0, "spine"), ([5000], 8, "permuted"),
+                                            ([0, 1, 2, 3], 2, "spine"), ([16000, 900], 0, "spine")]):
+    for kv_layout in (0, 1):
+        cases.append((k, ctxs, splits, layout, kv_layout))
+for k, ctxs, splits, layout, kv_layout in cases:                     # sixteen cases
+    c = W.make_attn_case("det", [W.tree_paper_geometry()] * len(ctxs), ctxs, seed=W.BASE_SEED + 300 + k, Hq=8, Hkv=2, Ns=32,
+                         layout=layout)
+    h = hashlib.sha256()
+    for rep in range(2):
+        dc = DeviceAttnCase(ctx, c, n_splits=splits, kv_layout=kv_layout)
+        dc.write(); dc.attend(); dc.publish()
+        torch.cuda.synchronize()
+        for name in ("out", "lse", "k_cache", "v_cache", "status"):
+            h.update(dc.t(name).cpu().contiguous().view(torch.uint8).numpy().tobytes())
+        h.update(dc.ctx_len_out.cpu().numpy().tobytes())
+        print(k, kv_layout, rep, h.hexdigest())
+"""
+
+
+def test_attention_sixteen_cases_repeat_bit_for_bit_within_and_across_processes():
+    """Sec. "Numerical and candidate-selection validation": the attention kernel's outputs and log-sum-exps
+    repeat bit for bit within each of sixteen cases, with matching digests across two processes.  (Written
+    KV entries, publication and status words are folded into the digests as well.)"""
+    outs = []
+    for _ in range(2):
+        r = subprocess.run([sys.executable, "-c", _ATTN_CHILD % ROOT], capture_output=True, text=True, timeout=600)
+        assert r.returncode == 0, r.stderr[-2000:]
+        outs.append(r.stdout.strip().splitlines())
+    assert outs[0] == outs[1] and len(outs[0]) == 32
+    # within a case the second run must extend the digest by the same bytes as the first: check the runs directly
+    c = W.make_attn_case("det", [W.tree_paper_geometry()] * 2, [700, 45], seed=W.BASE_SEED + 300, Hq=8, Hkv=2, Ns=32, layout="spine")
+    ref = None
+    for rep in range(3):
+        dc = DeviceAttnCase(ctx(), c, n_splits=0)
+        dc.write(); dc.attend()
+        torch.cuda.synchronize()
+        got = (dc.t("out").clone(), dc.t("lse").clone())
+        if ref is not None:
+            assert torch.equal(ref[0], got[0]) and torch.equal(ref[1], got[1])
+        ref = got
