@@ -340,7 +340,7 @@ def measure_extra_config(ctx, name, out_dtype, peak_gbs, steps=20, warmup=3, sna
     return out
 
 
-def measure_attention(ctx, peak_gbs, steps=30, warmup=4, B=8, context=16384, Hq=32, Hkv=8, n_sets=2):
+def measure_attention(ctx, peak_gbs, steps=30, warmup=4, B=8, context=16384, Hq=32, Hkv=8, n_sets=2, with_oracle=False):
     """The attention half of the verifier on the paper's tree geometry (28 candidates + root padded to 32
     rows, spine-first slots): tree KV write, ancestry-masked decode attention and KV publication of one
     full-attention layer, timed back to back over rotating cache sets larger than L2.  The paper states no
@@ -426,6 +426,36 @@ def measure_attention(ctx, peak_gbs, steps=30, warmup=4, B=8, context=16384, Hq=
            "timing": f"{steps} back-to-back calls between two CUDA events, {n_sets} cache sets of {kv // 2 ** 20} MiB each rotated (larger than L2)",
            "accepted": "even sequences accept six spine nodes (in place under the spine-first map: no bytes move), odd ones a rescue branch",
            "status_ok_and_finite": ok}
+    if with_oracle:
+        # error of the timed launch against the fp64 oracle on sampled (sequence, query head) pairs, every node
+        # (CPU-baseline leg only: the oracle is test infrastructure)
+        from oracle import attn_oracle as A
+        L = layers[0]
+        ctx.kv_write_tree(desc, packs[0])
+        ctx.tree_attention(desc, packs[0])
+        torch.cuda.synchronize()
+        f64 = lambda t: t.to(torch.float64).cpu().numpy()
+        outs, lses, q = f64(L.tensors["out"]), f64(L.tensors["lse"]), f64(L.tensors["q"])
+        G = Hq // Hkv
+        max_abs, max_ratio, max_lse_ulp, n_el = 0.0, 0.0, 0.0, 0
+        for b, h in ((0, 0), (B // 2, Hq // 2 + 1), (B - 1, Hq - 1)):
+            g = h // G
+            k1 = f64(L.tensors["k_cache"][b:b + 1, :, g:g + 1])
+            v1 = f64(L.tensors["v_cache"][b:b + 1, :, g:g + 1])
+            one = lambda a_: a_[b:b + 1]
+            args_ = (one(parent), one(slot), q[b:b + 1, :, h:h + 1], k1, v1, np.asarray([context]), np.zeros(1, np.int32), dh ** -0.5)
+            ref, rl = A.tree_attention(*args_)
+            bound, _ = A.tree_attention(args_[0], args_[1], args_[2], k1, np.abs(v1), *args_[5:])
+            err = np.abs(outs[b, :, h] - ref[0, :, 0])
+            max_abs = max(max_abs, float(err.max()))
+            max_ratio = max(max_ratio, float((err / (2.0 ** -8 * bound[0, :, 0] + 1e-30)).max()))
+            ulp = np.spacing(np.abs(rl[0, :, 0]).astype(np.float32)).astype(np.float64)
+            max_lse_ulp = max(max_lse_ulp, float((np.abs(lses[b, :, h] - rl[0, :, 0]) / ulp).max()))
+            n_el += err.size
+        out["error_vs_fp64_oracle"] = {"sampled_outputs": n_el, "max_abs_output_error": max_abs,
+                                       "max_error_over_bf16_probability_bound": max_ratio,
+                                       "max_lse_error_in_fp32_ulp": max_lse_ulp,
+                                       "bound": "2^-8 * sum_p softmax_p |v_p| per element (probabilities rounded to bf16)"}
     del layers, packs
     torch.cuda.empty_cache()
     return out
@@ -808,7 +838,7 @@ def main():
                 extra[key] = {"unavailable": f"{type(e).__name__}: {e}"[:200]}
         line["configs"] = extra
         try:
-            line["attention"] = measure_attention(ctx, peak_gbs)
+            line["attention"] = measure_attention(ctx, peak_gbs, with_oracle=not args.no_cpu_baseline)
         except Exception as e:
             line["attention"] = {"unavailable": f"{type(e).__name__}: {e}"[:200]}
     print(json.dumps(line), flush=True)
