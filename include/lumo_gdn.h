@@ -397,7 +397,8 @@ int lumo_kv_write_tree(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_att
  * by rounding.
  * Needs max_positions * Hkv * dh * 2 bytes < 2^40 per cache row.  Enqueues only; library scratch for
  * the partial results grows on the first call with a shape.  All attention calls of a context share that
- * scratch: enqueue them on one stream (or otherwise serialise them).  If a bounded device-side wait runs
+ * scratch: enqueue them on one stream (or otherwise serialise them).  After one call with a shape the call
+ * allocates nothing and can be captured into a CUDA graph.  If a bounded device-side wait runs
  * out, every sequence of the call gets LUMO_SEQ_TIMEOUT and the outputs of the call are invalid. */
 int lumo_tree_attention(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_attn_args* layers, int n_layers,
                         void* stream);

@@ -291,3 +291,51 @@ def test_host_side_refusals_enqueue_nothing():
     dc.write(); dc.attend()                                             # the context is still usable
     torch.cuda.synchronize()
     assert dc.t("status").tolist() == [0]
+
+
+def test_write_attend_publish_replayed_from_one_cuda_graph():
+    """The three calls captured once (after a warm-up that sizes the library's scratch) and replayed on new
+    contents of the same buffers: new tree entries and queries, advanced context lengths, another accepted
+    path.  Every replay must match the oracle run on the same contents (Sec. "Device-resident commitment":
+    fixed-shape device products feed captured publication)."""
+    parents = trees("paper", 2, 28, 0)
+    c = W.make_attn_case("graph0", parents, [300, 77], seed=W.BASE_SEED + 60, Hq=8, Hkv=2, Ns=32, layout="spine",
+                         max_positions=500)
+    cx = ctx()
+    dc = DeviceAttnCase(cx, c, n_splits=0)
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        dc.write(st); dc.attend(st); dc.publish(st)                 # warm-up outside capture (scratch, kernel attributes)
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            dc.write(st); dc.attend(st); dc.publish(st)
+        k_host, v_host = c.k_cache.copy(), c.v_cache.copy()
+        ctx_host = c.ctx_len.copy()
+        for rep in range(3):
+            cn = W.make_attn_case(f"graph{rep + 1}", parents, ctx_host.tolist(), seed=W.BASE_SEED + 61 + rep, Hq=8, Hkv=2,
+                                  Ns=32, layout="spine", max_positions=500)
+            cn.cache_row = c.cache_row
+            cn.k_cache, cn.v_cache = k_host, v_host
+            up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(torch.bfloat16).to(dc.dev)
+            for name, arr in (("q", cn.q), ("k_new", cn.k_new), ("v_new", cn.v_new), ("k_cache", k_host), ("v_cache", v_host)):
+                dc.t(name).copy_(up(arr))
+            dc.ctx_len.copy_(torch.from_numpy(ctx_host).to(dc.dev))
+            dc.accepted.fill_(-1)
+            dc.accepted[:, :cn.accepted.shape[1]].copy_(torch.from_numpy(cn.accepted).to(dc.dev))
+            dc.accepted_len.copy_(torch.from_numpy(cn.accepted_len).to(dc.dev))
+            dc.t("out").fill_(float("nan")); dc.t("status").fill_(-1)
+            g.replay()
+            st.synchronize()
+            k1, v1 = A.kv_write(cn.slot, cn.k_new, cn.v_new, k_host, v_host, ctx_host, cn.cache_row)
+            ref, _ = A.tree_attention(cn.parent, cn.slot, cn.q, k1, v1, ctx_host, cn.cache_row, cn.scale)
+            bound, _ = A.tree_attention(cn.parent, cn.slot, cn.q, k1, np.abs(v1), ctx_host, cn.cache_row, cn.scale)
+            err = np.abs(dc.np("out") - ref)
+            assert (err <= 1.05 * 2.0 ** -8 * bound + 2e-5 * (1.0 + np.abs(ref))).all(), f"replay {rep}"
+            acc = np.full((2, c.lmax), -1, dtype=np.int32)
+            acc[:, :cn.accepted.shape[1]] = cn.accepted
+            k2, v2, ctx2, stt = A.kv_publish(cn.parent, cn.slot, k1, v1, ctx_host, cn.cache_row, acc, cn.accepted_len)
+            assert dc.t("status").tolist() == stt.tolist() == [0, 0]
+            assert np.array_equal(dc.np("k_cache"), k2) and np.array_equal(dc.np("v_cache"), v2), f"replay {rep} publication"
+            assert dc.ctx_len_out.tolist() == ctx2.tolist()
+            k_host, v_host, ctx_host = k2.astype(np.float32), v2.astype(np.float32), ctx2.astype(np.int32)
