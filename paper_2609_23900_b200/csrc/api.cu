@@ -186,8 +186,8 @@ int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx) {
 
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo) {
   if (!ctx) return LUMO_ERR_ARG;
-  if (algo < 0 || algo > 3)
-    return fail(ctx, LUMO_ERR_ARG, "scan algo must be 0 (auto), 1 (rank-1), 2 (Gram form, forward substitution) or 3 (solved Gram form)");
+  if (algo < 0 || algo > 4)
+    return fail(ctx, LUMO_ERR_ARG, "scan algo must be 0 (auto), 1 (rank-1), 2 (Gram form, forward substitution), 3 (solved Gram form) or 4 (Gram form, closed-form tail)");
   ctx->scan_algo = algo;
   return LUMO_OK;
 }
@@ -524,7 +524,7 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
     e = timed(ctx, LUMO_K_SCAN, st, [&] {
       const bool pdl = use_overlap(ctx, s) && !state_fresh;
       return ctx->scan_algo == 3 ? launch_scan_solve(s, t, lb, ctx->sm_count, pdl, st)
-                                 : launch_scan_gram(s, t, lb, ctx->sm_count, pdl, st);
+                                 : launch_scan_gram(s, t, lb, ctx->sm_count, pdl, ctx->scan_algo == 4, st);
     });
     return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "Gram-form scan launch");
   }
@@ -679,7 +679,7 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
   }
   e = timed(ctx, LUMO_K_SCAN, st, [&] {
     return ctx->scan_algo == 3 ? launch_scan_solve_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st)
-                               : launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st);
+                               : launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, ctx->scan_algo == 4, st);
   });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "fused scan launch");
 }

@@ -53,7 +53,7 @@ struct lumo_ctx {
   size_t attn_scratch_bytes = 0;
   uint32_t attn_launch_id = 0;
   // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
-  int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form with forward substitution, 3 solved Gram form
+  int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form with forward substitution, 3 solved Gram form, 4 Gram form with closed-form tail
   bool timeout_drill = false;   // test aid: the tensor-core scan skips its tensor-core work (lumo_ctx_set_timeout_drill)
   bool overlap = true;          // programmatic dependent launch between conv -> scan -> commit
   // Kind of the previous call that launched on this context.  Kernels that read some of their inputs
@@ -284,11 +284,12 @@ cudaError_t launch_select(const void* logits, int dtype, int rows, int V, int sp
                           cudaStream_t st);
 // Gram-form scan on tcgen05 (scan_gram.cu)
 bool gram_supported(const Shape& s, int max_depth);
-cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
+// direct: closed-form tail (per-node back substitution, one output pass) instead of the level-by-level one
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl, bool direct,
                              cudaStream_t st);
 // same scan, first replaying the previous cycle's accepted path into the state it has just loaded
 cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
-                                   int sm_count, bool pdl, cudaStream_t st);
+                                   int sm_count, bool pdl, bool direct, cudaStream_t st);
 // solved Gram form on tcgen05 (scan_solve.cu): the triangular system solved on scalars, one state product
 cudaError_t launch_scan_solve(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
                               cudaStream_t st);

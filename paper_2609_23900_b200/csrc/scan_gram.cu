@@ -223,12 +223,146 @@ struct NodeOps {
   uint2 ao;        // first four ancestor offsets (16 bits each)
 };
 
+// Closed-form tail of one item, entered when the Gram block has been dumped to shared memory
+// (dump[R][c]: R < NT the products K_R . K_c, NT <= R < 2 NT the products Q_(R-NT) . K_c), the V rows
+// are on their way (cp.async) and S0 [K | Q]^T sits in tensor-memory columns [0, 2 NT).
+//
+// With a_0 .. a_(D-1) the path of node t (root first, t itself last), A[t][j] = beta_t G(t, a_j)
+// (k^_aj . k^_t) for the strict ancestors and W[t][j] = G(t, a_j) (k^_aj . q^_t) for all of them, the
+// deltas solve (I + A) delta = rhs with rhs_s = beta_s (v_s - g_s S0 k^_s), and
+//   o_t = g_t S0 q^_t + sum_j M[t][j] rhs_(a_j),   M = W (I + A)^-1.
+// A and (I + A)^-1 couple only nodes of one root path, so row t of M comes from a back substitution
+// over that path alone: m[j] = W[t][j] - sum_(i > j) m[i] A[a_i][j].  Nothing here waits for another
+// node: four barrier-separated phases, whatever the depth of the tree.
+template <int NT, class LY>
+__device__ __forceinline__ void direct_tail(const Shape& s, const LayerPtrs& L, Small& sm, unsigned char* smem, const float* dump,
+                                            const __nv_bfloat16* Vs, uint32_t tmem_lane, int N, int b, int hv, int tid) {
+  const int warp = tid >> 5, lane = tid & 31, grp = tid >> 7, vrow = tid & 127;
+  float* Am = reinterpret_cast<float*>(smem + LY::kRec);        // [node][16], in the place of the records
+  float* Wm = Am + NT * 16;
+  float* Mm = Wm + NT * 16;
+  static_assert(LY::kRec + NT * 16 * 4 * 3 <= LY::kV, "coefficient tables overflow the record area");
+  float* Pq = reinterpret_cast<float*>(smem);                   // S0 q products [node][row], in the place of the dump
+  float* Rh = reinterpret_cast<float*>(smem + LY::kKQ);         // right-hand sides [node][row], in the place of K and Q
+  // ---- A and W along each node's ancestry: sixteen lanes per node (lane j = path entry j); G(t, a_j)
+  //      is a suffix product of the alphas over the lanes ----------------------------------------------
+  {
+    const int j = tid & 15, ln = tid >> 4;
+#pragma unroll
+    for (int m = 0; m < NT / 16; ++m) {
+      if (16 * m >= N) break;                                       // uniform
+      const int pi = ln + 16 * m;
+      const int D = pi < N ? ((sm.meta[pi] >> 16) & 0xFF) : 0;      // depth, 1..16 (the same in all 16 lanes)
+      const bool in = j < D;
+      const int a = sm.anc[pi][j];                                  // 0 beyond the depth
+      float incl = in ? sm.alpha[a] : 1.f;
+#pragma unroll
+      for (int off = 1; off < 16; off <<= 1) {
+        const float v = __shfl_down_sync(0xffffffffu, incl, off, 16);
+        if (j + off < 16) incl *= v;
+      }
+      float excl = __shfl_down_sync(0xffffffffu, incl, 1, 16);      // product over the lanes above j
+      if (j == 15) excl = 1.f;
+      const float g_t = __shfl_sync(0xffffffffu, incl, 0, 16);      // product over the whole path
+      float ksa = 1.f;
+      if (s.l2norm && in) ksa = rsqrtf(dump[a * LY::kStride + a] + s.l2_eps);
+      const float ks_t = __shfl_sync(0xffffffffu, ksa, D > 0 ? D - 1 : 0, 16);
+      const float qs_t = s.l2norm ? s.scale * rsqrtf(sm.qq[pi] + s.l2_eps) : s.scale;
+      const float b_t = sm.beta[pi];
+      float kk = 0.f, qk = 0.f;
+      if (in) { kk = dump[pi * LY::kStride + a]; qk = dump[(NT + pi) * LY::kStride + a]; }
+      Am[pi * 16 + j] = j < D - 1 ? b_t * excl * ks_t * ksa * kk : 0.f;   // no entry for the node itself
+      Wm[pi * 16 + j] = in ? qs_t * excl * ksa * qk : 0.f;
+      if (j == 0) { sm.qs[pi] = g_t * qs_t; sm.ks[pi] = b_t * g_t * ks_t; }   // factors of S0 q and of S0 k
+    }
+  }
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");            // this thread's pieces of V
+  __syncthreads();                                                  // A, W, V in place; the dump is dead
+  // ---- M by back substitution, four lanes per node holding its sixteen entries ------------------------
+  if (tid < 4 * NT) {                                               // whole warps
+    const int pi = tid >> 2, q4 = tid & 3;
+    const int D = pi < N ? ((sm.meta[pi] >> 16) & 0xFF) : 0;
+    float4 w = *reinterpret_cast<const float4*>(Wm + pi * 16 + 4 * q4);
+    const int Dw = __reduce_max_sync(0xffffffffu, D);
+    for (int jh = Dw - 1; jh >= 1; --jh) {                          // bounded: <= 15 steps
+      const int e = jh & 3;
+      const float cand = e == 0 ? w.x : e == 1 ? w.y : e == 2 ? w.z : w.w;
+      const float mval = __shfl_sync(0xffffffffu, cand, (lane & ~3) | (jh >> 2));
+      if (jh < D) {
+        const float4 ar = *reinterpret_cast<const float4*>(Am + sm.anc[pi][jh] * 16 + 4 * q4);
+        w.x = fmaf(-mval, ar.x, w.x); w.y = fmaf(-mval, ar.y, w.y);
+        w.z = fmaf(-mval, ar.z, w.z); w.w = fmaf(-mval, ar.w, w.w);
+      }
+    }
+    *reinterpret_cast<float4*>(Mm + pi * 16 + 4 * q4) = w;
+  }
+  // ---- the S0 products leave tensor memory (lane = value row): the first half of the CTA turns the key
+  //      products into right-hand sides, the second half moves the query products ----------------------
+  if (grp == 0) {
+    for (int cb = 0; cb < (N + 31) / 32; ++cb) {                    // bounded: <= 2
+      uint32_t r0[16], r1[16];
+      tmem_ld16_issue(tmem_lane + cb * 32, r0);
+      tmem_ld16_issue(tmem_lane + cb * 32 + 16, r1);
+      tmem_ld_wait();
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        const int sn = cb * 32 + e;
+        const float pk = __uint_as_float(e < 16 ? r0[e & 15] : r1[e & 15]);
+        const float v = __bfloat162float(Vs[sn * kD + vrow]);       // rows of padding nodes hold stale bytes: never read back
+        Rh[sn * kD + vrow] = fmaf(sm.beta[sn], v, -sm.ks[sn] * pk);
+      }
+    }
+  } else {
+    for (int cb = 0; cb < (N + 31) / 32; ++cb)                      // bounded: <= 2
+      tmem_cols32_to_smem(tmem_lane + NT + cb * 32, Pq + (cb * 32) * kD + vrow, kD);
+  }
+  __syncthreads();
+  // ---- outputs: one warp per node, lane l carries value rows 4l .. 4l+3; a node that another group
+  //      emits is skipped altogether ----------------------------------------------------------------------
+  for (int pi = warp; pi < N; pi += kWarps) {                       // bounded: <= 8 rounds
+    const int meta = sm.meta[pi];
+    if (!((meta >> 24) & 1)) continue;
+    const int D = (meta >> 16) & 0xFF;
+    const float cq = sm.qs[pi];
+    const float4 pq = *reinterpret_cast<const float4*>(Pq + pi * kD + 4 * lane);
+    float2 o01 = make_float2(cq * pq.x, cq * pq.y), o23 = make_float2(cq * pq.z, cq * pq.w);
+    const int nblk = (D + 3) >> 2;
+    for (int blk = 0; blk < nblk; ++blk) {                          // bounded: <= 4 blocks of four path entries
+      const float4 mc = *reinterpret_cast<const float4*>(Mm + pi * 16 + 4 * blk);
+      const uint32_t a4 = *reinterpret_cast<const uint32_t*>(&sm.anc[pi][4 * blk]);
+      // entries beyond the depth (last block only) have m = 0 and read the node's own row: nothing of
+      // another branch can reach this output, not even as 0 x NaN
+      const int rem = D - 4 * blk;
+      const float4 d0 = *reinterpret_cast<const float4*>(Rh + (a4 & 0xFF) * kD + 4 * lane);
+      const float4 d1 = *reinterpret_cast<const float4*>(Rh + (rem > 1 ? (a4 >> 8) & 0xFF : pi) * kD + 4 * lane);
+      const float4 d2 = *reinterpret_cast<const float4*>(Rh + (rem > 2 ? (a4 >> 16) & 0xFF : pi) * kD + 4 * lane);
+      const float4 d3 = *reinterpret_cast<const float4*>(Rh + (rem > 3 ? a4 >> 24 : pi) * kD + 4 * lane);
+      auto step = [&](float m, const float4& dd) {
+        const float2 mm = make_float2(m, m);
+        o01 = __ffma2_rn(mm, make_float2(dd.x, dd.y), o01);
+        o23 = __ffma2_rn(mm, make_float2(dd.z, dd.w), o23);
+      };
+      step(mc.x, d0); step(mc.y, d1); step(mc.z, d2); step(mc.w, d3);
+    }
+    const size_t oi = (((size_t)b * s.Ns + (meta & 0xFFFF)) * s.Hv + hv) * kD + 4 * lane;
+    if (s.out_dtype == LUMO_BF16) {
+      __nv_bfloat162 b01 = __floats2bfloat162_rn(o01.x, o01.y), b23 = __floats2bfloat162_rn(o23.x, o23.y);
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(L.out) + oi) =
+          make_uint2(*reinterpret_cast<uint32_t*>(&b01), *reinterpret_cast<uint32_t*>(&b23));
+    } else {
+      *reinterpret_cast<float4*>(reinterpret_cast<float*>(L.out) + oi) = make_float4(o01.x, o01.y, o23.x, o23.y);
+    }
+  }
+}
+
 // NT = node tile of the MMAs: 64, or 32 when no group of the launch has more than 32 nodes (K rows
 // 0..NT-1 and Q rows NT..2NT-1 of the operand tile; the products occupy NT + NT + NT columns)
 // kFused: before anything else the previous cycle's accepted path is replayed into the state rows as
 // they pass through the registers (same per-token update as the commit kernel), and the rows are
 // written back in place; the scan then runs from the updated state.  One group per sequence only.
-template <int NT, bool kFused, bool kCompact = false>
+// kDirect: the triangular system is solved on scalars per node (M = W (I + A)^-1 along each ancestry, no
+// dependency between nodes) and every output is one pass over its path; no level-by-level substitution.
+template <int NT, bool kFused, bool kCompact = false, bool kDirect = false>
 __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t, const LayerBatch& lb, int n_items,
                                                const FusedPrev* fp) {
   extern __shared__ unsigned char smem_raw[];
@@ -625,6 +759,12 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     // both halves of the CTA read the Gram rows: 32 of the NT columns each (one half is enough for NT = 32)
     if (grp * 32 < NT) tmem_cols32_to_smem(tmem_lane + LY::kGramCol + grp * 32, dump + vrow * LY::kStride + grp * 32, 1);
     __syncthreads();
+    if constexpr (kDirect) {
+      direct_tail<NT, LY>(s, L, sm, smem, dump, Vs, tmem_lane, N, b, hv, tid);
+      tc_fence_before();
+      __syncthreads();      // tensor memory and the aliased shared memory are free for the next item
+      continue;
+    }
     // ---- h. normalisation factors ------------------------------------------------------------------
     if (tid < NT) sm.ks[tid] = s.l2norm ? rsqrtf(dump[tid * LY::kStride + tid] + s.l2_eps) : 1.f;
     else if (tid < 2 * NT) sm.qs[tid - NT] = s.l2norm ? s.scale * rsqrtf(sm.qq[tid - NT] + s.l2_eps) : s.scale;
@@ -768,22 +908,28 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(LY::kTmem) : "memory");
 }
 
-template <int NT>
+template <int NT, bool kDirect>
 __global__ void __launch_bounds__(kThreads, 2)
 scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
-  scan_gram_body<NT, false>(s, t, lb, n_items, nullptr);
+  scan_gram_body<NT, false, false, kDirect>(s, t, lb, n_items, nullptr);
 }
 
 // trees of at most 32 nodes, launches of several waves: three smaller CTAs per SM
+template <bool kDirect>
 __global__ void __launch_bounds__(kThreads, 3)
 scan_gram_compact_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
-  scan_gram_body<32, false, true>(s, t, lb, n_items, nullptr);
+  scan_gram_body<32, false, true, kDirect>(s, t, lb, n_items, nullptr);
 }
 
-template <int NT>
+template <int NT, bool kDirect>
 __global__ void __launch_bounds__(kThreads, 2)
 scan_gram_fused_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items, FusedPrev fp) {
-  scan_gram_body<NT, true>(s, t, lb, n_items, &fp);
+  scan_gram_body<NT, true, false, kDirect>(s, t, lb, n_items, &fp);
+}
+
+template <class K>
+cudaError_t allow_smem(K kernel, int bytes) {
+  return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
 
 }  // namespace
@@ -792,7 +938,7 @@ bool gram_supported(const Shape& s, int max_depth) {
   return s.d == kD && s.in_dtype == LUMO_BF16 && s.snapshot_mode == 0 && max_depth <= 16;
 }
 
-cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl, bool direct,
                              cudaStream_t st) {
   const int items = s.n_layers * t.n_groups * s.Hv;
   static bool configured[kMaxDevices] = {};      // the attribute is a per-device setting
@@ -801,11 +947,12 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
   if (e0 != cudaSuccess) return e0;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   if (!configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(scan_gram_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(scan_gram_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(scan_gram_compact_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GL<true>::kBytes);
+    cudaError_t e = allow_smem(scan_gram_kernel<64, false>, kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_kernel<32, false>, kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_kernel<64, true>, kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_kernel<32, true>, kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_compact_kernel<false>, GL<true>::kBytes);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_compact_kernel<true>, GL<true>::kBytes);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
@@ -814,16 +961,18 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
   // Compact CTAs (68 KB, 80 registers, 128 tensor-memory columns: three per SM) pay one more tensor-core
   // round trip per item: they win when a launch has several waves of items (the 48-layer stack: 205 ->
   // 190 us) and lose on a single wave (batch 1: 9.3 -> 10.5 us).
-  if (t.max_group_nodes <= 32 && items >= 4 * sm_count)
-    return launch_kernel(scan_gram_compact_kernel, dim3(3 * sm_count), dim3(kThreads), GL<true>::kBytes, st, pdl, s, t, lb, items);
+  if (t.max_group_nodes <= 32 && items >= 4 * sm_count) {
+    auto k = direct ? scan_gram_compact_kernel<true> : scan_gram_compact_kernel<false>;
+    return launch_kernel(k, dim3(3 * sm_count), dim3(kThreads), GL<true>::kBytes, st, pdl, s, t, lb, items);
+  }
   const int grid = items < 2 * sm_count ? items : 2 * sm_count;
-  if (t.max_group_nodes <= 32)
-    return launch_kernel(scan_gram_kernel<32>, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
-  return launch_kernel(scan_gram_kernel<64>, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
+  auto k = t.max_group_nodes <= 32 ? (direct ? scan_gram_kernel<32, true> : scan_gram_kernel<32, false>)
+                                   : (direct ? scan_gram_kernel<64, true> : scan_gram_kernel<64, false>);
+  return launch_kernel(k, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
 }
 
 cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
-                                   int sm_count, bool pdl, cudaStream_t st) {
+                                   int sm_count, bool pdl, bool direct, cudaStream_t st) {
   const int items = s.n_layers * t.n_groups * s.Hv;
   static bool configured[kMaxDevices] = {};      // the attribute is a per-device setting
   int dev = 0;
@@ -831,16 +980,17 @@ cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const Layer
   if (e0 != cudaSuccess) return e0;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   if (!configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(scan_gram_fused_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesFused);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(scan_gram_fused_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesFused);
+    cudaError_t e = allow_smem(scan_gram_fused_kernel<64, false>, kSmemBytesFused);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_fused_kernel<32, false>, kSmemBytesFused);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_fused_kernel<64, true>, kSmemBytesFused);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_fused_kernel<32, true>, kSmemBytesFused);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   const int grid = items < 2 * sm_count ? items : 2 * sm_count;
-  if (t.max_group_nodes <= 32)
-    return launch_kernel(scan_gram_fused_kernel<32>, dim3(grid), dim3(kThreads), kSmemBytesFused, st, pdl, s, t, lb, items, fp);
-  return launch_kernel(scan_gram_fused_kernel<64>, dim3(grid), dim3(kThreads), kSmemBytesFused, st, pdl, s, t, lb, items, fp);
+  auto k = t.max_group_nodes <= 32 ? (direct ? scan_gram_fused_kernel<32, true> : scan_gram_fused_kernel<32, false>)
+                                   : (direct ? scan_gram_fused_kernel<64, true> : scan_gram_fused_kernel<64, false>);
+  return launch_kernel(k, dim3(grid), dim3(kThreads), kSmemBytesFused, st, pdl, s, t, lb, items, fp);
 }
 
 }  // namespace lumo

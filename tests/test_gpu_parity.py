@@ -126,7 +126,7 @@ def test_conv_recorded_operands(name):
 # ------------------------------------------------------------------ scan
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("use_conv", [False, True])
-@pytest.mark.parametrize("algo", ["rank1", "gram", "solve"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct"])
 def test_scan_outputs_match_oracle(name, use_conv, algo):
     c = CASES[name]()
     if algo != "rank1" and not gram_eligible(c):
@@ -154,7 +154,7 @@ def test_scan_outputs_match_oracle(name, use_conv, algo):
     assert_close(dc16.np("out"), o_ref, bf16=True, what=f"{name} scan bf16 out")
 
 
-@pytest.mark.parametrize("algo", ["rank1", "gram", "solve"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct"])
 def test_scan_twice_is_bitwise_reproducible(algo):
     c = CASES["cfg2"]()
     dc = DeviceCase(ctx(algo), c)
@@ -166,7 +166,7 @@ def test_scan_twice_is_bitwise_reproducible(algo):
     assert torch.equal(a, dc.t("out")) and torch.equal(qa, dc.t("q"))
 
 
-@pytest.mark.parametrize("algo", ["rank1", "gram", "solve"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct"])
 def test_l2norm_flag_scale_and_f32_gates(algo):
     c = small(rand_parents(4, 20, 2), d=128, dtype="bf16")
     rs = np.random.default_rng(1)
@@ -280,7 +280,7 @@ def test_commit_controls_len0_poisoned_tail_invalid_paths_skipped_rows():
     assert torch.all(dc2.t("out")[2] == 0) and torch.all(dc2.t("out")[3] == 0) and torch.all(dc2.t("q")[2] == 0)
 
 
-@pytest.mark.parametrize("tc", ["gram", "solve"])
+@pytest.mark.parametrize("tc", ["gram", "solve", "direct"])
 def test_gram_scan_skipped_rows_padding_and_depth_16(tc):
     # a 16-deep chain plus side leaves (depth limit of the Gram form), padded and permuted rows,
     # one skipped sequence and one row outside the pool
@@ -311,7 +311,7 @@ def test_gram_scan_skipped_rows_padding_and_depth_16(tc):
     ctx("auto")
 
 
-@pytest.mark.parametrize("tc", ["gram", "solve"])
+@pytest.mark.parametrize("tc", ["gram", "solve", "direct"])
 def test_gram_groups_with_long_prefix_paths(tc):
     # caterpillar: a 10-node spine with 24 leaves under every spine node (250 nodes).  The tree is cut
     # into groups that each carry a prefix path of up to 10 recomputed nodes; every node must still be
@@ -371,7 +371,7 @@ def test_randomized_shapes_both_kernels():
                         beta_uniform=rng.random() < 0.5, with_bias=rng.random() < 0.3)
         use_conv = rng.random() < 0.5
         ref = None
-        for algo in ("solve", "gram", "rank1"):
+        for algo in ("solve", "gram", "direct", "rank1"):
             dc = DeviceCase(ctx(algo), c, use_conv=use_conv)
             dc.t("out").fill_(float("nan"))
             dc.verify()
@@ -473,14 +473,15 @@ def test_kernel_overlap_changes_nothing(name):
     assert not torch.equal(res[True][0][0], res[True][0][1])      # the cycles really advanced the state
 
 
+@pytest.mark.parametrize("algo", ["gram", "direct"])
 @pytest.mark.parametrize("name", ["cfg3_5layers", "paper_geometry_5layers"])
-def test_compact_three_cta_scan_matches_oracle(name):
+def test_compact_three_cta_scan_matches_oracle(name, algo):
     """Launches with several waves of items over trees of at most 32 nodes take the compact variant of the
     Gram scan (the state crosses shared memory in two 64-column halves, three CTAs per SM).  Every layer,
     every output, element by element against the oracle; padded and permuted rows in the second case."""
     c = W.config3(n_layers=5) if name == "cfg3_5layers" else W.config_paper(B=4, n_layers=5)
     assert len(c.layers) * c.B * c.Hv >= 4 * 148          # enough items for the compact kernel to be chosen
-    dc = DeviceCase(ctx("gram"), c)
+    dc = DeviceCase(ctx(algo), c)
     for l in range(len(c.layers)):
         dc.t("out", l).fill_(float("nan"))
     dc.verify()
