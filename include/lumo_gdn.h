@@ -120,9 +120,13 @@ int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx);
 /* Which scan kernel lumo_gdn_tree_verify uses: 0 = automatic (the tensor-core kernel when the shape
  * allows it: d = 128, bf16 operands, tree depth <= 16, no snapshots; trees of more than 64 nodes are
  * cut into node groups on the host; else rank-1), 1 = always the rank-1 fp32 kernel, 2 = the Gram form
- * with a forward substitution over value rows (what "automatic" picks: it measured faster), 3 = the
- * solved Gram form (the triangular system is solved on scalars per head and the state enters a single
- * product with "effective queries"); 2 and 3 return LUMO_ERR_UNSUPPORTED on other shapes. */
+ * with a forward substitution over value rows, level by level, 3 = the solved Gram form (the triangular
+ * system is solved on scalars per head and the state enters a single product with "effective queries"),
+ * 4 = the Gram form with a closed-form tail (the same two products as 2; then M = W (I + A)^-1 by a back
+ * substitution per node along its own root path and one pass that sums M x right-hand sides: no step
+ * waits for another node).  "Automatic" picks between 2 and 4 per descriptor from the shape of its trees
+ * (thin deep trees, a spine with small side branches, take 4; wide ones take 2: measured).  2, 3 and 4
+ * return LUMO_ERR_UNSUPPORTED on other shapes. */
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo);
 
 /* Test aid for the failure path of the tensor-core scan.  That kernel waits for its tensor-core work

@@ -304,6 +304,7 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   const bool attn = Ns <= kMaxAttnSlots;
   const size_t o_vis = attn ? reserve((size_t)B * N * 8) : 0, o_used = attn ? reserve((size_t)B * 8) : 0;
   size_t gi = 0;
+  long long subst_rounds = 0, group_nodes = 0;     // over all groups: rounds of the substitution, nodes
   for (int b = 0; b < B; ++b) {
     const HostTree& t = d->trees[b];
     if (attn) {
@@ -393,9 +394,15 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
           for (int j = dep - 2; j >= 0; --j) { anc[pi * 16 + j] = (uint8_t)pos[cur]; cur = parent[(size_t)b * N + cur]; }
           for (int dd = dep; dd < 20; ++dd) lvl[dd] += 1;      // lvl[d] = members of depth <= d
         }
+        for (int dd = 1; dd < 20; ++dd) subst_rounds += (lvl[dd] - lvl[dd - 1] + 7) / 8;
+        group_nodes += n;
       }
     }
   }
+  // measured on B200 (us per item): substitution 0.45 per round, closed form 1.7 + 0.08 per node; the
+  // closed form is taken when it wins by a margin (28-node spine trees of depth 12: 18.5 -> 17.0 us per
+  // launch at batch 8; 64-node trees of depth 8 stay with the substitution: 19.1 against 20.5 us)
+  d->closed_form_pays = tc && 100 * subst_rounds > 600 * (long long)G + 18 * group_nodes;
   if (ctx->device < 0) { *out = d; return LUMO_OK; }   // host-only: tables stay on the host
   DeviceGuard g(ctx->device);
   cudaError_t e = cudaMalloc(&d->dev, h.size() * sizeof(int32_t));
@@ -524,7 +531,7 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
     e = timed(ctx, LUMO_K_SCAN, st, [&] {
       const bool pdl = use_overlap(ctx, s) && !state_fresh;
       return ctx->scan_algo == 3 ? launch_scan_solve(s, t, lb, ctx->sm_count, pdl, st)
-                                 : launch_scan_gram(s, t, lb, ctx->sm_count, pdl, ctx->scan_algo == 4, st);
+                                 : launch_scan_gram(s, t, lb, ctx->sm_count, pdl, ctx->scan_algo == 4 || (ctx->scan_algo == 0 && desc->closed_form_pays), st);
     });
     return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "Gram-form scan launch");
   }
@@ -679,7 +686,7 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
   }
   e = timed(ctx, LUMO_K_SCAN, st, [&] {
     return ctx->scan_algo == 3 ? launch_scan_solve_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st)
-                               : launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, ctx->scan_algo == 4, st);
+                               : launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, ctx->scan_algo == 4 || (ctx->scan_algo == 0 && desc->closed_form_pays), st);
   });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "fused scan launch");
 }

@@ -95,6 +95,10 @@ struct lumo_tree_desc {
   int32_t* d_tc_meta = nullptr;   // [G, 64] physical row | depth << 16 | emit << 24 of the node at position pi
   uint8_t* d_tc_anc = nullptr;    // [G, 64, 16] positions of the ancestors, root first, then the node's own position
   uint8_t* d_tc_lvl = nullptr;    // [G, 20] lvl[d] = number of group nodes of depth <= d (lvl[0] = 0)
+  // Which tail the Gram-form scan takes by default.  The level-by-level substitution costs one round per
+  // eight nodes of a level, the closed-form tail a fixed part plus a part per node: thin, deep trees (a
+  // spine with small side branches) are cheaper in closed form, wide ones by levels.
+  bool closed_form_pays = false;
   uint32_t* d_vis = nullptr;      // [B, N, 8] attention visibility over physical slots (present when Ns <= 256)
   uint32_t* d_slot_used = nullptr;// [B, 8] slots that hold a node
 };

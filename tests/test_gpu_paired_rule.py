@@ -45,7 +45,7 @@ def test_paired_error_rule_counts():
     res = paired_rule(ctx(), W.config_paper(B=2))
     k = res["kernels"]
     assert k["rank1"]["passed_vs_sequential_kernel"] == res["cells"]
-    for algo in ("rank1", "gram", "solve"):
+    for algo in ("rank1", "gram", "direct", "solve"):
         assert k[algo]["max_abs_error"] < 2e-6 and k[algo]["median_cell_rms_error"] < 2e-7
     # the commit chain with a float64 output product is the more exact native side
     assert res["native"]["commit_chain"]["median_cell_rms_error"] <= res["native"]["sequential_kernel"]["median_cell_rms_error"]

@@ -166,6 +166,22 @@ def test_scan_twice_is_bitwise_reproducible(algo):
     assert torch.equal(a, dc.t("out")) and torch.equal(qa, dc.t("q"))
 
 
+def test_automatic_choice_between_the_two_tails_follows_the_tree_shape():
+    """Thin deep trees (the paper's geometry: 28 nodes over 12 levels) take the closed-form tail, wide ones
+    (64 nodes over 8 levels) the level-by-level substitution: the automatic choice reproduces the bits of
+    the kernel it is meant to pick, and the two kernels do differ in the last bits."""
+    for case, expect, other in ((W.config_paper(B=3), "direct", "gram"), (CASES["cfg2"](), "gram", "direct")):
+        outs = {}
+        for algo in ("auto", "gram", "direct"):
+            dc = DeviceCase(ctx(algo), case)
+            dc.verify()
+            torch.cuda.synchronize()
+            outs[algo] = dc.t("out").clone()
+        assert torch.equal(outs["auto"], outs[expect])
+        assert not torch.equal(outs["auto"], outs[other])
+    ctx("auto")
+
+
 @pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct"])
 def test_l2norm_flag_scale_and_f32_gates(algo):
     c = small(rand_parents(4, 20, 2), d=128, dtype="bf16")
