@@ -21,6 +21,9 @@
 // offset); a warp loads the record of its next node before the barrier that publishes the
 // previous level, so that only the ancestors' deltas are fetched after it.
 //
+// A second tail (kDirect, below) replaces the level-by-level walk by a closed form: M = W (I + A)^-1 per
+// node along its own root path, then one pass over right-hand sides; the host picks per descriptor.
+//
 // One CTA (256 threads) handles one (layer, sequence, value head) at a time; two CTAs per SM
 // overlap one item's loads with the other's arithmetic.  Limits of this
 // kernel: d = 128, bf16 operands, N <= 64 nodes, tree depth <= 16, no state snapshots; everything
