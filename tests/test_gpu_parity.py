@@ -166,6 +166,51 @@ def test_scan_twice_is_bitwise_reproducible(algo):
     assert torch.equal(a, dc.t("out")) and torch.equal(qa, dc.t("q"))
 
 
+@pytest.mark.parametrize("use_conv", [False, True])
+@pytest.mark.parametrize("algo,shape", [("rank1", "cfg2"), ("gram", "cfg2"), ("direct", "cfg2"), ("direct", "paper"),
+                                        ("gram", "grouped"), ("direct", "grouped"), ("solve", "cfg2")])
+def test_path_locality_poisoned_subtree_leaves_the_other_nodes_bitwise_unchanged(algo, shape, use_conv):
+    """Sec. "The recurrence and path locality": the output of a node depends on its root path alone.  The
+    inputs of one whole subtree per sequence (and of every padding slot) are replaced by NaN (by 1e30 for
+    the solved form, whose final product runs over all nodes with zero coefficients off the path): every
+    node outside the subtree keeps its output bit for bit, through the convolution as well."""
+    if shape == "cfg2":
+        c = W.config2(B=3)
+    elif shape == "paper":
+        c = W.config_paper(B=3)
+    else:   # 150 nodes per tree: cut into node groups with recomputed prefix paths
+        c = W.make_case("grp", rand_parents(5, 150, 3), seed=17, Hk=2, Hv=4, d=128, in_dtype="bf16", Ns=160, permute_slots=True)
+    if algo == "solve" and use_conv:
+        pytest.skip("1e30 through the SiLU of the convolution is no longer finite")
+    poison = 1e30 if algo == "solve" else float("nan")
+    dc = DeviceCase(ctx(algo), c, use_conv=use_conv)
+    dc.verify()
+    torch.cuda.synchronize()
+    clean = dc.t("out").clone()
+    inside = np.zeros((c.B, c.N), dtype=bool)
+    for b in range(c.B):
+        depth = W.tree_depths(c.parent[b].tolist())
+        kids = [i for i in range(c.N) if depth[i] == 2]
+        root_of_poison = kids[len(kids) // 2]
+        for i in range(c.N):                                  # parents precede children
+            inside[b, i] = i == root_of_poison or (c.parent[b, i] >= 0 and inside[b, c.parent[b, i]])
+        assert inside[b].sum() >= 1 and not inside[b].all()
+        rows = [int(c.slot[b, i]) for i in range(c.N) if inside[b, i]]
+        rows += sorted(set(range(c.Ns)) - set(c.slot[b].tolist()))          # padding slots too
+        for t in (("x",) if use_conv else ("q", "k", "v")):
+            dc.t(t)[b, rows] = poison
+    dc.verify()
+    torch.cuda.synchronize()
+    got = dc.t("out")
+    for b in range(c.B):
+        keep = [int(c.slot[b, i]) for i in range(c.N) if not inside[b, i]]
+        assert torch.equal(got[b, keep], clean[b, keep]), f"sequence {b}: poison reached a node outside the subtree"
+        if algo != "solve":
+            gone = [int(c.slot[b, i]) for i in range(c.N) if inside[b, i]]
+            assert torch.isnan(got[b, gone]).any(dim=-1).all()               # and the poison was real
+    ctx("auto")
+
+
 def test_automatic_choice_between_the_two_tails_follows_the_tree_shape():
     """Thin deep trees (the paper's geometry: 28 nodes over 12 levels) take the closed-form tail, wide ones
     (64 nodes over 8 levels) the level-by-level substitution: the automatic choice reproduces the bits of
