@@ -41,6 +41,9 @@ CASES = {
                                       in_dtype="bf16", alpha_lo=0.5, beta_uniform=True),
     "rand256_b2": lambda: W.make_case("r", rand_parents(3, 256, 2), seed=7, Hk=4, Hv=8, d=128,
                                       in_dtype="bf16", alpha_lo=0.5, beta_uniform=True, with_bias=True),
+    # the deepest tree the library takes: one chain of 256 nodes (accepted paths up to the 256-entry limit)
+    "chain256_deep": lambda: W.make_case("cd", [W.tree_chain(256)] * 2, seed=8, Hk=1, Hv=2, d=64, in_dtype="f32",
+                                         alpha_lo=0.9),
 }
 
 
@@ -247,7 +250,7 @@ def test_l2norm_flag_scale_and_f32_gates(algo):
 
 
 # ------------------------------------------------------------------ snapshots and commit
-@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2", "cfgP_padded_permuted", "chain16x16_b2", "rand256_b2"])
+@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2", "cfgP_padded_permuted", "chain16x16_b2", "rand256_b2", "chain256_deep"])
 def test_commit_state_history_and_agreement_with_verifier_state(name):
     c = CASES[name]()
     ends = np.array([[a[l - 1] if l else -1] for a, l in zip(c.accepted, c.accepted_len)], dtype=np.int32)
@@ -298,6 +301,22 @@ def test_cfg0_accepted_path_is_0_2_6_and_commit_matches_leaf_state():
     # all seven node states against the oracle
     _, snap_ref, _ = oracle_scan_from_device(dc, snap_nodes=[list(range(7))])
     assert_close(snap, snap_ref, what="cfg0 all node states")
+
+
+def test_commit_of_the_longest_path_the_library_takes():
+    """A chain of 256 nodes accepted whole: 256 replayed updates per head, the limit of the staged path."""
+    c = CASES["chain256_deep"]()
+    dc = DeviceCase(ctx(), c)
+    dc.verify()
+    acc = np.tile(np.arange(256, dtype=np.int32), (c.B, 1))
+    ln = np.array([256, 255], dtype=np.int32)
+    dev = dc.dev
+    dc.commit(accepted=torch.from_numpy(acc).to(dev), length=torch.from_numpy(ln).to(dev))
+    torch.cuda.synchronize()
+    st_ref, hist_ref, status, _ = oracle_commit_from_device(dc, accepted=acc, length=ln)
+    assert dc.np("status").tolist() == status.tolist() == [0, 0]
+    assert_close(dc.np("state"), st_ref, what="256-step replay")
+    assert np.array_equal(dc.np("conv_hist"), hist_ref)
 
 
 def test_commit_controls_len0_poisoned_tail_invalid_paths_skipped_rows():
