@@ -688,31 +688,38 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   }
   const int slot0 = t.x, nslot = t.y;
   const size_t base = (size_t)slot0 * kRows + r;
-  // Second round trip: four slots at a time, their log-sum-exps (one per lane) and their rows together; the
-  // combination itself runs in slot order against the maximum of all log-sum-exps.
+  // Second round trip: the log-sum-exps of all slots (one per lane) and, in the same flight, the rows of the
+  // first eight slots; further slots follow eight at a time.  The combination itself runs in slot order
+  // against the maximum of all log-sum-exps, whatever the grouping of the loads.
+  constexpr int kBatch = 8;
+  auto load_rows = [&](float4 (&v)[kBatch], int s0) {
+#pragma unroll
+    for (int k = 0; k < kBatch; ++k)
+      v[k] = s0 + k < nslot ? reinterpret_cast<const float4*>(a.part_o + (base + (size_t)(s0 + k) * kRows) * kDh)[lane]
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+  };
+  float4 v[kBatch];
+  load_rows(v, 0);
   float mx = -INFINITY;
+  float ls_lane = -INFINITY;                  // log-sum-exp of slot `lane` (slots beyond 32: reloaded below)
   for (int s0 = 0; s0 < nslot; s0 += 32) {
     const float ls = (s0 + lane < nslot) ? a.part_lse[base + (size_t)(s0 + lane) * kRows] : -INFINITY;
+    if (s0 == 0) ls_lane = ls;
     mx = fmaxf(mx, ls);
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
   float den = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s0 = 0; s0 < nslot; s0 += 4) {
-    float ls[4];
-    float4 v[4];
+  for (int s0 = 0; s0 < nslot; s0 += kBatch) {
+    if (s0) load_rows(v, s0);
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const bool in = s0 + k < nslot;
-      ls[k] = in ? a.part_lse[base + (size_t)(s0 + k) * kRows] : -INFINITY;
-      v[k] = in ? reinterpret_cast<const float4*>(a.part_o + (base + (size_t)(s0 + k) * kRows) * kDh)[lane]
-                : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      if (ls[k] == -INFINITY) continue;      // an empty slot (or none)
-      const float wgt = ex2(ls[k] - mx);
+    for (int k = 0; k < kBatch; ++k) {
+      const int sl = s0 + k;
+      float ls = __shfl_sync(0xffffffffu, ls_lane, sl & 31);
+      if (sl >= 32 && sl < nslot) ls = a.part_lse[base + (size_t)sl * kRows];
+      if (sl >= nslot || ls == -INFINITY) continue;      // none, or an empty slot
+      const float wgt = ex2(ls - mx);
       den += wgt;
       acc.x = fmaf(wgt, v[k].x, acc.x); acc.y = fmaf(wgt, v[k].y, acc.y);
       acc.z = fmaf(wgt, v[k].z, acc.z); acc.w = fmaf(wgt, v[k].w, acc.w);
