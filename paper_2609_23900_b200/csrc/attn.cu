@@ -79,6 +79,7 @@ struct Small {
   unsigned long long k_full[kStages], k_empty[kStages], v_full[kStages], v_empty[kStages];
   unsigned long long s_full[2], s_read[2], p_full;
   unsigned long long q_full, o_free;
+  unsigned long long q_req;           // the first segment's query loads have been issued (the rings may fill behind them)
   uint32_t tmem_base;
   uint32_t timed_out;
   int seq_ctx[kSeqCache], seq_row[kSeqCache], seq_nt[kSeqCache];   // ctx_len, cache_row and tile count of the first sequences
@@ -337,6 +338,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     mbar_init(&sm.s_read[1], kSoftmaxWarps);
     mbar_init(&sm.p_full, kSoftmaxWarps);        // one arrival per softmax warp
     mbar_init(&sm.q_full, kSoftmaxWarps);
+    mbar_init(&sm.q_req, kSoftmaxWarps);
     mbar_init(&sm.o_free, kSoftmaxWarps);
     sm.timed_out = 0;
     asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -372,8 +374,9 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
           if (use > 0 && ok) ok = mbar_wait(&empty[st], (use - 1) & 1u);
           // Start-up: the rings of all CTAs fill at once (28 MB in flight) and the first segment's query rows
           // would queue behind them (measured: 3.4 us for 256 bytes per thread).  Only the first K tile goes
-          // ahead of the queries; everything else waits for their arrival in tensor memory.
-          if (it == (is_v ? 0u : 1u) && ok) ok = mbar_wait(&sm.q_full, 0);
+          // ahead of the queries; everything else waits until their loads have been issued (requests are served
+          // roughly in order: the queries come back first, the rings fill behind them).
+          if (it == (is_v ? 0u : 1u) && ok) ok = mbar_wait(&sm.q_req, 0);
           if (!ok) continue;
           mbar_expect_tx(&full[st], kTileBytes);
           const uint32_t dst = ring + st * kTileBytes;
@@ -472,6 +475,8 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         const uint4 v = okq ? __ldg(qrow + half * 8 + c) : make_uint4(0u, 0u, 0u, 0u);
         qr[4 * c] = v.x; qr[4 * c + 1] = v.y; qr[4 * c + 2] = v.z; qr[4 * c + 3] = v.w;
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.q_req);     // every lane's loads are on their way
       tmem_st32(tmem_lane + kColQ + half * 32, qr);
       tmem_st_wait();
       tc_fence_before();
