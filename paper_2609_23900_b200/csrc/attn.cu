@@ -490,12 +490,14 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
       const int rg = sg.rt * kRows + row;
       const bool row_ok = rg < GN;
       const int hl = row_ok ? rg / a.N : 0, node = row_ok ? rg - hl * a.N : 0;
-      float* slot_o = a.part_o + ((size_t)sg.slot * kRows + row) * kDh + half * 64;
+      // a slot holds its rows by groups of four columns, [column group][row][4]: the 32 lanes of a store (32
+      // rows, one group) write 512 contiguous bytes, and the merge kernel reads them the same way
+      float4* slot_o = reinterpret_cast<float4*>(a.part_o + (size_t)sg.slot * kRows * kDh) + (size_t)(half * 16) * kRows + row;
       float* slot_l = a.part_lse + (size_t)sg.slot * kRows + row;
       if (sthread == 0) a.unit_slots[sg.unit] = make_int2(sg.slot0, sg.nslots);   // for the merge (same pair from every writer)
       if (sg.n == 0) {                           // empty partition (fixed mode): an empty slot
         if (row_ok) {
-          for (int e = 0; e < 16; ++e) reinterpret_cast<float4*>(slot_o)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int e = 0; e < 16; ++e) slot_o[(size_t)e * kRows] = make_float4(0.f, 0.f, 0.f, 0.f);
           if (half == 0) *slot_l = -INFINITY;
         }
         have = work.next(&sgn);                  // (an empty partition is a CTA's only segment)
@@ -640,7 +642,7 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         if (row_ok) {
 #pragma unroll
           for (int e = 0; e < 32; e += 4)
-            *reinterpret_cast<float4*>(slot_o + c + e) =
+            slot_o[(size_t)((c + e) >> 2) * kRows] =
                 make_float4(__uint_as_float(orr[e]) * inv, __uint_as_float(orr[e + 1]) * inv,
                             __uint_as_float(orr[e + 2]) * inv, __uint_as_float(orr[e + 3]) * inv);
         }
@@ -660,23 +662,26 @@ tree_attn_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
   if (warp == 2) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
 }
 
-// Combination of a unit's slots: one warp per output row, slots in order (so the result for a given
-// decomposition is reproducible), weights exp2(lse_s - max lse).
+// Combination of a unit's slots: a warp takes 32 rows of a unit and one group of four columns (the slots
+// hold [column group][row][4], so its loads are contiguous), a lane one row; slots in order (so the result
+// for a given decomposition is reproducible), weights exp2(lse_s - max lse).
+// kBatch: slots per flight of loads (8: few slots per unit and a small register footprint, so that the CTAs
+// are staged beside the draining attention kernel; 24: a unit spread over all SMs, about 19 slots at batch 1)
+template <int kBatch>
 __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   pdl_wait();          // launched as a programmatic dependent of the attention kernel: its slots are complete from here on
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int GN = a.G * a.N;
-  const long long w = (long long)blockIdx.x * 8 + warp;
-  if (w >= (long long)a.B * a.Hkv * GN) return;
-  const int b = (int)(w / ((long long)a.Hkv * GN));
-  const int rem = (int)(w - (long long)b * a.Hkv * GN);
-  const int hkv = rem / GN, rg = rem - hkv * GN;
-  const int rt = rg / kRows, r = rg - rt * kRows;
-  const int hl = rg / a.N, node = rg - hl * a.N;
-  const size_t out_row = (((size_t)b * a.N + node) * a.Hq + (size_t)hkv * a.G + hl);
-  float4* dst = reinterpret_cast<float4*>(a.out + out_row * kDh) + lane;
   const int upb = a.Hkv * a.RT;
-  const int u = b * upb + hkv * a.RT + rt;
+  const long long w = (long long)blockIdx.x * 8 + warp;
+  if (w >= (long long)a.B * upb * 128) return;
+  const int cg = (int)(w & 31), rq = (int)((w >> 5) & 3);
+  const int u = (int)(w >> 7);
+  const int b = u / upb;
+  const int rem = u - b * upb;
+  const int hkv = rem / a.RT, rt = rem - hkv * a.RT;
+  const int r = rq * 32 + lane;
+  const int rg = rt * kRows + r;
   // Three independent loads first (one round trip): the sequence's context length and cache row, and the slot
   // range the attention kernel recorded for this unit (meaningless for a sequence that fails its check).
   const int cx = a.ctx_len[b], cr = a.cache_row[b];
@@ -684,47 +689,46 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   const int st = seq_check(cx, cr, a.Ns, a.n_rows, a.max_pos);
   // status word of the sequence: its check, else whether any wait of this launch's attention kernel ran out
   // (then the outputs of the whole call are suspect)
-  if (a.status && lane == 0 && hkv == 0 && rg == 0)
+  if (a.status && lane == 0 && rem == 0 && rq == 0 && cg == 0)
     a.status[b] = st != LUMO_SEQ_OK ? st : (*a.fail_flag == a.launch_id ? (int)LUMO_SEQ_TIMEOUT : (int)LUMO_SEQ_OK);
+  if (rg >= GN) return;                      // rows beyond the group (no warp-wide operation follows)
+  const int hl = rg / a.N, node = rg - hl * a.N;
+  const size_t out_row = (((size_t)b * a.N + node) * a.Hq + (size_t)hkv * a.G + hl);
+  float4* dst = reinterpret_cast<float4*>(a.out + out_row * kDh) + cg;
   if (st != LUMO_SEQ_OK) {                   // the sequence owns no tiles: zeros
     *dst = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (a.lse && lane == 0) a.lse[out_row] = 0.f;
+    if (a.lse && cg == 0) a.lse[out_row] = 0.f;
     return;
   }
   const int slot0 = t.x, nslot = t.y;
-  const size_t base = (size_t)slot0 * kRows + r;
-  // Second round trip: the log-sum-exps of all slots (one per lane) and, in the same flight, the rows of the
-  // first eight slots; further slots follow eight at a time.  The combination itself runs in slot order
-  // against the maximum of all log-sum-exps, whatever the grouping of the loads.
-  constexpr int kBatch = 8;
-  auto load_rows = [&](float4 (&v)[kBatch], int s0) {
-#pragma unroll
-    for (int k = 0; k < kBatch; ++k)
-      v[k] = s0 + k < nslot ? reinterpret_cast<const float4*>(a.part_o + (base + (size_t)(s0 + k) * kRows) * kDh)[lane]
-                            : make_float4(0.f, 0.f, 0.f, 0.f);
-  };
+  const float* lse_p = a.part_lse + (size_t)slot0 * kRows + r;                          // + slot * kRows
+  const float4* row_p = reinterpret_cast<const float4*>(a.part_o) + ((size_t)slot0 * 32 + cg) * kRows + r;   // + slot * 32 * kRows
+  // Second round trip: the rows of the first kBatch slots together with all log-sum-exps; further slots follow
+  // kBatch at a time.  The combination runs in slot order against the maximum of all log-sum-exps, whatever the
+  // grouping of the loads.
   float4 v[kBatch];
-  load_rows(v, 0);
-  float mx = -INFINITY;
-  float ls_lane = -INFINITY;                  // log-sum-exp of slot `lane` (slots beyond 32: reloaded below)
-  for (int s0 = 0; s0 < nslot; s0 += 32) {
-    const float ls = (s0 + lane < nslot) ? a.part_lse[base + (size_t)(s0 + lane) * kRows] : -INFINITY;
-    if (s0 == 0) ls_lane = ls;
-    mx = fmaxf(mx, ls);
-  }
+  float ls[kBatch];
+  auto load_batch = [&](int s0) {
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    for (int k = 0; k < kBatch; ++k) {
+      const bool in = s0 + k < nslot;
+      ls[k] = in ? lse_p[(size_t)(s0 + k) * kRows] : -INFINITY;
+      v[k] = in ? row_p[(size_t)(s0 + k) * 32 * kRows] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  load_batch(0);
+  float mx = -INFINITY;
+#pragma unroll
+  for (int k = 0; k < kBatch; ++k) mx = fmaxf(mx, ls[k]);
+  for (int sl = kBatch; sl < nslot; ++sl) mx = fmaxf(mx, lse_p[(size_t)sl * kRows]);   // bounded: < 256 slots
   float den = 0.f;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   for (int s0 = 0; s0 < nslot; s0 += kBatch) {
-    if (s0) load_rows(v, s0);
+    if (s0) load_batch(s0);
 #pragma unroll
     for (int k = 0; k < kBatch; ++k) {
-      const int sl = s0 + k;
-      float ls = __shfl_sync(0xffffffffu, ls_lane, sl & 31);
-      if (sl >= 32 && sl < nslot) ls = a.part_lse[base + (size_t)sl * kRows];
-      if (sl >= nslot || ls == -INFINITY) continue;      // none, or an empty slot
-      const float wgt = ex2(ls - mx);
+      if (ls[k] == -INFINITY) continue;      // none, or an empty slot
+      const float wgt = ex2(ls[k] - mx);
       den += wgt;
       acc.x = fmaf(wgt, v[k].x, acc.x); acc.y = fmaf(wgt, v[k].y, acc.y);
       acc.z = fmaf(wgt, v[k].z, acc.z); acc.w = fmaf(wgt, v[k].w, acc.w);
@@ -732,7 +736,7 @@ __global__ void __launch_bounds__(256) attn_merge_kernel(const AttnArgs a) {
   }
   const float inv = den > 0.f ? 1.f / den : 0.f;
   *dst = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
-  if (a.lse && lane == 0) a.lse[out_row] = den > 0.f ? (mx + log2f(den)) * kLn2 : -INFINITY;
+  if (a.lse && cg == 0) a.lse[out_row] = den > 0.f ? (mx + log2f(den)) * kLn2 : -INFINITY;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -826,9 +830,14 @@ cudaError_t launch_attn(const AttnPlan& plan, cudaStream_t st) {
 }
 
 cudaError_t launch_attn_merge(const AttnPlan& plan, cudaStream_t st) {
-  const long long rows = (long long)plan.a.B * plan.a.Hkv * plan.a.G * plan.a.N;
+  // one warp per (unit, 32 rows, group of four columns): 128 warps per unit, 16 CTAs
+  const long long ctas = (long long)plan.a.B * plan.a.Hkv * plan.a.RT * 16;
   // dependent launch: the CTAs are staged while the attention kernel drains and wait on the device for its end
-  return launch_kernel(attn_merge_kernel, dim3((unsigned)((rows + 7) / 8)), dim3(256), 0, st, true, plan.a);
+  const long long units = (long long)plan.a.B * plan.a.Hkv * plan.a.RT;
+  const long long slots_per_unit = plan.a.S > 0 ? plan.a.S : ((long long)plan.grid.x + units - 1) / units + 1;
+  if (slots_per_unit > 12)
+    return launch_kernel(attn_merge_kernel<24>, dim3((unsigned)ctas), dim3(256), 0, st, true, plan.a);
+  return launch_kernel(attn_merge_kernel<8>, dim3((unsigned)ctas), dim3(256), 0, st, true, plan.a);
 }
 
 }  // namespace lumo
