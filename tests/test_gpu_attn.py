@@ -61,6 +61,9 @@ CASES = [
     ("wide_suffix", "star", 1, 200, 256, 2, 2, [130], "permuted", 2),             # suffix of four key tiles
     ("deep_chain", "chain", 2, 64, 64, 4, 2, [0, 1], "permuted", 1),
     ("more_splits_than_tiles", "random", 2, 8, 8, 4, 2, [10, 100], "identity", 8),
+    # a unit spread over many CTAs: the merge takes more slots than one flight of its wide variant holds
+    ("long_b1_auto", "paper", 1, 28, 32, 8, 2, [16384], "spine", 0),
+    ("split32", "paper", 1, 28, 32, 4, 1, [5000], "spine", 32),
 ]
 
 
