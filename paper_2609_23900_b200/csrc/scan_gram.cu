@@ -407,7 +407,12 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     const int hv = item % s.Hv;
     const int gi = (item / s.Hv) % t.n_groups;                     // node group
     const int layer = item / (s.Hv * t.n_groups);
-    const int4 ginfo = *reinterpret_cast<const int4*>(t.tc_group + gi * 4);
+    // A tree of one group (every tree when there are as many groups as sequences) needs no look-up: group =
+    // sequence, all nodes, first group.  That takes one dependent load off the head of the item's chain
+    // (group -> state row -> state).
+    const bool one_group = t.n_groups == s.B;
+    int4 ginfo = make_int4(gi, s.N, 1, 0);
+    if (!one_group) ginfo = *reinterpret_cast<const int4*>(t.tc_group + gi * 4);
     const int b = ginfo.x, N = ginfo.y;                            // sequence, nodes in this group
     const bool first_group = ginfo.z != 0;                         // writes the per-sequence zero rows
     const LayerPtrs& L = lb.l[layer];
@@ -424,7 +429,7 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
       n_hv = nxt % s.Hv;
       const int n_gi = (nxt / s.Hv) % t.n_groups;
       n_layer = nxt / (s.Hv * t.n_groups);
-      const int4 gi4 = *reinterpret_cast<const int4*>(t.tc_group + n_gi * 4);
+      const int4 gi4 = one_group ? make_int4(n_gi, s.N, 1, 0) : *reinterpret_cast<const int4*>(t.tc_group + n_gi * 4);
       n_b = gi4.x;
       if (tid < gi4.y) n_meta = t.tc_meta[n_gi * kNT + tid];
       n_row = lb.l[n_layer].state_row[n_b];
