@@ -502,7 +502,7 @@ def main():
                     help="also measure configs 3 (recomputed and cached) and 4 (three shapes) in the same run "
                          "(default: on for the default workload)")
     ap.add_argument("--no-extra-configs", dest="extra_configs", action="store_false")
-    ap.add_argument("--scan-algo", default="auto", choices=["auto", "rank1", "gram", "solve", "direct"],
+    ap.add_argument("--scan-algo", default="auto", choices=["auto", "rank1", "gram", "solve", "direct", "tensor"],
                     help="which scan kernel verify uses (auto = the library's choice)")
     ap.add_argument("--attention-only", action="store_true",
                     help="time only the attention layer (the 'attention' block of the default line) and print it as its own JSON line")

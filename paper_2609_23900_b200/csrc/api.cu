@@ -186,8 +186,8 @@ int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx) {
 
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo) {
   if (!ctx) return LUMO_ERR_ARG;
-  if (algo < 0 || algo > 4)
-    return fail(ctx, LUMO_ERR_ARG, "scan algo must be 0 (auto), 1 (rank-1), 2 (Gram form, forward substitution), 3 (solved Gram form) or 4 (Gram form, closed-form tail)");
+  if (algo < 0 || algo > 5)
+    return fail(ctx, LUMO_ERR_ARG, "scan algo must be 0 (auto), 1 (rank-1), 2 (Gram form, forward substitution), 3 (solved Gram form), 4 (Gram form, closed-form tail) or 5 (closed-form tail, output sum on the tensor core)");
   ctx->scan_algo = algo;
   return LUMO_OK;
 }
@@ -403,6 +403,10 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   // closed form is taken when it wins by a margin (28-node spine trees of depth 12: 18.5 -> 17.0 us per
   // launch at batch 8; 64-node trees of depth 8 stay with the substitution: 19.1 against 20.5 us)
   d->closed_form_pays = tc && 100 * subst_rounds > 600 * (long long)G + 18 * group_nodes;
+  // measured with the tensor-core sum (launch times, us, substitution against it): 48 layers of 32-node trees
+  // 190 -> 182, 256-node chains 225 -> 196, random 256-node trees 236 -> 228; a 255-child star 177 -> 200 and
+  // single-wave launches (64-node trees at batch 8: 18.8 against 18.7, but the whole step 38.7 against 39.5) stay
+  d->tensor_tail_pays = tc && 450 * subst_rounds > 300 * (long long)G + 78 * group_nodes;
   if (ctx->device < 0) { *out = d; return LUMO_OK; }   // host-only: tables stay on the host
   DeviceGuard g(ctx->device);
   cudaError_t e = cudaMalloc(&d->dev, h.size() * sizeof(int32_t));
@@ -503,6 +507,18 @@ int lumo_select_spine_top3(lumo_ctx* ctx, const lumo_select_args* a, int32_t* sp
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "select launch");
 }
 
+// Which tail the Gram-form scan takes: 0 level-by-level substitution, 1 closed form, 2 closed form with the output
+// sum on the tensor core.  Automatic: thin deep trees take 2 (equal to 1 there, measured); other trees take 2 when
+// the descriptor says it pays and the launch has several waves of items; everything else takes 0.
+static int scan_tail(const lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo::Shape& s) {
+  if (ctx->scan_algo == 5) return 2;
+  if (ctx->scan_algo == 4) return 1;
+  if (ctx->scan_algo != 0) return 0;
+  if (desc->closed_form_pays) return 2;
+  const long long items = (long long)s.n_layers * desc->n_groups * s.Hv;
+  return desc->tensor_tail_pays && items > 2LL * ctx->sm_count ? 2 : 0;
+}
+
 int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_gdn_args* layers, int n_layers,
                          void* stream) {
   Shape s;
@@ -531,7 +547,7 @@ int lumo_gdn_tree_verify(lumo_ctx* ctx, const lumo_tree_desc* desc, const lumo_g
     e = timed(ctx, LUMO_K_SCAN, st, [&] {
       const bool pdl = use_overlap(ctx, s) && !state_fresh;
       return ctx->scan_algo == 3 ? launch_scan_solve(s, t, lb, ctx->sm_count, pdl, st)
-                                 : launch_scan_gram(s, t, lb, ctx->sm_count, pdl, ctx->scan_algo == 4 || (ctx->scan_algo == 0 && desc->closed_form_pays), st);
+                                 : launch_scan_gram(s, t, lb, ctx->sm_count, pdl, scan_tail(ctx, desc, s), st);
     });
     return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "Gram-form scan launch");
   }

@@ -53,7 +53,7 @@ struct lumo_ctx {
   size_t attn_scratch_bytes = 0;
   uint32_t attn_launch_id = 0;
   // optional per-launch timing (lumo_ctx_timing_*): a fixed pool of event pairs
-  int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form with forward substitution, 3 solved Gram form, 4 Gram form with closed-form tail
+  int scan_algo = 0;            // 0 auto, 1 rank-1, 2 Gram form with forward substitution, 3 solved Gram form, 4 Gram form with closed-form tail, 5 the same with the output sum on the tensor core
   bool timeout_drill = false;   // test aid: the tensor-core scan skips its tensor-core work (lumo_ctx_set_timeout_drill)
   bool overlap = true;          // programmatic dependent launch between conv -> scan -> commit
   // Kind of the previous call that launched on this context.  Kernels that read some of their inputs
@@ -99,6 +99,10 @@ struct lumo_tree_desc {
   // eight nodes of a level, the closed-form tail a fixed part plus a part per node: thin, deep trees (a
   // spine with small side branches) are cheaper in closed form, wide ones by levels.
   bool closed_form_pays = false;
+  // the same comparison for the closed form whose output sum is one tensor-core product (0.3 + 0.078 per node):
+  // it pays on more trees, but only in launches of several waves, where an item's instruction count rather than
+  // its latency sets the pace
+  bool tensor_tail_pays = false;
   uint32_t* d_vis = nullptr;      // [B, N, 8] attention visibility over physical slots (present when Ns <= 256)
   uint32_t* d_slot_used = nullptr;// [B, 8] slots that hold a node
 };
@@ -288,8 +292,9 @@ cudaError_t launch_select(const void* logits, int dtype, int rows, int V, int sp
                           cudaStream_t st);
 // Gram-form scan on tcgen05 (scan_gram.cu)
 bool gram_supported(const Shape& s, int max_depth);
-// direct: closed-form tail (per-node back substitution, one output pass) instead of the level-by-level one
-cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl, bool direct,
+// tail: 0 level-by-level substitution, 1 closed form (per-node back substitution, one output pass over the path),
+// 2 closed form with the output sum as one tensor-core product
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl, int tail,
                              cudaStream_t st);
 // same scan, first replaying the previous cycle's accepted path into the state it has just loaded
 cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,

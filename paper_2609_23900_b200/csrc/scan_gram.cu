@@ -82,6 +82,8 @@ struct Small {
   uint8_t anc[kNT][16];              // positions of the ancestors, root first
   float qq[kNT];                     // |q|^2 of each node when normalising
   uint8_t lvl[20];                   // lvl[d] = number of nodes of depth <= d
+  uint32_t bad[2];                   // tensor-core tail: nodes whose right-hand side is not finite (bit per node; rare)
+  alignas(16) uint32_t out_off[kNT]; // tensor-core tail: element offset of each node's output row, ~0u when another group emits it
   unsigned long long mbar;
   uint32_t tmem_base;
   uint32_t timed_out;
@@ -358,6 +360,231 @@ __device__ __forceinline__ void direct_tail(const Shape& s, const LayerPtrs& L, 
   }
 }
 
+// Closed-form tail with the output sum on the tensor core.  Same scalar part as direct_tail (A, W, then
+// M = W (I + A)^-1 per node along its own root path); the sum o_t = g_t |q scale| S0 q_t + sum_s M[t][s] rhs_s
+// is then ONE product over all nodes of the group, O[row][t] = sum_s RHS[row][s] M[t][s] (M is zero off the
+// path), with both operands split into bf16 hi + lo (three products: hi.hi + hi.lo + lo.hi, relative error
+// 2^-16).  RHS [128 rows x NT nodes] and M [NT x NT] are K-major tiles with the 128-byte swizzle (a row of 64
+// nodes is one swizzle row; with NT = 32 the hi and lo halves share a row).  The result lands in the tensor-
+// memory columns of the Gram block and leaves lane = value row together with the query products.
+// A dense product would let a non-finite right-hand side of ANY node reach every output of the group (0 x NaN),
+// where the recurrence confines it to the node's subtree.  So a right-hand side that is not finite (or overflows
+// bf16) enters the product as zero and marks its node; when any node is marked (rare), the outputs of exactly the
+// nodes with a marked node on their path are written as NaN.  Non-finite keys, queries and gates need no such
+// care: they reach M only in the rows of the node's descendants, and the query products only the node itself.
+// Returns false when the bounded wait for the product ran out.
+template <int NT, class LY, bool kCompact>
+__device__ __forceinline__ bool direct_tail_tc(const Shape& s, const LayerPtrs& L, Small& sm, unsigned char* smem, uint32_t sbase,
+                                               const float* dump, const __nv_bfloat16* Vs, uint32_t tmem, uint32_t tmem_lane,
+                                               int N, int b, int hv, int tid, uint32_t& phase) {
+  const int lane = tid & 31, grp = tid >> 7, vrow = tid & 127;
+  float* Am = reinterpret_cast<float*>(smem + LY::kRec);        // [node][16], in the place of the records
+  float* Wm = Am + NT * 16;
+  static_assert(LY::kRec + NT * 16 * 4 * 2 <= LY::kV, "coefficient tables overflow the record area");
+  constexpr int kRt = kCompact ? LY::kKQ : 0;                   // RHS tiles: over the dead Gram dump, or (compact) over K and Q
+  constexpr int kMt = kCompact ? LY::kKQ + 16384 : LY::kKQ;     // M tiles: over the dead K and Q rows
+  constexpr int kRtTerm = NT == 64 ? 16384 : 64;                // byte distance from the hi to the lo operand
+  constexpr int kMtTerm = NT == 64 ? 8192 : 64;
+  constexpr int kMtBytes = NT == 64 ? 16384 : 4096;
+  static_assert(kCompact || (NT == 64 ? 32768 : 16384) <= LY::kRec, "right-hand-side tiles overflow the dump area");
+  // byte offset of element (row, col) of operand term 0 (hi) or 1 (lo): with NT = 64 the lo operand is a tile of
+  // its own `term_bytes` on, with NT = 32 it is the upper half (k bytes 64..127) of the same swizzled rows
+  auto tile_off = [](int row, int col, int term, int term_bytes) {
+    const int chunk = NT == 64 ? (col >> 3) : term * 4 + (col >> 3);
+    return (NT == 64 ? term * term_bytes : 0) + (int)sw128_offset(row, chunk) + (col & 7) * 2;
+  };
+  // ---- A and W along each node's ancestry (sixteen lanes per node); meanwhile the M tiles are cleared ----
+  for (int i = tid; i < kMtBytes / 16; i += kThreads)             // bounded: <= 4 rounds
+    *reinterpret_cast<uint4*>(smem + kMt + i * 16) = make_uint4(0u, 0u, 0u, 0u);
+  if (tid < 2) sm.bad[tid] = 0u;
+  {
+    const int j = tid & 15, ln = tid >> 4;
+#pragma unroll
+    for (int m = 0; m < NT / 16; ++m) {
+      if (16 * m >= N) break;                                       // uniform
+      const int pi = ln + 16 * m;
+      const int meta = sm.meta[pi];
+      const int D = pi < N ? ((meta >> 16) & 0xFF) : 0;             // depth, 1..16 (the same in all 16 lanes)
+      const bool in = j < D;
+      const int a = sm.anc[pi][j];                                  // 0 beyond the depth
+      float incl = in ? sm.alpha[a] : 1.f;
+#pragma unroll
+      for (int off = 1; off < 16; off <<= 1) {
+        const float v = __shfl_down_sync(0xffffffffu, incl, off, 16);
+        if (j + off < 16) incl *= v;
+      }
+      float excl = __shfl_down_sync(0xffffffffu, incl, 1, 16);      // product over the lanes above j
+      if (j == 15) excl = 1.f;
+      const float g_t = __shfl_sync(0xffffffffu, incl, 0, 16);      // product over the whole path
+      float ksa = 1.f;
+      if (s.l2norm && in) ksa = rsqrtf(dump[a * LY::kStride + a] + s.l2_eps);
+      const float ks_t = __shfl_sync(0xffffffffu, ksa, D > 0 ? D - 1 : 0, 16);
+      const float qs_t = s.l2norm ? s.scale * rsqrtf(sm.qq[pi] + s.l2_eps) : s.scale;
+      const float b_t = sm.beta[pi];
+      float kk = 0.f, qk = 0.f;
+      if (in) { kk = dump[pi * LY::kStride + a]; qk = dump[(NT + pi) * LY::kStride + a]; }
+      Am[pi * 16 + j] = j < D - 1 ? b_t * excl * ks_t * ksa * kk : 0.f;   // no entry for the node itself
+      Wm[pi * 16 + j] = in ? qs_t * excl * ksa * qk : 0.f;
+      if (j == 0) {
+        sm.qs[pi] = g_t * qs_t;                                     // factor of S0 q
+        sm.ks[pi] = b_t * g_t * ks_t;                               // factor of S0 k
+        sm.out_off[pi] = (pi < N && ((meta >> 24) & 1)) ? (uint32_t)((((size_t)b * s.Ns + (meta & 0xFFFF)) * s.Hv + hv) * kD) : 0xFFFFFFFFu;
+      }
+    }
+  }
+  asm volatile("cp.async.wait_group 0;\n" ::: "memory");            // this thread's pieces of V
+  tc_fence_before();                                                // the Gram columns were read: they take the product below
+  __syncthreads();                                                  // A, W, V, cleared M tiles in place; the dump is dead
+  // ---- M by back substitution (four lanes per node), scattered as bf16 hi + lo into the M tiles -----------
+  if (tid < 4 * NT) {                                               // whole warps
+    const int pi = tid >> 2, q4 = tid & 3;
+    const int D = pi < N ? ((sm.meta[pi] >> 16) & 0xFF) : 0;
+    float4 w = *reinterpret_cast<const float4*>(Wm + pi * 16 + 4 * q4);
+    const int Dw = __reduce_max_sync(0xffffffffu, D);
+    for (int jh = Dw - 1; jh >= 1; --jh) {                          // bounded: <= 15 steps
+      const int e = jh & 3;
+      const float cand = e == 0 ? w.x : e == 1 ? w.y : e == 2 ? w.z : w.w;
+      const float mval = __shfl_sync(0xffffffffu, cand, (lane & ~3) | (jh >> 2));
+      if (jh < D) {
+        const float4 ar = *reinterpret_cast<const float4*>(Am + sm.anc[pi][jh] * 16 + 4 * q4);
+        w.x = fmaf(-mval, ar.x, w.x); w.y = fmaf(-mval, ar.y, w.y);
+        w.z = fmaf(-mval, ar.z, w.z); w.w = fmaf(-mval, ar.w, w.w);
+      }
+    }
+    const uint32_t a4 = *reinterpret_cast<const uint32_t*>(&sm.anc[pi][4 * q4]);
+    const float mv[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (4 * q4 + e < D) {
+        const int sidx = (a4 >> (8 * e)) & 0xFF;
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(mv[e]);
+        const __nv_bfloat16 h1 = __float2bfloat16_rn(mv[e] - __bfloat162float(h0));
+        *reinterpret_cast<__nv_bfloat16*>(smem + kMt + tile_off(pi, sidx, 0, kMtTerm)) = h0;
+        *reinterpret_cast<__nv_bfloat16*>(smem + kMt + tile_off(pi, sidx, 1, kMtTerm)) = h1;
+      }
+    }
+  }
+  // ---- right-hand sides: lane = value row, each half of the CTA half of the nodes, eight nodes per 16-byte
+  //      store; padding nodes are written as zeros (their V bytes are stale) ----------------------------------
+  {
+    constexpr int kPer = NT / 2;                                    // nodes per thread
+    const int n0 = grp * kPer;
+    uint32_t pk[kPer];
+    tmem_ld16_issue(tmem_lane + n0, pk);
+    if constexpr (kPer == 32) tmem_ld16_issue(tmem_lane + n0 + 16, pk + 16);
+    tmem_ld_wait();
+#pragma unroll
+    for (int c = 0; c < kPer / 8; ++c) {
+      const int s0 = n0 + 8 * c;
+      const float4 b0 = *reinterpret_cast<const float4*>(&sm.beta[s0]), b1 = *reinterpret_cast<const float4*>(&sm.beta[s0 + 4]);
+      const float4 c0 = *reinterpret_cast<const float4*>(&sm.ks[s0]), c1 = *reinterpret_cast<const float4*>(&sm.ks[s0 + 4]);
+      const float bt[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+      const float ck[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+      float r8[8];
+      uint32_t hi[4], lo[4];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int sn = s0 + e;
+        const float v = __bfloat162float(Vs[sn * kD + vrow]);
+        r8[e] = sn < N ? fmaf(bt[e], v, -ck[e] * __uint_as_float(pk[8 * c + e])) : 0.f;
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(r8[2 * e], r8[2 * e + 1]);
+        hi[e] = *reinterpret_cast<uint32_t*>(&h);
+      }
+      // inf or NaN among the eight (as rounded to bf16)?  One test on the OR of the words: an exponent field of all
+      // ones shows as 0x7F80; the OR can show it where no single value has it, which only costs the exact look below
+      if ((((hi[0] | hi[1] | hi[2] | hi[3]) & 0x7F807F80u) + 0x00800080u) & 0x80008000u) {      // rare
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          if (((hi[e >> 1] >> (16 * (e & 1))) & 0x7F80u) == 0x7F80u) {
+            const int sn = s0 + e;
+            atomicOr(&sm.bad[sn >> 5], 1u << (sn & 31));
+            r8[e] = 0.f;
+            hi[e >> 1] &= (e & 1) ? 0x0000FFFFu : 0xFFFF0000u;
+          }
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float2 hf = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&hi[e]));
+        __nv_bfloat162 l = __floats2bfloat162_rn(r8[2 * e] - hf.x, r8[2 * e + 1] - hf.y);
+        lo[e] = *reinterpret_cast<uint32_t*>(&l);
+      }
+      *reinterpret_cast<uint4*>(smem + kRt + tile_off(vrow, s0, 0, kRtTerm)) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+      *reinterpret_cast<uint4*>(smem + kRt + tile_off(vrow, s0, 1, kRtTerm)) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    }
+  }
+  fence_async_proxy();          // generic-proxy writes -> visible to the tensor core's async proxy
+  __syncthreads();
+  // ---- O = RHS M^T: hi.hi + hi.lo + lo.hi, NT / 16 contraction steps each ----------------------------------
+  if (tid == 0) {
+    tc_fence_after();
+    constexpr uint32_t idesc = umma_idesc(128, NT);
+    const uint64_t d_r = umma_desc(sbase + kRt), d_m = umma_desc(sbase + kMt);
+    constexpr uint64_t r_lo = (uint64_t)(kRtTerm >> 4), m_lo = (uint64_t)(kMtTerm >> 4);
+#pragma unroll
+    for (int ks = 0; ks < NT / 16; ++ks) {
+      const uint64_t koff = (uint64_t)((ks * 32) >> 4);
+      umma(tmem + LY::kGramCol, d_r + koff, d_m + koff, idesc, ks ? 1u : 0u);
+      umma(tmem + LY::kGramCol, d_r + koff, d_m + m_lo + koff, idesc, 1u);
+      umma(tmem + LY::kGramCol, d_r + r_lo + koff, d_m + koff, idesc, 1u);
+    }
+    umma_commit(&sm.mbar);
+  }
+  const bool done = mbar_wait(&sm.mbar, phase);
+  phase ^= 1;
+  tc_fence_after();
+  if (!done) return false;
+  // ---- outputs: lane = value row, each half of the CTA half of the nodes -------------------------------------
+  {
+    constexpr int kPer = NT / 2;
+    const int n0 = grp * kPer;
+    uint32_t oo[kPer], pq[kPer];
+    tmem_ld16_issue(tmem_lane + LY::kGramCol + n0, oo);
+    tmem_ld16_issue(tmem_lane + NT + n0, pq);
+    if constexpr (kPer == 32) {
+      tmem_ld16_issue(tmem_lane + LY::kGramCol + n0 + 16, oo + 16);
+      tmem_ld16_issue(tmem_lane + NT + n0 + 16, pq + 16);
+    }
+    tmem_ld_wait();
+    if (sm.bad[0] | sm.bad[1]) {                                    // uniform over the CTA; rare
+      for (int e = 0; e < kPer; ++e) {                              // bounded: <= 32
+        const int pi = n0 + e;
+        if (pi >= N) break;
+        const int D = (sm.meta[pi] >> 16) & 0xFF;
+        bool hit = false;
+        for (int j = 0; j < D; ++j) {                               // bounded: <= 16
+          const int a = sm.anc[pi][j];
+          hit = hit || ((sm.bad[a >> 5] >> (a & 31)) & 1u);
+        }
+        if (hit) {                                                  // dynamic index into the register array is avoided
+#pragma unroll
+          for (int k = 0; k < kPer; ++k)
+            if (k == e) oo[k] = 0x7FC00000u;
+        }
+      }
+    }
+#pragma unroll
+    for (int e4 = 0; e4 < kPer; e4 += 4) {
+      const float4 cq4 = *reinterpret_cast<const float4*>(&sm.qs[n0 + e4]);
+      const uint4 of4 = *reinterpret_cast<const uint4*>(&sm.out_off[n0 + e4]);
+      const float cqs[4] = {cq4.x, cq4.y, cq4.z, cq4.w};
+      const uint32_t ofs[4] = {of4.x, of4.y, of4.z, of4.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        if (n0 + e4 + k < N && ofs[k] != 0xFFFFFFFFu) {
+          const float o = fmaf(cqs[k], __uint_as_float(pq[e4 + k]), __uint_as_float(oo[e4 + k]));
+          if (s.out_dtype == LUMO_BF16) reinterpret_cast<__nv_bfloat16*>(L.out)[(size_t)ofs[k] + vrow] = __float2bfloat16_rn(o);
+          else reinterpret_cast<float*>(L.out)[(size_t)ofs[k] + vrow] = o;
+        }
+      }
+    }
+  }
+  return true;
+}
+
 // NT = node tile of the MMAs: 64, or 32 when no group of the launch has more than 32 nodes (K rows
 // 0..NT-1 and Q rows NT..2NT-1 of the operand tile; the products occupy NT + NT + NT columns)
 // kFused: before anything else the previous cycle's accepted path is replayed into the state rows as
@@ -365,7 +592,8 @@ __device__ __forceinline__ void direct_tail(const Shape& s, const LayerPtrs& L, 
 // written back in place; the scan then runs from the updated state.  One group per sequence only.
 // kDirect: the triangular system is solved on scalars per node (M = W (I + A)^-1 along each ancestry, no
 // dependency between nodes) and every output is one pass over its path; no level-by-level substitution.
-template <int NT, bool kFused, bool kCompact = false, bool kDirect = false>
+// kTensor (with kDirect): the output sum of the closed form runs on the tensor core (direct_tail_tc).
+template <int NT, bool kFused, bool kCompact = false, bool kDirect = false, bool kTensor = false>
 __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t, const LayerBatch& lb, int n_items,
                                                const FusedPrev* fp) {
   extern __shared__ unsigned char smem_raw[];
@@ -767,7 +995,16 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
     // both halves of the CTA read the Gram rows: 32 of the NT columns each (one half is enough for NT = 32)
     if (grp * 32 < NT) tmem_cols32_to_smem(tmem_lane + LY::kGramCol + grp * 32, dump + vrow * LY::kStride + grp * 32, 1);
     __syncthreads();
-    if constexpr (kDirect) {
+    if constexpr (kDirect && kTensor) {
+      if (!direct_tail_tc<NT, LY, kCompact>(s, L, sm, smem, sbase, dump, Vs, tmem, tmem_lane, N, b, hv, tid, phase)) sm.timed_out = 1;
+      tc_fence_before();
+      __syncthreads();      // tensor memory and the aliased shared memory are free for the next item
+      if (sm.timed_out) {
+        if (L.status && tid == 0) L.status[b] = LUMO_SEQ_TIMEOUT;
+        break;
+      }
+      continue;
+    } else if constexpr (kDirect) {
       direct_tail<NT, LY>(s, L, sm, smem, dump, Vs, tmem_lane, N, b, hv, tid);
       tc_fence_before();
       __syncthreads();      // tensor memory and the aliased shared memory are free for the next item
@@ -916,17 +1153,17 @@ __device__ __forceinline__ void scan_gram_body(const Shape& s, const TreeDev& t,
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(LY::kTmem) : "memory");
 }
 
-template <int NT, bool kDirect>
+template <int NT, bool kDirect, bool kTensor = false>
 __global__ void __launch_bounds__(kThreads, 2)
 scan_gram_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
-  scan_gram_body<NT, false, false, kDirect>(s, t, lb, n_items, nullptr);
+  scan_gram_body<NT, false, false, kDirect, kTensor>(s, t, lb, n_items, nullptr);
 }
 
 // trees of at most 32 nodes, launches of several waves: three smaller CTAs per SM
-template <bool kDirect>
+template <bool kDirect, bool kTensor = false>
 __global__ void __launch_bounds__(kThreads, 3)
 scan_gram_compact_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
-  scan_gram_body<32, false, true, kDirect>(s, t, lb, n_items, nullptr);
+  scan_gram_body<32, false, true, kDirect, kTensor>(s, t, lb, n_items, nullptr);
 }
 
 template <int NT, bool kDirect>
@@ -946,8 +1183,9 @@ bool gram_supported(const Shape& s, int max_depth) {
   return s.d == kD && s.in_dtype == LUMO_BF16 && s.snapshot_mode == 0 && max_depth <= 16;
 }
 
-cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl, bool direct,
+cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl, int tail,
                              cudaStream_t st) {
+  const bool direct = tail != 0;
   const int items = s.n_layers * t.n_groups * s.Hv;
   static bool configured[kMaxDevices] = {};      // the attribute is a per-device setting
   int dev = 0;
@@ -961,6 +1199,9 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
     if (e == cudaSuccess) e = allow_smem(scan_gram_kernel<32, true>, kSmemBytes);
     if (e == cudaSuccess) e = allow_smem(scan_gram_compact_kernel<false>, GL<true>::kBytes);
     if (e == cudaSuccess) e = allow_smem(scan_gram_compact_kernel<true>, GL<true>::kBytes);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_kernel<64, true, true>, kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_kernel<32, true, true>, kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_compact_kernel<true, true>, GL<true>::kBytes);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
@@ -970,12 +1211,13 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
   // round trip per item: they win when a launch has several waves of items (the 48-layer stack: 205 ->
   // 190 us) and lose on a single wave (batch 1: 9.3 -> 10.5 us).
   if (t.max_group_nodes <= 32 && items >= 4 * sm_count) {
-    auto k = direct ? scan_gram_compact_kernel<true> : scan_gram_compact_kernel<false>;
+    auto k = tail == 2 ? scan_gram_compact_kernel<true, true> : direct ? scan_gram_compact_kernel<true> : scan_gram_compact_kernel<false>;
     return launch_kernel(k, dim3(3 * sm_count), dim3(kThreads), GL<true>::kBytes, st, pdl, s, t, lb, items);
   }
   const int grid = items < 2 * sm_count ? items : 2 * sm_count;
   auto k = t.max_group_nodes <= 32 ? (direct ? scan_gram_kernel<32, true> : scan_gram_kernel<32, false>)
                                    : (direct ? scan_gram_kernel<64, true> : scan_gram_kernel<64, false>);
+  if (tail == 2) k = t.max_group_nodes <= 32 ? scan_gram_kernel<32, true, true> : scan_gram_kernel<64, true, true>;
   return launch_kernel(k, dim3(grid), dim3(kThreads), kSmemBytes, st, pdl, s, t, lb, items);
 }
 

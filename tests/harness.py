@@ -11,7 +11,7 @@ _ctx = None
 
 
 def ctx(algo="auto"):
-    """Shared context; `algo` selects the scan kernel ("auto", "rank1", "gram", "solve", "direct") for the calls that follow."""
+    """Shared context; `algo` selects the scan kernel ("auto", "rank1", "gram", "solve", "direct", "tensor") for the calls that follow."""
     global _ctx
     if _ctx is None:
         _ctx = binding.Context(0)

@@ -62,7 +62,7 @@ def _cell_errors(x, ref):
     return np.sqrt((e ** 2).mean(-1)), np.abs(e).max(-1)
 
 
-def paired_rule(ctx, case, algos=("gram", "direct", "solve"), layer=0, with_commit_chain=True):
+def paired_rule(ctx, case, algos=("gram", "direct", "tensor", "solve"), layer=0, with_commit_chain=True):
     """Per scan kernel: cells (sequence, node, value head) inside the paired bound against each native
     side, with the error levels behind the counts."""
     active = np.zeros((case.B, case.Ns), dtype=bool)

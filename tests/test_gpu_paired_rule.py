@@ -47,5 +47,8 @@ def test_paired_error_rule_counts():
     assert k["rank1"]["passed_vs_sequential_kernel"] == res["cells"]
     for algo in ("rank1", "gram", "direct", "solve"):
         assert k[algo]["max_abs_error"] < 2e-6 and k[algo]["median_cell_rms_error"] < 2e-7
+    # the closed form with the tensor-core sum carries its right-hand sides and coefficients as bf16 hi + lo:
+    # relative 2^-16 on that sum, still three orders of magnitude inside the gate and below bf16 output rounding
+    assert k["tensor"]["max_abs_error"] < 2e-5 and k["tensor"]["median_cell_rms_error"] < 2e-6
     # the commit chain with a float64 output product is the more exact native side
     assert res["native"]["commit_chain"]["median_cell_rms_error"] <= res["native"]["sequential_kernel"]["median_cell_rms_error"]

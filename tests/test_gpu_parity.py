@@ -129,7 +129,7 @@ def test_conv_recorded_operands(name):
 # ------------------------------------------------------------------ scan
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("use_conv", [False, True])
-@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct", "tensor"])
 def test_scan_outputs_match_oracle(name, use_conv, algo):
     c = CASES[name]()
     if algo != "rank1" and not gram_eligible(c):
@@ -157,7 +157,7 @@ def test_scan_outputs_match_oracle(name, use_conv, algo):
     assert_close(dc16.np("out"), o_ref, bf16=True, what=f"{name} scan bf16 out")
 
 
-@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct", "tensor"])
 def test_scan_twice_is_bitwise_reproducible(algo):
     c = CASES["cfg2"]()
     dc = DeviceCase(ctx(algo), c)
@@ -171,7 +171,8 @@ def test_scan_twice_is_bitwise_reproducible(algo):
 
 @pytest.mark.parametrize("use_conv", [False, True])
 @pytest.mark.parametrize("algo,shape", [("rank1", "cfg2"), ("gram", "cfg2"), ("direct", "cfg2"), ("direct", "paper"),
-                                        ("gram", "grouped"), ("direct", "grouped"), ("solve", "cfg2")])
+                                        ("gram", "grouped"), ("direct", "grouped"), ("solve", "cfg2"),
+                                        ("tensor", "cfg2"), ("tensor", "paper"), ("tensor", "grouped")])
 def test_path_locality_poisoned_subtree_leaves_the_other_nodes_bitwise_unchanged(algo, shape, use_conv):
     """Sec. "The recurrence and path locality": the output of a node depends on its root path alone.  The
     inputs of one whole subtree per sequence (and of every padding slot) are replaced by NaN (by 1e30 for
@@ -183,9 +184,11 @@ def test_path_locality_poisoned_subtree_leaves_the_other_nodes_bitwise_unchanged
         c = W.config_paper(B=3)
     else:   # 150 nodes per tree: cut into node groups with recomputed prefix paths
         c = W.make_case("grp", rand_parents(5, 150, 3), seed=17, Hk=2, Hv=4, d=128, in_dtype="bf16", Ns=160, permute_slots=True)
-    if algo == "solve" and use_conv:
+    dense = algo == "solve"       # its last product runs over all nodes with zero coefficients off the path (the other
+                                  # tensor-core tail marks non-finite right-hand sides and keeps them out of its product)
+    if dense and use_conv:
         pytest.skip("1e30 through the SiLU of the convolution is no longer finite")
-    poison = 1e30 if algo == "solve" else float("nan")
+    poison = 1e30 if dense else float("nan")
     dc = DeviceCase(ctx(algo), c, use_conv=use_conv)
     dc.verify()
     torch.cuda.synchronize()
@@ -208,29 +211,32 @@ def test_path_locality_poisoned_subtree_leaves_the_other_nodes_bitwise_unchanged
     for b in range(c.B):
         keep = [int(c.slot[b, i]) for i in range(c.N) if not inside[b, i]]
         assert torch.equal(got[b, keep], clean[b, keep]), f"sequence {b}: poison reached a node outside the subtree"
-        if algo != "solve":
+        if not dense:
             gone = [int(c.slot[b, i]) for i in range(c.N) if inside[b, i]]
             assert torch.isnan(got[b, gone]).any(dim=-1).all()               # and the poison was real
     ctx("auto")
 
 
-def test_automatic_choice_between_the_two_tails_follows_the_tree_shape():
-    """Thin deep trees (the paper's geometry: 28 nodes over 12 levels) take the closed-form tail, wide ones
-    (64 nodes over 8 levels) the level-by-level substitution: the automatic choice reproduces the bits of
-    the kernel it is meant to pick, and the two kernels do differ in the last bits."""
-    for case, expect, other in ((W.config_paper(B=3), "direct", "gram"), (CASES["cfg2"](), "gram", "direct")):
+def test_automatic_choice_of_the_tail_follows_the_tree_shape_and_the_launch_size():
+    """Thin deep trees (the paper's geometry: 28 nodes over 12 levels) take the closed-form tail with the
+    tensor-core sum; wide ones in a launch of one wave (64 nodes over 8 levels, batch 8) the level-by-level
+    substitution; the same kind of tree in a launch of several waves (five layers of 32-node trees) the
+    closed form again.  The automatic choice reproduces the bits of the kernel it is meant to pick, and the
+    kernels do differ in the last bits."""
+    for case, expect, other in ((W.config_paper(B=3), "tensor", "gram"), (CASES["cfg2"](), "gram", "tensor"),
+                                (W.config3(n_layers=5), "tensor", "gram")):
         outs = {}
-        for algo in ("auto", "gram", "direct"):
+        for algo in ("auto", "gram", "tensor"):
             dc = DeviceCase(ctx(algo), case)
             dc.verify()
             torch.cuda.synchronize()
-            outs[algo] = dc.t("out").clone()
-        assert torch.equal(outs["auto"], outs[expect])
-        assert not torch.equal(outs["auto"], outs[other])
+            outs[algo] = [dc.t("out", l).clone() for l in range(len(case.layers))]
+        assert all(torch.equal(x, y) for x, y in zip(outs["auto"], outs[expect]))
+        assert not all(torch.equal(x, y) for x, y in zip(outs["auto"], outs[other]))
     ctx("auto")
 
 
-@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct"])
+@pytest.mark.parametrize("algo", ["rank1", "gram", "solve", "direct", "tensor"])
 def test_l2norm_flag_scale_and_f32_gates(algo):
     c = small(rand_parents(4, 20, 2), d=128, dtype="bf16")
     rs = np.random.default_rng(1)
@@ -360,7 +366,7 @@ def test_commit_controls_len0_poisoned_tail_invalid_paths_skipped_rows():
     assert torch.all(dc2.t("out")[2] == 0) and torch.all(dc2.t("out")[3] == 0) and torch.all(dc2.t("q")[2] == 0)
 
 
-@pytest.mark.parametrize("tc", ["gram", "solve", "direct"])
+@pytest.mark.parametrize("tc", ["gram", "solve", "direct", "tensor"])
 def test_gram_scan_skipped_rows_padding_and_depth_16(tc):
     # a 16-deep chain plus side leaves (depth limit of the Gram form), padded and permuted rows,
     # one skipped sequence and one row outside the pool
@@ -391,7 +397,7 @@ def test_gram_scan_skipped_rows_padding_and_depth_16(tc):
     ctx("auto")
 
 
-@pytest.mark.parametrize("tc", ["gram", "solve", "direct"])
+@pytest.mark.parametrize("tc", ["gram", "solve", "direct", "tensor"])
 def test_gram_groups_with_long_prefix_paths(tc):
     # caterpillar: a 10-node spine with 24 leaves under every spine node (250 nodes).  The tree is cut
     # into groups that each carry a prefix path of up to 10 recomputed nodes; every node must still be
@@ -451,7 +457,7 @@ def test_randomized_shapes_both_kernels():
                         beta_uniform=rng.random() < 0.5, with_bias=rng.random() < 0.3)
         use_conv = rng.random() < 0.5
         ref = None
-        for algo in ("solve", "gram", "direct", "rank1"):
+        for algo in ("solve", "gram", "direct", "tensor", "rank1"):
             dc = DeviceCase(ctx(algo), c, use_conv=use_conv)
             dc.t("out").fill_(float("nan"))
             dc.verify()
@@ -553,7 +559,7 @@ def test_kernel_overlap_changes_nothing(name):
     assert not torch.equal(res[True][0][0], res[True][0][1])      # the cycles really advanced the state
 
 
-@pytest.mark.parametrize("algo", ["gram", "direct"])
+@pytest.mark.parametrize("algo", ["gram", "direct", "tensor"])
 @pytest.mark.parametrize("name", ["cfg3_5layers", "paper_geometry_5layers"])
 def test_compact_three_cta_scan_matches_oracle(name, algo):
     """Launches with several waves of items over trees of at most 32 nodes take the compact variant of the

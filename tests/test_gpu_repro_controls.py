@@ -30,7 +30,7 @@ from synthetic import workload as W
 from synthetic.device_case import DeviceAttnCase, DeviceCase
 ctx = binding.Context(0)
 h = hashlib.sha256()
-for algo in ("gram", "direct", "solve", "rank1"):
+for algo in ("gram", "direct", "tensor", "solve", "rank1"):
     ctx.set_scan_algo(algo)
     for rep in range(2):
         dc = DeviceCase(ctx, W.config_paper(B=4), out_dtype="bf16")
@@ -49,7 +49,7 @@ def test_two_fresh_processes_two_runs_each_reproduce_bit_for_bit():
         r = subprocess.run([sys.executable, "-c", _CHILD % ROOT], capture_output=True, text=True, timeout=600)
         assert r.returncode == 0, r.stderr[-2000:]
         outs.append(r.stdout.strip().splitlines())
-    assert outs[0] == outs[1] and len(outs[0]) == 8          # digests chain over kernels and repeats: equal line by line
+    assert outs[0] == outs[1] and len(outs[0]) == 10          # digests chain over kernels and repeats: equal line by line
     # within a process the second run of a kernel extends the digest by the same bytes as the first:
     # checked directly as well
     c = W.config_paper(B=4)
