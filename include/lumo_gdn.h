@@ -124,9 +124,12 @@ int64_t lumo_ctx_scratch_bytes(const lumo_ctx* ctx);
  * system is solved on scalars per head and the state enters a single product with "effective queries"),
  * 4 = the Gram form with a closed-form tail (the same two products as 2; then M = W (I + A)^-1 by a back
  * substitution per node along its own root path and one pass that sums M x right-hand sides: no step
- * waits for another node).  "Automatic" picks between 2 and 4 per descriptor from the shape of its trees
- * (thin deep trees, a spine with small side branches, take 4; wide ones take 2: measured).  2, 3 and 4
- * return LUMO_ERR_UNSUPPORTED on other shapes. */
+ * waits for another node), 5 = the closed form of 4 with that sum as one more tensor-core product over all
+ * nodes of a group (right-hand sides and coefficients as bf16 hi + lo: relative 2^-16 on the sum; a right-hand
+ * side that is not finite is kept out of the product and turns the outputs of its own subtree into NaN, as the
+ * recurrence would).  "Automatic" picks between 2 and 5 per descriptor and launch (thin deep trees, a spine with
+ * small side branches, take 5; other trees take 5 in launches of several waves where it measured faster; the
+ * rest take 2).  2 to 5 return LUMO_ERR_UNSUPPORTED on other shapes. */
 int lumo_ctx_set_scan_algo(lumo_ctx* ctx, int algo);
 
 /* Test aid for the failure path of the tensor-core scan.  That kernel waits for its tensor-core work

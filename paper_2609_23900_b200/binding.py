@@ -169,7 +169,8 @@ class Context:
         return _lib.lumo_ctx_scratch_bytes(self._h)
 
     def set_scan_algo(self, algo: str = "auto"):
-        """"auto" | "rank1" | "gram" | "solve" | "direct" (Gram form with the closed-form tail): which scan kernel verify uses."""
+        """"auto" | "rank1" | "gram" | "solve" | "direct" (Gram form with the closed-form tail) | "tensor" (the same with
+        the output sum on the tensor core): which scan kernel verify uses."""
         self._check(_lib.lumo_ctx_set_scan_algo(self._h, {"auto": 0, "rank1": 1, "gram": 2, "solve": 3, "direct": 4, "tensor": 5}[algo]))
 
     def set_timeout_drill(self, on: bool):
