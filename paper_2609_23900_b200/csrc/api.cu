@@ -404,8 +404,8 @@ int lumo_tree_desc_create(lumo_ctx* ctx, int batch, int n_nodes, int n_slots, co
   // launch at batch 8; 64-node trees of depth 8 stay with the substitution: 19.1 against 20.5 us)
   d->closed_form_pays = tc && 100 * subst_rounds > 600 * (long long)G + 18 * group_nodes;
   // measured with the tensor-core sum (launch times, us, substitution against it): 48 layers of 32-node trees
-  // 190 -> 182, 256-node chains 225 -> 196, random 256-node trees 236 -> 228; a 255-child star 177 -> 200 and
-  // single-wave launches (64-node trees at batch 8: 18.8 against 18.7, but the whole step 38.7 against 39.5) stay
+  // 190 -> 175, 256-node chains 225 -> 190, random 256-node trees 236 -> 218; a 255-child star 177 -> 200 and
+  // single-wave launches (64-node trees at batch 8: equal within 1%, at four times the error) stay
   d->tensor_tail_pays = tc && 450 * subst_rounds > 300 * (long long)G + 78 * group_nodes;
   if (ctx->device < 0) { *out = d; return LUMO_OK; }   // host-only: tables stay on the host
   DeviceGuard g(ctx->device);

@@ -537,7 +537,10 @@ __device__ __forceinline__ bool direct_tail_tc(const Shape& s, const LayerPtrs& 
   phase ^= 1;
   tc_fence_after();
   if (!done) return false;
-  // ---- outputs: lane = value row, each half of the CTA half of the nodes -------------------------------------
+  // ---- outputs: they leave tensor memory lane = value row, cross shared memory [node][row] (over the dead
+  //      right-hand-side tiles) and are written one node per warp, 256 or 512 contiguous bytes at a time -----------
+  float* stage = reinterpret_cast<float*>(smem + kRt);
+  static_assert(kCompact || NT * kD * 4 <= LY::kRec, "output staging overflows the dump area");
   {
     constexpr int kPer = NT / 2;
     const int n0 = grp * kPer;
@@ -549,37 +552,37 @@ __device__ __forceinline__ bool direct_tail_tc(const Shape& s, const LayerPtrs& 
       tmem_ld16_issue(tmem_lane + NT + n0 + 16, pq + 16);
     }
     tmem_ld_wait();
-    if (sm.bad[0] | sm.bad[1]) {                                    // uniform over the CTA; rare
-      for (int e = 0; e < kPer; ++e) {                              // bounded: <= 32
-        const int pi = n0 + e;
-        if (pi >= N) break;
-        const int D = (sm.meta[pi] >> 16) & 0xFF;
-        bool hit = false;
-        for (int j = 0; j < D; ++j) {                               // bounded: <= 16
-          const int a = sm.anc[pi][j];
-          hit = hit || ((sm.bad[a >> 5] >> (a & 31)) & 1u);
-        }
-        if (hit) {                                                  // dynamic index into the register array is avoided
-#pragma unroll
-          for (int k = 0; k < kPer; ++k)
-            if (k == e) oo[k] = 0x7FC00000u;
-        }
-      }
-    }
 #pragma unroll
     for (int e4 = 0; e4 < kPer; e4 += 4) {
       const float4 cq4 = *reinterpret_cast<const float4*>(&sm.qs[n0 + e4]);
-      const uint4 of4 = *reinterpret_cast<const uint4*>(&sm.out_off[n0 + e4]);
       const float cqs[4] = {cq4.x, cq4.y, cq4.z, cq4.w};
-      const uint32_t ofs[4] = {of4.x, of4.y, of4.z, of4.w};
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        if (n0 + e4 + k < N && ofs[k] != 0xFFFFFFFFu) {
-          const float o = fmaf(cqs[k], __uint_as_float(pq[e4 + k]), __uint_as_float(oo[e4 + k]));
-          if (s.out_dtype == LUMO_BF16) reinterpret_cast<__nv_bfloat16*>(L.out)[(size_t)ofs[k] + vrow] = __float2bfloat16_rn(o);
-          else reinterpret_cast<float*>(L.out)[(size_t)ofs[k] + vrow] = o;
-        }
+      for (int k = 0; k < 4; ++k)
+        stage[(n0 + e4 + k) * kD + vrow] = fmaf(cqs[k], __uint_as_float(pq[e4 + k]), __uint_as_float(oo[e4 + k]));
+    }
+  }
+  __syncthreads();
+  const bool any_bad = (sm.bad[0] | sm.bad[1]) != 0u;               // uniform over the CTA; rare
+  const int warp = tid >> 5;
+  for (int pi = warp; pi < N; pi += kWarps) {                       // bounded: <= 8 rounds
+    const uint32_t off = sm.out_off[pi];
+    if (off == 0xFFFFFFFFu) continue;
+    float4 o = *reinterpret_cast<const float4*>(stage + pi * kD + 4 * lane);
+    if (any_bad) {
+      const int D = (sm.meta[pi] >> 16) & 0xFF;
+      bool hit = false;
+      for (int j = 0; j < D; ++j) {                                 // bounded: <= 16
+        const int a = sm.anc[pi][j];
+        hit = hit || ((sm.bad[a >> 5] >> (a & 31)) & 1u);
       }
+      if (hit) o = make_float4(__uint_as_float(0x7FC00000u), __uint_as_float(0x7FC00000u), __uint_as_float(0x7FC00000u), __uint_as_float(0x7FC00000u));
+    }
+    if (s.out_dtype == LUMO_BF16) {
+      __nv_bfloat162 b01 = __floats2bfloat162_rn(o.x, o.y), b23 = __floats2bfloat162_rn(o.z, o.w);
+      *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(L.out) + (size_t)off + 4 * lane) =
+          make_uint2(*reinterpret_cast<uint32_t*>(&b01), *reinterpret_cast<uint32_t*>(&b23));
+    } else {
+      *reinterpret_cast<float4*>(reinterpret_cast<float*>(L.out) + (size_t)off + 4 * lane) = o;
     }
   }
   return true;
