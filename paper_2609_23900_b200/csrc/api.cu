@@ -702,7 +702,7 @@ int lumo_gdn_commit_verify(lumo_ctx* ctx, const lumo_tree_desc* prev_desc, const
   }
   e = timed(ctx, LUMO_K_SCAN, st, [&] {
     return ctx->scan_algo == 3 ? launch_scan_solve_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, st)
-                               : launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, ctx->scan_algo == 4 || (ctx->scan_algo == 0 && desc->closed_form_pays), st);
+                               : launch_scan_gram_fused(s, t, lb, fp, ctx->sm_count, pdl_scan, scan_tail(ctx, desc, s), st);
   });
   return e == cudaSuccess ? LUMO_OK : cuda_fail(ctx, e, "fused scan launch");
 }

@@ -298,7 +298,7 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
                              cudaStream_t st);
 // same scan, first replaying the previous cycle's accepted path into the state it has just loaded
 cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
-                                   int sm_count, bool pdl, bool direct, cudaStream_t st);
+                                   int sm_count, bool pdl, int tail, cudaStream_t st);
 // solved Gram form on tcgen05 (scan_solve.cu): the triangular system solved on scalars, one state product
 cudaError_t launch_scan_solve(const Shape& s, const TreeDev& t, const LayerBatch& lb, int sm_count, bool pdl,
                               cudaStream_t st);

@@ -1169,10 +1169,10 @@ scan_gram_compact_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items) {
   scan_gram_body<32, false, true, kDirect, kTensor>(s, t, lb, n_items, nullptr);
 }
 
-template <int NT, bool kDirect>
+template <int NT, bool kDirect, bool kTensor = false>
 __global__ void __launch_bounds__(kThreads, 2)
 scan_gram_fused_kernel(Shape s, TreeDev t, LayerBatch lb, int n_items, FusedPrev fp) {
-  scan_gram_body<NT, true, false, kDirect>(s, t, lb, n_items, &fp);
+  scan_gram_body<NT, true, false, kDirect, kTensor>(s, t, lb, n_items, &fp);
 }
 
 template <class K>
@@ -1225,7 +1225,8 @@ cudaError_t launch_scan_gram(const Shape& s, const TreeDev& t, const LayerBatch&
 }
 
 cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const LayerBatch& lb, const FusedPrev& fp,
-                                   int sm_count, bool pdl, bool direct, cudaStream_t st) {
+                                   int sm_count, bool pdl, int tail, cudaStream_t st) {
+  const bool direct = tail != 0;
   const int items = s.n_layers * t.n_groups * s.Hv;
   static bool configured[kMaxDevices] = {};      // the attribute is a per-device setting
   int dev = 0;
@@ -1237,12 +1238,15 @@ cudaError_t launch_scan_gram_fused(const Shape& s, const TreeDev& t, const Layer
     if (e == cudaSuccess) e = allow_smem(scan_gram_fused_kernel<32, false>, kSmemBytesFused);
     if (e == cudaSuccess) e = allow_smem(scan_gram_fused_kernel<64, true>, kSmemBytesFused);
     if (e == cudaSuccess) e = allow_smem(scan_gram_fused_kernel<32, true>, kSmemBytesFused);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_fused_kernel<64, true, true>, kSmemBytesFused);
+    if (e == cudaSuccess) e = allow_smem(scan_gram_fused_kernel<32, true, true>, kSmemBytesFused);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
   const int grid = items < 2 * sm_count ? items : 2 * sm_count;
   auto k = t.max_group_nodes <= 32 ? (direct ? scan_gram_fused_kernel<32, true> : scan_gram_fused_kernel<32, false>)
                                    : (direct ? scan_gram_fused_kernel<64, true> : scan_gram_fused_kernel<64, false>);
+  if (tail == 2) k = t.max_group_nodes <= 32 ? scan_gram_fused_kernel<32, true, true> : scan_gram_fused_kernel<64, true, true>;
   return launch_kernel(k, dim3(grid), dim3(kThreads), kSmemBytesFused, st, pdl, s, t, lb, items, fp);
 }
 

@@ -63,7 +63,7 @@ def _oracle(P, C, dcP, layersC, l, accepted, length):
     return st1, hist1, status, y, o_ref
 
 
-@pytest.fixture(params=["auto", "solve", "direct"])
+@pytest.fixture(params=["auto", "solve", "direct", "tensor"])
 def algo(request):
     """Both tensor-core scans have a fused variant; every fused test runs on each."""
     yield request.param
